@@ -1,0 +1,443 @@
+#!/usr/bin/env python
+"""Throughput of the DPSGD gradient-privatisation step (examples/s through per-example weight
+gradients + clip + noise) on synthetic inputs, with the roofline fraction of the dominant kernel
+and the float64 CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload small_cnn|flat|sweep|per_layer]
+    python bench.py --impl reference ...        # times the CPU oracle on a bounded sample
+
+One "step" is one pass of the whole path over one batch: for `small_cnn` 256 examples through
+four weight-gradient calls, one clip-accumulate and one noise-average.  Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "examples/s through per-example wgrad+clip+noise"
+UNIT = "examples/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]), bf16_sustained=float(d["bf16_tflops_sustained"]),
+                    source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- workloads (device side)
+class SmallCnn:
+    """configs[1]: 3 convs + classifier on 32x32x3, B=256, fp32, whole-model clip C=1.5, sigma=1."""
+    name = "small_cnn"
+
+    def __init__(self, torch, rank):
+        from paper_2109_12191_b200 import synth
+        from paper_2109_12191_b200.step import GlobalClipStep
+        self.torch, self.synth = torch, synth
+        self.cfg = synth.small_cnn()
+        self.layers, self.B = self.cfg["layers"], self.cfg["B"]
+        self.step_obj = GlobalClipStep(self.layers, self.B, "f32", self.cfg["C"], self.cfg["sigma"])
+        self.examples_per_step = self.B
+        # inputs rotate over several sets so that consecutive steps never find their inputs in L2
+        self.n_sets = 3
+        g = torch.Generator(device="cuda"); g.manual_seed(1000 + rank)
+        self.sets = [[(torch.randn(l.x_shape(self.B), device="cuda", generator=g),
+                       torch.randn(l.dy_shape(self.B), device="cuda", generator=g)) for l in self.layers]
+                     for _ in range(self.n_sets)]
+        self.in_bytes = sum(x.numel() * 4 + y.numel() * 4 for x, y in self.sets[0])
+        self.host_sets = None
+        self.call_names = [f"wgrad:{l.name}" for l in self.layers] + ["clip_accumulate", "noise_average"]
+
+    def describe(self):
+        return {"workload": "small_cnn: conv3x3 3->32 s1, 32->64 s2, 64->128 s2, dense 8192->10 (all with bias) on 32x32x3, "
+                            "B=256 fp32, global clip C=1.5, sigma=1.0, |B|=256",
+                "examples_per_step": self.B, "params": self.step_obj.P,
+                "l2": f"inputs rotate over {self.n_sets} resident sets ({self.n_sets * self.in_bytes / 1e6:.0f} MB) and "
+                      f"{self.step_obj.P * self.B * 4 / 1e6:.0f} MB of per-example gradients are written and re-read per step; both exceed the 126 MB L2"}
+
+    def run(self, i, rec=None):
+        st = self.step_obj
+        ins = self.sets[i % self.n_sets]
+        st.begin()
+        for li, (X, dY) in enumerate(ins):
+            if rec: rec.start(li)
+            st.wgrad(li, X, dY)
+            if rec: rec.stop(li)
+        k = len(ins)
+        if rec: rec.start(k)
+        st.clip_accumulate()
+        if rec: rec.stop(k)
+        if rec: rec.start(k + 1)
+        st.finish(seed=0, step=i)
+        if rec: rec.stop(k + 1)
+
+    def algorithmic_bytes(self, call):
+        """Bytes each call must move: inputs once, per-example gradients once (written by wgrad, read by clip)."""
+        st = self.step_obj
+        if call < len(self.layers):
+            l = self.layers[call]
+            x = math.prod(l.x_shape(self.B)) * 4
+            y = math.prod(l.dy_shape(self.B)) * 4
+            return x + y + (l.n_weight + l.n_bias) * self.B * 4
+        if call == len(self.layers):
+            return st.P * self.B * 4 + 2 * st.P * 4
+        return 2 * st.P * 4
+
+    def e2e_prepare(self):
+        t = self.torch
+        self.host_sets = [[(x.cpu().pin_memory(), y.cpu().pin_memory()) for x, y in s] for s in self.sets]
+        self.stage = [(t.empty_like(x), t.empty_like(y)) for x, y in self.sets[0]]
+        self.host_out = t.empty(self.step_obj.P, dtype=t.float32).pin_memory()
+        return self.in_bytes, self.step_obj.P * 4
+
+    def e2e_run(self, i):
+        st = self.step_obj
+        hs = self.host_sets[i % self.n_sets]
+        for (dx, dy), (hx, hy) in zip(self.stage, hs):
+            dx.copy_(hx, non_blocking=True); dy.copy_(hy, non_blocking=True)
+        st.begin()
+        for li, (X, dY) in enumerate(self.stage):
+            st.wgrad(li, X, dY)
+        st.clip_accumulate()
+        out = st.finish(seed=0, step=i)
+        self.host_out.copy_(out, non_blocking=True)
+
+    def cpu_sample(self, budget_s):
+        """The oracle on the first examples of one batch: wgrad + norms + clip + sum + noise + average."""
+        import numpy as np
+        import oracle
+        n = self.B
+        ins = [self.synth.layer_inputs(l, n, "f32", 1, li, 0) for li, l in enumerate(self.layers)]
+        reps, t0 = 0, time.perf_counter()
+        while reps < 16 and (reps == 0 or time.perf_counter() - t0 < budget_s):
+            groups = []
+            for l, i in zip(self.layers, ins):
+                if l.kind == "conv":
+                    dW, db = oracle.conv_wgrad(i["X"], i["dY"], l.R, l.S, l.stride, l.pad, bias=l.bias)
+                else:
+                    dW, db = oracle.dense_wgrad(i["X"], i["dY"], bias=l.bias)
+                groups += [dW.reshape(n, -1), db.reshape(n, -1)]
+            oracle.privatise([groups], self.cfg["C"], self.cfg["sigma"], "global", 0, 0)
+            reps += 1
+        dt = time.perf_counter() - t0
+        return n * reps / dt, f"one whole batch of {n} examples, whole path (wgrad, norms, clip, sum, noise, average), repeated {reps} times"
+
+
+class FlatGrad:
+    """configs[3]: flattened ResNet-50 gradients, P=25,557,032, B=64 per chunk, 16 chunks, C=1, sigma=1."""
+    name = "flat"
+
+    def __init__(self, torch, rank):
+        from paper_2109_12191_b200 import synth
+        from paper_2109_12191_b200.step import FlatClipStep
+        self.torch, self.synth = torch, synth
+        self.cfg = synth.resnet50_flat()
+        self.P, self.B, self.G = self.cfg["P"], self.cfg["B"], self.cfg["G"]
+        self.step_obj = FlatClipStep(self.P, self.B, self.cfg["C"], self.cfg["sigma"])
+        self.examples_per_step = self.B * self.G
+        g = torch.Generator(device="cuda"); g.manual_seed(2000 + rank)
+        self.bufs = []
+        for _ in range(2):                                   # two resident chunks (13 GB), alternated
+            t = torch.empty((self.B, self.P), device="cuda")
+            t.normal_(0.0, self.cfg["grad_std"], generator=g)
+            self.bufs.append(t)
+        self.call_names = ["clip_accumulate(norms computed)", "noise_average"]
+
+    def describe(self):
+        return {"workload": "flat: ResNet-50 (GroupNorm) flattened per-example gradients, P=25,557,032 fp32 ~N(0,1e-6), "
+                            "B=64 per chunk x 16 chunks = |B| 1024, global clip C=1.0, sigma=1.0; norms computed by the library",
+                "examples_per_step": self.examples_per_step, "params": self.P,
+                "l2": "each chunk is 6.54 GB, far larger than L2; two resident chunks alternate"}
+
+    def run(self, i, rec=None):
+        st = self.step_obj
+        st.begin()
+        for c in range(self.G):
+            if rec: rec.start(0)
+            st.chunk(self.bufs[c & 1])
+            if rec: rec.stop(0)
+        if rec: rec.start(1)
+        st.finish(seed=0, step=i)
+        if rec: rec.stop(1)
+
+    def algorithmic_bytes(self, call):
+        if call == 0:
+            return 2 * self.B * self.P * 4 + 2 * self.P * 4   # norm pass + clip pass over the chunk, accumulator r+w
+        return 2 * self.P * 4
+
+    def e2e_prepare(self):
+        t = self.torch
+        self.host_chunk = t.empty((self.B, self.P), dtype=t.float32).pin_memory()
+        self.host_chunk.copy_(self.bufs[0])
+        self.host_out = t.empty(self.P, dtype=t.float32).pin_memory()
+        return self.B * self.P * 4 * self.G, self.P * 4
+
+    def e2e_run(self, i):
+        st = self.step_obj
+        st.begin()
+        for c in range(self.G):
+            self.bufs[c & 1].copy_(self.host_chunk, non_blocking=True)
+            st.chunk(self.bufs[c & 1])
+        self.host_out.copy_(st.finish(seed=0, step=i), non_blocking=True)
+
+    def cpu_sample(self, budget_s):
+        import numpy as np
+        import oracle
+        n, P = 8, self.P
+        G = self.synth.normal_f32((n, P), 3, 0, 0, scale=self.cfg["grad_std"])
+        t0 = time.perf_counter()
+        acc, _, _ = oracle.clipped_sum([G], self.cfg["C"], "global")
+        oracle.noise_average(acc[0], 0, self.cfg["sigma"], self.cfg["C"], n, 0, 0)
+        dt = time.perf_counter() - t0
+        return n / dt, f"{n} examples of one 64-example chunk at full P (norms, clip, sum) plus one noise+average pass"
+
+
+WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad}
+
+
+class CallTimer:
+    """CUDA-event pairs around each C-ABI call, recorded on the stream the kernels are launched on."""
+
+    def __init__(self, torch, n_calls):
+        self.torch, self.n = torch, n_calls
+        self.pairs = [[] for _ in range(n_calls)]
+        self._open = {}
+
+    def start(self, k):
+        e = self.torch.cuda.Event(enable_timing=True)
+        e.record()
+        self._open[k] = e
+
+    def stop(self, k):
+        e = self.torch.cuda.Event(enable_timing=True)
+        e.record()
+        self.pairs[k].append((self._open.pop(k), e))
+
+    def totals_ms(self):
+        return [sum(a.elapsed_time(b) for a, b in p) for p in self.pairs]
+
+    def counts(self):
+        return [len(p) for p in self.pairs]
+
+
+def run_ours(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    import __graft_entry__
+    if rank == 0:
+        __graft_entry__.build()
+    if dist:
+        dist.barrier()
+    from paper_2109_12191_b200 import binding as b
+
+    wl = WORKLOADS[args.workload](torch, rank)
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for i in range(warmup):
+        wl.run(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    rec = CallTimer(torch, len(wl.call_names))
+    launches0 = b.dp_debug_launch_count()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(steps):
+        wl.run(warmup + i, rec)
+    t_end.record()
+    barrier()
+    launches = b.dp_debug_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = t_start.elapsed_time(t_end)
+    if dist:
+        t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = t.item()
+    value = wl.examples_per_step * steps * world / (ms / 1e3)
+
+    # ---- end to end: pinned host inputs -> device, the step, result -> host, every step
+    h2d, d2h = wl.e2e_prepare()
+    e2e_steps = max(3, min(steps, args.e2e_steps))
+    for i in range(2):
+        wl.e2e_run(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        wl.e2e_run(i)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist:
+        t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = t.item()
+    e2e_value = wl.examples_per_step * e2e_steps * world / (e2e_ms / 1e3)
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant call (largest share of device time)
+    peaks = measured_peaks()
+    totals, counts = rec.totals_ms(), rec.counts()
+    dom = max(range(len(totals)), key=lambda k: totals[k])
+    avg_ms = totals[dom] / counts[dom]
+    achieved = wl.algorithmic_bytes(dom) / (avg_ms / 1e3) / 1e9
+    roofline = {"bound": "hbm", "kernel": wl.call_names[dom], "achieved": round(achieved, 1), "peak": peaks["hbm"],
+                "peak_source": peaks["source"], "unit": "GB/s", "frac": round(achieved / peaks["hbm"], 4),
+                "avg_ms_per_launch": round(avg_ms, 5), "traffic": None,
+                "shares": {n: round(t / sum(totals), 4) for n, t in zip(wl.call_names, totals)}}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        v, sample = wl.cpu_sample(10.0)
+        cpu = {"value": round(v, 3), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample}
+
+    line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": round(ms / steps, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": wl.describe(),
+            "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The oracle, as it stands, on this machine's host cores; each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import __graft_entry__
+    import oracle
+    oracle.build()
+
+    class _NoTorch:
+        pass
+    cls = WORKLOADS[args.workload]
+    wl = cls.__new__(cls)
+    from paper_2109_12191_b200 import synth
+    wl.synth = synth
+    if args.workload == "small_cnn":
+        wl.cfg = synth.small_cnn(); wl.layers = wl.cfg["layers"]; wl.B = wl.cfg["B"]
+        config = {"workload": "small_cnn (CPU oracle, whole batches)", "examples_per_step": 256}
+    else:
+        wl.cfg = synth.resnet50_flat(); wl.P, wl.B, wl.G = wl.cfg["P"], wl.cfg["B"], wl.cfg["G"]
+        config = {"workload": "flat (CPU oracle on a sample)", "examples_per_step": 8}
+    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
+    for _ in range(warmup):
+        wl.cpu_sample(1.0)
+    vals, sample = [], ""
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        v, sample = wl.cpu_sample(5.0)
+        vals.append(v)
+    dt = time.perf_counter() - t0
+    v = statistics.mean(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": round(v, 3), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": steps, "warmup": warmup, "ms_per_step": round(dt / steps * 1e3, 3), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": round(v, 3), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(v, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    defaults = {"small_cnn": (400, 10), "flat": (8, 3)}
+    if args.steps is None:
+        args.steps = defaults[args.workload][0]
+    if args.warmup is None:
+        args.warmup = defaults[args.workload][1]
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,188 @@
+/*
+ * dpstep.h -- C ABI of the DPSGD gradient-privatisation step for one NVIDIA B200 (sm_100a).
+ *
+ * The step (paper section 2, "Algorithm", equation for g_t):
+ *
+ *     g_t = ( N(0, sigma^2 C^2 I) + sum_{x_j in B} clip(grad L(theta, x_j), C) ) / |B|
+ *
+ * with clip(g, C) = g * min(1, C / ||g||_2), the batch B reached by accumulating chunks
+ * of examples (section 2, "gradient accumulation"), and optionally each of M parameter
+ * groups clipped on its own to C / sqrt(M) (section 3.5).
+ *
+ * General rules for every entry point
+ *   - Every data pointer is a DEVICE pointer unless its comment says "host".  All device
+ *     buffers are allocated, owned and freed by the caller; the library allocates no
+ *     device memory and keeps no state between calls (scratch comes in as `workspace`).
+ *   - Device pointers must be 16-byte aligned; tensors are dense, row-major, channels-last:
+ *       conv   X [B,H,W,C_in]   dY [B,OH,OW,K_out]   G_w [B,K_out,R,S,C_in]   G_b [B,K_out]
+ *       dense  X [B,C_in]       dY [B,K_out]         G_w [B,K_out,C_in]       G_b [B,K_out]
+ *       norm   X = normalised activation [B,H,W,C_in], dY [B,H,W,C_in], G_w = dgamma [B,C_in],
+ *              G_b = dbeta [B,C_in]
+ *     with OH = (H + 2*pad - R)/stride + 1 (integer division), likewise OW.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronising.  Arguments are validated on the host
+ *     before anything is launched; on error nothing has been launched.
+ *   - Functions return a dp_status; they never abort, throw or print.
+ */
+#ifndef DPSTEP_H
+#define DPSTEP_H
+
+#include <stddef.h>
+
+#if defined(__GNUC__)
+#define DP_API __attribute__((visibility("default")))
+#else
+#define DP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DP_OK = 0,
+    DP_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, non-positive size, bad enum, bad C or sigma */
+    DP_ERR_UNSUPPORTED = 2,   /* a valid request this build has no kernel for */
+    DP_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or smaller than dp_workspace_bytes() */
+    DP_ERR_CUDA = 4,          /* a CUDA runtime / driver call or a launch failed */
+    DP_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up (reported through dp_wgrad_check) */
+} dp_status;
+
+typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;            /* type of X and dY; every output is fp32 */
+typedef enum { DP_LAYER_DENSE = 0, DP_LAYER_CONV2D = 1, DP_LAYER_NORM_AFFINE = 2 } dp_layer_kind;
+typedef enum { DP_CLIP_GLOBAL = 0, DP_CLIP_PER_LAYER = 1 } dp_clip_mode;
+typedef enum {
+    DP_EPI_STORE_NORM = 0,    /* write per-example gradients G_w (and G_b) and sqnorm[B]          */
+    DP_EPI_NORM_ONLY = 1,     /* write sqnorm[B] only; no per-example gradient reaches memory     */
+    DP_EPI_CLIP_ACCUM = 2     /* clip each example of this layer to C_l and add the sum to acc    */
+} dp_epilogue;
+typedef enum {
+    DP_IMPL_AUTO = 0,         /* tensor-core kernel when the shape allows it, else the CUDA-core one */
+    DP_IMPL_CUDA_CORE = 1,    /* force the fp32 FMA kernel (any shape)                              */
+    DP_IMPL_TENSOR_CORE = 2   /* force the tcgen05 kernel; DP_ERR_UNSUPPORTED if the shape is not eligible */
+} dp_impl;
+
+typedef struct {
+    int kind;                 /* dp_layer_kind */
+    int dtype;                /* dp_dtype of X and dY */
+    int B;                    /* examples in this chunk, >= 1 */
+    int C_in, H, W;           /* input channels and spatial size (dense: H = W = 1) */
+    int K_out, R, S;          /* output channels and filter size (dense: R = S = 1; norm: K_out = C_in, R = S = 1) */
+    int stride, pad;          /* conv only (dense / norm: 1, 0); dilation 1 and groups 1 are the only ones built */
+    int has_bias;             /* conv / dense: 1 if a bias gradient is wanted; norm: ignored, dbeta always exists */
+    int bias_separate;        /* 0: weight and bias form ONE parameter group (one norm, one clip factor per example);
+                                 1: they are TWO groups (section 3.5 counts parameter tensors), so sqnorm and
+                                    clip_out carry two values per example: (weight, bias) */
+    int impl;                 /* dp_impl */
+} dp_layer_desc;
+
+/* Number of parameter groups the layer reports per example: 2 when bias_separate != 0 and the
+ * layer has a bias-like tensor, else 1 (0 for an invalid descriptor). */
+DP_API int dp_layer_groups(const dp_layer_desc *desc);
+
+/* Bytes of device scratch dp_per_example_wgrad needs for this layer and epilogue
+ * (0 for an invalid descriptor).  The scratch holds per-tile partial squared norms and,
+ * for some paths, per-example bias gradients or clip factors. */
+DP_API size_t dp_workspace_bytes(const dp_layer_desc *desc, int epilogue);
+
+/* Per-example weight gradients of one layer for a chunk of B examples
+ * (section 2: "per-example gradients are computed"; the layer formulas are the standard
+ * weight gradients given X and dY):
+ *     conv   G_w[n,k,r,s,c] = sum_{oh,ow} dY[n,oh,ow,k] * Xpad[n, oh*stride+r-pad, ow*stride+s-pad, c]
+ *            G_b[n,k]       = sum_{oh,ow} dY[n,oh,ow,k]
+ *     dense  G_w[n,o,i] = dY[n,o] * X[n,i];   G_b[n,o] = dY[n,o]
+ *     norm   G_w[n,c] = sum_{h,w} dY[n,h,w,c] * X[n,h,w,c];   G_b[n,c] = sum_{h,w} dY[n,h,w,c]
+ * and the squared L2 norm of each example's gradient of this layer, taken from the accumulators
+ * before they leave the chip (for the rank-1 dense gradient: the closed form |dY_n|^2 |X_n|^2).
+ *
+ *   X, dY      inputs, type desc->dtype.
+ *   G_w, G_b   [B, P_w], [B, P_b] fp32 outputs; required for DP_EPI_STORE_NORM (G_b only when
+ *              the layer has a bias), ignored otherwise.
+ *   sqnorm     fp32 output, always written: sqnorm[n*sqnorm_stride + g] for example n and group g
+ *              (g < dp_layer_groups()); sqnorm_stride >= groups lets a layer write its column(s) of the
+ *              [B, L] table dp_clip_accumulate reads.
+ *   C_l        clip threshold of this layer, used by DP_EPI_CLIP_ACCUM only (> 0, +inf allowed).
+ *   acc_w/b    [P_w], [P_b] fp32, read-modify-write; DP_EPI_CLIP_ACCUM only:
+ *              acc += sum_n min(1, C_l/||g_n||) * g_n  (section 3.5, one group = this layer).
+ *   clip_out   optional [B, groups] fp32: the factors that were applied (DP_EPI_CLIP_ACCUM).
+ *   workspace  at least dp_workspace_bytes(desc, epilogue) bytes, 256-byte aligned.
+ *
+ * Results are bit-reproducible from run to run (fixed reduction orders, no float atomics).
+ * Errors: DP_ERR_INVALID_ARG, DP_ERR_UNSUPPORTED, DP_ERR_WORKSPACE, DP_ERR_CUDA. */
+DP_API dp_status dp_per_example_wgrad(const dp_layer_desc *desc, const void *X, const void *dY,
+                               float *G_w, float *G_b, float *sqnorm, long long sqnorm_stride,
+                               int epilogue, float C_l, float *acc_w, float *acc_b, float *clip_out,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Bytes of device scratch dp_clip_accumulate needs (per-block partial norms and factors). */
+DP_API size_t dp_clip_workspace_bytes(int B, int L, const long long *P_l /* host, [L] */);
+
+/* Norm, clip and accumulate over materialised per-example gradients
+ * (section 2, the sum over x_j in B of clip(.,C); section 3.5 for the per-layer mode):
+ *     GLOBAL     s_n = sum_l ||G_l[n]||^2,  f_n = min(1, C/sqrt(s_n)),            acc_l += sum_n f_n * G_l[n]
+ *     PER_LAYER  s_{n,l} = ||G_l[n]||^2,    f_{n,l} = min(1, (C/sqrt(L))/sqrt(s_{n,l})), acc_l += sum_n f_{n,l} * G_l[n]
+ * The factor is exactly 1 when s <= threshold^2 (so a zero gradient and C = +inf are safe).
+ * Calling it once per chunk accumulates over chunks (section 2, gradient accumulation).
+ *
+ *   G        host array of L device pointers, G[l] = [B, P_l] fp32.  L = 1 is a flat [B, P] matrix.
+ *   P_l      host array of L sizes (> 0).
+ *   sqnorm   device [B, L] fp32 (row n holds the L per-tensor squared norms of example n, as
+ *            written by dp_per_example_wgrad) or NULL, in which case the norms are computed
+ *            here with one extra pass over G.
+ *   C        clip norm of the whole gradient, > 0, +inf allowed.
+ *   acc      host array of L device pointers, acc[l] = [P_l] fp32, read-modify-write.
+ *   norms_out  optional device fp32: GLOBAL [B] whole-gradient L2 norms; PER_LAYER [B, L].
+ *   clip_out   optional device fp32, same shape: the factors applied.
+ *   workspace  at least dp_clip_workspace_bytes(B, L, P_l) bytes, 256-byte aligned. */
+DP_API dp_status dp_clip_accumulate(int mode, int B, int L, const float *const *G, const long long *P_l,
+                             const float *sqnorm, float C, float *const *acc,
+                             float *norms_out, float *clip_out,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Noise and average (section 2): out[i] = (acc[i] + sigma * C * z_{param_offset+i}) / total_batch,
+ * one pass, `out` may alias `acc`.  z is a standard normal that depends only on
+ * (seed, step, global parameter index g = param_offset + i):
+ *   Philox4x32-10 (Salmon et al., SC'11) with counter (lo32(g/4), hi32(g/4), lo32(step), hi32(step))
+ *   and key (lo32(seed), hi32(seed)) gives words r0..r3;  for the pair (a,b) = (0,1) resp. (2,3):
+ *   u1 = ((r_a >> 9) + 0.5) * 2^-23, u2 = (r_b >> 8) * 2^-24, radius = sqrt(-2 ln u1),
+ *   lane g%4 = 0,2 takes radius*cos(2 pi u2), lane 1,3 takes radius*sin(2 pi u2).
+ * sigma = 0 adds nothing, whatever C is; with sigma > 0, C must be finite.
+ * In per-layer mode C is still the whole-gradient bound (the per-group thresholds are chosen so
+ * that the whole gradient keeps sensitivity C).
+ * Errors: DP_ERR_INVALID_ARG for P <= 0, param_offset < 0, total_batch <= 0, sigma < 0, C <= 0. */
+DP_API dp_status dp_noise_average(const float *acc, long long P, long long param_offset,
+                           float sigma, float C, long long total_batch,
+                           unsigned long long seed, unsigned long long step,
+                           float *out, void *cuda_stream);
+
+/* Test hook: the raw Philox words of blocks first_block .. first_block+n_blocks-1 of the
+ * (seed, step) stream described above, out4 = [n_blocks, 4] uint32 on the device. */
+DP_API dp_status dp_debug_philox_raw(unsigned int *out4, long long n_blocks, long long first_block,
+                              unsigned long long seed, unsigned long long step, void *cuda_stream);
+
+/* Test hook: the standard normals z_g for g = first_index .. first_index+count-1, fp32 on the device. */
+DP_API dp_status dp_debug_noise_z(float *z, long long count, long long first_index,
+                           unsigned long long seed, unsigned long long step, void *cuda_stream);
+
+/* Reads (with a synchronising copy) the device status word some tensor-core launches keep at
+ * the start of `workspace`: DP_OK, or DP_ERR_TIMEOUT when a bounded wait inside the kernel
+ * expired (the kernel then returned early and its outputs are invalid). */
+DP_API dp_status dp_wgrad_check(const void *workspace, void *cuda_stream);
+
+/* 1 if dp_per_example_wgrad would run this layer on the tcgen05 tensor-core kernel under
+ * DP_IMPL_AUTO, else 0 (also 0 for an invalid descriptor). */
+DP_API int dp_wgrad_uses_tensor_cores(const dp_layer_desc *desc, int epilogue);
+
+DP_API const char *dp_status_string(int status);
+
+/* Text of the last CUDA error this thread's calls ran into ("" if none). Host memory owned by the library. */
+DP_API const char *dp_last_cuda_error(void);
+
+/* Number of kernels this process has launched through the library so far (a host-side counter;
+ * benchmarks report the difference over their timed region). */
+DP_API unsigned long long dp_debug_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPSTEP_H */

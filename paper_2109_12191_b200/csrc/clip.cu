@@ -1,0 +1,281 @@
+// Norm, clip and accumulate over materialised per-example gradients
+// (paper section 2: sum over the batch of clip(g_j, C); section 3.5: per-group threshold C/sqrt(M)).
+//
+// Three memory-bound stages, all with fixed reduction orders:
+//   1. (only when the caller has no norms) per-block partial sums of squares of every example row,
+//      then one block per (tensor, example) folds the partials;
+//   2. one small kernel turns squared norms into clip factors;
+//   3. every thread owns four neighbouring parameters, streams the B example rows through
+//      registers with 128-bit loads, and touches the accumulator once.
+#include "common.cuh"
+#include <math.h>
+
+namespace dp {
+
+constexpr int kMaxSeg = 40;          // tensors per launch (table travels as a kernel parameter)
+constexpr int kNormChunk = 8192;     // floats of one example row reduced by one block (stage 1)
+constexpr int kAccCols = 1024;       // parameters per block in stage 3 (256 threads x float4)
+
+struct SegTable {
+    const float *G[kMaxSeg];         // [B, P] per tensor
+    float *acc[kMaxSeg];             // [P] per tensor
+    long long P[kMaxSeg];
+    int blk_start[kMaxSeg + 1];      // first block of each tensor within this launch
+    int col[kMaxSeg];                // index l of the tensor in the [B, L] norm / factor tables
+    long long part_start[kMaxSeg];   // first partial slot of each tensor within one example's row of partials
+    int nseg;
+};
+
+__device__ __forceinline__ int find_seg(const SegTable &t, int blk) {
+    int s = 0;
+    while (s + 1 < t.nseg && blk >= t.blk_start[s + 1]) ++s;
+    return s;
+}
+
+// stage 1a: partial[n][part_start[seg] + j] = sum of squares of G_seg[n, j*chunk .. (j+1)*chunk)
+__global__ void __launch_bounds__(256)
+sqnorm_partial_kernel(const __grid_constant__ SegTable tab, float *__restrict__ partial, long long parts_per_example) {
+    __shared__ float scratch[32];
+    const int seg = find_seg(tab, blockIdx.x);
+    const int j = blockIdx.x - tab.blk_start[seg];
+    const int n = blockIdx.y;
+    const long long P = tab.P[seg];
+    const long long c0 = (long long)j * kNormChunk;
+    const int len = (int)min((long long)kNormChunk, P - c0);
+    const float *row = tab.G[seg] + (long long)n * P + c0;
+    float a = 0.f;
+    if ((reinterpret_cast<uintptr_t>(row) & 15) == 0) {
+        const float4 *row4 = reinterpret_cast<const float4 *>(row);
+        const int n4 = len >> 2;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+        for (int i = threadIdx.x; i < n4; i += 256) {
+            const float4 v = __ldg(row4 + i);
+            a0 = fmaf(v.x, v.x, a0); a1 = fmaf(v.y, v.y, a1); a2 = fmaf(v.z, v.z, a2); a3 = fmaf(v.w, v.w, a3);
+        }
+        a = (a0 + a1) + (a2 + a3);
+        for (int i = (n4 << 2) + threadIdx.x; i < len; i += 256) a = fmaf(row[i], row[i], a);
+    } else {
+        for (int i = threadIdx.x; i < len; i += 256) a = fmaf(row[i], row[i], a);
+    }
+    a = block_sum(a, scratch);
+    if (threadIdx.x == 0) partial[(long long)n * parts_per_example + tab.part_start[seg] + j] = a;
+}
+
+// stage 1b: sq[n][col[seg]] = sum over the tensor's partials, in index order, in double
+__global__ void __launch_bounds__(128)
+sqnorm_fold_kernel(const __grid_constant__ SegTable tab, const float *__restrict__ partial,
+                   long long parts_per_example, float *__restrict__ sq, int L) {
+    __shared__ double scratch[32];
+    const int seg = blockIdx.x, n = blockIdx.y;
+    const long long nparts = (tab.P[seg] + kNormChunk - 1) / kNormChunk;
+    const float *p = partial + (long long)n * parts_per_example + tab.part_start[seg];
+    double a = 0.0;
+    for (long long i = threadIdx.x; i < nparts; i += 128) a += (double)p[i];
+    a = block_sum(a, scratch);
+    if (threadIdx.x == 0) sq[(long long)n * L + tab.col[seg]] = (float)a;
+}
+
+// stage 2: factors.  GLOBAL: one factor per example from the sum over its L tensors (thread per example).
+// PER_LAYER: one factor per (example, tensor) against C/sqrt(L).
+__global__ void clip_factor_kernel(const float *__restrict__ sq, int B, int L, int per_layer, float C,
+                                   float *__restrict__ factor, float *norms_out, float *clip_out) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (per_layer) {
+        if (idx >= B * L) return;
+        const float thr = (float)((double)C / sqrt((double)L));
+        const double s = (double)sq[idx];
+        const float f = clip_factor(s, thr);
+        factor[idx] = f;
+        if (norms_out) norms_out[idx] = (float)sqrt(s);
+        if (clip_out) clip_out[idx] = f;
+    } else {
+        if (idx >= B) return;
+        double s = 0.0;
+        for (int l = 0; l < L; ++l) s += (double)sq[(long long)idx * L + l];
+        const float f = clip_factor(s, C);
+        factor[idx] = f;
+        if (norms_out) norms_out[idx] = (float)sqrt(s);
+        if (clip_out) clip_out[idx] = f;
+    }
+}
+
+// stage 3: acc[i] += sum_n factor * G[n, i].  factor index: GLOBAL n, PER_LAYER n*L + col.
+template <int UNROLL>
+__global__ void __launch_bounds__(256)
+scale_accumulate_kernel(const __grid_constant__ SegTable tab, const float *__restrict__ factor, int B, int L,
+                        int per_layer) {
+    __shared__ float f_sh[256];
+    const int seg = find_seg(tab, blockIdx.x);
+    const long long P = tab.P[seg];
+    const long long c0 = (long long)(blockIdx.x - tab.blk_start[seg]) * kAccCols;
+    const float *G = tab.G[seg];
+    float *acc = tab.acc[seg];
+    const int f_stride = per_layer ? L : 1;
+    const int f_off = per_layer ? tab.col[seg] : 0;
+    // vector path needs every row start 16-byte aligned: base aligned and P a multiple of 4
+    const bool vec = ((P & 3) == 0) && ((reinterpret_cast<uintptr_t>(G) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(acc) & 15) == 0);
+    if (vec) {
+        const long long i = c0 + 4 * threadIdx.x;
+        const bool live = i < P;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int n0 = 0; n0 < B; n0 += 256) {
+            const int nb = min(256, B - n0);
+            __syncthreads();
+            if (threadIdx.x < nb) f_sh[threadIdx.x] = factor[(long long)(n0 + threadIdx.x) * f_stride + f_off];
+            __syncthreads();
+            if (live) {
+                const float *g = G + (long long)n0 * P + i;
+                int n = 0;
+                for (; n + UNROLL <= nb; n += UNROLL) {
+                    float4 v[UNROLL];
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u)
+                        v[u] = __ldcs(reinterpret_cast<const float4 *>(g + (long long)(n + u) * P));
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const float f = f_sh[n + u];
+                        s.x = fmaf(f, v[u].x, s.x); s.y = fmaf(f, v[u].y, s.y);
+                        s.z = fmaf(f, v[u].z, s.z); s.w = fmaf(f, v[u].w, s.w);
+                    }
+                }
+                for (; n < nb; ++n) {
+                    const float4 v = __ldcs(reinterpret_cast<const float4 *>(g + (long long)n * P));
+                    const float f = f_sh[n];
+                    s.x = fmaf(f, v.x, s.x); s.y = fmaf(f, v.y, s.y); s.z = fmaf(f, v.z, s.z); s.w = fmaf(f, v.w, s.w);
+                }
+            }
+        }
+        if (live) {
+            float4 a = *reinterpret_cast<const float4 *>(acc + i);
+            a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
+            *reinterpret_cast<float4 *>(acc + i) = a;
+        }
+    } else {
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int n0 = 0; n0 < B; n0 += 256) {
+            const int nb = min(256, B - n0);
+            __syncthreads();
+            if (threadIdx.x < nb) f_sh[threadIdx.x] = factor[(long long)(n0 + threadIdx.x) * f_stride + f_off];
+            __syncthreads();
+            for (int n = 0; n < nb; ++n) {
+                const float f = f_sh[n];
+                const float *g = G + (long long)(n0 + n) * P + c0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const long long i = threadIdx.x + 256 * q;
+                    if (c0 + i < P) s[q] = fmaf(f, g[i], s[q]);
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const long long i = c0 + threadIdx.x + 256 * q;
+            if (i < P) acc[i] += s[q];
+        }
+    }
+}
+
+struct ClipPlan {
+    size_t partial_off, sq_off, factor_off, total;
+    long long parts_per_example;
+};
+
+static bool plan(int B, int L, const long long *P_l, ClipPlan &pl) {
+    long long parts = 0;
+    for (int l = 0; l < L; ++l) {
+        if (P_l[l] <= 0) return false;
+        parts += (P_l[l] + kNormChunk - 1) / kNormChunk;
+    }
+    pl.parts_per_example = parts;
+    size_t off = 0;
+    pl.partial_off = off; off = round_up(off + sizeof(float) * (size_t)parts * B, 256);
+    pl.sq_off = off;      off = round_up(off + sizeof(float) * (size_t)B * L, 256);
+    pl.factor_off = off;  off = round_up(off + sizeof(float) * (size_t)B * L, 256);
+    pl.total = off;
+    return true;
+}
+
+}  // namespace dp
+
+extern "C" size_t dp_clip_workspace_bytes(int B, int L, const long long *P_l) {
+    dp::ClipPlan pl;
+    if (B <= 0 || L <= 0 || !P_l || !dp::plan(B, L, P_l, pl)) return 0;
+    return pl.total;
+}
+
+extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                        const float *sqnorm, float C, float *const *acc, float *norms_out,
+                                        float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    using namespace dp;
+    if (mode != DP_CLIP_GLOBAL && mode != DP_CLIP_PER_LAYER) return DP_ERR_INVALID_ARG;
+    if (B <= 0 || L <= 0 || !G || !P_l || !acc || !(C > 0.0f)) return DP_ERR_INVALID_ARG;
+    if (B > 65535) return DP_ERR_UNSUPPORTED;
+    ClipPlan pl;
+    if (!plan(B, L, P_l, pl)) return DP_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l) {
+        if (!G[l] || !acc[l] || !aligned(G[l], 4) || !aligned(acc[l], 4)) return DP_ERR_INVALID_ARG;
+        if ((P_l[l] + kAccCols - 1) / kAccCols > 0x3fffffffll) return DP_ERR_UNSUPPORTED;
+    }
+    if (sqnorm && !aligned(sqnorm, 4)) return DP_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < pl.total) return DP_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    float *partial = reinterpret_cast<float *>(ws + pl.partial_off);
+    float *sq_ws = reinterpret_cast<float *>(ws + pl.sq_off);
+    float *factor = reinterpret_cast<float *>(ws + pl.factor_off);
+    const int per_layer = (mode == DP_CLIP_PER_LAYER);
+
+    // tensors go to the kernels in tables of at most kMaxSeg entries
+    auto fill = [&](int l0, SegTable &t, bool norm_blocks, long long &part_cursor) {
+        t.nseg = 0;
+        int blk = 0;
+        for (int l = l0; l < L && t.nseg < kMaxSeg; ++l) {
+            const int s = t.nseg++;
+            t.G[s] = G[l]; t.acc[s] = acc[l]; t.P[s] = P_l[l]; t.col[s] = l;
+            t.blk_start[s] = blk;
+            t.part_start[s] = part_cursor;
+            const long long nparts = (P_l[l] + kNormChunk - 1) / kNormChunk;
+            part_cursor += nparts;
+            const long long nb = norm_blocks ? nparts : (P_l[l] + kAccCols - 1) / kAccCols;
+            if ((long long)blk + nb > 0x7fffffffll) { --t.nseg; part_cursor -= nparts; break; }
+            blk += (int)nb;
+        }
+        t.blk_start[t.nseg] = blk;
+        return blk;
+    };
+
+    const float *sq = sqnorm;
+    if (!sq) {
+        long long cursor = 0;
+        for (int l0 = 0; l0 < L;) {
+            SegTable t;
+            const int blocks = fill(l0, t, true, cursor);
+            if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
+            sqnorm_partial_kernel<<<dim3((unsigned)blocks, (unsigned)B), 256, 0, stream>>>(t, partial, pl.parts_per_example);
+            DP_LAUNCH_CHECK("sqnorm_partial_kernel");
+            sqnorm_fold_kernel<<<dim3((unsigned)t.nseg, (unsigned)B), 128, 0, stream>>>(t, partial, pl.parts_per_example, sq_ws, L);
+            DP_LAUNCH_CHECK("sqnorm_fold_kernel");
+            l0 += t.nseg;
+        }
+        sq = sq_ws;
+    }
+    {
+        const long long count = per_layer ? (long long)B * L : B;
+        clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, stream>>>(sq, B, L, per_layer, C, factor, norms_out, clip_out);
+        DP_LAUNCH_CHECK("clip_factor_kernel");
+    }
+    {
+        long long cursor = 0;
+        for (int l0 = 0; l0 < L;) {
+            SegTable t;
+            const int blocks = fill(l0, t, false, cursor);
+            if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
+            scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
+            DP_LAUNCH_CHECK("scale_accumulate_kernel");
+            l0 += t.nseg;
+        }
+    }
+    return DP_OK;
+}

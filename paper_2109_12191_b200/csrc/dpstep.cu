@@ -1,0 +1,218 @@
+// Host side of dp_per_example_wgrad: argument checks, workspace layout, and the choice between
+// the tcgen05 tensor-core kernel and the CUDA-core kernels.
+#include "wgrad_simple.cuh"
+#include "wgrad_tc.cuh"
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+#include <atomic>
+
+namespace dp {
+
+static thread_local char g_last_error[256] = "";
+static std::atomic<unsigned long long> g_launches{0};
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+dp_status cuda_fail(cudaError_t e, const char *where) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+    return DP_ERR_CUDA;
+}
+
+static bool valid_desc(const dp_layer_desc *d) {
+    if (!d) return false;
+    if (d->kind != DP_LAYER_DENSE && d->kind != DP_LAYER_CONV2D && d->kind != DP_LAYER_NORM_AFFINE) return false;
+    if (d->dtype != DP_F32 && d->dtype != DP_BF16) return false;
+    if (d->impl != DP_IMPL_AUTO && d->impl != DP_IMPL_CUDA_CORE && d->impl != DP_IMPL_TENSOR_CORE) return false;
+    if (d->B <= 0 || d->C_in <= 0 || d->K_out <= 0 || d->H <= 0 || d->W <= 0) return false;
+    if (d->kind == DP_LAYER_CONV2D) {
+        if (d->R <= 0 || d->S <= 0 || d->stride <= 0 || d->pad < 0) return false;
+        if (d->H + 2 * d->pad < d->R || d->W + 2 * d->pad < d->S) return false;
+    } else {
+        if (d->R != 1 || d->S != 1 || d->stride != 1 || d->pad != 0) return false;
+        if (d->kind == DP_LAYER_DENSE && (d->H != 1 || d->W != 1)) return false;
+        if (d->kind == DP_LAYER_NORM_AFFINE && d->K_out != d->C_in) return false;
+    }
+    return true;
+}
+
+static ConvGeom geom_of(const dp_layer_desc *d) {
+    ConvGeom g;
+    g.B = d->B; g.H = d->H; g.W = d->W; g.Cin = d->C_in; g.Kout = d->K_out; g.R = d->R; g.S = d->S;
+    g.stride = d->stride; g.pad = d->pad;
+    g.OH = (d->H + 2 * d->pad - d->R) / d->stride + 1;
+    g.OW = (d->W + 2 * d->pad - d->S) / d->stride + 1;
+    g.M = d->K_out; g.N = d->R * d->S * d->C_in; g.K = g.OH * g.OW;
+    return g;
+}
+
+static bool has_bias_tensor(const dp_layer_desc *d) { return d->kind == DP_LAYER_NORM_AFFINE || d->has_bias != 0; }
+static int groups_of(const dp_layer_desc *d) { return (d->bias_separate && has_bias_tensor(d)) ? 2 : 1; }
+
+struct WgradPlan {
+    bool use_tc;
+    int slots, w_slots;
+    size_t status_off, partial_off, factor_off, db_off, chunk_off, dg_off, tc_off, total;
+};
+
+static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
+    const ConvGeom g = geom_of(d);
+    const size_t B = (size_t)d->B;
+    pl.use_tc = false;
+    if (d->kind == DP_LAYER_CONV2D && d->impl != DP_IMPL_CUDA_CORE) pl.use_tc = tc_eligible(d->dtype, g, epi);
+    size_t off = 0;
+    pl.status_off = off; off += 256;
+    if (d->kind == DP_LAYER_CONV2D) {
+        const int tiles = pl.use_tc ? tc_norm_slots(d->dtype, g, epi) : fma_tiles_m(g) * fma_tiles_n(g);
+        pl.w_slots = tiles;
+        pl.slots = tiles + (d->has_bias ? bias_blocks(g) : 0);
+    } else {
+        pl.w_slots = 1; pl.slots = 2;
+    }
+    pl.partial_off = off; off = round_up(off + sizeof(float) * B * pl.slots, 256);
+    pl.factor_off = off;  off = round_up(off + sizeof(float) * B * 2, 256);
+    pl.db_off = off;
+    if (d->kind != DP_LAYER_NORM_AFFINE && d->has_bias) off = round_up(off + sizeof(float) * B * d->K_out, 256);
+    pl.chunk_off = off; pl.dg_off = off;
+    if (d->kind == DP_LAYER_NORM_AFFINE) {
+        off = round_up(off + sizeof(float) * B * norm_chunks(d->H * d->W) * 2 * d->C_in, 256);
+        pl.dg_off = off;
+        off = round_up(off + sizeof(float) * B * 2 * d->C_in, 256);
+    }
+    pl.tc_off = off;
+    if (pl.use_tc) off = round_up(off + tc_workspace_bytes(d->dtype, g, epi), 256);
+    pl.total = off;
+    return true;
+}
+
+}  // namespace dp
+
+using namespace dp;
+
+extern "C" int dp_layer_groups(const dp_layer_desc *desc) { return valid_desc(desc) ? groups_of(desc) : 0; }
+
+extern "C" size_t dp_workspace_bytes(const dp_layer_desc *desc, int epilogue) {
+    if (!valid_desc(desc) || epilogue < 0 || epilogue > 2) return 0;
+    WgradPlan pl;
+    make_plan(desc, epilogue, pl);
+    return pl.total;
+}
+
+extern "C" int dp_wgrad_uses_tensor_cores(const dp_layer_desc *desc, int epilogue) {
+    if (!valid_desc(desc) || epilogue < 0 || epilogue > 2) return 0;
+    WgradPlan pl;
+    make_plan(desc, epilogue, pl);
+    return pl.use_tc ? 1 : 0;
+}
+
+extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X, const void *dY, float *G_w, float *G_b,
+                                          float *sqnorm, long long sqnorm_stride, int epi, float C_l, float *acc_w,
+                                          float *acc_b, float *clip_out, void *workspace, size_t workspace_bytes,
+                                          void *cuda_stream) {
+    if (!valid_desc(d) || epi < 0 || epi > 2) return DP_ERR_INVALID_ARG;
+    if (!X || !dY || !sqnorm || !aligned(X, 16) || !aligned(dY, 16) || !aligned(sqnorm, 4)) return DP_ERR_INVALID_ARG;
+    const int groups = groups_of(d);
+    const bool bias = has_bias_tensor(d);
+    if (sqnorm_stride < groups) return DP_ERR_INVALID_ARG;
+    if (epi == DP_EPI_STORE_NORM) {
+        if (!G_w || !aligned(G_w, 16) || (bias && (!G_b || !aligned(G_b, 16)))) return DP_ERR_INVALID_ARG;
+    }
+    if (epi == DP_EPI_CLIP_ACCUM) {
+        if (!(C_l > 0.0f)) return DP_ERR_INVALID_ARG;
+        if (!acc_w || !aligned(acc_w, 16) || (bias && (!acc_b || !aligned(acc_b, 16)))) return DP_ERR_INVALID_ARG;
+        if (clip_out && !aligned(clip_out, 4)) return DP_ERR_INVALID_ARG;
+    }
+    WgradPlan pl;
+    make_plan(d, epi, pl);
+    if (d->impl == DP_IMPL_TENSOR_CORE && !pl.use_tc) return DP_ERR_UNSUPPORTED;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < pl.total) return DP_ERR_WORKSPACE;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    float *partial = reinterpret_cast<float *>(ws + pl.partial_off);
+    float *factor = reinterpret_cast<float *>(ws + pl.factor_off);
+    float *db_ws = reinterpret_cast<float *>(ws + pl.db_off);
+    const ConvGeom g = geom_of(d);
+    const int clip = (epi == DP_EPI_CLIP_ACCUM);
+    dp_status rc;
+    DP_CUDA_TRY(cudaMemsetAsync(ws + pl.status_off, 0, 16, st));
+
+    if (d->kind == DP_LAYER_CONV2D) {
+        float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;
+        if (d->has_bias) {
+            rc = launch_bias(d->dtype, dY, g, db, partial, pl.slots, pl.w_slots, st);
+            if (rc != DP_OK) return rc;
+        }
+        if (epi != DP_EPI_CLIP_ACCUM) {
+            if (pl.use_tc) rc = launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
+            else rc = launch_conv_fma(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, st);
+            if (rc != DP_OK) return rc;
+            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
+        }
+        // per-layer clipping: norms of every example first, then the clipped sum with the factors known
+        if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
+        else rc = launch_conv_fma(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, st);
+        if (rc != DP_OK) return rc;
+        rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st);
+        if (rc != DP_OK) return rc;
+        if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
+        else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, st);
+        if (rc != DP_OK) return rc;
+        if (d->has_bias) return launch_bias_accum(db, d->B, d->K_out, factor, acc_b, st);
+        return DP_OK;
+    }
+
+    if (d->kind == DP_LAYER_DENSE) {
+        if (epi == DP_EPI_STORE_NORM) {
+            rc = launch_dense_store(d->dtype, X, dY, d->B, d->C_in, d->K_out, G_w, d->has_bias ? G_b : nullptr, st);
+            if (rc != DP_OK) return rc;
+        }
+        rc = launch_dense_norm(d->dtype, X, dY, d->B, d->C_in, d->K_out, d->has_bias, partial,
+                               (clip && d->has_bias) ? db_ws : nullptr, st);
+        if (rc != DP_OK) return rc;
+        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st);
+        if (rc != DP_OK || !clip) return rc;
+        // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
+        rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, 2, factor, acc_w, st);
+        if (rc != DP_OK) return rc;
+        if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
+        return DP_OK;
+    }
+
+    // normalisation affine
+    {
+        float *chunk_partial = reinterpret_cast<float *>(ws + pl.chunk_off);
+        float *dg = (epi == DP_EPI_STORE_NORM) ? G_w : reinterpret_cast<float *>(ws + pl.dg_off);
+        float *dbt = (epi == DP_EPI_STORE_NORM) ? G_b : reinterpret_cast<float *>(ws + pl.dg_off) + (size_t)d->B * d->C_in;
+        rc = launch_norm_affine(d->dtype, X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
+        if (rc != DP_OK) return rc;
+        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st);
+        if (rc != DP_OK || !clip) return rc;
+        return launch_affine_accum(dg, dbt, d->B, d->C_in, factor, acc_w, acc_b, st);
+    }
+}
+
+extern "C" dp_status dp_wgrad_check(const void *workspace, void *cuda_stream) {
+    if (!workspace) return DP_ERR_INVALID_ARG;
+    int status = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DP_CUDA_TRY(cudaMemcpyAsync(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost, st));
+    DP_CUDA_TRY(cudaStreamSynchronize(st));
+    return status == 0 ? DP_OK : DP_ERR_TIMEOUT;
+}
+
+extern "C" const char *dp_status_string(int status) {
+    switch (status) {
+        case DP_OK: return "ok";
+        case DP_ERR_INVALID_ARG: return "invalid argument";
+        case DP_ERR_UNSUPPORTED: return "unsupported";
+        case DP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case DP_ERR_CUDA: return "CUDA error";
+        case DP_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char *dp_last_cuda_error(void) { return dp::g_last_error; }
+
+extern "C" unsigned long long dp_debug_launch_count(void) { return dp::g_launches.load(std::memory_order_relaxed); }

@@ -1,0 +1,453 @@
+// CUDA-core (fp32 FMA) per-example weight gradients: the any-shape path for convolutions, the
+// dense outer product, the normalisation-affine reduction, bias sums, and the small kernels that
+// fold per-tile squared norms into per-example norms and clip factors.
+// Formulas: paper section 2 (per-example gradient, its L2 norm, clip) and section 3.5 (per-layer threshold).
+#include "wgrad_simple.cuh"
+#include <math.h>
+
+namespace dp {
+
+constexpr int TM = kFmaTile, TN = kFmaTile, TK = 16;
+
+// Per-example gradient matrix D_n[m, j] = sum_q A[q, m] * Bm[q, j] with
+//   A[q, m]  = dY[n, pix, m]                       q = n*K + pix
+//   Bm[q, j] = Xpad[n, oh*st + r - pad, ow*st + s - pad, c],  j = (r*S + s)*Cin + c
+// MODE 0/1: the block owns one example (blockIdx.z) and reduces q over that example's pixels.
+// MODE 2:   the block owns the tile for ALL examples: q runs over B*K and A is scaled by the
+//           example's clip factor, so the accumulator ends as sum_n f_n D_n[m, j].
+template <typename T, int MODE>
+__global__ void __launch_bounds__(256)
+conv_wgrad_fma_kernel(const T *__restrict__ X, const T *__restrict__ dY, const ConvGeom g, float *__restrict__ G_w,
+                      float *__restrict__ partial, int slots, const float *__restrict__ factor,
+                      float *__restrict__ acc_w) {
+    __shared__ __align__(16) float sA[TK][TM];
+    __shared__ __align__(16) float sB[TK][TN];
+    __shared__ float scratch[32];
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.y * TM, j0 = blockIdx.x * TN;
+    const int n_fixed = (MODE == 2) ? 0 : blockIdx.z;
+    const long long q_begin = (MODE == 2) ? 0 : (long long)n_fixed * g.K;
+    const long long q_end = (MODE == 2) ? (long long)g.B * g.K : q_begin + g.K;
+
+    // loader role: this thread fills column lm of sA and column lj of sB for rows lp, lp+4, lp+8, lp+12
+    const int lcol = tid & 63, lp = tid >> 6;
+    const bool a_ok = (m0 + lcol) < g.M;
+    const int jj = j0 + lcol;
+    const bool b_ok = jj < g.N;
+    const int c = b_ok ? jj % g.Cin : 0;
+    const int rs = b_ok ? jj / g.Cin : 0;
+    const int r = rs / g.S, s = rs % g.S;
+
+    float ra[4], rb[4];
+    auto fetch = [&](long long qc) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const long long q = qc + lp + 4 * i;
+            ra[i] = 0.f; rb[i] = 0.f;
+            if (q < q_end) {
+                const int n = (int)(q / g.K);
+                const int pix = (int)(q - (long long)n * g.K);
+                if (a_ok) {
+                    float v = to_float(dY[q * g.Kout + m0 + lcol]);
+                    if (MODE == 2) v *= factor[2 * n];
+                    ra[i] = v;
+                }
+                if (b_ok) {
+                    const int oh = pix / g.OW, ow = pix - oh * g.OW;
+                    const int ih = oh * g.stride + r - g.pad, iw = ow * g.stride + s - g.pad;
+                    if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W)
+                        rb[i] = to_float(X[(((long long)n * g.H + ih) * g.W + iw) * g.Cin + c]);
+                }
+            }
+        }
+    };
+
+    const int ty = tid >> 4, tx = tid & 15;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[i][k] = 0.f;
+
+    fetch(q_begin);
+    for (long long qc = q_begin; qc < q_end; qc += TK) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { sA[lp + 4 * i][lcol] = ra[i]; sB[lp + 4 * i][lcol] = rb[i]; }
+        __syncthreads();
+        if (qc + TK < q_end) fetch(qc + TK);
+#pragma unroll
+        for (int kk = 0; kk < TK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4 *>(&sA[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4 *>(&sB[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) acc[i][k] = fmaf(av[i], bv[k], acc[i][k]);
+        }
+        __syncthreads();
+    }
+
+    const int jb = j0 + tx * 4;
+    if (MODE == 0 || MODE == 1) {
+        float sq = 0.f;   // rows / columns outside the matrix hold exact zeros, no masking needed
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) sq = fmaf(acc[i][k], acc[i][k], sq);
+        sq = block_sum(sq, scratch);
+        if (tid == 0) partial[(long long)n_fixed * slots + blockIdx.y * gridDim.x + blockIdx.x] = sq;
+    }
+    if (MODE == 0 || MODE == 2) {
+        float *base = (MODE == 0) ? G_w + (long long)n_fixed * g.M * g.N : acc_w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int m = m0 + ty * 4 + i;
+            if (m >= g.M) continue;
+            float *row = base + (long long)m * g.N;
+            if ((g.N & 3) == 0) {
+                if (jb < g.N) {
+                    float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                    if (MODE == 2) {
+                        const float4 o = *reinterpret_cast<const float4 *>(row + jb);
+                        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                    }
+                    *reinterpret_cast<float4 *>(row + jb) = v;
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (jb + k < g.N) row[jb + k] = (MODE == 2) ? row[jb + k] + acc[i][k] : acc[i][k];
+            }
+        }
+    }
+}
+
+// db[n, k] = sum over pixels of dY[n, pix, k]; 64 channels x 4 pixel lanes per block, lanes folded in order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bias_kernel(const T *__restrict__ dY, int K, int Kout, float *__restrict__ db, float *__restrict__ partial, int slots,
+            int slot0) {
+    __shared__ float lanes[4][kBiasCols];
+    __shared__ float scratch[32];
+    const int n = blockIdx.y, col = threadIdx.x & 63, lane = threadIdx.x >> 6;
+    const int k = blockIdx.x * kBiasCols + col;
+    float a = 0.f;
+    if (k < Kout) {
+        const T *p = dY + (long long)n * K * Kout + k;
+        for (int pix = lane; pix < K; pix += 4) a += to_float(p[(long long)pix * Kout]);
+    }
+    lanes[lane][col] = a;
+    __syncthreads();
+    float sq = 0.f;
+    if (lane == 0 && k < Kout) {
+        const float v = (lanes[0][col] + lanes[1][col]) + (lanes[2][col] + lanes[3][col]);
+        db[(long long)n * Kout + k] = v;
+        sq = v * v;
+    }
+    sq = block_sum(sq, scratch);
+    if (threadIdx.x == 0) partial[(long long)n * slots + slot0 + blockIdx.x] = sq;
+}
+
+// One block per example: weight slots [0, w_slots) and bias slots [w_slots, slots) summed in index order.
+__global__ void __launch_bounds__(128)
+finalize_norm_kernel(const float *__restrict__ partial, int slots, int w_slots, int separate, float *__restrict__ sqnorm,
+                     long long sq_stride, int clip, float C_l, float *__restrict__ factor, float *clip_out) {
+    __shared__ double scratch[32];
+    const int n = blockIdx.x;
+    const float *p = partial + (long long)n * slots;
+    double sw = 0.0, sb = 0.0;
+    for (int i = threadIdx.x; i < w_slots; i += 128) sw += (double)p[i];
+    for (int i = w_slots + threadIdx.x; i < slots; i += 128) sb += (double)p[i];
+    sw = block_sum(sw, scratch);
+    sb = block_sum(sb, scratch);
+    if (threadIdx.x != 0) return;
+    if (separate) {
+        sqnorm[n * sq_stride] = (float)sw;
+        sqnorm[n * sq_stride + 1] = (float)sb;
+        if (clip) {
+            const float fw = clip_factor(sw, C_l), fb = clip_factor(sb, C_l);
+            factor[2 * n] = fw; factor[2 * n + 1] = fb;
+            if (clip_out) { clip_out[2 * n] = fw; clip_out[2 * n + 1] = fb; }
+        }
+    } else {
+        const double s = sw + sb;
+        sqnorm[n * sq_stride] = (float)s;
+        if (clip) {
+            const float f = clip_factor(s, C_l);
+            factor[2 * n] = f; factor[2 * n + 1] = f;
+            if (clip_out) clip_out[n] = f;
+        }
+    }
+}
+
+__global__ void bias_accum_kernel(const float *__restrict__ db, int B, int Kout, const float *__restrict__ factor,
+                                  float *__restrict__ acc_b) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= Kout) return;
+    float a = 0.f;
+    for (int n = 0; n < B; ++n) a = fmaf(factor[2 * n + 1], db[(long long)n * Kout + k], a);
+    acc_b[k] += a;
+}
+
+// ------------------------------------------------------------------ dense layer
+// G_w[n, o, i] = dY[n, o] * X[n, i]: pure store stream, four columns per thread when Cin % 4 == 0.
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(256)
+dense_store_kernel(const T *__restrict__ X, const T *__restrict__ dY, long long total, int Cin, int Kout,
+                   float *__restrict__ G_w) {
+    const int per_row = VEC ? (Cin >> 2) : Cin;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const long long row = idx / per_row;             // n * Kout + o
+        const int i = (int)(idx - row * per_row);
+        const long long n = row / Kout;
+        const float gy = to_float(dY[row]);
+        if (VEC) {
+            const T *x = X + n * Cin + 4 * i;
+            const float4 v = make_float4(gy * to_float(x[0]), gy * to_float(x[1]), gy * to_float(x[2]), gy * to_float(x[3]));
+            __stcs(reinterpret_cast<float4 *>(G_w + row * Cin) + i, v);
+        } else {
+            G_w[row * Cin + i] = gy * to_float(X[n * Cin + i]);
+        }
+    }
+}
+
+template <typename T>
+__global__ void widen_kernel(const T *__restrict__ src, long long count, float *__restrict__ dst) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) dst[i] = to_float(src[i]);
+}
+
+// rank-1 closed form: |dY_n^T X_n|_F^2 = |dY_n|^2 |X_n|^2, bias part |dY_n|^2
+template <typename T>
+__global__ void __launch_bounds__(256)
+dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, int Kout, int has_bias,
+                  float *__restrict__ partial) {
+    __shared__ double scratch[32];
+    const int n = blockIdx.x;
+    double sx = 0.0, sy = 0.0;
+    for (int i = threadIdx.x; i < Cin; i += 256) { const double v = to_float(X[(long long)n * Cin + i]); sx += v * v; }
+    for (int i = threadIdx.x; i < Kout; i += 256) { const double v = to_float(dY[(long long)n * Kout + i]); sy += v * v; }
+    sx = block_sum(sx, scratch);
+    sy = block_sum(sy, scratch);
+    if (threadIdx.x == 0) {
+        partial[2 * n] = (float)(sx * sy);
+        partial[2 * n + 1] = has_bias ? (float)sy : 0.f;
+    }
+}
+
+// ------------------------------------------------------------------ normalisation affine
+// stage 1: block = (channel-vector block, pixel chunk, example); thread = (pixel row, channel vector).
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, int HW, int C, int tcv,
+                           float *__restrict__ chunk_partial, int chunks) {
+    extern __shared__ float red[];                       // [rows][tcv*VEC*2]
+    const int n = blockIdx.z, chunk = blockIdx.y;
+    const int rows = 256 / tcv;
+    const int prow = threadIdx.x / tcv, cvi = threadIdx.x - prow * tcv;
+    const int c0 = (blockIdx.x * tcv + cvi) * VEC;
+    const bool live = prow < rows && c0 < C;
+    float sg[VEC], sb[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { sg[v] = 0.f; sb[v] = 0.f; }
+    const int p_end = min(HW, (chunk + 1) * kNormPix);
+    if (live) {
+        for (int p = chunk * kNormPix + prow; p < p_end; p += rows) {
+            const long long off = ((long long)n * HW + p) * C + c0;
+            T xv[VEC], gv[VEC];
+            if (VEC * sizeof(T) == 16) {
+                *reinterpret_cast<uint4 *>(xv) = __ldcs(reinterpret_cast<const uint4 *>(X + off));
+                *reinterpret_cast<uint4 *>(gv) = __ldcs(reinterpret_cast<const uint4 *>(dY + off));
+            } else {
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) { xv[v] = X[off + v]; gv[v] = dY[off + v]; }
+            }
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) {
+                const float gg = to_float(gv[v]);
+                sg[v] = fmaf(gg, to_float(xv[v]), sg[v]);
+                sb[v] += gg;
+            }
+        }
+    }
+    const int width = tcv * VEC * 2;
+    if (prow < rows) {
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            red[prow * width + cvi * VEC + v] = sg[v];
+            red[prow * width + tcv * VEC + cvi * VEC + v] = sb[v];
+        }
+    }
+    __syncthreads();
+    if (prow == 0 && c0 < C) {
+        float *out = chunk_partial + (((long long)n * chunks + chunk) * 2) * C;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            float a = 0.f, b = 0.f;
+            for (int rr = 0; rr < rows; ++rr) {
+                a += red[rr * width + cvi * VEC + v];
+                b += red[rr * width + tcv * VEC + cvi * VEC + v];
+            }
+            out[c0 + v] = a;
+            out[C + c0 + v] = b;
+        }
+    }
+}
+
+// stage 2: fold chunks in index order, store dgamma / dbeta, squared norms of both
+__global__ void __launch_bounds__(256)
+norm_affine_fold_kernel(const float *__restrict__ chunk_partial, int chunks, int C, float *__restrict__ dgamma,
+                        float *__restrict__ dbeta, float *__restrict__ partial2) {
+    __shared__ double scratch[32];
+    const int n = blockIdx.x;
+    double qg = 0.0, qb = 0.0;
+    for (int c = threadIdx.x; c < C; c += 256) {
+        float a = 0.f, b = 0.f;
+        for (int k = 0; k < chunks; ++k) {
+            const float *p = chunk_partial + (((long long)n * chunks + k) * 2) * C;
+            a += p[c];
+            b += p[C + c];
+        }
+        dgamma[(long long)n * C + c] = a;
+        dbeta[(long long)n * C + c] = b;
+        qg += (double)a * a;
+        qb += (double)b * b;
+    }
+    qg = block_sum(qg, scratch);
+    qb = block_sum(qb, scratch);
+    if (threadIdx.x == 0) { partial2[2 * n] = (float)qg; partial2[2 * n + 1] = (float)qb; }
+}
+
+__global__ void affine_accum_kernel(const float *__restrict__ dgamma, const float *__restrict__ dbeta, int B, int C,
+                                    const float *__restrict__ factor, float *__restrict__ acc_w,
+                                    float *__restrict__ acc_b) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    float a = 0.f, b = 0.f;
+    for (int n = 0; n < B; ++n) {
+        a = fmaf(factor[2 * n], dgamma[(long long)n * C + c], a);
+        b = fmaf(factor[2 * n + 1], dbeta[(long long)n * C + c], b);
+    }
+    acc_w[c] += a;
+    acc_b[c] += b;
+}
+
+// ------------------------------------------------------------------ host launchers
+template <typename T>
+static dp_status conv_fma_t(int mode, const T *X, const T *dY, const ConvGeom &g, float *G_w, float *partial, int slots,
+                            const float *factor, float *acc_w, cudaStream_t st) {
+    const dim3 grid(fma_tiles_n(g), fma_tiles_m(g), mode == 2 ? 1 : g.B);
+    if (grid.y > 65535 || grid.z > 65535) return DP_ERR_UNSUPPORTED;
+    if (mode == 0) conv_wgrad_fma_kernel<T, 0><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w);
+    else if (mode == 1) conv_wgrad_fma_kernel<T, 1><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w);
+    else conv_wgrad_fma_kernel<T, 2><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w);
+    DP_LAUNCH_CHECK("conv_wgrad_fma_kernel");
+    return DP_OK;
+}
+
+dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, const ConvGeom &g, float *G_w,
+                          float *partial, int slots, const float *factor, float *acc_w, cudaStream_t st) {
+    if (dtype == DP_F32)
+        return conv_fma_t(mode, static_cast<const float *>(X), static_cast<const float *>(dY), g, G_w, partial, slots, factor, acc_w, st);
+    return conv_fma_t(mode, static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), g, G_w, partial, slots, factor, acc_w, st);
+}
+
+dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
+                      cudaStream_t st) {
+    const dim3 grid(bias_blocks(g), g.B);
+    if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
+    if (dtype == DP_F32) bias_kernel<<<grid, 256, 0, st>>>(static_cast<const float *>(dY), g.K, g.Kout, db, partial, slots, slot0);
+    else bias_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), g.K, g.Kout, db, partial, slots, slot0);
+    DP_LAUNCH_CHECK("bias_kernel");
+    return DP_OK;
+}
+
+dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
+                          long long sq_stride, int clip, float C_l, float *factor, float *clip_out, cudaStream_t st) {
+    finalize_norm_kernel<<<B, 128, 0, st>>>(partial, slots, w_slots, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
+    DP_LAUNCH_CHECK("finalize_norm_kernel");
+    return DP_OK;
+}
+
+dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st) {
+    bias_accum_kernel<<<(Kout + 127) / 128, 128, 0, st>>>(db, B, Kout, factor, acc_b);
+    DP_LAUNCH_CHECK("bias_accum_kernel");
+    return DP_OK;
+}
+
+template <typename T>
+static dp_status dense_store_t(const T *X, const T *dY, int B, int Cin, int Kout, float *G_w, float *G_b, cudaStream_t st) {
+    const bool vec = (Cin & 3) == 0;
+    const long long total = (long long)B * Kout * (vec ? Cin / 4 : Cin);
+    const unsigned grid = (unsigned)min((long long)148 * 16, (total + 255) / 256);
+    if (vec) dense_store_kernel<T, true><<<grid, 256, 0, st>>>(X, dY, total, Cin, Kout, G_w);
+    else dense_store_kernel<T, false><<<grid, 256, 0, st>>>(X, dY, total, Cin, Kout, G_w);
+    DP_LAUNCH_CHECK("dense_store_kernel");
+    if (G_b) {
+        const long long cnt = (long long)B * Kout;
+        widen_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(dY, cnt, G_b);
+        DP_LAUNCH_CHECK("widen_kernel");
+    }
+    return DP_OK;
+}
+
+dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, float *G_w, float *G_b,
+                             cudaStream_t st) {
+    if (dtype == DP_F32) return dense_store_t(static_cast<const float *>(X), static_cast<const float *>(dY), B, Cin, Kout, G_w, G_b, st);
+    return dense_store_t(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, Cin, Kout, G_w, G_b, st);
+}
+
+dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias,
+                            float *partial, float *db, cudaStream_t st) {
+    const long long cnt = (long long)B * Kout;
+    if (dtype == DP_F32) {
+        dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), Cin, Kout, has_bias, partial);
+        DP_LAUNCH_CHECK("dense_norm_kernel");
+        if (db) { widen_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(static_cast<const float *>(dY), cnt, db); DP_LAUNCH_CHECK("widen_kernel"); }
+    } else {
+        dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), Cin, Kout, has_bias, partial);
+        DP_LAUNCH_CHECK("dense_norm_kernel");
+        if (db) { widen_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), cnt, db); DP_LAUNCH_CHECK("widen_kernel"); }
+    }
+    return DP_OK;
+}
+
+template <typename T, int VEC>
+static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, float *chunk_partial, cudaStream_t st) {
+    const int cv = (C + VEC - 1) / VEC;
+    const int tcv = cv < 256 ? cv : 256;
+    const int chunks = norm_chunks(HW);
+    const dim3 grid((cv + tcv - 1) / tcv, chunks, B);
+    if (grid.y > 65535 || grid.z > 65535) return DP_ERR_UNSUPPORTED;
+    const size_t smem = sizeof(float) * (size_t)(256 / tcv) * tcv * VEC * 2;
+    norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, chunk_partial, chunks);
+    DP_LAUNCH_CHECK("norm_affine_partial_kernel");
+    return DP_OK;
+}
+
+dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
+                             float *dgamma, float *dbeta, float *partial2, cudaStream_t st) {
+    dp_status rc;
+    if (dtype == DP_F32) {
+        if ((C & 3) == 0) rc = norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, st);
+        else rc = norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, st);
+    } else {
+        if ((C & 7) == 0) rc = norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, st);
+        else rc = norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, st);
+    }
+    if (rc != DP_OK) return rc;
+    norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, norm_chunks(HW), C, dgamma, dbeta, partial2);
+    DP_LAUNCH_CHECK("norm_affine_fold_kernel");
+    return DP_OK;
+}
+
+dp_status launch_affine_accum(const float *dgamma, const float *dbeta, int B, int C, const float *factor, float *acc_w,
+                              float *acc_b, cudaStream_t st) {
+    affine_accum_kernel<<<(C + 127) / 128, 128, 0, st>>>(dgamma, dbeta, B, C, factor, acc_w, acc_b);
+    DP_LAUNCH_CHECK("affine_accum_kernel");
+    return DP_OK;
+}
+
+}  // namespace dp

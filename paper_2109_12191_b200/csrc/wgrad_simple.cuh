@@ -1,0 +1,50 @@
+// Internal launch interface of the CUDA-core per-example weight-gradient kernels.
+#pragma once
+#include "common.cuh"
+
+namespace dp {
+
+struct ConvGeom {
+    int B, H, W, Cin, Kout, R, S, stride, pad, OH, OW;
+    int M;   // Kout                     (rows of the per-example gradient matrix)
+    int N;   // R*S*Cin                  (columns)
+    int K;   // OH*OW                    (reduction length per example)
+};
+
+constexpr int kFmaTile = 64;          // output tile edge of the CUDA-core kernel
+constexpr int kBiasCols = 64;         // output channels per bias-reduction block
+constexpr int kNormPix = 256;         // pixels per block in the norm-affine reduction
+
+inline int fma_tiles_m(const ConvGeom &g) { return (g.M + kFmaTile - 1) / kFmaTile; }
+inline int fma_tiles_n(const ConvGeom &g) { return (g.N + kFmaTile - 1) / kFmaTile; }
+inline int bias_blocks(const ConvGeom &g) { return (g.Kout + kBiasCols - 1) / kBiasCols; }
+
+// mode: 0 store + norm partials, 1 norm partials only, 2 clip-accumulate (factor[n*2] scales example n)
+dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, const ConvGeom &g, float *G_w,
+                          float *partial, int slots, const float *factor, float *acc_w, cudaStream_t stream);
+// db[n,k] = sum over pixels of dY; also sum_k db^2 per block into partial[n*slots + slot0 + block]
+dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
+                      cudaStream_t stream);
+// folds the partial slots of every example into sqnorm (and clip factors when clip != 0)
+dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
+                          long long sq_stride, int clip, float C_l, float *factor, float *clip_out,
+                          cudaStream_t stream);
+// acc_b[k] += sum_n factor[n*2+1] * db[n,k]
+dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream);
+
+dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, float *G_w,
+                             float *G_b, cudaStream_t stream);
+// writes partial[n*2+0] = |dY_n|^2 |X_n|^2 and partial[n*2+1] = |dY_n|^2 (0 without bias); db (optional) = dY as fp32
+dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias,
+                            float *partial, float *db, cudaStream_t stream);
+
+// stage 1: per pixel-chunk partial sums; stage 2: fold, store, squared norms into partial2[n*2 + {0,1}]
+dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
+                             float *dgamma, float *dbeta, float *partial2, cudaStream_t stream);
+// acc_w[c] += sum_n factor[n*2] dgamma[n,c]; acc_b[c] += sum_n factor[n*2+1] dbeta[n,c]
+dp_status launch_affine_accum(const float *dgamma, const float *dbeta, int B, int C, const float *factor,
+                              float *acc_w, float *acc_b, cudaStream_t stream);
+
+inline int norm_chunks(int HW) { return (HW + kNormPix - 1) / kNormPix; }
+
+}  // namespace dp

@@ -1,0 +1,17 @@
+// Internal launch interface of the tcgen05 (5th-generation tensor core) per-example conv weight-gradient kernel.
+#pragma once
+#include "wgrad_simple.cuh"
+
+namespace dp {
+
+// true when the layer can run on the tensor-core kernel (channel counts, sizes and TMA alignment rules)
+bool tc_eligible(int dtype, const ConvGeom &g, int epilogue);
+// number of per-example partial squared-norm slots the kernel writes
+int tc_norm_slots(int dtype, const ConvGeom &g, int epilogue);
+size_t tc_workspace_bytes(int dtype, const ConvGeom &g, int epilogue);
+// epilogue as dp_epilogue; factor[n*2] scales example n (CLIP_ACCUM); status: device word set to nonzero on a timed-out wait
+dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
+                         float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace,
+                         int *status, cudaStream_t stream);
+
+}  // namespace dp

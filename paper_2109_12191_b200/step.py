@@ -1,0 +1,171 @@
+"""Buffer ownership and call sequencing for one privatisation step.
+
+Nothing is computed here: these classes allocate device tensors with PyTorch and issue the
+C-ABI calls of ``binding`` in the order of the paper's section 2 (per-example gradients ->
+norms -> clip -> sum over the chunk, repeated per accumulation chunk -> noise -> average) or,
+for per-layer clipping (section 3.5), with the clip fused into the weight-gradient call.
+"""
+from __future__ import annotations
+
+import math
+import torch
+
+from . import binding as b
+from .synth import Layer
+
+_KIND = {"conv": b.DP_LAYER_CONV2D, "dense": b.DP_LAYER_DENSE, "norm": b.DP_LAYER_NORM_AFFINE}
+
+
+def layer_desc(layer: Layer, B: int, dtype: str, impl=b.DP_IMPL_AUTO, bias_separate=1):
+    return b.make_desc(_KIND[layer.kind], b.DP_BF16 if dtype == "bf16" else b.DP_F32, B, layer.Cin, layer.Kout,
+                       layer.H, layer.W, layer.R, layer.S, layer.stride, layer.pad, int(layer.bias), bias_separate, impl)
+
+
+def _tensors_of(layers):
+    """[(layer index, 'w' | 'b', size)] in parameter order: weight then bias-like tensor of each layer."""
+    out = []
+    for li, l in enumerate(layers):
+        out.append((li, "w", l.n_weight))
+        if l.n_bias:
+            out.append((li, "b", l.n_bias))
+    return out
+
+
+class GlobalClipStep:
+    """Whole-model clipping: per-example gradients are materialised per layer (STORE+NORM epilogue),
+    one dp_clip_accumulate call per chunk consumes them with the norms the epilogues produced."""
+
+    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda"):
+        self.layers, self.B, self.dtype, self.C, self.sigma = list(layers), B, dtype, float(C), float(sigma)
+        self.tensors = _tensors_of(self.layers)
+        self.L = len(self.tensors)
+        self.P_l = [t[2] for t in self.tensors]
+        self.P = sum(self.P_l)
+        self.descs = [layer_desc(l, B, dtype, impl, 1) for l in self.layers]
+        self.G = [torch.empty((B, p), dtype=torch.float32, device=device) for p in self.P_l]
+        self.sq = torch.zeros((B, self.L), dtype=torch.float32, device=device)
+        self.acc = torch.zeros(self.P, dtype=torch.float32, device=device)
+        self.out = torch.empty(self.P, dtype=torch.float32, device=device)
+        offs, o = [], 0
+        for p in self.P_l:
+            offs.append(o)
+            o += p
+        self.offsets = offs
+        self.acc_views = [self.acc[o:o + p] for o, p in zip(offs, self.P_l)]
+        self.norms = torch.empty(B, dtype=torch.float32, device=device)
+        self.clip = torch.empty(B, dtype=torch.float32, device=device)
+        ws = max([b.dp_workspace_bytes(d, b.DP_EPI_STORE_NORM) for d in self.descs] + [256])
+        self.ws = torch.empty(ws, dtype=torch.uint8, device=device)
+        self.clip_ws = torch.empty(max(b.dp_clip_workspace_bytes(B, self.P_l), 256), dtype=torch.uint8, device=device)
+        # column of each layer's first tensor in the [B, L] norm table, and its G buffers
+        self._col, col = [], 0
+        for l in self.layers:
+            self._col.append(col)
+            col += 2 if l.n_bias else 1
+        self.chunks_done = 0
+
+    def begin(self):
+        self.acc.zero_()
+        self.chunks_done = 0
+
+    def wgrad(self, li, X, dY):
+        col = self._col[li]
+        G_w = self.G[col]
+        G_b = self.G[col + 1] if self.layers[li].n_bias else None
+        b.check(b.dp_per_example_wgrad(self.descs[li], X, dY, G_w, G_b, self.sq.data_ptr() + 4 * col, self.L,
+                                       b.DP_EPI_STORE_NORM, 0.0, None, None, None, self.ws), "dp_per_example_wgrad")
+
+    def clip_accumulate(self, use_epilogue_norms=True):
+        b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, self.G, self.P_l, self.sq if use_epilogue_norms else None,
+                                     self.C, self.acc_views, self.norms, self.clip, self.clip_ws), "dp_clip_accumulate")
+        self.chunks_done += 1
+
+    def chunk(self, inputs):
+        """inputs: list of (X, dY) device tensors, one pair per layer."""
+        for li, (X, dY) in enumerate(inputs):
+            self.wgrad(li, X, dY)
+        self.clip_accumulate()
+
+    def finish(self, seed=0, step=0):
+        total = self.B * self.chunks_done
+        b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, total, seed, step, self.out), "dp_noise_average")
+        return self.out
+
+
+class FlatClipStep:
+    """Flattened per-example gradients [B, P] handed in directly (no weight-gradient stage)."""
+
+    def __init__(self, P, B, C, sigma, device="cuda"):
+        self.P, self.B, self.C, self.sigma = P, B, float(C), float(sigma)
+        self.acc = torch.zeros(P, dtype=torch.float32, device=device)
+        self.out = torch.empty(P, dtype=torch.float32, device=device)
+        self.norms = torch.empty(B, dtype=torch.float32, device=device)
+        self.clip = torch.empty(B, dtype=torch.float32, device=device)
+        self.ws = torch.empty(max(b.dp_clip_workspace_bytes(B, [P]), 256), dtype=torch.uint8, device=device)
+        self.chunks_done = 0
+
+    def begin(self):
+        self.acc.zero_()
+        self.chunks_done = 0
+
+    def chunk(self, G, sqnorm=None):
+        b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, [G], [self.P], sqnorm, self.C, [self.acc], self.norms,
+                                     self.clip, self.ws), "dp_clip_accumulate")
+        self.chunks_done += 1
+
+    def finish(self, seed=0, step=0):
+        b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, self.B * self.chunks_done, seed, step, self.out),
+                "dp_noise_average")
+        return self.out
+
+
+class PerLayerClipStep:
+    """Per-layer clipping (threshold C/sqrt(L) per parameter tensor) fused into the weight-gradient call:
+    no per-example gradient is written to memory."""
+
+    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda"):
+        self.layers, self.B, self.dtype, self.C, self.sigma = list(layers), B, dtype, float(C), float(sigma)
+        self.tensors = _tensors_of(self.layers)
+        self.L = len(self.tensors)
+        self.C_l = self.C / math.sqrt(self.L)
+        self.descs = [layer_desc(l, B, dtype, impl, 1) for l in self.layers]
+        self.acc_w = [torch.zeros(l.n_weight, dtype=torch.float32, device=device) for l in self.layers]
+        self.acc_b = [torch.zeros(l.n_bias, dtype=torch.float32, device=device) if l.n_bias else None for l in self.layers]
+        self.sq = torch.zeros((B, self.L), dtype=torch.float32, device=device)
+        ws = max([b.dp_workspace_bytes(d, b.DP_EPI_CLIP_ACCUM) for d in self.descs] + [256])
+        self.ws = torch.empty(ws, dtype=torch.uint8, device=device)
+        self._col, col = [], 0
+        for l in self.layers:
+            self._col.append(col)
+            col += 2 if l.n_bias else 1
+        self.P = sum(t[2] for t in self.tensors)
+        self.chunks_done = 0
+
+    def begin(self):
+        for a in self.acc_w:
+            a.zero_()
+        for a in self.acc_b:
+            if a is not None:
+                a.zero_()
+        self.chunks_done = 0
+
+    def wgrad(self, li, X, dY):
+        b.check(b.dp_per_example_wgrad(self.descs[li], X, dY, None, None, self.sq.data_ptr() + 4 * self._col[li], self.L,
+                                       b.DP_EPI_CLIP_ACCUM, self.C_l, self.acc_w[li], self.acc_b[li], None, self.ws),
+                "dp_per_example_wgrad")
+
+    def chunk(self, inputs):
+        for li, (X, dY) in enumerate(inputs):
+            self.wgrad(li, X, dY)
+        self.chunks_done += 1
+
+    def finish(self, seed=0, step=0):
+        """Noise uses the whole-gradient bound C (the per-tensor thresholds keep the sensitivity at C)."""
+        total, off = self.B * self.chunks_done, 0
+        for aw, ab in zip(self.acc_w, self.acc_b):
+            for a in (aw, ab):
+                if a is None:
+                    continue
+                b.check(b.dp_noise_average(a, a.numel(), off, self.sigma, self.C, total, seed, step, a), "dp_noise_average")
+                off += a.numel()
+        return self.acc_w, self.acc_b

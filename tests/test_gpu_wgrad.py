@@ -1,0 +1,136 @@
+"""GPU parity of dp_per_example_wgrad (every layer kind, epilogue and implementation) against the oracle."""
+import math
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2109_12191_b200 import synth
+from gpu_util import (B, rel_l2, gpu_layer, oracle_layer, scaled_inputs, make_desc, TOL_NORM, TOL_FMA, TOL_ACC_BF16,
+                      TOL_ACC_F32)
+
+pytestmark = pytest.mark.gpu
+
+STORE, NORM, CLIP = 0, 1, 2
+AUTO, CUDA_CORE, TENSOR_CORE = 0, 1, 2
+
+
+def tol_for(out, dtype):
+    """Accumulated / stored gradient tolerance: plain fp32 rounding on the CUDA-core path and for bf16
+    inputs (their products are exact in fp32); the TF32-class bound for fp32 inputs on tensor cores."""
+    if not out["uses_tc"]:
+        return TOL_FMA
+    return TOL_ACC_BF16 if dtype == "bf16" else TOL_ACC_F32
+
+
+def check_layer(layer, Bn, dtype, impl, key, bias_separate=0, spread=False):
+    inp = scaled_inputs(layer, Bn, dtype, *key, spread=spread)
+    dW, db = oracle_layer(layer, inp)
+    sq_w = oracle.sqnorm(dW)
+    sq_b = oracle.sqnorm(db) if db is not None else np.zeros(Bn)
+    groups = 2 if (bias_separate and db is not None) else 1
+    ref_sq = np.stack([sq_w, sq_b], 1) if groups == 2 else (sq_w + sq_b)[:, None]
+
+    out = gpu_layer(layer, inp, dtype, STORE, impl, bias_separate)
+    tol = tol_for(out, dtype)
+    for n in range(Bn):
+        assert rel_l2(out["G_w"][n], dW[n]) <= tol, (layer.name, n)
+    if db is not None:
+        for n in range(Bn):
+            assert rel_l2(out["G_b"][n], db[n]) <= tol
+    np.testing.assert_allclose(out["sq"], ref_sq, rtol=TOL_NORM)
+
+    out_n = gpu_layer(layer, inp, dtype, NORM, impl, bias_separate)
+    np.testing.assert_allclose(out_n["sq"], ref_sq, rtol=TOL_NORM)
+
+    # per-layer clip + accumulate, threshold at the median norm so both branches occur when norms spread
+    C_l = float(np.sqrt(np.median(ref_sq)))
+    f = oracle.clip_factor(ref_sq, C_l).reshape(Bn, groups)
+    ref_acc_w = np.einsum("n,np->p", f[:, 0], dW)
+    out_c = gpu_layer(layer, inp, dtype, CLIP, impl, bias_separate, C_l=C_l)
+    np.testing.assert_allclose(out_c["clip"], f, rtol=TOL_NORM)
+    np.testing.assert_allclose(out_c["sq"], ref_sq, rtol=TOL_NORM)
+    assert rel_l2(out_c["acc_w"], ref_acc_w) <= tol_for(out_c, dtype)
+    if db is not None:
+        ref_acc_b = np.einsum("n,np->p", f[:, groups - 1], db)
+        assert rel_l2(out_c["acc_b"], ref_acc_b) <= tol_for(out_c, dtype)
+    return out
+
+
+FMA_CONVS = [
+    # Cin, Kout, R, stride, pad, H, bias
+    (3, 32, 3, 1, 1, 32, True),      # first conv of the small CNN: 27 columns
+    (32, 64, 3, 2, 1, 32, True),
+    (64, 128, 3, 2, 1, 16, True),
+    (3, 64, 7, 2, 3, 30, False),     # stem-like: 147 columns (not a multiple of 4), stride 2, pad 3
+    (5, 7, 3, 1, 0, 9, True),        # nothing aligned
+    (16, 8, 1, 2, 0, 8, False),      # strided 1x1
+    (8, 70, 5, 1, 2, 7, True),       # K = 49 pixels, ragged tile rows
+    (2, 3, 3, 1, 1, 1, False),       # 1x1 image with padding: only the centre tap sees data
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", FMA_CONVS)
+def test_conv_cuda_core(case, dtype):
+    Cin, Kout, R, stride, pad, H, bias = case
+    layer = synth.conv(Cin, Kout, R, stride, pad, H, bias, name=str(case))
+    check_layer(layer, 5, dtype, CUDA_CORE, (930, sum(case[:6])), spread=True)
+
+
+def test_conv_non_square_image_and_filter():
+    layer = synth.Layer("conv", 6, 9, R=3, S=5, stride=2, pad=1, H=11, W=14, bias=True, name="3x5")
+    check_layer(layer, 3, "f32", CUDA_CORE, (931,), spread=True)
+
+
+@pytest.mark.parametrize("bias_separate", [0, 1])
+def test_bias_group_handling(bias_separate):
+    layer = synth.conv(8, 16, 3, 1, 1, 10, True, "bias groups")
+    check_layer(layer, 6, "f32", CUDA_CORE, (932,), bias_separate=bias_separate, spread=True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("Cin,Kout,bias", [(256, 64, True), (8192, 10, True), (13, 7, False), (2048, 1000, False)])
+def test_dense(Cin, Kout, bias, dtype):
+    layer = synth.dense(Cin, Kout, bias, "dense")
+    Bn = 8 if Cin * Kout < 1_000_000 else 3
+    check_layer(layer, Bn, dtype, AUTO, (933, Cin), spread=True)
+    check_layer(layer, Bn, dtype, AUTO, (933, Cin), bias_separate=1, spread=True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("C,H", [(64, 12), (256, 7), (2048, 3), (24, 20), (5, 6), (512, 17)])
+def test_norm_affine(C, H, dtype):
+    layer = synth.norm(C, H, "gn")
+    check_layer(layer, 4, dtype, AUTO, (934, C), bias_separate=1, spread=True)
+    check_layer(layer, 4, dtype, AUTO, (934, C), bias_separate=0, spread=True)
+
+
+def test_rerun_gives_identical_bits():
+    layer = synth.conv(32, 64, 3, 2, 1, 32, True)
+    inp = synth.layer_inputs(layer, 6, "f32", 935)
+    a = gpu_layer(layer, inp, "f32", STORE, CUDA_CORE)
+    b = gpu_layer(layer, inp, "f32", STORE, CUDA_CORE)
+    np.testing.assert_array_equal(a["G_w"], b["G_w"])
+    np.testing.assert_array_equal(a["sq"], b["sq"])
+
+
+def test_sqnorm_stride_writes_one_column_of_a_table():
+    layer = synth.conv(8, 16, 3, 1, 1, 10, True)
+    inp = synth.layer_inputs(layer, 4, "f32", 936)
+    table = torch.full((4, 5), -1.0, device="cuda")
+    gpu_layer(layer, inp, "f32", NORM, CUDA_CORE, bias_separate=1, sq=table, sq_stride=5, sq_col=2)
+    t = table.cpu().numpy()
+    dW, db = oracle_layer(layer, inp)
+    np.testing.assert_allclose(t[:, 2], oracle.sqnorm(dW), rtol=TOL_NORM)
+    np.testing.assert_allclose(t[:, 3], oracle.sqnorm(db), rtol=TOL_NORM)
+    assert np.all(t[:, [0, 1, 4]] == -1.0)
+
+
+def test_dense_norm_is_the_rank1_closed_form():
+    layer = synth.dense(300, 40, True)
+    inp = synth.layer_inputs(layer, 7, "f32", 937)
+    out = gpu_layer(layer, inp, "f32", NORM)
+    x2 = (inp["X"].astype(np.float64) ** 2).sum(1)
+    y2 = (inp["dY"].astype(np.float64) ** 2).sum(1)
+    np.testing.assert_allclose(out["sq"][:, 0], y2 * x2 + y2, rtol=1e-6)
