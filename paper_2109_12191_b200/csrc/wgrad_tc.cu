@@ -1,9 +1,443 @@
-// placeholder until the tcgen05 kernel lands: nothing is eligible, so every layer takes the CUDA-core path
+// Per-example convolution weight gradients on the 5th-generation tensor cores (tcgen05 + TMEM),
+// operands staged by TMA.  One (example, output tile) at a time per CTA, persistent CTAs.
+//
+// For example n the gradient is the matrix product  D_n = dY_n^T * Xcol_n  over the output pixels:
+//     dY_n   [pixels, K_out]          (channels-last: K_out contiguous)
+//     Xcol_n [pixels, R*S*C_in]       (column j = (r*S+s)*C_in + c is the input shifted by tap (r,s))
+// Both operands have the reduction index (pixel) as the slow axis, i.e. they are "MN-major" for the
+// tensor core.  A TMA box {64 channels, OWt, OHt, 1 example} lands in shared memory as OWt*OHt rows of
+// 128 bytes with the 128-byte swizzle, which is exactly the canonical MN-major operand slab; the tap
+// shift and the zero padding come from the box start coordinate and TMA's out-of-bounds zero fill.
+//
+// Roles (192 threads): warp 0 issues TMA loads, warp 1 allocates TMEM and issues tcgen05.mma,
+// warps 2-5 read accumulators back with tcgen05.ld, square-sum them (the per-example norm) and store.
+// Two accumulator buffers in TMEM let the epilogue of one tile overlap the main loop of the next.
+// Every wait is bounded: on expiry the CTA sets a status word, drains and returns.
 #include "wgrad_tc.cuh"
+#include <cuda.h>
+#include <mutex>
+#include <algorithm>
+#include <array>
+#include <map>
+
 namespace dp {
-bool tc_eligible(int, const ConvGeom &, int) { return false; }
-int tc_norm_slots(int, const ConvGeom &, int) { return 0; }
+
+constexpr int kSlabCh = 64;            // bf16 channels per 128-byte row
+constexpr int kRowBytes = 128;
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 200 * 1024;
+constexpr uint32_t kWaitPolls = 1u << 21;   // x ~1 us suspend hint: about two seconds before a wait gives up
+
+struct TcPlan {
+    bool ok;
+    int a_is_x;                 // 1: rows of D are columns j of Xcol, columns of D are output channels k
+    int a_ext, b_ext;           // operand extents (multiples of 64)
+    int m_tiles, n_tiles, NT;   // NT: nominal columns per tile (multiple of 64, <= 256)
+    int OWt, OHt, tiles_w, tiles_h, Kt, k_tiles;
+    int stages, stage_bytes, a_bytes;
+    size_t smem;
+};
+
+struct TcParams {
+    int B, Kout, Ng, Cin, S, stride, pad;
+    int a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT;
+    int OWt, OHt, tiles_w, Kt, k_tiles, stages, stage_bytes, a_bytes;
+    int mode;                   // 0 store + norm, 1 norm only
+    float *G_w;
+    float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
+    int slots;
+    int *status;
+    long long total_tiles;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                 "selp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this or another wait expired).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t it = 0; it < kWaitPolls; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate, issued by one thread
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory operand descriptor: MN-major slab(s) with the 128-byte swizzle.
+//   start address >> 4 | leading byte offset (between 64-channel slabs) >> 4 at bit 16 |
+//   stride byte offset (between groups of 8 reduction rows = 1024 B) >> 4 at bit 32 |
+//   descriptor version 1 at bit 46 | layout type 2 (128-byte swizzle) at bit 61
+__device__ __forceinline__ uint64_t operand_desc(uint32_t addr, uint32_t slab_stride_bytes) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((slab_stride_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both MN-major, M = 128, N = n_cols.
+__device__ __forceinline__ uint32_t instr_desc(int n_cols) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n_cols >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// TMA start coordinates of 64-channel slab `slab` of an operand for the pixel tile at (oh0, ow0)
+__device__ __forceinline__ void slab_coords(bool is_x, int slab, const TcParams &p, int oh0, int ow0, int &c0, int &c1, int &c2) {
+    if (is_x) {
+        const int j0 = slab * kSlabCh;
+        const int tap = j0 / p.Cin;
+        c0 = j0 - tap * p.Cin;
+        const int r = tap / p.S, s = tap - r * p.S;
+        c1 = ow0 * p.stride + s - p.pad;
+        c2 = oh0 * p.stride + r - p.pad;
+    } else {
+        c0 = slab * kSlabCh;
+        c1 = ow0;
+        c2 = oh0;
+    }
+}
+
+__global__ void __launch_bounds__(192, 1)
+conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t tiles_u32 = smem_u32(tiles);
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int *abort_p = &abort_flag;
+
+    const int tiles_per_example = p.m_tiles * p.n_tiles;
+    const int slab_bytes = p.Kt * kRowBytes;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one lane)
+        if (lane == 0) {
+            const CUtensorMap *mapA = p.a_is_x ? &tmX : &tmY, *mapB = p.a_is_x ? &tmY : &tmX;
+            int stage = 0; uint32_t phase = 0;
+            bool live = true;
+            for (long long t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+                const int n = (int)(t / tiles_per_example);
+                const int rem = (int)(t - (long long)n * tiles_per_example);
+                const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+                const int a_slab0 = mt * 2, a_slabs = min(2, p.a_ext / kSlabCh - a_slab0);
+                const int b_slab0 = nt * (p.NT / kSlabCh), b_slabs = min(p.NT / kSlabCh, p.b_ext / kSlabCh - b_slab0);
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    const int th = kt / p.tiles_w, tw = kt - th * p.tiles_w;
+                    const int oh0 = th * p.OHt, ow0 = tw * p.OWt;
+                    if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p)) { live = false; break; }
+                    const uint32_t bar = smem_u32(&full_bar[stage]);
+                    mbar_expect_tx(bar, (uint32_t)((a_slabs + b_slabs) * slab_bytes));
+                    const uint32_t a_dst = tiles_u32 + stage * p.stage_bytes, b_dst = a_dst + p.a_bytes;
+                    int c0, c1, c2;
+                    for (int s = 0; s < a_slabs; ++s) {
+                        slab_coords(p.a_is_x != 0, a_slab0 + s, p, oh0, ow0, c0, c1, c2);
+                        tma_load_4d(a_dst + s * slab_bytes, mapA, bar, c0, c1, c2, n);
+                    }
+                    for (int s = 0; s < b_slabs; ++s) {
+                        slab_coords(p.a_is_x == 0, b_slab0 + s, p, oh0, ow0, c0, c1, c2);
+                        tma_load_4d(b_dst + s * slab_bytes, mapB, bar, c0, c1, c2, n);
+                    }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            uint32_t acc_phase = 0;  // bit b: phase of accumulator buffer b
+            int buf = 0;
+            bool live = true;
+            for (long long t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+                const int rem = (int)(t % tiles_per_example);
+                const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+                const int a_slabs = min(2, p.a_ext / kSlabCh - mt * 2);
+                const int b_slabs = min(p.NT / kSlabCh, p.b_ext / kSlabCh - nt * (p.NT / kSlabCh));
+                const uint32_t idesc = instr_desc(b_slabs * kSlabCh);
+                // a single live slab is read twice (leading offset 0): rows 64..127 of D repeat rows 0..63 and are ignored
+                const uint32_t a_lbo = (a_slabs == 2) ? (uint32_t)slab_bytes : 0u;
+                if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p)) { live = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p)) { live = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_src = tiles_u32 + stage * p.stage_bytes, b_src = a_src + p.a_bytes;
+                    for (int ks = 0; ks < p.Kt / 16; ++ks) {
+                        const uint64_t ad = operand_desc(a_src + ks * 2048, a_lbo);
+                        const uint64_t bd = operand_desc(b_src + ks * 2048, (uint32_t)slab_bytes);
+                        umma_bf16(d_tmem, ad, bd, idesc, (kt | ks) ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&empty_bar[stage]));      // frees the stage once these MMAs have read it
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (!live) break;
+                umma_commit(smem_u32(&tmem_full[buf]));            // accumulator complete
+                acc_phase ^= 1u << buf;
+                buf ^= 1;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        uint32_t full_phase = 0;     // bit b: parity to wait for on accumulator buffer b
+        int buf = 0;
+        bool live = true;
+        for (long long t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+            const int n = (int)(t / tiles_per_example);
+            const int rem = (int)(t - (long long)n * tiles_per_example);
+            const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+            const int a_rows = min(128, p.a_ext - mt * 128);
+            const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
+            const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p);
+            if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }   // the whole warp leaves together
+            full_phase ^= 1u << buf;
+            tc_fence_after();
+            const bool row_ok = row < a_rows;
+            const int a_idx = mt * 128 + row;            // index along the A operand's extent
+            float sq = 0.f;
+            float *Gn = p.G_w + (long long)n * p.Kout * p.Ng;
+            for (int cc = 0; cc < n_cols; cc += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (uint32_t)(buf * 256 + cc) + ((uint32_t)(q * 32) << 16), v);
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq = fmaf(f, f, sq); }
+                    if (p.mode == 0) {
+                        const int b_idx = nt * p.NT + cc;
+                        if (p.a_is_x) {          // row = column j of G, tile column = output channel k: lanes write consecutive j
+                            float *dst = Gn + (long long)b_idx * p.Ng + a_idx;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) __stcs(dst + (long long)i * p.Ng, __uint_as_float(v[i]));
+                        } else {                 // row = output channel k, tile columns = 32 consecutive j
+                            float4 *dst = reinterpret_cast<float4 *>(Gn + (long long)a_idx * p.Ng + b_idx);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                __stcs(dst + i, make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                            __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            sq = warp_sum(sq);
+            if (lane == 0) p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
+            buf ^= 1;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag) {
+        // give copies still in flight time to land before shared memory is released
+        if (threadIdx.x == 0) { *p.status = DP_ERR_TIMEOUT; __threadfence(); }
+        __nanosleep(200000);
+        __syncthreads();
+    }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+static int step_cycles(int n_cols) {     // per 16-pixel MMA step: tensor pipe vs shared-memory operand reads
+    const int pipe = n_cols / 2, smem = 32 + n_cols / 4;
+    return pipe > smem ? pipe : smem;
+}
+
+static TcPlan search_plan(int dtype, const ConvGeom &g);
+
+// The tiling search is pure; its results are memoised per layer geometry (host side only).
+static TcPlan make_plan(int dtype, const ConvGeom &g) {
+    static std::mutex mu;
+    static std::map<std::array<int, 10>, TcPlan> memo;
+    const std::array<int, 10> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, 0};
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find(key);
+    if (it != memo.end()) return it->second;
+    const TcPlan pl = search_plan(dtype, g);
+    memo.emplace(key, pl);
+    return pl;
+}
+
+static TcPlan search_plan(int dtype, const ConvGeom &g) {
+    TcPlan best; best.ok = false;
+    if (dtype != DP_BF16) return best;
+    if (g.stride != 1) return best;
+    if (g.Cin % kSlabCh || g.Kout % kSlabCh) return best;
+    if (g.OW > 256 || g.OH > 65535 || g.K < 1) return best;
+    double best_cost = 1e300;
+    for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
+        const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
+        for (int NT = 64; NT <= 256; NT += 64) {
+            if (NT > b_ext && NT != 64 * ((b_ext + 63) / 64)) continue;
+            const int nt_cols = NT < b_ext ? NT : b_ext;
+            const int m_tiles = (a_ext + 127) / 128, n_tiles = (b_ext + nt_cols - 1) / nt_cols;
+            const int slabs = 2 + nt_cols / kSlabCh;
+            long long mma = 0;
+            for (int t = 0; t < n_tiles; ++t) mma += step_cycles(std::min(nt_cols, b_ext - t * nt_cols));
+            mma *= m_tiles;
+            for (int OHt = 1; OHt <= g.OH && OHt <= g.H && OHt <= 256; ++OHt)
+                for (int OWt = 1; OWt <= g.OW && OWt <= g.W; ++OWt) {
+                    const int Kt = OHt * OWt;
+                    if (Kt % 16 || Kt > 256) continue;
+                    const int stage_bytes = slabs * Kt * kRowBytes;
+                    int stages = kSmemBudget / stage_bytes;
+                    if (stages < 2) continue;
+                    if (stages > kMaxStages) stages = kMaxStages;
+                    const int tw = (g.OW + OWt - 1) / OWt, th = (g.OH + OHt - 1) / OHt;
+                    const long long steps = (long long)tw * th * (Kt / 16);
+                    // cost: tensor-pipe cycles, a fixed toll per stage hand-over, and a penalty for shallow pipelines
+                    double cost = (double)mma * steps + 60.0 * tw * th * m_tiles * n_tiles;
+                    if (stages < 3) cost *= 1.25;
+                    cost *= 1.0 + 0.02 * (256 - nt_cols) / 64;
+                    if (cost < best_cost) {
+                        best_cost = cost;
+                        best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
+                        best.m_tiles = m_tiles; best.n_tiles = n_tiles; best.NT = nt_cols;
+                        best.OWt = OWt; best.OHt = OHt; best.tiles_w = tw; best.tiles_h = th; best.Kt = Kt;
+                        best.k_tiles = tw * th; best.stages = stages; best.stage_bytes = stage_bytes;
+                        best.a_bytes = 2 * Kt * kRowBytes;
+                        best.smem = (size_t)stages * stage_bytes + 1024;
+                    }
+                }
+        }
+    }
+    return best;
+}
+
+bool tc_eligible(int dtype, const ConvGeom &g, int epilogue) {
+    if (epilogue == DP_EPI_CLIP_ACCUM) return false;
+    return make_plan(dtype, g).ok && encode_fn() != nullptr;
+}
+
+int tc_norm_slots(int dtype, const ConvGeom &g, int) {
+    const TcPlan pl = make_plan(dtype, g);
+    return pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
+}
+
 size_t tc_workspace_bytes(int, const ConvGeom &, int) { return 0; }
-dp_status launch_conv_tc(int, int, const void *, const void *, const ConvGeom &, float *, float *, int, const float *,
-                         float *, void *, int *, cudaStream_t) { return DP_ERR_UNSUPPORTED; }
+
+static bool encode_nhwc(CUtensorMap *map, const void *base, int C, int W, int H, int Bn, int boxW, int boxH) {
+    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)Bn};
+    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kSlabCh, (cuuint32_t)boxW, (cuuint32_t)boxH, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
+                         float *partial, int slots, const float *, float *, void *, int *status, cudaStream_t stream) {
+    const TcPlan pl = make_plan(dtype, g);
+    if (!pl.ok || !encode_fn() || epilogue == DP_EPI_CLIP_ACCUM) return DP_ERR_UNSUPPORTED;
+    CUtensorMap tmX, tmY;
+    if (!encode_nhwc(&tmX, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    TcParams p;
+    p.B = g.B; p.Kout = g.Kout; p.Ng = g.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
+    p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
+    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
+    p.mode = (epilogue == DP_EPI_STORE_NORM) ? 0 : 1;
+    p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
+    p.total_tiles = (long long)g.B * pl.m_tiles * pl.n_tiles;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
+    int dev = 0, sms = 148;
+    DP_CUDA_TRY(cudaGetDevice(&dev));
+    DP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const unsigned grid = (unsigned)std::min<long long>(p.total_tiles, sms);
+    conv_wgrad_tc_kernel<<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+    DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
+    return DP_OK;
+}
+
 }  // namespace dp

@@ -23,7 +23,7 @@ def tol_for(out, dtype):
     return TOL_ACC_BF16 if dtype == "bf16" else TOL_ACC_F32
 
 
-def check_layer(layer, Bn, dtype, impl, key, bias_separate=0, spread=False):
+def check_layer(layer, Bn, dtype, impl, key, bias_separate=0, spread=False, clip_impl=None):
     inp = scaled_inputs(layer, Bn, dtype, *key, spread=spread)
     dW, db = oracle_layer(layer, inp)
     sq_w = oracle.sqnorm(dW)
@@ -47,7 +47,7 @@ def check_layer(layer, Bn, dtype, impl, key, bias_separate=0, spread=False):
     C_l = float(np.sqrt(np.median(ref_sq)))
     f = oracle.clip_factor(ref_sq, C_l).reshape(Bn, groups)
     ref_acc_w = np.einsum("n,np->p", f[:, 0], dW)
-    out_c = gpu_layer(layer, inp, dtype, CLIP, impl, bias_separate, C_l=C_l)
+    out_c = gpu_layer(layer, inp, dtype, CLIP, clip_impl if clip_impl is not None else impl, bias_separate, C_l=C_l)
     np.testing.assert_allclose(out_c["clip"], f, rtol=TOL_NORM)
     np.testing.assert_allclose(out_c["sq"], ref_sq, rtol=TOL_NORM)
     assert rel_l2(out_c["acc_w"], ref_acc_w) <= tol_for(out_c, dtype)
@@ -134,3 +134,47 @@ def test_dense_norm_is_the_rank1_closed_form():
     x2 = (inp["X"].astype(np.float64) ** 2).sum(1)
     y2 = (inp["dY"].astype(np.float64) ** 2).sum(1)
     np.testing.assert_allclose(out["sq"][:, 0], y2 * x2 + y2, rtol=1e-6)
+
+
+# ------------------------------------------------------------------ tcgen05 path (bf16, 64-channel multiples)
+TC_CONVS = [
+    # Cin, Kout, R, stride, pad, H, bias
+    (64, 64, 1, 1, 0, 8, False),       # both extents 64: a single operand slab read twice
+    (64, 64, 3, 1, 1, 8, True),        # 576 columns: tiles of 256, 256, 64
+    (128, 128, 3, 1, 1, 8, False),
+    (64, 256, 1, 1, 0, 14, False),     # 14x14: pixel tiles hang over the image edge (zero filled)
+    (256, 64, 1, 1, 0, 14, False),
+    (128, 192, 3, 1, 1, 12, True),
+    (64, 64, 3, 1, 1, 7, False),       # 49 pixels inside an 8x8 pixel tile
+    (64, 128, 3, 1, 0, 10, False),     # no padding: 8x8 outputs from a 10x10 input
+    (320, 64, 1, 1, 0, 6, False),      # extent 320 = 2.5 row tiles
+    (64, 64, 5, 1, 2, 9, False),       # 5x5 taps
+]
+
+
+@pytest.mark.parametrize("case", TC_CONVS)
+def test_conv_tensor_core(case):
+    Cin, Kout, R, stride, pad, H, bias = case
+    layer = synth.conv(Cin, Kout, R, stride, pad, H, bias, name=str(case))
+    out = check_layer(layer, 5, "bf16", TENSOR_CORE, (940, sum(case[:6])), spread=True, clip_impl=AUTO)
+    assert out["uses_tc"]
+
+
+def test_tensor_core_matches_cuda_core_bitwise_norm_inputs():
+    """Same layer through both implementations: bf16 products are exact in fp32, so the two differ by
+    accumulation order only."""
+    layer = synth.conv(128, 128, 3, 1, 1, 14, name="tc vs fma")
+    inp = synth.layer_inputs(layer, 4, "bf16", 941)
+    a = gpu_layer(layer, inp, "bf16", STORE, TENSOR_CORE)
+    b = gpu_layer(layer, inp, "bf16", STORE, CUDA_CORE)
+    assert rel_l2(a["G_w"], b["G_w"]) <= 1e-5
+    np.testing.assert_allclose(a["sq"], b["sq"], rtol=1e-5)
+
+
+def test_tensor_core_rerun_is_bit_identical():
+    layer = synth.conv(64, 128, 3, 1, 1, 14, name="tc rerun")
+    inp = synth.layer_inputs(layer, 6, "bf16", 942)
+    a = gpu_layer(layer, inp, "bf16", STORE, TENSOR_CORE)
+    b = gpu_layer(layer, inp, "bf16", STORE, TENSOR_CORE)
+    np.testing.assert_array_equal(a["G_w"], b["G_w"])
+    np.testing.assert_array_equal(a["sq"], b["sq"])
