@@ -418,16 +418,77 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_sweep(args):
+    """configs[2] / any layer list: time dp_per_example_wgrad per layer with both epilogues.
+    L2 is flushed (a 512 MB buffer is overwritten) before every timed launch."""
+    import torch
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2109_12191_b200 import binding as b, synth
+    from paper_2109_12191_b200.step import layer_desc
+    peaks = measured_peaks()
+    cfg = synth.resnet50_sweep() if args.workload == "sweep" else None
+    layers = cfg["layers"]
+    if args.workload == "sweep_all":
+        layers = [l for l in synth.resnet50_gn_layers() if l.kind != "norm"]
+    if args.layers:
+        layers = [layers[int(i)] for i in args.layers.split(",")]
+    Bn, dtype = 32, "bf16"
+    flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")
+    rows, reps = [], max(3, args.steps or 10)
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    for l in layers:
+        X = torch.randn(l.x_shape(Bn), device="cuda", generator=g).to(torch.bfloat16)
+        dY = torch.randn(l.dy_shape(Bn), device="cuda", generator=g).to(torch.bfloat16)
+        G_w = torch.empty((Bn, l.n_weight), device="cuda")
+        sq = torch.empty((Bn, 1), device="cuda")
+        row = {"layer": l.name, "M": l.Kout, "N": l.R * l.S * l.Cin, "K": l.OH * l.OW}
+        in_bytes = (X.numel() + dY.numel()) * 2
+        flops = l.flops() * Bn
+        for epi, tag, out_bytes in ((b.DP_EPI_STORE_NORM, "store", G_w.numel() * 4), (b.DP_EPI_NORM_ONLY, "norm", 0)):
+            d = layer_desc(l, Bn, dtype, b.DP_IMPL_AUTO, 0)
+            ws = torch.empty(max(b.dp_workspace_bytes(d, epi), 256), dtype=torch.uint8, device="cuda")
+            call = lambda: b.check(b.dp_per_example_wgrad(d, X, dY, G_w, None, sq, 1, epi, 0.0, None, None, None, ws))
+            for _ in range(3):
+                call()
+            times = []
+            for _ in range(reps):
+                flush.fill_(1.0)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); call(); e1.record()
+                torch.cuda.synchronize()
+                times.append(e0.elapsed_time(e1))
+            b.check(b.dp_wgrad_check(ws))
+            ms = statistics.median(times)
+            t_hbm = (in_bytes + out_bytes) / (peaks["hbm"] * 1e9) * 1e3
+            t_tc = flops / (peaks["bf16"] * 1e12) * 1e3
+            row[tag] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1), "gbs": round((in_bytes + out_bytes) / ms / 1e6, 1),
+                        "bound": "hbm" if t_hbm > t_tc else "tensor", "frac_of_bound": round(max(t_hbm, t_tc) / ms, 3),
+                        "tc": bool(b.dp_wgrad_uses_tensor_cores(d, epi)), "ex_per_s": round(Bn / ms * 1e3, 1)}
+        rows.append(row)
+        del X, dY, G_w
+    tot_store = sum(r["store"]["ms"] for r in rows)
+    tot_norm = sum(r["norm"]["ms"] for r in rows)
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "workload": args.workload, "B": Bn, "dtype": "bf16", "peaks": peaks,
+                      "store_total_ms": round(tot_store, 3), "norm_total_ms": round(tot_norm, 3),
+                      "store_ex_per_s": round(Bn / tot_store * 1e3, 1), "norm_ex_per_s": round(Bn / tot_norm * 1e3, 1),
+                      "layers": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS) + ["sweep", "sweep_all"])
     ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--layers", default="", help="sweep workloads: comma-separated layer indices")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload in ("sweep", "sweep_all"):
+        return run_sweep(args)
     defaults = {"small_cnn": (400, 10), "flat": (8, 3)}
     if args.steps is None:
         args.steps = defaults[args.workload][0]

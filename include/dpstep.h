@@ -178,6 +178,12 @@ DP_API const char *dp_status_string(int status);
 /* Text of the last CUDA error this thread's calls ran into ("" if none). Host memory owned by the library. */
 DP_API const char *dp_last_cuda_error(void);
 
+/* Test / report hook: the tiling the tensor-core kernel would use for a conv layer, as up to 12 ints
+ * {rows-are-input-columns, row extent, column extent, row tiles, column tiles, columns per tile,
+ *  pixel-tile width, pixel-tile height, pixels per stage, pixel tiles, pipeline stages, bytes per stage}.
+ * Returns the number of values available (0 when the layer is not eligible). `out` is host memory. */
+DP_API int dp_debug_wgrad_plan(const dp_layer_desc *desc, int *out, int n);
+
 /* Number of kernels this process has launched through the library so far (a host-side counter;
  * benchmarks report the difference over their timed region). */
 DP_API unsigned long long dp_debug_launch_count(void);

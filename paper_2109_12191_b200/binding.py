@@ -27,7 +27,7 @@ DP_IMPL_AUTO, DP_IMPL_CUDA_CORE, DP_IMPL_TENSOR_CORE = 0, 1, 2
 EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_clip_workspace_bytes",
            "dp_clip_accumulate", "dp_noise_average", "dp_debug_philox_raw", "dp_debug_noise_z",
            "dp_wgrad_check", "dp_wgrad_uses_tensor_cores", "dp_status_string", "dp_last_cuda_error",
-           "dp_debug_launch_count"]
+           "dp_debug_launch_count", "dp_debug_wgrad_plan"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -66,6 +66,7 @@ _lib.dp_wgrad_check.argtypes = [_vp, _vp]; _lib.dp_wgrad_check.restype = _i
 _lib.dp_status_string.argtypes = [_i]; _lib.dp_status_string.restype = ctypes.c_char_p
 _lib.dp_last_cuda_error.argtypes = []; _lib.dp_last_cuda_error.restype = ctypes.c_char_p
 _lib.dp_debug_launch_count.argtypes = []; _lib.dp_debug_launch_count.restype = _ull
+_lib.dp_debug_wgrad_plan.argtypes = [_dp, ctypes.POINTER(_i), _i]; _lib.dp_debug_wgrad_plan.restype = _i
 
 
 def _ptr(t):
@@ -158,3 +159,12 @@ def dp_last_cuda_error():
 
 def dp_debug_launch_count():
     return _lib.dp_debug_launch_count()
+
+
+PLAN_FIELDS = ("a_is_x", "a_ext", "b_ext", "m_tiles", "n_tiles", "NT", "OWt", "OHt", "Kt", "k_tiles", "stages", "stage_bytes")
+
+
+def dp_debug_wgrad_plan(desc):
+    out = (_i * 12)()
+    n = _lib.dp_debug_wgrad_plan(ctypes.byref(desc), out, 12)
+    return dict(zip(PLAN_FIELDS, list(out)[:n])) if n else None

@@ -192,6 +192,11 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
     }
 }
 
+extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int *out, int n) {
+    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || !out || n <= 0) return 0;
+    return tc_describe_plan(desc->dtype, geom_of(desc), out, n);
+}
+
 extern "C" dp_status dp_wgrad_check(const void *workspace, void *cuda_stream) {
     if (!workspace) return DP_ERR_INVALID_ARG;
     int status = 0;

@@ -22,8 +22,7 @@
 
 namespace dp {
 
-constexpr int kSlabCh = 64;            // bf16 channels per 128-byte row
-constexpr int kRowBytes = 128;
+constexpr int kRowBytes = 128;         // one pixel's slab of channels: 64 bf16 or 32 fp32/tf32
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 200 * 1024;
 constexpr uint32_t kWaitPolls = 1u << 21;   // x ~1 us suspend hint: about two seconds before a wait gives up
@@ -31,8 +30,8 @@ constexpr uint32_t kWaitPolls = 1u << 21;   // x ~1 us suspend hint: about two s
 struct TcPlan {
     bool ok;
     int a_is_x;                 // 1: rows of D are columns j of Xcol, columns of D are output channels k
-    int a_ext, b_ext;           // operand extents (multiples of 64)
-    int m_tiles, n_tiles, NT;   // NT: nominal columns per tile (multiple of 64, <= 256)
+    int a_ext, b_ext;           // operand extents in elements (multiples of the slab width)
+    int m_tiles, n_tiles, NT;   // NT: nominal columns per tile (<= 256)
     int OWt, OHt, tiles_w, tiles_h, Kt, k_tiles;
     int stages, stage_bytes, a_bytes;
     size_t smem;
@@ -40,6 +39,8 @@ struct TcPlan {
 
 struct TcParams {
     int B, Kout, Ng, Cin, S, stride, pad;
+    int slab_ch;                // channels per 128-byte row: 64 (bf16) or 32 (fp32 as tf32)
+    int krows;                  // reduction rows per MMA: 16 (bf16) or 8 (tf32)
     int a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT;
     int OWt, OHt, tiles_w, Kt, k_tiles, stages, stage_bytes, a_bytes;
     int mode;                   // 0 store + norm, 1 norm only
@@ -47,7 +48,7 @@ struct TcParams {
     float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
     int slots;
     int *status;
-    long long total_tiles;
+    int total_tiles;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -95,11 +96,17 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate, issued by one thread
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+// D[tmem] (+)= A[smem] * B[smem], fp32 accumulate, issued by one thread; TF32 selects kind::tf32 (fp32 inputs)
+template <bool TF32>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    if (TF32)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -113,39 +120,26 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// Shared-memory operand descriptor: MN-major slab(s) with the 128-byte swizzle.
-//   start address >> 4 | leading byte offset (between 64-channel slabs) >> 4 at bit 16 |
-//   stride byte offset (between groups of 8 reduction rows = 1024 B) >> 4 at bit 32 |
-//   descriptor version 1 at bit 46 | layout type 2 (128-byte swizzle) at bit 61
-__device__ __forceinline__ uint64_t operand_desc(uint32_t addr, uint32_t slab_stride_bytes) {
-    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((slab_stride_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;
+// Shared-memory operand descriptor without the start address, for MN-major slabs of 128-byte rows.
+//   leading byte offset (between slabs) >> 4 at bit 16 | stride byte offset (between groups of reduction rows) >> 4
+//   at bit 32 | descriptor version 1 at bit 46 | layout type at bit 61.
+// 16-bit operands use the plain 128-byte swizzle (type 2: 16-byte chunks, pattern repeats every 8 rows = 1024 B).
+// 32-bit (tf32) MN-major operands only exist with the 128-byte swizzle of 32-byte chunks (type 1: pattern
+// repeats every 4 rows = 512 B); the tensor map then uses the matching SWIZZLE_128B_ATOM_32B mode.
+template <bool TF32>
+__device__ __forceinline__ uint64_t operand_desc_base(uint32_t slab_stride_bytes) {
+    uint64_t d = (uint64_t)((slab_stride_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(((TF32 ? 512u : 1024u) >> 4) & 0x3FFFu) << 32;
     d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
+    d |= (uint64_t)(TF32 ? 1 : 2) << 61;
     return d;
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both MN-major, M = 128, N = n_cols.
-__device__ __forceinline__ uint32_t instr_desc(int n_cols) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n_cols >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: fp32 accumulator, A and B of one type (bf16 = 1, tf32 = 2), both MN-major, M = 128, N = n_cols.
+__device__ __forceinline__ uint32_t instr_desc(int n_cols, uint32_t fmt) {
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n_cols >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// TMA start coordinates of 64-channel slab `slab` of an operand for the pixel tile at (oh0, ow0)
-__device__ __forceinline__ void slab_coords(bool is_x, int slab, const TcParams &p, int oh0, int ow0, int &c0, int &c1, int &c2) {
-    if (is_x) {
-        const int j0 = slab * kSlabCh;
-        const int tap = j0 / p.Cin;
-        c0 = j0 - tap * p.Cin;
-        const int r = tap / p.S, s = tap - r * p.S;
-        c1 = ow0 * p.stride + s - p.pad;
-        c2 = oh0 * p.stride + r - p.pad;
-    } else {
-        c0 = slab * kSlabCh;
-        c1 = ow0;
-        c2 = oh0;
-    }
-}
-
+template <bool TF32>
 __global__ void __launch_bounds__(192, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -158,6 +152,9 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const uint32_t tiles_u32 = smem_u32(tiles);
 
     if (threadIdx.x == 0) {
+        // pull both tensor maps into the TMA descriptor cache before the first copy needs them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
@@ -172,37 +169,54 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
     const int tiles_per_example = p.m_tiles * p.n_tiles;
     const int slab_bytes = p.Kt * kRowBytes;
+    const int a_slabs_tile = 128 / p.slab_ch, b_slabs_tile = p.NT / p.slab_ch;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer (one lane)
-        if (lane == 0) {
-            const CUtensorMap *mapA = p.a_is_x ? &tmX : &tmY, *mapB = p.a_is_x ? &tmY : &tmX;
-            int stage = 0; uint32_t phase = 0;
-            bool live = true;
-            for (long long t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-                const int n = (int)(t / tiles_per_example);
-                const int rem = (int)(t - (long long)n * tiles_per_example);
-                const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
-                const int a_slab0 = mt * 2, a_slabs = min(2, p.a_ext / kSlabCh - a_slab0);
-                const int b_slab0 = nt * (p.NT / kSlabCh), b_slabs = min(p.NT / kSlabCh, p.b_ext / kSlabCh - b_slab0);
-                for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    const int th = kt / p.tiles_w, tw = kt - th * p.tiles_w;
-                    const int oh0 = th * p.OHt, ow0 = tw * p.OWt;
-                    if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p)) { live = false; break; }
-                    const uint32_t bar = smem_u32(&full_bar[stage]);
-                    mbar_expect_tx(bar, (uint32_t)((a_slabs + b_slabs) * slab_bytes));
-                    const uint32_t a_dst = tiles_u32 + stage * p.stage_bytes, b_dst = a_dst + p.a_bytes;
-                    int c0, c1, c2;
-                    for (int s = 0; s < a_slabs; ++s) {
-                        slab_coords(p.a_is_x != 0, a_slab0 + s, p, oh0, ow0, c0, c1, c2);
-                        tma_load_4d(a_dst + s * slab_bytes, mapA, bar, c0, c1, c2, n);
-                    }
-                    for (int s = 0; s < b_slabs; ++s) {
-                        slab_coords(p.a_is_x == 0, b_slab0 + s, p, oh0, ow0, c0, c1, c2);
-                        tma_load_4d(b_dst + s * slab_bytes, mapB, bar, c0, c1, c2, n);
-                    }
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        // ------------------------------------------------------------ TMA producer
+        // Lane L owns slab L of the stage (A slabs first, then B slabs): it works out its tap shift and channel
+        // offset once per tile and then only adds the pixel-tile origin, so no division sits in the stage loop.
+        int stage = 0; uint32_t phase = 0;
+        bool live = true;
+        for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+            const int n = t / tiles_per_example;
+            const int rem = t - n * tiles_per_example;
+            const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+            const int a_slab0 = mt * a_slabs_tile, a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - a_slab0);
+            const int b_slab0 = nt * b_slabs_tile, b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - b_slab0);
+            const bool is_a = lane < a_slabs_tile;
+            const int local = is_a ? lane : lane - a_slabs_tile;
+            const bool active = is_a ? (local < a_slabs) : (local < b_slabs);
+            const bool is_x = is_a ? (p.a_is_x != 0) : (p.a_is_x == 0);
+            const int slab = (is_a ? a_slab0 : b_slab0) + local;
+            int c0, dw = 0, dh = 0, mul = 1;
+            if (is_x) {
+                const int j0 = slab * p.slab_ch;
+                const int tap = j0 / p.Cin;
+                c0 = j0 - tap * p.Cin;
+                const int r = tap / p.S;
+                dw = (tap - r * p.S) - p.pad;
+                dh = r - p.pad;
+                mul = p.stride;
+            } else {
+                c0 = slab * p.slab_ch;
+            }
+            const CUtensorMap *map = is_x ? &tmX : &tmY;
+            const uint32_t dst_off = (is_a ? 0u : (uint32_t)p.a_bytes) + (uint32_t)(local * slab_bytes);
+            const uint32_t tx_bytes = (uint32_t)((a_slabs + b_slabs) * slab_bytes);
+            int ow0 = 0, oh0 = 0, tw = 0;
+            for (int kt = 0; kt < p.k_tiles; ++kt) {
+                bool ok = true;
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p);
+                    if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { live = false; break; }
+                if (active)
+                    tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
+                                ow0 * mul + dw, oh0 * mul + dh, n);
+                if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -212,25 +226,30 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             uint32_t acc_phase = 0;  // bit b: phase of accumulator buffer b
             int buf = 0;
             bool live = true;
-            for (long long t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-                const int rem = (int)(t % tiles_per_example);
-                const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
-                const int a_slabs = min(2, p.a_ext / kSlabCh - mt * 2);
-                const int b_slabs = min(p.NT / kSlabCh, p.b_ext / kSlabCh - nt * (p.NT / kSlabCh));
-                const uint32_t idesc = instr_desc(b_slabs * kSlabCh);
-                // a single live slab is read twice (leading offset 0): rows 64..127 of D repeat rows 0..63 and are ignored
-                const uint32_t a_lbo = (a_slabs == 2) ? (uint32_t)slab_bytes : 0u;
+            const uint64_t desc_hi = operand_desc_base<TF32>((uint32_t)slab_bytes);
+            const int ksteps = p.Kt / p.krows;
+            const uint32_t kadvance = (uint32_t)(p.krows * kRowBytes) >> 4;     // descriptor start-address units of 16 B
+            for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+                const int rem = t % tiles_per_example;
+                const int nt = rem % p.n_tiles;
+                const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
+                const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, TF32 ? 2u : 1u);
                 if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p)) { live = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                uint32_t accumulate = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
                     if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p)) { live = false; break; }
                     tc_fence_after();
-                    const uint32_t a_src = tiles_u32 + stage * p.stage_bytes, b_src = a_src + p.a_bytes;
-                    for (int ks = 0; ks < p.Kt / 16; ++ks) {
-                        const uint64_t ad = operand_desc(a_src + ks * 2048, a_lbo);
-                        const uint64_t bd = operand_desc(b_src + ks * 2048, (uint32_t)slab_bytes);
-                        umma_bf16(d_tmem, ad, bd, idesc, (kt | ks) ? 1u : 0u);
+                    const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
+                    uint64_t ad = desc_hi | (uint64_t)((a_src & 0x3FFFFu) >> 4);
+                    uint64_t bd = desc_hi | (uint64_t)(((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
+                    // rows of the A tile past the operand's extent hold whatever the stage held before:
+                    // they only feed rows of D that the epilogue never reads
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        umma<TF32>(d_tmem, ad, bd, idesc, accumulate);
+                        accumulate = 1;
+                        ad += kadvance; bd += kadvance;
                     }
                     umma_commit(smem_u32(&empty_bar[stage]));      // frees the stage once these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -248,9 +267,9 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         uint32_t full_phase = 0;     // bit b: parity to wait for on accumulator buffer b
         int buf = 0;
         bool live = true;
-        for (long long t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-            const int n = (int)(t / tiles_per_example);
-            const int rem = (int)(t - (long long)n * tiles_per_example);
+        for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+            const int n = t / tiles_per_example;
+            const int rem = t - n * tiles_per_example;
             const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
             const int a_rows = min(128, p.a_ext - mt * 128);
             const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
@@ -322,7 +341,20 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-static int step_cycles(int n_cols) {     // per 16-pixel MMA step: tensor pipe vs shared-memory operand reads
+static int sm_count() {
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            sms = v;
+        else
+            return 148;
+    }
+    return sms;
+}
+
+// cycles of one MMA step (one instruction): tensor pipe (N/2) against shared-memory operand reads (4 KB of A + N*32 B of B at 128 B/clk)
+static int step_cycles(int n_cols) {
     const int pipe = n_cols / 2, smem = 32 + n_cols / 4;
     return pipe > smem ? pipe : smem;
 }
@@ -333,7 +365,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g);
 static TcPlan make_plan(int dtype, const ConvGeom &g) {
     static std::mutex mu;
     static std::map<std::array<int, 10>, TcPlan> memo;
-    const std::array<int, 10> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, 0};
+    const std::array<int, 10> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B};
     std::lock_guard<std::mutex> lock(mu);
     auto it = memo.find(key);
     if (it != memo.end()) return it->second;
@@ -344,45 +376,51 @@ static TcPlan make_plan(int dtype, const ConvGeom &g) {
 
 static TcPlan search_plan(int dtype, const ConvGeom &g) {
     TcPlan best; best.ok = false;
-    if (dtype != DP_BF16) return best;
-    if (g.stride != 1) return best;
-    if (g.Cin % kSlabCh || g.Kout % kSlabCh) return best;
-    if (g.OW > 256 || g.OH > 65535 || g.K < 1) return best;
+    if (dtype != DP_BF16) return best;   // fp32 inputs stay on the CUDA cores until the split-tf32 path lands
+    const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
+    const int krows = (dtype == DP_BF16) ? 16 : 8;
+    if (g.Cin % slab_ch || g.Kout % slab_ch) return best;
+    if (g.stride > 8 || g.K < 1 || g.OH > 65535) return best;
+    const int sms = sm_count();
+    const int a_slabs_tile = 128 / slab_ch;
     double best_cost = 1e300;
     for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
         const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
-        for (int NT = 64; NT <= 256; NT += 64) {
-            if (NT > b_ext && NT != 64 * ((b_ext + 63) / 64)) continue;
-            const int nt_cols = NT < b_ext ? NT : b_ext;
-            const int m_tiles = (a_ext + 127) / 128, n_tiles = (b_ext + nt_cols - 1) / nt_cols;
-            const int slabs = 2 + nt_cols / kSlabCh;
-            long long mma = 0;
-            for (int t = 0; t < n_tiles; ++t) mma += step_cycles(std::min(nt_cols, b_ext - t * nt_cols));
-            mma *= m_tiles;
-            for (int OHt = 1; OHt <= g.OH && OHt <= g.H && OHt <= 256; ++OHt)
-                for (int OWt = 1; OWt <= g.OW && OWt <= g.W; ++OWt) {
+        for (int NT = slab_ch; NT <= 256; NT += slab_ch) {
+            if (NT != 32 && NT % 64) continue;
+            if (NT > b_ext) break;
+            const int m_tiles = (a_ext + 127) / 128, n_tiles = (b_ext + NT - 1) / NT;
+            const int slabs = a_slabs_tile + NT / slab_ch;
+            const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
+            if (total_tiles > 0x7fffffffLL) continue;
+            const long long waves = (total_tiles + sms - 1) / sms;
+            for (int OHt = 1; OHt <= g.OH; ++OHt) {
+                if (OHt * g.stride > 256 || OHt * g.stride > g.H) break;
+                for (int OWt = 1; OWt <= g.OW; ++OWt) {
+                    if (OWt * g.stride > 256 || OWt * g.stride > g.W) break;
                     const int Kt = OHt * OWt;
-                    if (Kt % 16 || Kt > 256) continue;
+                    if (Kt % krows || Kt > 256) continue;
                     const int stage_bytes = slabs * Kt * kRowBytes;
                     int stages = kSmemBudget / stage_bytes;
                     if (stages < 2) continue;
                     if (stages > kMaxStages) stages = kMaxStages;
                     const int tw = (g.OW + OWt - 1) / OWt, th = (g.OH + OHt - 1) / OHt;
-                    const long long steps = (long long)tw * th * (Kt / 16);
-                    // cost: tensor-pipe cycles, a fixed toll per stage hand-over, and a penalty for shallow pipelines
-                    double cost = (double)mma * steps + 60.0 * tw * th * m_tiles * n_tiles;
-                    if (stages < 3) cost *= 1.25;
-                    cost *= 1.0 + 0.02 * (256 - nt_cols) / 64;
+                    // a stage costs the larger of its tensor time and the fixed hand-over work of the issuing threads
+                    const double stage_cost = std::max((double)(Kt / krows) * step_cycles(NT), 450.0);
+                    double tile_cost = stage_cost * tw * th + 600.0;
+                    if (stages < 3) tile_cost *= 1.3;
+                    const double cost = tile_cost * (double)waves;
                     if (cost < best_cost) {
                         best_cost = cost;
                         best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
-                        best.m_tiles = m_tiles; best.n_tiles = n_tiles; best.NT = nt_cols;
+                        best.m_tiles = m_tiles; best.n_tiles = n_tiles; best.NT = NT;
                         best.OWt = OWt; best.OHt = OHt; best.tiles_w = tw; best.tiles_h = th; best.Kt = Kt;
                         best.k_tiles = tw * th; best.stages = stages; best.stage_bytes = stage_bytes;
-                        best.a_bytes = 2 * Kt * kRowBytes;
+                        best.a_bytes = a_slabs_tile * Kt * kRowBytes;
                         best.smem = (size_t)stages * stage_bytes + 1024;
                     }
                 }
+            }
         }
     }
     return best;
@@ -400,13 +438,27 @@ int tc_norm_slots(int dtype, const ConvGeom &g, int) {
 
 size_t tc_workspace_bytes(int, const ConvGeom &, int) { return 0; }
 
-static bool encode_nhwc(CUtensorMap *map, const void *base, int C, int W, int H, int Bn, int boxW, int boxH) {
+int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n) {
+    const TcPlan pl = make_plan(dtype, g);
+    if (!pl.ok) return 0;
+    const int v[12] = {pl.a_is_x, pl.a_ext, pl.b_ext, pl.m_tiles, pl.n_tiles, pl.NT, pl.OWt, pl.OHt, pl.Kt, pl.k_tiles,
+                       pl.stages, pl.stage_bytes};
+    for (int i = 0; i < n && i < 12; ++i) out[i] = v[i];
+    return 12;
+}
+
+// channels-last [B, H, W, C] tensor, box = {one slab of channels, boxW, boxH, 1 example}; `step` > 1 walks every
+// step-th pixel (the box then spans boxW*step pixels and delivers boxW of them)
+static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, int W, int H, int Bn, int boxW, int boxH, int step) {
+    const cuuint64_t es = (dtype == DP_BF16) ? 2 : 4;
     const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)Bn};
-    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)kSlabCh, (cuuint32_t)boxW, (cuuint32_t)boxH, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    const cuuint64_t strides[3] = {(cuuint64_t)C * es, (cuuint64_t)W * C * es, (cuuint64_t)H * W * C * es};
+    const cuuint32_t box[4] = {(cuuint32_t)(kRowBytes / es), (cuuint32_t)(boxW * step), (cuuint32_t)(boxH * step), 1};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)step, (cuuint32_t)step, 1};
+    return encode_fn()(map, dtype == DP_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+                       const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       dtype == DP_BF16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -415,27 +467,28 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     const TcPlan pl = make_plan(dtype, g);
     if (!pl.ok || !encode_fn() || epilogue == DP_EPI_CLIP_ACCUM) return DP_ERR_UNSUPPORTED;
     CUtensorMap tmX, tmY;
-    if (!encode_nhwc(&tmX, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
-    if (!encode_nhwc(&tmY, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
     TcParams p;
     p.B = g.B; p.Kout = g.Kout; p.Ng = g.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.slab_ch = (dtype == DP_BF16) ? 64 : 32; p.krows = (dtype == DP_BF16) ? 16 : 8;
     p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
     p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
     p.mode = (epilogue == DP_EPI_STORE_NORM) ? 0 : 1;
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
-    p.total_tiles = (long long)g.B * pl.m_tiles * pl.n_tiles;
+    p.total_tiles = g.B * pl.m_tiles * pl.n_tiles;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
-    int dev = 0, sms = 148;
-    DP_CUDA_TRY(cudaGetDevice(&dev));
-    DP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const unsigned grid = (unsigned)std::min<long long>(p.total_tiles, sms);
-    conv_wgrad_tc_kernel<<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+    const unsigned grid = (unsigned)std::min(p.total_tiles, sm_count());
+    if (dtype == DP_BF16) conv_wgrad_tc_kernel<false><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+    else conv_wgrad_tc_kernel<true><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
     return DP_OK;
 }

@@ -136,27 +136,30 @@ def test_dense_norm_is_the_rank1_closed_form():
     np.testing.assert_allclose(out["sq"][:, 0], y2 * x2 + y2, rtol=1e-6)
 
 
-# ------------------------------------------------------------------ tcgen05 path (bf16, 64-channel multiples)
+# ------------------------------------------------------------------ tcgen05 path
 TC_CONVS = [
-    # Cin, Kout, R, stride, pad, H, bias
-    (64, 64, 1, 1, 0, 8, False),       # both extents 64: a single operand slab read twice
-    (64, 64, 3, 1, 1, 8, True),        # 576 columns: tiles of 256, 256, 64
-    (128, 128, 3, 1, 1, 8, False),
-    (64, 256, 1, 1, 0, 14, False),     # 14x14: pixel tiles hang over the image edge (zero filled)
-    (256, 64, 1, 1, 0, 14, False),
-    (128, 192, 3, 1, 1, 12, True),
-    (64, 64, 3, 1, 1, 7, False),       # 49 pixels inside an 8x8 pixel tile
-    (64, 128, 3, 1, 0, 10, False),     # no padding: 8x8 outputs from a 10x10 input
-    (320, 64, 1, 1, 0, 6, False),      # extent 320 = 2.5 row tiles
-    (64, 64, 5, 1, 2, 9, False),       # 5x5 taps
+    # dtype, Cin, Kout, R, stride, pad, H, bias        (bf16: channels in multiples of 64; fp32 runs as tf32: multiples of 32)
+    ("bf16", 64, 64, 1, 1, 0, 8, False),       # both extents 64: half of the 128-row tile is unused
+    ("bf16", 64, 64, 3, 1, 1, 8, True),        # 576 columns: ragged last tile
+    ("bf16", 128, 128, 3, 1, 1, 8, False),
+    ("bf16", 64, 256, 1, 1, 0, 14, False),     # 14x14: pixel tiles hang over the image edge (zero filled)
+    ("bf16", 256, 64, 1, 1, 0, 14, False),
+    ("bf16", 128, 192, 3, 1, 1, 12, True),
+    ("bf16", 64, 64, 3, 1, 1, 7, False),       # 49 pixels
+    ("bf16", 64, 128, 3, 1, 0, 10, False),     # no padding: 8x8 outputs from a 10x10 input
+    ("bf16", 320, 64, 1, 1, 0, 6, False),      # extent 320 = 2.5 row tiles
+    ("bf16", 64, 64, 5, 1, 2, 9, False),       # 5x5 taps
+    ("bf16", 128, 128, 3, 2, 1, 14, False),    # stride 2 through the tensor map's element stride
+    ("bf16", 64, 128, 1, 2, 0, 14, False),     # strided 1x1 (projection shortcut)
+    ("bf16", 64, 64, 3, 2, 1, 15, True),       # odd input size with stride 2
 ]
 
 
 @pytest.mark.parametrize("case", TC_CONVS)
 def test_conv_tensor_core(case):
-    Cin, Kout, R, stride, pad, H, bias = case
+    dtype, Cin, Kout, R, stride, pad, H, bias = case
     layer = synth.conv(Cin, Kout, R, stride, pad, H, bias, name=str(case))
-    out = check_layer(layer, 5, "bf16", TENSOR_CORE, (940, sum(case[:6])), spread=True, clip_impl=AUTO)
+    out = check_layer(layer, 5, dtype, TENSOR_CORE, (940, sum(case[1:7])), spread=True, clip_impl=AUTO)
     assert out["uses_tc"]
 
 
