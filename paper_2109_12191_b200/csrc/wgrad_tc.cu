@@ -13,6 +13,11 @@
 // warps 2-5 read accumulators back with tcgen05.ld, square-sum them (the per-example norm) and store.
 // Two accumulator buffers in TMEM let the epilogue of one tile overlap the main loop of the next.
 // Every wait is bounded: on expiry the CTA sets a status word, drains and returns.
+//
+// fp32 inputs run as split tf32: the tensor core truncates fp32 to tf32, which biases every norm by about
+// 1e-3, so four more warps split each landed stage into hi = x with the low 13 mantissa bits cleared (kept
+// in place) and lo = x - hi (a second buffer of the same layout), and the issuer accumulates
+// hi*hi + lo*hi + hi*lo per step.  What is dropped (lo*lo and the truncation of lo) is below 2^-20 relative.
 #include "wgrad_tc.cuh"
 #include <cuda.h>
 #include <mutex>
@@ -43,6 +48,7 @@ struct TcParams {
     int krows;                  // reduction rows per MMA: 16 (bf16) or 8 (tf32)
     int a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT;
     int OWt, OHt, tiles_w, Kt, k_tiles, stages, stage_bytes, a_bytes;
+    int lo_offset;              // split tf32: byte offset of the lo copy inside a stage
     int mode;                   // 0 store + norm, 1 norm only
     float *G_w;
     float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
@@ -140,10 +146,10 @@ __device__ __forceinline__ uint32_t instr_desc(int n_cols, uint32_t fmt) {
 }
 
 template <bool TF32>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(TF32 ? 320 : 192, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], ready_bar[kMaxStages], tmem_full[2], tmem_empty[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -156,7 +162,9 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
         abort_flag = 0;
-        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 4);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -239,17 +247,28 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
                 uint32_t accumulate = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p)) { live = false; break; }
+                    if (!mbar_wait(smem_u32(TF32 ? &ready_bar[stage] : &full_bar[stage]), phase, abort_p)) { live = false; break; }
                     tc_fence_after();
                     const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
                     uint64_t ad = desc_hi | (uint64_t)((a_src & 0x3FFFFu) >> 4);
                     uint64_t bd = desc_hi | (uint64_t)(((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
                     // rows of the A tile past the operand's extent hold whatever the stage held before:
                     // they only feed rows of D that the epilogue never reads
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        umma<TF32>(d_tmem, ad, bd, idesc, accumulate);
-                        accumulate = 1;
-                        ad += kadvance; bd += kadvance;
+                    if (TF32) {
+                        const uint64_t lo = (uint64_t)((uint32_t)p.lo_offset >> 4);
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            umma<TF32>(d_tmem, ad + lo, bd, idesc, accumulate);      // lo(A) * hi(B)
+                            umma<TF32>(d_tmem, ad, bd + lo, idesc, 1u);              // hi(A) * lo(B)
+                            umma<TF32>(d_tmem, ad, bd, idesc, 1u);                   // hi(A) * hi(B)
+                            accumulate = 1;
+                            ad += kadvance; bd += kadvance;
+                        }
+                    } else {
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            umma<TF32>(d_tmem, ad, bd, idesc, accumulate);
+                            accumulate = 1;
+                            ad += kadvance; bd += kadvance;
+                        }
                     }
                     umma_commit(smem_u32(&empty_bar[stage]));      // frees the stage once these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -258,6 +277,40 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 umma_commit(smem_u32(&tmem_full[buf]));            // accumulator complete
                 acc_phase ^= 1u << buf;
                 buf ^= 1;
+            }
+        }
+    } else if (TF32 && warp >= 6) {
+        // ------------------------------------------------------------ split warps (fp32 inputs only)
+        // hi stays where TMA put it, lo goes to the same offset of the stage's second half; both keep the
+        // swizzled layout because the split is element-wise on identical relative addresses.
+        const int tid = threadIdx.x - 192;
+        int stage = 0; uint32_t phase = 0;
+        bool live = true;
+        for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
+            const int rem = t % tiles_per_example;
+            const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+            const int a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - mt * a_slabs_tile);
+            const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
+            const int a_chunks = a_slabs * (slab_bytes >> 4), chunks = a_chunks + b_slabs * (slab_bytes >> 4);
+            for (int kt = 0; kt < p.k_tiles; ++kt) {
+                const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p);
+                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+                uint8_t *base = tiles + (size_t)stage * p.stage_bytes;
+                for (int i = tid; i < chunks; i += 128) {
+                    uint8_t *ptr = (i < a_chunks) ? base + ((size_t)i << 4) : base + p.a_bytes + ((size_t)(i - a_chunks) << 4);
+                    const float4 x = *reinterpret_cast<const float4 *>(ptr);
+                    float4 hi, lo;
+                    hi.x = __uint_as_float(__float_as_uint(x.x) & 0xFFFFE000u); lo.x = x.x - hi.x;
+                    hi.y = __uint_as_float(__float_as_uint(x.y) & 0xFFFFE000u); lo.y = x.y - hi.y;
+                    hi.z = __uint_as_float(__float_as_uint(x.z) & 0xFFFFE000u); lo.z = x.z - hi.z;
+                    hi.w = __uint_as_float(__float_as_uint(x.w) & 0xFFFFE000u); lo.w = x.w - hi.w;
+                    *reinterpret_cast<float4 *>(ptr) = hi;
+                    *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ready_bar[stage]));
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
     } else {
@@ -376,13 +429,14 @@ static TcPlan make_plan(int dtype, const ConvGeom &g) {
 
 static TcPlan search_plan(int dtype, const ConvGeom &g) {
     TcPlan best; best.ok = false;
-    if (dtype != DP_BF16) return best;   // fp32 inputs stay on the CUDA cores until the split-tf32 path lands
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
     if (g.Cin % slab_ch || g.Kout % slab_ch) return best;
     if (g.stride > 8 || g.K < 1 || g.OH > 65535) return best;
     const int sms = sm_count();
     const int a_slabs_tile = 128 / slab_ch;
+    const int copies = (dtype == DP_BF16) ? 1 : 2;      // split tf32 keeps a hi and a lo copy of every stage
+    const int mma_per_step = (dtype == DP_BF16) ? 1 : 3;
     double best_cost = 1e300;
     for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
         const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
@@ -400,13 +454,13 @@ static TcPlan search_plan(int dtype, const ConvGeom &g) {
                     if (OWt * g.stride > 256 || OWt * g.stride > g.W) break;
                     const int Kt = OHt * OWt;
                     if (Kt % krows || Kt > 256) continue;
-                    const int stage_bytes = slabs * Kt * kRowBytes;
+                    const int stage_bytes = slabs * Kt * kRowBytes * copies;
                     int stages = kSmemBudget / stage_bytes;
                     if (stages < 2) continue;
                     if (stages > kMaxStages) stages = kMaxStages;
                     const int tw = (g.OW + OWt - 1) / OWt, th = (g.OH + OHt - 1) / OHt;
                     // a stage costs the larger of its tensor time and the fixed hand-over work of the issuing threads
-                    const double stage_cost = std::max((double)(Kt / krows) * step_cycles(NT), 450.0);
+                    const double stage_cost = std::max((double)(Kt / krows) * step_cycles(NT) * mma_per_step, 450.0);
                     double tile_cost = stage_cost * tw * th + 600.0;
                     if (stages < 3) tile_cost *= 1.3;
                     const double cost = tile_cost * (double)waves;
@@ -475,6 +529,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
     p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
+    p.lo_offset = pl.stage_bytes / 2;
     p.mode = (epilogue == DP_EPI_STORE_NORM) ? 0 : 1;
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
     p.total_tiles = g.B * pl.m_tiles * pl.n_tiles;
@@ -488,7 +543,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
     const unsigned grid = (unsigned)std::min(p.total_tiles, sm_count());
     if (dtype == DP_BF16) conv_wgrad_tc_kernel<false><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
-    else conv_wgrad_tc_kernel<true><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+    else conv_wgrad_tc_kernel<true><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
     return DP_OK;
 }

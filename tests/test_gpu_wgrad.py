@@ -18,9 +18,9 @@ AUTO, CUDA_CORE, TENSOR_CORE = 0, 1, 2
 def tol_for(out, dtype):
     """Accumulated / stored gradient tolerance: plain fp32 rounding on the CUDA-core path and for bf16
     inputs (their products are exact in fp32); the TF32-class bound for fp32 inputs on tensor cores."""
-    if not out["uses_tc"]:
-        return TOL_FMA
-    return TOL_ACC_BF16 if dtype == "bf16" else TOL_ACC_F32
+    # bf16 products are exact in fp32 and fp32 inputs run as split tf32, so both implementations are held
+    # to plain fp32 rounding here -- far inside the 1e-2 / 2e-3 bounds the workload tests apply
+    return TOL_FMA
 
 
 def check_layer(layer, Bn, dtype, impl, key, bias_separate=0, spread=False, clip_impl=None):
@@ -152,6 +152,10 @@ TC_CONVS = [
     ("bf16", 128, 128, 3, 2, 1, 14, False),    # stride 2 through the tensor map's element stride
     ("bf16", 64, 128, 1, 2, 0, 14, False),     # strided 1x1 (projection shortcut)
     ("bf16", 64, 64, 3, 2, 1, 15, True),       # odd input size with stride 2
+    ("f32", 32, 64, 3, 2, 1, 32, True),        # second conv of the small CNN
+    ("f32", 64, 128, 3, 2, 1, 16, True),       # third conv of the small CNN
+    ("f32", 32, 32, 1, 1, 0, 8, False),
+    ("f32", 96, 160, 3, 1, 1, 9, False),       # extents that are multiples of 32 but not of 64 or 128
 ]
 
 
