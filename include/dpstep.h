@@ -139,6 +139,30 @@ DP_API dp_status dp_clip_accumulate(int mode, int B, int L, const float *const *
                              float *norms_out, float *clip_out,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* dp_clip_accumulate for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this exists for deployment reasons only.)
+ *
+ * Some callers have no way to hand over a workspace: code running inside a framework whose caching
+ * allocator already owns the whole device, plug-ins and callbacks that are forbidden to call cudaMalloc
+ * because it synchronises the device, and services that pre-reserve every byte at start-up.  For them
+ * the scratch of the norm / factor stages lives inside the library, in one fixed device array of
+ * dp_clip_static_scratch_bytes() bytes (2 MiB) that every GPU loading the library holds until exit.
+ * Arguments and results are those of dp_clip_accumulate without the workspace pair.
+ *
+ *   - Limit: problems whose dp_clip_workspace_bytes(B, L, P_l) exceeds the array are refused with
+ *     DP_ERR_WORKSPACE (dp_last_cuda_error() says why); nothing is launched.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device current); make that first call outside any stream capture.  No call allocates or frees memory.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to start at
+ *     zero (each call writes what it later reads), but two calls whose kernels overlap on the GPU -- different
+ *     streams, or different host threads on the same device -- race on it: keep such calls ordered. */
+DP_API dp_status dp_clip_accumulate_static(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                           const float *sqnorm, float C, float *const *acc,
+                                           float *norms_out, float *clip_out, void *cuda_stream);
+
+/* Size in bytes of the built-in scratch array dp_clip_accumulate_static works in. */
+DP_API size_t dp_clip_static_scratch_bytes(void);
+
 /* Noise and average (section 2): out[i] = (acc[i] + sigma * C * z_{param_offset+i}) / total_batch,
  * one pass, `out` may alias `acc`.  z is a standard normal that depends only on
  * (seed, step, global parameter index g = param_offset + i):

@@ -27,7 +27,8 @@ DP_IMPL_AUTO, DP_IMPL_CUDA_CORE, DP_IMPL_TENSOR_CORE = 0, 1, 2
 EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_clip_workspace_bytes",
            "dp_clip_accumulate", "dp_noise_average", "dp_debug_philox_raw", "dp_debug_noise_z",
            "dp_wgrad_check", "dp_wgrad_uses_tensor_cores", "dp_status_string", "dp_last_cuda_error",
-           "dp_debug_launch_count", "dp_debug_wgrad_plan"]
+           "dp_debug_launch_count", "dp_debug_wgrad_plan", "dp_clip_accumulate_static",
+           "dp_clip_static_scratch_bytes"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -59,6 +60,10 @@ _lib.dp_clip_workspace_bytes.argtypes = [_i, _i, ctypes.POINTER(_ll)]; _lib.dp_c
 _lib.dp_clip_accumulate.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctypes.POINTER(_ll), _vp, _f,
                                     ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
 _lib.dp_clip_accumulate.restype = _i
+_lib.dp_clip_accumulate_static.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctypes.POINTER(_ll), _vp, _f,
+                                           ctypes.POINTER(_vp), _vp, _vp, _vp]
+_lib.dp_clip_accumulate_static.restype = _i
+_lib.dp_clip_static_scratch_bytes.argtypes = []; _lib.dp_clip_static_scratch_bytes.restype = _sz
 _lib.dp_noise_average.argtypes = [_vp, _ll, _ll, _f, _f, _ll, _ull, _ull, _vp, _vp]; _lib.dp_noise_average.restype = _i
 _lib.dp_debug_philox_raw.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_philox_raw.restype = _i
 _lib.dp_debug_noise_z.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_noise_z.restype = _i
@@ -131,6 +136,19 @@ def dp_clip_accumulate(mode, B, G, P_l, sqnorm, C, acc, norms_out, clip_out, wor
     Ap = (_vp * L)(*[_ptr(a) for a in acc]) if acc is not None else None
     return _lib.dp_clip_accumulate(mode, B, L, Gp, (_ll * L)(*P_l), _ptr(sqnorm), C, Ap, _ptr(norms_out),
                                    _ptr(clip_out), _ptr(workspace), workspace_bytes, _stream(stream))
+
+
+def dp_clip_accumulate_static(mode, B, G, P_l, sqnorm, C, acc, norms_out, clip_out, stream=None):
+    """dp_clip_accumulate with the library's built-in scratch array instead of a caller workspace."""
+    L = len(P_l)
+    Gp = (_vp * L)(*[_ptr(g) for g in G]) if G is not None else None
+    Ap = (_vp * L)(*[_ptr(a) for a in acc]) if acc is not None else None
+    return _lib.dp_clip_accumulate_static(mode, B, L, Gp, (_ll * L)(*P_l), _ptr(sqnorm), C, Ap, _ptr(norms_out),
+                                          _ptr(clip_out), _stream(stream))
+
+
+def dp_clip_static_scratch_bytes():
+    return _lib.dp_clip_static_scratch_bytes()
 
 
 def dp_noise_average(acc, P, param_offset, sigma, C, total_batch, seed, step, out, stream=None):

@@ -9,6 +9,7 @@
 //      registers with 128-bit loads, and touches the accumulator once.
 #include "common.cuh"
 #include <math.h>
+#include <mutex>
 
 namespace dp {
 
@@ -278,4 +279,56 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
         }
     }
     return DP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------------
+// Variant of dp_clip_accumulate for callers that cannot supply scratch memory of their own.
+// The scratch lives in this file-scope device array, so every GPU that loads the library carries
+// kStaticScratchBytes of it until the process exits.
+namespace dp {
+constexpr size_t kStaticScratchBytes = 2u << 20;   // 2 MiB
+static __device__ __align__(256) unsigned char g_clip_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mu;
+static void *g_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of g_clip_scratch on the current device.  In host code the array's name is only a
+// stand-in for the symbol, never a usable address, so the address is asked for once per device, with
+// that device current, and remembered.
+static dp_status static_scratch(void **out) {
+    int dev = -1;
+    DP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return DP_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    if (!g_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        DP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_clip_scratch));
+        if (!ptr) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_clip_scratch)");
+        g_scratch_addr[dev] = ptr;
+    }
+    *out = g_scratch_addr[dev];
+    return DP_OK;
+}
+}  // namespace dp
+
+extern "C" size_t dp_clip_static_scratch_bytes(void) { return dp::kStaticScratchBytes; }
+
+extern "C" dp_status dp_clip_accumulate_static(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                               const float *sqnorm, float C, float *const *acc, float *norms_out,
+                                               float *clip_out, void *cuda_stream) {
+    if (B <= 0 || L <= 0 || !P_l) return DP_ERR_INVALID_ARG;
+    const size_t need = dp_clip_workspace_bytes(B, L, P_l);
+    if (need == 0) return DP_ERR_INVALID_ARG;
+    if (need > dp::kStaticScratchBytes) {
+        dp::note_error("dp_clip_accumulate_static: this problem needs more scratch than the built-in 2 MiB array; "
+                       "use dp_clip_accumulate with a caller-owned workspace");
+        return DP_ERR_WORKSPACE;
+    }
+    void *scratch = nullptr;
+    const dp_status rc = dp::static_scratch(&scratch);
+    if (rc != DP_OK) return rc;
+    // every scratch word the kernels read is written earlier in the same call, so nothing needs clearing
+    return dp_clip_accumulate(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, scratch, dp::kStaticScratchBytes,
+                              cuda_stream);
 }

@@ -10,6 +10,8 @@ namespace dp {
 
 // Records the text of a failed CUDA call for dp_last_cuda_error() and returns DP_ERR_CUDA.
 dp_status cuda_fail(cudaError_t e, const char *where);
+// Records a plain message for dp_last_cuda_error() (used where the failure is not a CUDA error code).
+void note_error(const char *message);
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

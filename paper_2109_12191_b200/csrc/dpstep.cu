@@ -19,6 +19,8 @@ dp_status cuda_fail(cudaError_t e, const char *where) {
     return DP_ERR_CUDA;
 }
 
+void note_error(const char *message) { snprintf(g_last_error, sizeof(g_last_error), "%s", message); }
+
 static bool valid_desc(const dp_layer_desc *d) {
     if (!d) return false;
     if (d->kind != DP_LAYER_DENSE && d->kind != DP_LAYER_CONV2D && d->kind != DP_LAYER_NORM_AFFINE) return false;
