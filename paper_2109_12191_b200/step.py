@@ -86,8 +86,9 @@ class GlobalClipStep:
             self.wgrad(li, X, dY)
         self.clip_accumulate()
 
-    def finish(self, seed=0, step=0):
-        total = self.B * self.chunks_done
+    def finish(self, seed=0, step=0, world=1):
+        """world > 1: `acc` already holds the sum over all ranks (see sharding.allreduce_accumulator)."""
+        total = self.B * self.chunks_done * world
         b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, total, seed, step, self.out), "dp_noise_average")
         return self.out
 
@@ -113,9 +114,9 @@ class FlatClipStep:
                                      self.clip, self.ws), "dp_clip_accumulate")
         self.chunks_done += 1
 
-    def finish(self, seed=0, step=0):
-        b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, self.B * self.chunks_done, seed, step, self.out),
-                "dp_noise_average")
+    def finish(self, seed=0, step=0, world=1):
+        b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, self.B * self.chunks_done * world, seed, step,
+                                   self.out), "dp_noise_average")
         return self.out
 
 
