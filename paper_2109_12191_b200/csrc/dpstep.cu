@@ -81,8 +81,13 @@ static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
         pl.dg_off = off;
         off = round_up(off + sizeof(float) * B * 2 * d->C_in, 256);
     }
-    pl.tc_off = off;
-    if (pl.use_tc) off = round_up(off + tc_workspace_bytes(d->dtype, g, epi), 256);
+    pl.tc_off = off;       // partial sums of the clipped-sum pass (either implementation)
+    if (epi == DP_EPI_CLIP_ACCUM && d->kind != DP_LAYER_NORM_AFFINE) {
+        size_t bytes = 0;
+        if (pl.use_tc) bytes = tc_workspace_bytes(d->dtype, g, epi);
+        else { const int sp = fma_clip_splits(g); bytes = sp > 1 ? sizeof(float) * (size_t)sp * g.M * g.N : 0; }
+        off = round_up(off + bytes, 256);
+    }
     pl.total = off;
     return true;
 }
@@ -147,18 +152,18 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         }
         if (epi != DP_EPI_CLIP_ACCUM) {
             if (pl.use_tc) rc = launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
-            else rc = launch_conv_fma(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, st);
+            else rc = launch_conv_fma(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, nullptr, st);
             if (rc != DP_OK) return rc;
             return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
         }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
-        else rc = launch_conv_fma(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, st);
+        else rc = launch_conv_fma(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
         if (rc != DP_OK) return rc;
         rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st);
         if (rc != DP_OK) return rc;
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
-        else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, st);
+        else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
@@ -175,7 +180,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
-        rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, 2, factor, acc_w, st);
+        rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, 2, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;

@@ -13,21 +13,24 @@ constexpr int TM = kFmaTile, TN = kFmaTile, TK = 16;
 //   A[q, m]  = dY[n, pix, m]                       q = n*K + pix
 //   Bm[q, j] = Xpad[n, oh*st + r - pad, ow*st + s - pad, c],  j = (r*S + s)*Cin + c
 // MODE 0/1: the block owns one example (blockIdx.z) and reduces q over that example's pixels.
-// MODE 2:   the block owns the tile for ALL examples: q runs over B*K and A is scaled by the
-//           example's clip factor, so the accumulator ends as sum_n f_n D_n[m, j].
+// MODE 2:   the block owns the tile for a RANGE of examples (blockIdx.z picks the range): q runs over
+//           those examples' pixels and A is scaled by the example's clip factor, so the accumulator ends
+//           as sum_n f_n D_n[m, j].  With one range the sum is added to acc_w; with several, range z
+//           writes its partial sum to sum_ws[z] and a fold kernel adds them in order.
 template <typename T, int MODE>
 __global__ void __launch_bounds__(256)
 conv_wgrad_fma_kernel(const T *__restrict__ X, const T *__restrict__ dY, const ConvGeom g, float *__restrict__ G_w,
                       float *__restrict__ partial, int slots, const float *__restrict__ factor,
-                      float *__restrict__ acc_w) {
+                      float *__restrict__ acc_w, int per_split, float *__restrict__ sum_ws) {
     __shared__ __align__(16) float sA[TK][TM];
     __shared__ __align__(16) float sB[TK][TN];
     __shared__ float scratch[32];
     const int tid = threadIdx.x;
     const int m0 = blockIdx.y * TM, j0 = blockIdx.x * TN;
     const int n_fixed = (MODE == 2) ? 0 : blockIdx.z;
-    const long long q_begin = (MODE == 2) ? 0 : (long long)n_fixed * g.K;
-    const long long q_end = (MODE == 2) ? (long long)g.B * g.K : q_begin + g.K;
+    const long long q_begin = (MODE == 2) ? (long long)blockIdx.z * per_split * g.K : (long long)n_fixed * g.K;
+    const long long q_end = (MODE == 2) ? (long long)min(g.B, ((int)blockIdx.z + 1) * per_split) * g.K : q_begin + g.K;
+    const bool add_to_acc = (MODE == 2) && gridDim.z == 1;
 
     // loader role: this thread fills column lm of sA and column lj of sB for rows lp, lp+4, lp+8, lp+12
     const int lcol = tid & 63, lp = tid >> 6;
@@ -99,7 +102,8 @@ conv_wgrad_fma_kernel(const T *__restrict__ X, const T *__restrict__ dY, const C
         if (tid == 0) partial[(long long)n_fixed * slots + blockIdx.y * gridDim.x + blockIdx.x] = sq;
     }
     if (MODE == 0 || MODE == 2) {
-        float *base = (MODE == 0) ? G_w + (long long)n_fixed * g.M * g.N : acc_w;
+        float *base = (MODE == 0) ? G_w + (long long)n_fixed * g.M * g.N
+                                  : (add_to_acc ? acc_w : sum_ws + (long long)blockIdx.z * g.M * g.N);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int m = m0 + ty * 4 + i;
@@ -108,7 +112,7 @@ conv_wgrad_fma_kernel(const T *__restrict__ X, const T *__restrict__ dY, const C
             if ((g.N & 3) == 0) {
                 if (jb < g.N) {
                     float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                    if (MODE == 2) {
+                    if (add_to_acc) {
                         const float4 o = *reinterpret_cast<const float4 *>(row + jb);
                         v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
                     }
@@ -117,7 +121,7 @@ conv_wgrad_fma_kernel(const T *__restrict__ X, const T *__restrict__ dY, const C
             } else {
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    if (jb + k < g.N) row[jb + k] = (MODE == 2) ? row[jb + k] + acc[i][k] : acc[i][k];
+                    if (jb + k < g.N) row[jb + k] = add_to_acc ? row[jb + k] + acc[i][k] : acc[i][k];
             }
         }
     }
@@ -335,23 +339,48 @@ __global__ void affine_accum_kernel(const float *__restrict__ dgamma, const floa
 }
 
 // ------------------------------------------------------------------ host launchers
+int fma_clip_splits(const ConvGeom &g) {
+    const int tiles = fma_tiles_m(g) * fma_tiles_n(g);
+    int want = (2 * 148) / tiles;
+    if (want < 1) want = 1;
+    if (want > g.B) want = g.B;
+    const int per = (g.B + want - 1) / want;
+    return (g.B + per - 1) / per;
+}
+
+// acc[i] += sum_s ws[s][i], splits in index order
+__global__ void fold_sums_kernel(const float *__restrict__ ws, int splits, long long P, float *__restrict__ acc) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= P) return;
+    float a = acc[i];
+    for (int s = 0; s < splits; ++s) a += ws[(long long)s * P + i];
+    acc[i] = a;
+}
+
 template <typename T>
 static dp_status conv_fma_t(int mode, const T *X, const T *dY, const ConvGeom &g, float *G_w, float *partial, int slots,
-                            const float *factor, float *acc_w, cudaStream_t st) {
-    const dim3 grid(fma_tiles_n(g), fma_tiles_m(g), mode == 2 ? 1 : g.B);
+                            const float *factor, float *acc_w, float *sum_ws, cudaStream_t st) {
+    const int splits = (mode == 2) ? fma_clip_splits(g) : 1;
+    const int per = (g.B + splits - 1) / splits;
+    const dim3 grid(fma_tiles_n(g), fma_tiles_m(g), mode == 2 ? splits : g.B);
     if (grid.y > 65535 || grid.z > 65535) return DP_ERR_UNSUPPORTED;
-    if (mode == 0) conv_wgrad_fma_kernel<T, 0><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w);
-    else if (mode == 1) conv_wgrad_fma_kernel<T, 1><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w);
-    else conv_wgrad_fma_kernel<T, 2><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w);
+    if (mode == 0) conv_wgrad_fma_kernel<T, 0><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w, per, sum_ws);
+    else if (mode == 1) conv_wgrad_fma_kernel<T, 1><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w, per, sum_ws);
+    else conv_wgrad_fma_kernel<T, 2><<<grid, 256, 0, st>>>(X, dY, g, G_w, partial, slots, factor, acc_w, per, sum_ws);
     DP_LAUNCH_CHECK("conv_wgrad_fma_kernel");
+    if (mode == 2 && splits > 1) {
+        const long long P = (long long)g.M * g.N;
+        fold_sums_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(sum_ws, splits, P, acc_w);
+        DP_LAUNCH_CHECK("fold_sums_kernel");
+    }
     return DP_OK;
 }
 
 dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, const ConvGeom &g, float *G_w,
-                          float *partial, int slots, const float *factor, float *acc_w, cudaStream_t st) {
+                          float *partial, int slots, const float *factor, float *acc_w, float *sum_ws, cudaStream_t st) {
     if (dtype == DP_F32)
-        return conv_fma_t(mode, static_cast<const float *>(X), static_cast<const float *>(dY), g, G_w, partial, slots, factor, acc_w, st);
-    return conv_fma_t(mode, static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), g, G_w, partial, slots, factor, acc_w, st);
+        return conv_fma_t(mode, static_cast<const float *>(X), static_cast<const float *>(dY), g, G_w, partial, slots, factor, acc_w, sum_ws, st);
+    return conv_fma_t(mode, static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), g, G_w, partial, slots, factor, acc_w, sum_ws, st);
 }
 
 dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,

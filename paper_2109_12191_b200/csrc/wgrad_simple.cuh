@@ -19,9 +19,13 @@ inline int fma_tiles_m(const ConvGeom &g) { return (g.M + kFmaTile - 1) / kFmaTi
 inline int fma_tiles_n(const ConvGeom &g) { return (g.N + kFmaTile - 1) / kFmaTile; }
 inline int bias_blocks(const ConvGeom &g) { return (g.Kout + kBiasCols - 1) / kBiasCols; }
 
-// mode: 0 store + norm partials, 1 norm partials only, 2 clip-accumulate (factor[n*2] scales example n)
+// mode: 0 store + norm partials, 1 norm partials only, 2 clip-accumulate (factor[n*2] scales example n).
+// Mode 2 cuts the batch into fma_clip_splits(g) example ranges; with more than one range the partial sums go
+// through sum_ws ([splits][M*N] floats) and are folded into acc_w in range order.
+int fma_clip_splits(const ConvGeom &g);
 dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, const ConvGeom &g, float *G_w,
-                          float *partial, int slots, const float *factor, float *acc_w, cudaStream_t stream);
+                          float *partial, int slots, const float *factor, float *acc_w, float *sum_ws,
+                          cudaStream_t stream);
 // db[n,k] = sum over pixels of dY; also sum_k db^2 per block into partial[n*slots + slot0 + block]
 dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
                       cudaStream_t stream);

@@ -49,13 +49,30 @@ struct TcParams {
     int a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT;
     int OWt, OHt, tiles_w, Kt, k_tiles, stages, stage_bytes, a_bytes;
     int lo_offset;              // split tf32: byte offset of the lo copy inside a stage
-    int mode;                   // 0 store + norm, 1 norm only
+    int mode;                   // 0 store + norm, 1 norm only, 2 clipped sum over a range of examples
     float *G_w;
     float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
     int slots;
     int *status;
-    int total_tiles;
+    int total_tiles;            // work items: (example, tile) pairs, or (example range, tile) pairs in mode 2
+    // mode 2: item = (split, tile); the CTA walks examples [split*per_split, ...) and keeps sum_n f_n D_n in registers
+    int splits, per_split;
+    const float *factor;        // [B][2], element 0 = weight factor
+    float *sum_out;             // splits == 1: the accumulator (added to); else partial sums [splits][Kout*Ng]
 };
+
+struct Item { int mt, nt, n_lo, n_hi, split; };
+__device__ __forceinline__ Item decode_item(const TcParams &p, int item) {
+    Item it;
+    const int tpe = p.m_tiles * p.n_tiles;
+    const int outer = item / tpe;          // the example, or in mode 2 the example range
+    const int rem = item - outer * tpe;
+    it.mt = rem / p.n_tiles;
+    it.nt = rem - it.mt * p.n_tiles;
+    if (p.mode == 2) { it.split = outer; it.n_lo = outer * p.per_split; it.n_hi = min(p.B, it.n_lo + p.per_split); }
+    else { it.split = 0; it.n_lo = outer; it.n_hi = outer + 1; }
+    return it;
+}
 
 // ----------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -145,7 +162,7 @@ __device__ __forceinline__ uint32_t instr_desc(int n_cols, uint32_t fmt) {
     return (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n_cols >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-template <bool TF32>
+template <bool TF32, bool CLIP>
 __global__ void __launch_bounds__(TF32 ? 320 : 192, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -175,7 +192,6 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const uint32_t tmem_base = tmem_base_slot;
     volatile int *abort_p = &abort_flag;
 
-    const int tiles_per_example = p.m_tiles * p.n_tiles;
     const int slab_bytes = p.Kt * kRowBytes;
     const int a_slabs_tile = 128 / p.slab_ch, b_slabs_tile = p.NT / p.slab_ch;
 
@@ -185,10 +201,9 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         // offset once per tile and then only adds the pixel-tile origin, so no division sits in the stage loop.
         int stage = 0; uint32_t phase = 0;
         bool live = true;
-        for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-            const int n = t / tiles_per_example;
-            const int rem = t - n * tiles_per_example;
-            const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+        for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
+            const Item it = decode_item(p, item);
+            const int mt = it.mt, nt = it.nt;
             const int a_slab0 = mt * a_slabs_tile, a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - a_slab0);
             const int b_slab0 = nt * b_slabs_tile, b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - b_slab0);
             const bool is_a = lane < a_slabs_tile;
@@ -211,20 +226,22 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const CUtensorMap *map = is_x ? &tmX : &tmY;
             const uint32_t dst_off = (is_a ? 0u : (uint32_t)p.a_bytes) + (uint32_t)(local * slab_bytes);
             const uint32_t tx_bytes = (uint32_t)((a_slabs + b_slabs) * slab_bytes);
-            int ow0 = 0, oh0 = 0, tw = 0;
-            for (int kt = 0; kt < p.k_tiles; ++kt) {
-                bool ok = true;
-                if (lane == 0) {
-                    ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p);
-                    if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+            for (int n = it.n_lo; n < it.n_hi && live; ++n) {
+                int ow0 = 0, oh0 = 0, tw = 0;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    bool ok = true;
+                    if (lane == 0) {
+                        ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p);
+                        if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { live = false; break; }
+                    if (active)
+                        tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
+                                    ow0 * mul + dw, oh0 * mul + dh, n);
+                    if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) { live = false; break; }
-                if (active)
-                    tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
-                                ow0 * mul + dw, oh0 * mul + dh, n);
-                if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -237,11 +254,11 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const uint64_t desc_hi = operand_desc_base<TF32>((uint32_t)slab_bytes);
             const int ksteps = p.Kt / p.krows;
             const uint32_t kadvance = (uint32_t)(p.krows * kRowBytes) >> 4;     // descriptor start-address units of 16 B
-            for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-                const int rem = t % tiles_per_example;
-                const int nt = rem % p.n_tiles;
-                const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
-                const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, TF32 ? 2u : 1u);
+            for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
+              const Item it = decode_item(p, item);
+              const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - it.nt * b_slabs_tile);
+              const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, TF32 ? 2u : 1u);
+              for (int n = it.n_lo; n < it.n_hi && live; ++n) {
                 if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p)) { live = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
@@ -277,6 +294,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 umma_commit(smem_u32(&tmem_full[buf]));            // accumulator complete
                 acc_phase ^= 1u << buf;
                 buf ^= 1;
+              }
             }
         }
     } else if (TF32 && warp >= 6) {
@@ -286,13 +304,13 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         const int tid = threadIdx.x - 192;
         int stage = 0; uint32_t phase = 0;
         bool live = true;
-        for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-            const int rem = t % tiles_per_example;
-            const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
-            const int a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - mt * a_slabs_tile);
-            const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
+        for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
+            const Item it = decode_item(p, item);
+            const int a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - it.mt * a_slabs_tile);
+            const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - it.nt * b_slabs_tile);
             const int a_chunks = a_slabs * (slab_bytes >> 4), chunks = a_chunks + b_slabs * (slab_bytes >> 4);
-            for (int kt = 0; kt < p.k_tiles; ++kt) {
+            const int stage_count = (it.n_hi - it.n_lo) * p.k_tiles;
+            for (int kt = 0; kt < stage_count; ++kt) {
                 const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p);
                 if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
                 uint8_t *base = tiles + (size_t)stage * p.stage_bytes;
@@ -320,48 +338,101 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         uint32_t full_phase = 0;     // bit b: parity to wait for on accumulator buffer b
         int buf = 0;
         bool live = true;
-        for (int t = blockIdx.x; t < p.total_tiles && live; t += gridDim.x) {
-            const int n = t / tiles_per_example;
-            const int rem = t - n * tiles_per_example;
-            const int mt = rem / p.n_tiles, nt = rem - mt * p.n_tiles;
+        for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
+            const Item it = decode_item(p, item);
+            const int mt = it.mt, nt = it.nt;
             const int a_rows = min(128, p.a_ext - mt * 128);
             const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
-            const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p);
-            if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }   // the whole warp leaves together
-            full_phase ^= 1u << buf;
-            tc_fence_after();
             const bool row_ok = row < a_rows;
             const int a_idx = mt * 128 + row;            // index along the A operand's extent
-            float sq = 0.f;
-            float *Gn = p.G_w + (long long)n * p.Kout * p.Ng;
-            for (int cc = 0; cc < n_cols; cc += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem_base + (uint32_t)(buf * 256 + cc) + ((uint32_t)(q * 32) << 16), v);
-                if (row_ok) {
+            float run[CLIP ? 128 : 1];                   // clip mode: this thread's row of sum_n f_n D_n (NT <= 128)
+            if (CLIP) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq = fmaf(f, f, sq); }
-                    if (p.mode == 0) {
-                        const int b_idx = nt * p.NT + cc;
-                        if (p.a_is_x) {          // row = column j of G, tile column = output channel k: lanes write consecutive j
-                            float *dst = Gn + (long long)b_idx * p.Ng + a_idx;
+                for (int i = 0; i < 128; ++i) run[CLIP ? i : 0] = 0.f;
+            }
+            for (int n = it.n_lo; n < it.n_hi; ++n) {
+                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p);
+                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }   // the whole warp leaves together
+                full_phase ^= 1u << buf;
+                tc_fence_after();
+                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256) + ((uint32_t)(q * 32) << 16);
+                if (CLIP) {
+                    const float f = p.factor[2 * n];
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) __stcs(dst + (long long)i * p.Ng, __uint_as_float(v[i]));
-                        } else {                 // row = output channel k, tile columns = 32 consecutive j
-                            float4 *dst = reinterpret_cast<float4 *>(Gn + (long long)a_idx * p.Ng + b_idx);
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        if (c4 * 32 < n_cols) {
+                            uint32_t v[32];
+                            tmem_ld32(t_addr + (uint32_t)(c4 * 32), v);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                __stcs(dst + i, make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                                            __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
+                            for (int i = 0; i < 32; ++i)
+                                run[CLIP ? c4 * 32 + i : 0] = fmaf(f, __uint_as_float(v[i]), run[CLIP ? c4 * 32 + i : 0]);
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+                } else {
+                    float sq = 0.f;
+                    float *Gn = p.G_w + (long long)n * p.Kout * p.Ng;
+                    for (int cc = 0; cc < n_cols; cc += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(t_addr + (uint32_t)cc, v);
+                        if (row_ok) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq = fmaf(f, f, sq); }
+                            if (p.mode == 0) {
+                                const int b_idx = nt * p.NT + cc;
+                                if (p.a_is_x) {      // row = column j of G, tile column = output channel k: lanes write consecutive j
+                                    float *dst = Gn + (long long)b_idx * p.Ng + a_idx;
+#pragma unroll
+                                    for (int i = 0; i < 32; ++i) __stcs(dst + (long long)i * p.Ng, __uint_as_float(v[i]));
+                                } else {             // row = output channel k, tile columns = 32 consecutive j
+                                    float4 *dst = reinterpret_cast<float4 *>(Gn + (long long)a_idx * p.Ng + b_idx);
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i)
+                                        __stcs(dst + i, make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                                    __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
+                                }
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+                    sq = warp_sum(sq);
+                    if (lane == 0) p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
+                }
+                buf ^= 1;
+            }
+            if (CLIP && live && row_ok) {
+                // one owner per output element: add straight into the accumulator, or leave a partial sum for the fold
+                const bool add = p.splits == 1;
+                float *base = p.sum_out + (add ? 0ll : (long long)it.split * p.Kout * p.Ng);
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    if (c4 * 32 < n_cols) {
+                        const int b_idx = nt * p.NT + c4 * 32;
+                        if (p.a_is_x) {
+                            float *dst = base + (long long)b_idx * p.Ng + a_idx;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                float *e = dst + (long long)i * p.Ng;
+                                const float r = run[CLIP ? c4 * 32 + i : 0];
+                                *e = add ? *e + r : r;
+                            }
+                        } else {
+                            float4 *dst = reinterpret_cast<float4 *>(base + (long long)a_idx * p.Ng + b_idx);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                float4 r = make_float4(run[CLIP ? c4 * 32 + 4 * i : 0], run[CLIP ? c4 * 32 + 4 * i + 1 : 0],
+                                                       run[CLIP ? c4 * 32 + 4 * i + 2 : 0], run[CLIP ? c4 * 32 + 4 * i + 3 : 0]);
+                                if (add) { const float4 o = dst[i]; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
+                                dst[i] = r;
+                            }
                         }
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
-            sq = warp_sum(sq);
-            if (lane == 0) p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
-            buf ^= 1;
         }
     }
 
@@ -374,6 +445,26 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         __syncthreads();
     }
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
+// acc[i] += sum over splits of part[s][i], splits in index order (P a multiple of 4, both 16-byte aligned)
+__global__ void __launch_bounds__(256)
+fold_partial_sums_kernel(const float *__restrict__ part, int splits, long long P, float *__restrict__ acc) {
+    const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= P) return;
+    float4 a = *reinterpret_cast<const float4 *>(acc + i);
+    for (int s = 0; s < splits; ++s) {
+        const float4 v = __ldcs(reinterpret_cast<const float4 *>(part + (long long)s * P + i));
+        a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    *reinterpret_cast<float4 *>(acc + i) = a;
+}
+
+dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream) {
+    if (P % 4) return DP_ERR_UNSUPPORTED;
+    fold_partial_sums_kernel<<<(unsigned)((P / 4 + 255) / 256), 256, 0, stream>>>(part, splits, P, acc);
+    DP_LAUNCH_CHECK("fold_partial_sums_kernel");
+    return DP_OK;
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -412,22 +503,24 @@ static int step_cycles(int n_cols) {
     return pipe > smem ? pipe : smem;
 }
 
-static TcPlan search_plan(int dtype, const ConvGeom &g);
+static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt);
 
 // The tiling search is pure; its results are memoised per layer geometry (host side only).
-static TcPlan make_plan(int dtype, const ConvGeom &g) {
+static TcPlan make_plan(int dtype, const ConvGeom &g, int max_nt = 256) {
     static std::mutex mu;
-    static std::map<std::array<int, 10>, TcPlan> memo;
-    const std::array<int, 10> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B};
+    static std::map<std::array<int, 11>, TcPlan> memo;
+    const std::array<int, 11> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, max_nt};
     std::lock_guard<std::mutex> lock(mu);
     auto it = memo.find(key);
     if (it != memo.end()) return it->second;
-    const TcPlan pl = search_plan(dtype, g);
+    const TcPlan pl = search_plan(dtype, g, max_nt);
     memo.emplace(key, pl);
     return pl;
 }
 
-static TcPlan search_plan(int dtype, const ConvGeom &g) {
+// max_nt = 128 plans the clipped-sum mode: its running sum lives in registers (128 columns per thread) and the
+// work items are (example range, tile) pairs, so the wave count no longer depends on the batch size
+static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
     TcPlan best; best.ok = false;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
@@ -440,14 +533,16 @@ static TcPlan search_plan(int dtype, const ConvGeom &g) {
     double best_cost = 1e300;
     for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
         const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
-        for (int NT = slab_ch; NT <= 256; NT += slab_ch) {
+        for (int NT = slab_ch; NT <= max_nt; NT += slab_ch) {
             if (NT != 32 && NT % 64) continue;
             if (NT > b_ext) break;
             const int m_tiles = (a_ext + 127) / 128, n_tiles = (b_ext + NT - 1) / NT;
             const int slabs = a_slabs_tile + NT / slab_ch;
             const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
             if (total_tiles > 0x7fffffffLL) continue;
-            const long long waves = (total_tiles + sms - 1) / sms;
+            // per-CTA share of (example, tile) units: whole waves of tiles, or in clipped-sum mode an even share of the examples
+            const double waves = (max_nt == 256) ? (double)((total_tiles + sms - 1) / sms)
+                                                 : std::max(1.0, (double)total_tiles / sms);
             for (int OHt = 1; OHt <= g.OH; ++OHt) {
                 if (OHt * g.stride > 256 || OHt * g.stride > g.H) break;
                 for (int OWt = 1; OWt <= g.OW; ++OWt) {
@@ -463,7 +558,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g) {
                     const double stage_cost = std::max((double)(Kt / krows) * step_cycles(NT) * mma_per_step, 450.0);
                     double tile_cost = stage_cost * tw * th + 600.0;
                     if (stages < 3) tile_cost *= 1.3;
-                    const double cost = tile_cost * (double)waves;
+                    const double cost = tile_cost * waves;
                     if (cost < best_cost) {
                         best_cost = cost;
                         best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
@@ -481,8 +576,18 @@ static TcPlan search_plan(int dtype, const ConvGeom &g) {
 }
 
 bool tc_eligible(int dtype, const ConvGeom &g, int epilogue) {
-    if (epilogue == DP_EPI_CLIP_ACCUM) return false;
-    return make_plan(dtype, g).ok && encode_fn() != nullptr;
+    if (!encode_fn() || !make_plan(dtype, g).ok) return false;
+    return epilogue != DP_EPI_CLIP_ACCUM || make_plan(dtype, g, 128).ok;
+}
+
+// clipped-sum mode: how many example ranges each tile is cut into so that every SM has an item
+static void clip_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &per_split) {
+    const int tiles = pl.m_tiles * pl.n_tiles;
+    int want = sm_count() / tiles;
+    if (want < 1) want = 1;
+    if (want > g.B) want = g.B;
+    per_split = (g.B + want - 1) / want;
+    splits = (g.B + per_split - 1) / per_split;
 }
 
 int tc_norm_slots(int dtype, const ConvGeom &g, int) {
@@ -490,7 +595,14 @@ int tc_norm_slots(int dtype, const ConvGeom &g, int) {
     return pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
 }
 
-size_t tc_workspace_bytes(int, const ConvGeom &, int) { return 0; }
+size_t tc_workspace_bytes(int dtype, const ConvGeom &g, int epilogue) {
+    if (epilogue != DP_EPI_CLIP_ACCUM) return 0;
+    const TcPlan pl = make_plan(dtype, g, 128);
+    if (!pl.ok) return 0;
+    int splits, per;
+    clip_split(g, pl, splits, per);
+    return splits > 1 ? sizeof(float) * (size_t)splits * g.M * g.N : 0;
+}
 
 int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n) {
     const TcPlan pl = make_plan(dtype, g);
@@ -517,9 +629,11 @@ static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, in
 }
 
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
-                         float *partial, int slots, const float *, float *, void *, int *status, cudaStream_t stream) {
-    const TcPlan pl = make_plan(dtype, g);
-    if (!pl.ok || !encode_fn() || epilogue == DP_EPI_CLIP_ACCUM) return DP_ERR_UNSUPPORTED;
+                         float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace, int *status,
+                         cudaStream_t stream) {
+    const bool clip = epilogue == DP_EPI_CLIP_ACCUM;
+    const TcPlan pl = make_plan(dtype, g, clip ? 128 : 256);
+    if (!pl.ok || !encode_fn()) return DP_ERR_UNSUPPORTED;
     CUtensorMap tmX, tmY;
     if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
     if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
@@ -530,21 +644,36 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
     p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
     p.lo_offset = pl.stage_bytes / 2;
-    p.mode = (epilogue == DP_EPI_STORE_NORM) ? 0 : 1;
+    p.mode = clip ? 2 : (epilogue == DP_EPI_STORE_NORM ? 0 : 1);
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
-    p.total_tiles = g.B * pl.m_tiles * pl.n_tiles;
+    p.splits = 1; p.per_split = g.B; p.factor = factor; p.sum_out = acc_w;
+    if (clip) {
+        clip_split(g, pl, p.splits, p.per_split);
+        if (p.splits > 1) p.sum_out = static_cast<float *>(tc_workspace);
+        p.total_tiles = p.splits * pl.m_tiles * pl.n_tiles;
+    } else {
+        p.total_tiles = g.B * pl.m_tiles * pl.n_tiles;
+    }
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        const int bytes = kSmemBudget + 2048;
+        attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (attr_err == cudaSuccess) attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (attr_err == cudaSuccess) attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (attr_err == cudaSuccess) attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
     const unsigned grid = (unsigned)std::min(p.total_tiles, sm_count());
-    if (dtype == DP_BF16) conv_wgrad_tc_kernel<false><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
-    else conv_wgrad_tc_kernel<true><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
+    if (dtype == DP_BF16) {
+        if (clip) conv_wgrad_tc_kernel<false, true><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+        else conv_wgrad_tc_kernel<false, false><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+    } else {
+        if (clip) conv_wgrad_tc_kernel<true, true><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
+        else conv_wgrad_tc_kernel<true, false><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
+    }
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
+    if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g.M * g.N, acc_w, stream);
     return DP_OK;
 }
 

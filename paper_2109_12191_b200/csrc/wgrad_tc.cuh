@@ -10,6 +10,8 @@ bool tc_eligible(int dtype, const ConvGeom &g, int epilogue);
 int tc_norm_slots(int dtype, const ConvGeom &g, int epilogue);
 size_t tc_workspace_bytes(int dtype, const ConvGeom &g, int epilogue);
 // tiling chosen for the layer: {a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT, OWt, OHt, Kt, k_tiles, stages, stage_bytes}
+// acc[i] += sum_s part[s][i] in index order of s (P a multiple of 4)
+dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream);
 int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n);
 // epilogue as dp_epilogue; factor[n*2] scales example n (CLIP_ACCUM); status: device word set to nonzero on a timed-out wait
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,

@@ -163,8 +163,31 @@ TC_CONVS = [
 def test_conv_tensor_core(case):
     dtype, Cin, Kout, R, stride, pad, H, bias = case
     layer = synth.conv(Cin, Kout, R, stride, pad, H, bias, name=str(case))
-    out = check_layer(layer, 5, dtype, TENSOR_CORE, (940, sum(case[1:7])), spread=True, clip_impl=AUTO)
+    out = check_layer(layer, 5, dtype, TENSOR_CORE, (940, sum(case[1:7])), spread=True)
     assert out["uses_tc"]
+
+
+@pytest.mark.parametrize("Bn", [1, 37])
+def test_clipped_sum_example_ranges(Bn):
+    """Fused clip + accumulate cuts the batch into example ranges (ragged for 37) whose partial sums are folded
+    in order; both implementations, accumulating on top of a non-zero accumulator."""
+    b = B()
+    for impl, dtype, layer in ((TENSOR_CORE, "bf16", synth.conv(64, 64, 3, 1, 1, 8, name="tc ranges")),
+                               (TENSOR_CORE, "f32", synth.conv(32, 64, 3, 2, 1, 16, name="tf32 ranges")),
+                               (CUDA_CORE, "f32", synth.conv(3, 16, 3, 1, 1, 12, True, name="fma ranges"))):
+        inp = scaled_inputs(layer, Bn, dtype, 943, Bn, spread=Bn > 1)
+        dW, db = oracle_layer(layer, inp)
+        sq = oracle.sqnorm(dW) + (oracle.sqnorm(db) if db is not None else 0.0)
+        C_l = float(np.sqrt(np.median(sq)))
+        f = oracle.clip_factor(sq, C_l)
+        start_w = synth.normal_f32((layer.n_weight,), 944)
+        acc_w = torch.from_numpy(start_w.copy()).cuda()
+        acc_b = torch.zeros(layer.n_bias, device="cuda") if layer.n_bias else None
+        out = gpu_layer(layer, inp, dtype, CLIP, impl, 0, C_l=C_l, acc_w=acc_w, acc_b=acc_b)
+        np.testing.assert_allclose(out["clip"][:, 0], f, rtol=TOL_NORM)
+        assert rel_l2(out["acc_w"], start_w + np.einsum("n,np->p", f, dW)) <= TOL_FMA
+        if db is not None:
+            assert rel_l2(out["acc_b"], np.einsum("n,np->p", f, db)) <= TOL_FMA
 
 
 def test_tensor_core_matches_cuda_core_bitwise_norm_inputs():
