@@ -258,7 +258,111 @@ class FlatGrad:
         return n / dt, f"{n} examples of one 64-example chunk at full P (norms, clip, sum) plus one noise+average pass"
 
 
-WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad}
+class PerLayer:
+    """configs[4]: ResNet-50 (GroupNorm) per-layer clipping over all 161 tensors, bf16 inputs, B=32 per chunk,
+    32 chunks, C_l = C/sqrt(161), clip + accumulate fused into the weight-gradient call."""
+    name = "per_layer"
+    dtype_name = "bf16"
+
+    def __init__(self, torch, rank, dist=None, world=1):
+        from paper_2109_12191_b200 import synth, binding
+        from paper_2109_12191_b200.step import PerLayerClipStep
+        self.torch, self.synth, self.dist, self.world, self.b = torch, synth, dist, world, binding
+        self.cfg = synth.resnet50_per_layer()
+        self.layers, self.B, self.G = self.cfg["layers"], self.cfg["B"], self.cfg["G"]
+        self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"])
+        self.examples_per_step = self.B * self.G
+        g = torch.Generator(device="cuda"); g.manual_seed(4000 + rank)
+        self.inputs = []
+        for l in self.layers:                             # one resident chunk of inputs (2.8 GB), reused by every chunk
+            X = torch.empty(l.x_shape(self.B), device="cuda", dtype=torch.bfloat16).normal_(generator=g)
+            dY = torch.empty(l.dy_shape(self.B), device="cuda", dtype=torch.bfloat16).normal_(generator=g)
+            self.inputs.append((X, dY))
+        self.in_bytes = sum((x.numel() + y.numel()) * 2 for x, y in self.inputs)
+        self.call_names = ["wgrad:conv (tensor core)", "wgrad:conv (cuda core)", "wgrad:norm_affine", "wgrad:dense", "noise_average"]
+        self.kind_of = []
+        for l, d in zip(self.layers, self.step_obj.descs):
+            if l.kind == "conv":
+                self.kind_of.append(0 if binding.dp_wgrad_uses_tensor_cores(d, binding.DP_EPI_CLIP_ACCUM) else 1)
+            else:
+                self.kind_of.append(2 if l.kind == "norm" else 3)
+        self.flops_tc = sum(l.flops() for l, k in zip(self.layers, self.kind_of) if k == 0) * self.B
+        self.bytes_kind = [sum((x.numel() + y.numel()) * 2 for (x, y), k in zip(self.inputs, self.kind_of) if k == kk) for kk in range(4)]
+
+    def describe(self):
+        return {"workload": "per_layer: ResNet-50 (GroupNorm 32) at 224x224, all 161 parameter tensors (53 conv, 53x2 norm, fc "
+                            "weight + bias), bf16 X/dY ~N(0,1), B=32 per chunk x 32 chunks = |B| 1024, C=1.0 (C_l = C/sqrt(161)), "
+                            "sigma=1.0; clip + accumulate fused into dp_per_example_wgrad",
+                "examples_per_step": self.examples_per_step, "params": self.step_obj.P,
+                "l2": f"one chunk of inputs is {self.in_bytes / 1e9:.2f} GB, far larger than L2"}
+
+    def run(self, i, rec=None):
+        st = self.step_obj
+        st.begin()
+        for c in range(self.G):
+            for li, (X, dY) in enumerate(self.inputs):
+                k = self.kind_of[li]
+                if rec: rec.start(k)
+                st.wgrad(li, X, dY)
+                if rec: rec.stop(k)
+            st.chunks_done += 1
+        if rec: rec.start(4)
+        st.finish(seed=0, step=i)
+        if rec: rec.stop(4)
+
+    def algorithmic_bytes(self, call):
+        return self.bytes_kind[call] if call < 4 else 2 * self.step_obj.P * 4
+
+    def roofline(self, dom, avg_ms_total_per_chunk, peaks):
+        """Tensor-core convs are reported against the bf16 tensor peak (flops counted once although the two-pass
+        scheme executes them twice); everything else against HBM."""
+        if dom != 0:
+            return None
+        tf = self.flops_tc / (avg_ms_total_per_chunk / 1e3) / 1e12
+        return {"bound": "tensor", "achieved": round(tf, 1), "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                "frac": round(tf / peaks["bf16_sustained"], 4)}
+
+    def e2e_prepare(self):
+        t = self.torch
+        self.host_inputs = [(x.cpu().pin_memory(), y.cpu().pin_memory()) for x, y in self.inputs]
+        self.host_sum = t.empty(1, dtype=t.float32).pin_memory()
+        return self.in_bytes * self.G, 4 * self.step_obj.P
+
+    def e2e_run(self, i):
+        st = self.step_obj
+        st.begin()
+        for c in range(self.G):
+            for li, ((X, dY), (hx, hy)) in enumerate(zip(self.inputs, self.host_inputs)):
+                X.copy_(hx, non_blocking=True); dY.copy_(hy, non_blocking=True)
+                st.wgrad(li, X, dY)
+            st.chunks_done += 1
+        acc_w, acc_b = st.finish(seed=0, step=i)
+        for a in acc_w:
+            a.cpu()
+
+    def cpu_sample(self, budget_s):
+        import oracle
+        import math
+        n = 2
+        picks = [l for l in self.layers if l.kind == "conv" and l.H <= 14][:3] + [l for l in self.layers if l.kind == "norm" and l.H <= 28][:3]
+        t0 = time.perf_counter(); flops = 0
+        for li, l in enumerate(picks):
+            inp = self.synth.layer_inputs(l, n, "bf16", 4, li, 0)
+            if l.kind == "conv":
+                dW, _ = oracle.conv_wgrad(inp["X"], inp["dY"], l.R, l.S, l.stride, l.pad, bias=False)
+                groups = [dW.reshape(n, -1)]
+            else:
+                dg, dbt = oracle.norm_affine_wgrad(inp["X"], inp["dY"])
+                groups = [dg, dbt]
+            oracle.clipped_sum(groups, 1.0 / math.sqrt(161), "per_layer")
+            flops += l.flops() * n
+        dt = time.perf_counter() - t0
+        total = sum(l.flops() for l in self.layers)
+        return (flops / dt) / total, (f"{n} examples through {len(picks)} layers (3 convs, 3 norm layers), scaled to one example's "
+                                      f"{total / 1e9:.2f} Gflop by the flop ratio")
+
+
+WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad, "per_layer": PerLayer}
 
 
 class CallTimer:
@@ -367,6 +471,10 @@ def run_ours(args):
                 "peak_source": peaks["source"], "unit": "GB/s", "frac": round(achieved / peaks["hbm"], 4),
                 "avg_ms_per_launch": round(avg_ms, 5), "traffic": None,
                 "shares": {n: round(t / sum(totals), 4) for n, t in zip(wl.call_names, totals)}}
+    if hasattr(wl, "roofline"):
+        own = wl.roofline(dom, totals[dom] / (steps * wl.G), peaks)
+        if own:
+            roofline.update(own)
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -376,7 +484,7 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": round(ms / steps, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic", "config": dict(wl.describe(), parallelism=("single GPU" if world == 1 else f"batch sharded over {world} GPUs, one all-reduce of the accumulator per step")),
+            "dtype": getattr(wl, "dtype_name", "f32"), "data": "synthetic", "config": dict(wl.describe(), parallelism=("single GPU" if world == 1 else f"batch sharded over {world} GPUs, one all-reduce of the accumulator per step")),
             "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
@@ -495,7 +603,7 @@ def main():
     args = ap.parse_args()
     if args.workload in ("sweep", "sweep_all"):
         return run_sweep(args)
-    defaults = {"small_cnn": (400, 10), "flat": (8, 3)}
+    defaults = {"small_cnn": (400, 10), "flat": (8, 3), "per_layer": (2, 3)}
     if args.steps is None:
         args.steps = defaults[args.workload][0]
     if args.warmup is None:

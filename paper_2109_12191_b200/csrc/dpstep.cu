@@ -81,11 +81,12 @@ static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
         pl.dg_off = off;
         off = round_up(off + sizeof(float) * B * 2 * d->C_in, 256);
     }
-    pl.tc_off = off;       // partial sums of the clipped-sum pass (either implementation)
-    if (epi == DP_EPI_CLIP_ACCUM && d->kind != DP_LAYER_NORM_AFFINE) {
+    off = round_up(off, 1024);
+    pl.tc_off = off;       // tensor-core scratch (unfolded input, partial sums) or the CUDA-core path's partial sums
+    if (d->kind != DP_LAYER_NORM_AFFINE) {
         size_t bytes = 0;
         if (pl.use_tc) bytes = tc_workspace_bytes(d->dtype, g, epi);
-        else { const int sp = fma_clip_splits(g); bytes = sp > 1 ? sizeof(float) * (size_t)sp * g.M * g.N : 0; }
+        else if (epi == DP_EPI_CLIP_ACCUM) { const int sp = fma_clip_splits(g); bytes = sp > 1 ? sizeof(float) * (size_t)sp * g.M * g.N : 0; }
         off = round_up(off + bytes, 256);
     }
     pl.total = off;
@@ -162,7 +163,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         if (rc != DP_OK) return rc;
         rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st);
         if (rc != DP_OK) return rc;
-        if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
+        if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true);
         else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db, d->B, d->K_out, factor, acc_b, st);

@@ -43,7 +43,8 @@ struct TcPlan {
 };
 
 struct TcParams {
-    int B, Kout, Ng, Cin, S, stride, pad;
+    int B, Kout, Ng, Cin, S, stride, pad;   // Ng: row length of G in memory = number of real gradient columns
+    int n_pad_cols;             // 1 when the column extent carries zero padding beyond Ng (im2col'd small-channel layers)
     int slab_ch;                // channels per 128-byte row: 64 (bf16) or 32 (fp32 as tf32)
     int krows;                  // reduction rows per MMA: 16 (bf16) or 8 (tf32)
     int a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT;
@@ -343,8 +344,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const int mt = it.mt, nt = it.nt;
             const int a_rows = min(128, p.a_ext - mt * 128);
             const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
-            const bool row_ok = row < a_rows;
             const int a_idx = mt * 128 + row;            // index along the A operand's extent
+            const bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
             float run[CLIP ? 128 : 1];                   // clip mode: this thread's row of sum_n f_n D_n (NT <= 128)
             if (CLIP) {
 #pragma unroll
@@ -386,12 +387,17 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                     float *dst = Gn + (long long)b_idx * p.Ng + a_idx;
 #pragma unroll
                                     for (int i = 0; i < 32; ++i) __stcs(dst + (long long)i * p.Ng, __uint_as_float(v[i]));
-                                } else {             // row = output channel k, tile columns = 32 consecutive j
+                                } else if (!p.n_pad_cols) {   // row = output channel k, tile columns = 32 consecutive j
                                     float4 *dst = reinterpret_cast<float4 *>(Gn + (long long)a_idx * p.Ng + b_idx);
 #pragma unroll
                                     for (int i = 0; i < 8; ++i)
                                         __stcs(dst + i, make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
                                                                     __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
+                                } else {             // padded columns: rows are not 16-byte aligned, and j stops at Ng
+                                    float *dst = Gn + (long long)a_idx * p.Ng + b_idx;
+#pragma unroll
+                                    for (int i = 0; i < 32; ++i)
+                                        if (b_idx + i < p.Ng) dst[i] = __uint_as_float(v[i]);
                                 }
                             }
                         }
@@ -420,7 +426,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                 const float r = run[CLIP ? c4 * 32 + i : 0];
                                 *e = add ? *e + r : r;
                             }
-                        } else {
+                        } else if (!p.n_pad_cols) {
                             float4 *dst = reinterpret_cast<float4 *>(base + (long long)a_idx * p.Ng + b_idx);
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
@@ -429,6 +435,11 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                 if (add) { const float4 o = dst[i]; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
                                 dst[i] = r;
                             }
+                        } else {
+                            float *dst = base + (long long)a_idx * p.Ng + b_idx;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (b_idx + i < p.Ng) dst[i] = add ? dst[i] + run[CLIP ? c4 * 32 + i : 0] : run[CLIP ? c4 * 32 + i : 0];
                         }
                     }
                 }
@@ -460,11 +471,52 @@ fold_partial_sums_kernel(const float *__restrict__ part, int splits, long long P
     *reinterpret_cast<float4 *>(acc + i) = a;
 }
 
+__global__ void fold_partial_sums_scalar_kernel(const float *__restrict__ part, int splits, long long P, float *__restrict__ acc) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= P) return;
+    float a = acc[i];
+    for (int s = 0; s < splits; ++s) a += part[(long long)s * P + i];
+    acc[i] = a;
+}
+
 dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream) {
-    if (P % 4) return DP_ERR_UNSUPPORTED;
-    fold_partial_sums_kernel<<<(unsigned)((P / 4 + 255) / 256), 256, 0, stream>>>(part, splits, P, acc);
+    if (P % 4 == 0 && aligned(part, 16) && aligned(acc, 16))
+        fold_partial_sums_kernel<<<(unsigned)((P / 4 + 255) / 256), 256, 0, stream>>>(part, splits, P, acc);
+    else
+        fold_partial_sums_scalar_kernel<<<(unsigned)((P + 255) / 256), 256, 0, stream>>>(part, splits, P, acc);
     DP_LAUNCH_CHECK("fold_partial_sums_kernel");
     return DP_OK;
+}
+
+// Layers whose input has too few channels for a TMA slab (C_in = 3 stems) are first unfolded:
+// Xcol[n, oh, ow, j] = Xpad[n, oh*st + r - pad, ow*st + s - pad, c], j = (r*S + s)*C_in + c, zero for j >= R*S*C_in,
+// with rows padded to a whole number of slabs.  The layer then is a 1x1 convolution over Xcol for the kernel above.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+unfold_small_channels_kernel(const T *__restrict__ X, T *__restrict__ Xcol, const ConvGeom g, int n_pad, long long total) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;       // one 16-byte group of columns each
+    if (idx >= total) return;
+    const int groups = n_pad / VEC;
+    const long long pixel = idx / groups;                                        // (n*OH + oh)*OW + ow
+    const int j0 = (int)(idx - pixel * groups) * VEC;
+    const int ow = (int)(pixel % g.OW);
+    const long long t = pixel / g.OW;
+    const int oh = (int)(t % g.OH);
+    const long long n = t / g.OH;
+    T v[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        const int j = j0 + e;
+        T x = T(0.f);
+        if (j < g.N) {
+            const int c = j % g.Cin, rs = j / g.Cin;
+            const int r = rs / g.S, s = rs - r * g.S;
+            const int ih = oh * g.stride + r - g.pad, iw = ow * g.stride + s - g.pad;
+            if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) x = X[((n * g.H + ih) * g.W + iw) * g.Cin + c];
+        }
+        v[e] = x;
+    }
+    *reinterpret_cast<uint4 *>(Xcol + pixel * n_pad + j0) = *reinterpret_cast<const uint4 *>(v);
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -495,6 +547,30 @@ static int sm_count() {
             return 148;
     }
     return sms;
+}
+
+// What the tensor-core kernel is actually given: the layer itself, or its unfolded 1x1 form.
+struct TcProblem {
+    bool ok, unfold;
+    ConvGeom eff;       // geometry the kernel tiles
+    int n_pad;          // unfolded row length (columns incl. zero padding)
+};
+
+static TcProblem tc_problem(int dtype, const ConvGeom &g) {
+    TcProblem pr; pr.ok = false; pr.unfold = false; pr.eff = g; pr.n_pad = g.N;
+    const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
+    if (g.Kout % slab_ch) return pr;
+    if (g.Cin % slab_ch == 0) { pr.ok = true; return pr; }
+    // small-channel layers only: the unfolded copy costs N/C_in times the input, which is only worth it for thin inputs
+    if (g.Cin > 8 || g.N > 512) return pr;
+    pr.unfold = true;
+    pr.n_pad = (g.N + slab_ch - 1) / slab_ch * slab_ch;
+    ConvGeom e = g;
+    e.H = g.OH; e.W = g.OW; e.Cin = pr.n_pad; e.R = 1; e.S = 1; e.stride = 1; e.pad = 0;
+    e.N = pr.n_pad;
+    pr.eff = e;
+    pr.ok = true;
+    return pr;
 }
 
 // cycles of one MMA step (one instruction): tensor pipe (N/2) against shared-memory operand reads (4 KB of A + N*32 B of B at 128 B/clk)
@@ -575,9 +651,10 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
     return best;
 }
 
-bool tc_eligible(int dtype, const ConvGeom &g, int epilogue) {
-    if (!encode_fn() || !make_plan(dtype, g).ok) return false;
-    return epilogue != DP_EPI_CLIP_ACCUM || make_plan(dtype, g, 128).ok;
+bool tc_eligible(int dtype, const ConvGeom &g0, int epilogue) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    if (!pr.ok || !encode_fn() || !make_plan(dtype, pr.eff).ok) return false;
+    return epilogue != DP_EPI_CLIP_ACCUM || make_plan(dtype, pr.eff, 128).ok;
 }
 
 // clipped-sum mode: how many example ranges each tile is cut into so that every SM has an item
@@ -590,22 +667,37 @@ static void clip_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &pe
     splits = (g.B + per_split - 1) / per_split;
 }
 
-int tc_norm_slots(int dtype, const ConvGeom &g, int) {
-    const TcPlan pl = make_plan(dtype, g);
+int tc_norm_slots(int dtype, const ConvGeom &g0, int) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    if (!pr.ok) return 0;
+    const TcPlan pl = make_plan(dtype, pr.eff);
     return pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
 }
 
-size_t tc_workspace_bytes(int dtype, const ConvGeom &g, int epilogue) {
-    if (epilogue != DP_EPI_CLIP_ACCUM) return 0;
-    const TcPlan pl = make_plan(dtype, g, 128);
-    if (!pl.ok) return 0;
-    int splits, per;
-    clip_split(g, pl, splits, per);
-    return splits > 1 ? sizeof(float) * (size_t)splits * g.M * g.N : 0;
+static size_t unfold_bytes(int dtype, const ConvGeom &g0, const TcProblem &pr) {
+    if (!pr.unfold) return 0;
+    return round_up((size_t)g0.B * g0.OH * g0.OW * pr.n_pad * (dtype == DP_BF16 ? 2 : 4), 1024);
 }
 
-int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n) {
-    const TcPlan pl = make_plan(dtype, g);
+// layout: [unfolded input, if any][partial sums of the clipped-sum mode, if any]
+size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    if (!pr.ok) return 0;
+    size_t bytes = unfold_bytes(dtype, g0, pr);
+    if (epilogue == DP_EPI_CLIP_ACCUM) {
+        const TcPlan pl = make_plan(dtype, pr.eff, 128);
+        if (!pl.ok) return 0;
+        int splits, per;
+        clip_split(pr.eff, pl, splits, per);
+        if (splits > 1) bytes += sizeof(float) * (size_t)splits * g0.M * g0.N;
+    }
+    return bytes;
+}
+
+int tc_describe_plan(int dtype, const ConvGeom &g0, int *out, int n) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    if (!pr.ok) return 0;
+    const TcPlan pl = make_plan(dtype, pr.eff);
     if (!pl.ok) return 0;
     const int v[12] = {pl.a_is_x, pl.a_ext, pl.b_ext, pl.m_tiles, pl.n_tiles, pl.NT, pl.OWt, pl.OHt, pl.Kt, pl.k_tiles,
                        pl.stages, pl.stage_bytes};
@@ -628,17 +720,41 @@ static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, in
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
+dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g_in, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace, int *status,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, bool skip_unfold) {
     const bool clip = epilogue == DP_EPI_CLIP_ACCUM;
+    const ConvGeom &g0 = g_in;
+    const TcProblem pr = tc_problem(dtype, g0);
+    if (!pr.ok || !encode_fn()) return DP_ERR_UNSUPPORTED;
+    const ConvGeom &g = pr.eff;
     const TcPlan pl = make_plan(dtype, g, clip ? 128 : 256);
-    if (!pl.ok || !encode_fn()) return DP_ERR_UNSUPPORTED;
+    if (!pl.ok) return DP_ERR_UNSUPPORTED;
+    char *ws_bytes = static_cast<char *>(tc_workspace);
+    if (pr.unfold) {
+        // in a fused clip call this function runs twice (norm pass, then clipped-sum pass): the unfolded input is
+        // rebuilt only by the first of them
+        if (!(clip && skip_unfold)) {
+            const int vec = (dtype == DP_BF16) ? 8 : 4;
+            const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / vec);
+            const unsigned blocks = (unsigned)((total + 255) / 256);
+            if (dtype == DP_BF16)
+                unfold_small_channels_kernel<__nv_bfloat16, 8><<<blocks, 256, 0, stream>>>(
+                    static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad, total);
+            else
+                unfold_small_channels_kernel<float, 4><<<blocks, 256, 0, stream>>>(
+                    static_cast<const float *>(X), reinterpret_cast<float *>(ws_bytes), g0, pr.n_pad, total);
+            DP_LAUNCH_CHECK("unfold_small_channels_kernel");
+        }
+        X = ws_bytes;
+    }
+    float *part_ws = reinterpret_cast<float *>(ws_bytes + unfold_bytes(dtype, g0, pr));
     CUtensorMap tmX, tmY;
     if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
     if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
     TcParams p;
-    p.B = g.B; p.Kout = g.Kout; p.Ng = g.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.B = g.B; p.Kout = g.Kout; p.Ng = g0.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.n_pad_cols = (g.N != g0.N) ? 1 : 0;
     p.slab_ch = (dtype == DP_BF16) ? 64 : 32; p.krows = (dtype == DP_BF16) ? 16 : 8;
     p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
@@ -649,7 +765,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.splits = 1; p.per_split = g.B; p.factor = factor; p.sum_out = acc_w;
     if (clip) {
         clip_split(g, pl, p.splits, p.per_split);
-        if (p.splits > 1) p.sum_out = static_cast<float *>(tc_workspace);
+        if (p.splits > 1) p.sum_out = part_ws;
         p.total_tiles = p.splits * pl.m_tiles * pl.n_tiles;
     } else {
         p.total_tiles = g.B * pl.m_tiles * pl.n_tiles;
@@ -673,7 +789,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
         else conv_wgrad_tc_kernel<true, false><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
     }
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
-    if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g.M * g.N, acc_w, stream);
+    if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g0.M * g0.N, acc_w, stream);
     return DP_OK;
 }
 

@@ -156,6 +156,10 @@ TC_CONVS = [
     ("f32", 64, 128, 3, 2, 1, 16, True),       # third conv of the small CNN
     ("f32", 32, 32, 1, 1, 0, 8, False),
     ("f32", 96, 160, 3, 1, 1, 9, False),       # extents that are multiples of 32 but not of 64 or 128
+    ("bf16", 3, 64, 7, 2, 3, 30, False),       # stem: 3 input channels are unfolded to 147 (+45 zero) columns first
+    ("f32", 3, 32, 3, 1, 1, 32, True),         # first conv of the small CNN: 27 (+5 zero) columns
+    ("bf16", 4, 128, 3, 1, 1, 9, True),        # 36 columns, rows of the gradient not 16-byte aligned
+    ("f32", 1, 64, 5, 2, 2, 13, False),        # single input channel
 ]
 
 
