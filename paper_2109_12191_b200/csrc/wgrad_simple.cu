@@ -153,6 +153,43 @@ bias_kernel(const T *__restrict__ dY, int K, int Kout, float *__restrict__ db, f
     if (threadIdx.x == 0) partial[(long long)n * slots + slot0 + blockIdx.x] = sq;
 }
 
+// Vectorised variant for channel counts that are a multiple of one 16-byte vector (and at most 256 vectors):
+// one block per example, thread = (pixel row, channel vector), 16-byte loads, pixel rows folded in order.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+bias_vec_kernel(const T *__restrict__ dY, int K, int Kout, float *__restrict__ db, float *__restrict__ partial, int slots,
+                int slot0, int bias_slots) {
+    extern __shared__ float red[];                     // [rows][Kout]
+    __shared__ float scratch[32];
+    const int n = blockIdx.x;
+    const int lanes_k = Kout / VEC, rows = 256 / lanes_k;
+    const int prow = threadIdx.x / lanes_k, kv = threadIdx.x - prow * lanes_k;
+    float a[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) a[v] = 0.f;
+    if (prow < rows) {
+        const T *base = dY + (long long)n * K * Kout + kv * VEC;
+        for (int pix = prow; pix < K; pix += rows) {
+            T g[VEC];
+            *reinterpret_cast<uint4 *>(g) = __ldcs(reinterpret_cast<const uint4 *>(base + (long long)pix * Kout));
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) a[v] += to_float(g[v]);
+        }
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) red[prow * Kout + kv * VEC + v] = a[v];
+    }
+    __syncthreads();
+    float sq = 0.f;
+    for (int k = threadIdx.x; k < Kout; k += 256) {
+        float v = 0.f;
+        for (int r = 0; r < rows; ++r) v += red[r * Kout + k];
+        db[(long long)n * Kout + k] = v;
+        sq = fmaf(v, v, sq);
+    }
+    sq = block_sum(sq, scratch);
+    if (threadIdx.x < bias_slots) partial[(long long)n * slots + slot0 + threadIdx.x] = (threadIdx.x == 0) ? sq : 0.f;
+}
+
 // One block per example: weight slots [0, w_slots) and bias slots [w_slots, slots) summed in index order.
 __global__ void __launch_bounds__(128)
 finalize_norm_kernel(const float *__restrict__ partial, int slots, int w_slots, int separate, float *__restrict__ sqnorm,
@@ -195,24 +232,26 @@ __global__ void bias_accum_kernel(const float *__restrict__ db, int B, int Kout,
 }
 
 // ------------------------------------------------------------------ dense layer
-// G_w[n, o, i] = dY[n, o] * X[n, i]: pure store stream, four columns per thread when Cin % 4 == 0.
+// G_w[n, o, i] = dY[n, o] * X[n, i]: pure store stream.  One block per (example, output) row of the result,
+// four columns per thread when Cin % 4 == 0.
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(256)
-dense_store_kernel(const T *__restrict__ X, const T *__restrict__ dY, long long total, int Cin, int Kout,
-                   float *__restrict__ G_w) {
-    const int per_row = VEC ? (Cin >> 2) : Cin;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const long long row = idx / per_row;             // n * Kout + o
-        const int i = (int)(idx - row * per_row);
+dense_store_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, int Kout, int rows_per_block,
+                   long long total_rows, float *__restrict__ G_w) {
+    for (int rr = 0; rr < rows_per_block; ++rr) {
+        const long long row = (long long)blockIdx.x * rows_per_block + rr;      // n * Kout + o
+        if (row >= total_rows) return;
         const long long n = row / Kout;
         const float gy = to_float(dY[row]);
+        const T *x = X + n * Cin;
+        float *out = G_w + row * Cin;
         if (VEC) {
-            const T *x = X + n * Cin + 4 * i;
-            const float4 v = make_float4(gy * to_float(x[0]), gy * to_float(x[1]), gy * to_float(x[2]), gy * to_float(x[3]));
-            __stcs(reinterpret_cast<float4 *>(G_w + row * Cin) + i, v);
+            for (int i = threadIdx.x * 4; i < Cin; i += 1024) {
+                const float4 v = make_float4(gy * to_float(x[i]), gy * to_float(x[i + 1]), gy * to_float(x[i + 2]), gy * to_float(x[i + 3]));
+                __stcs(reinterpret_cast<float4 *>(out + i), v);
+            }
         } else {
-            G_w[row * Cin + i] = gy * to_float(X[n * Cin + i]);
+            for (int i = threadIdx.x; i < Cin; i += 256) out[i] = gy * to_float(x[i]);
         }
     }
 }
@@ -385,6 +424,16 @@ dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, co
 
 dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
                       cudaStream_t st) {
+    const int vec = (dtype == DP_F32) ? 4 : 8;
+    if (g.Kout % vec == 0 && g.Kout / vec <= 256 && bias_blocks(g) <= 256) {
+        const size_t smem = sizeof(float) * (size_t)(256 / (g.Kout / vec)) * g.Kout;
+        if (dtype == DP_F32)
+            bias_vec_kernel<float, 4><<<g.B, 256, smem, st>>>(static_cast<const float *>(dY), g.K, g.Kout, db, partial, slots, slot0, bias_blocks(g));
+        else
+            bias_vec_kernel<__nv_bfloat16, 8><<<g.B, 256, smem, st>>>(static_cast<const __nv_bfloat16 *>(dY), g.K, g.Kout, db, partial, slots, slot0, bias_blocks(g));
+        DP_LAUNCH_CHECK("bias_vec_kernel");
+        return DP_OK;
+    }
     const dim3 grid(bias_blocks(g), g.B);
     if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
     if (dtype == DP_F32) bias_kernel<<<grid, 256, 0, st>>>(static_cast<const float *>(dY), g.K, g.Kout, db, partial, slots, slot0);
@@ -409,10 +458,13 @@ dp_status launch_bias_accum(const float *db, int B, int Kout, const float *facto
 template <typename T>
 static dp_status dense_store_t(const T *X, const T *dY, int B, int Cin, int Kout, float *G_w, float *G_b, cudaStream_t st) {
     const bool vec = (Cin & 3) == 0;
-    const long long total = (long long)B * Kout * (vec ? Cin / 4 : Cin);
-    const unsigned grid = (unsigned)min((long long)148 * 16, (total + 255) / 256);
-    if (vec) dense_store_kernel<T, true><<<grid, 256, 0, st>>>(X, dY, total, Cin, Kout, G_w);
-    else dense_store_kernel<T, false><<<grid, 256, 0, st>>>(X, dY, total, Cin, Kout, G_w);
+    const long long rows = (long long)B * Kout;
+    // short rows share a block so that every block still moves a few KB
+    const int per_block = Cin >= 1024 ? 1 : (1024 + Cin - 1) / Cin;
+    const long long blocks = (rows + per_block - 1) / per_block;
+    if (blocks > 0x7fffffffLL) return DP_ERR_UNSUPPORTED;
+    if (vec) dense_store_kernel<T, true><<<(unsigned)blocks, 256, 0, st>>>(X, dY, Cin, Kout, per_block, rows, G_w);
+    else dense_store_kernel<T, false><<<(unsigned)blocks, 256, 0, st>>>(X, dY, Cin, Kout, per_block, rows, G_w);
     DP_LAUNCH_CHECK("dense_store_kernel");
     if (G_b) {
         const long long cnt = (long long)B * Kout;

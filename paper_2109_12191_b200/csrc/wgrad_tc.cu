@@ -519,6 +519,45 @@ unfold_small_channels_kernel(const T *__restrict__ X, T *__restrict__ Xcol, cons
     *reinterpret_cast<uint4 *>(Xcol + pixel * n_pad + j0) = *reinterpret_cast<const uint4 *>(v);
 }
 
+// Same unfolding, one block per (output row, example): the R input rows the output row touches are staged in
+// shared memory (zero rows for the padding), then every thread assembles 16-byte groups of columns from them.
+// Within one filter row r the (s, c) columns of a pixel are a contiguous run of the input row.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+unfold_rows_kernel(const T *__restrict__ X, T *__restrict__ Xcol, const ConvGeom g, int n_pad) {
+    extern __shared__ __align__(16) unsigned char unfold_smem[];
+    T *rows = reinterpret_cast<T *>(unfold_smem);          // [R][W*Cin]
+    const int oh = blockIdx.x, n = blockIdx.y;
+    const int row_len = g.W * g.Cin;
+    for (int r = 0; r < g.R; ++r) {
+        const int ih = oh * g.stride + r - g.pad;
+        const bool inside = ih >= 0 && ih < g.H;
+        const T *src = X + ((long long)n * g.H + (inside ? ih : 0)) * row_len;
+        for (int i = threadIdx.x; i < row_len; i += 256) rows[r * row_len + i] = inside ? src[i] : T(0.f);
+    }
+    __syncthreads();
+    const int groups = n_pad / VEC, tap_row = g.S * g.Cin;
+    T *dst = Xcol + ((long long)n * g.OH + oh) * g.OW * n_pad;
+    for (int chunk = threadIdx.x; chunk < g.OW * groups; chunk += 256) {
+        const int ow = chunk / groups;
+        const int j0 = (chunk - ow * groups) * VEC;
+        const int base = (ow * g.stride - g.pad) * g.Cin;
+        int r = j0 / tap_row, jj = j0 - r * tap_row;
+        T v[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            T x = T(0.f);
+            if (j0 + e < g.N) {
+                const int col = base + jj;
+                if (col >= 0 && col < row_len) x = rows[r * row_len + col];
+            }
+            v[e] = x;
+            if (++jj == tap_row) { jj = 0; ++r; }
+        }
+        *reinterpret_cast<uint4 *>(dst + (long long)chunk * VEC) = *reinterpret_cast<const uint4 *>(v);
+    }
+}
+
 // ----------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -738,7 +777,16 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
             const int vec = (dtype == DP_BF16) ? 8 : 4;
             const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / vec);
             const unsigned blocks = (unsigned)((total + 255) / 256);
-            if (dtype == DP_BF16)
+            const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * (dtype == DP_BF16 ? 2 : 4);
+            if (row_smem <= 40 * 1024 && g0.OH <= 0x7fffffff && g0.B <= 65535) {
+                const dim3 grid_rows(g0.OH, g0.B);
+                if (dtype == DP_BF16)
+                    unfold_rows_kernel<__nv_bfloat16, 8><<<grid_rows, 256, row_smem, stream>>>(
+                        static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad);
+                else
+                    unfold_rows_kernel<float, 4><<<grid_rows, 256, row_smem, stream>>>(
+                        static_cast<const float *>(X), reinterpret_cast<float *>(ws_bytes), g0, pr.n_pad);
+            } else if (dtype == DP_BF16)
                 unfold_small_channels_kernel<__nv_bfloat16, 8><<<blocks, 256, 0, stream>>>(
                     static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad, total);
             else
