@@ -134,6 +134,20 @@ class SmallCnn:
         st.finish(seed=0, step=i, world=self.world)
         if rec: rec.stop(k + 1)
 
+    def capture(self):
+        """One CUDA graph per input set, each holding a whole step (the noise step index is baked in: it does
+        not change the work)."""
+        t = self.torch
+        self.graphs = []
+        for k in range(self.n_sets):
+            g = t.cuda.CUDAGraph()
+            with t.cuda.graph(g):
+                self.run(k)
+            self.graphs.append(g)
+
+    def run_graphed(self, i):
+        self.graphs[i % self.n_sets].replay()
+
     def algorithmic_bytes(self, call):
         """Bytes each call must move: inputs once, per-example gradients once (written by wgrad, read by clip)."""
         st = self.step_obj
@@ -310,6 +324,22 @@ class PerLayer:
         st.finish(seed=0, step=i)
         if rec: rec.stop(4)
 
+    def capture(self):
+        """One CUDA graph holding one chunk (all 107 layer calls); a step replays it G times, then adds the noise."""
+        t, st = self.torch, self.step_obj
+        self.chunk_graph = t.cuda.CUDAGraph()
+        with t.cuda.graph(self.chunk_graph):
+            for li, (X, dY) in enumerate(self.inputs):
+                st.wgrad(li, X, dY)
+
+    def run_graphed(self, i):
+        st = self.step_obj
+        st.begin()
+        for c in range(self.G):
+            self.chunk_graph.replay()
+            st.chunks_done += 1
+        st.finish(seed=0, step=i)
+
     def algorithmic_bytes(self, call):
         return self.bytes_kind[call] if call < 4 else 2 * self.step_obj.P * 4
 
@@ -424,17 +454,37 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    # The step's launch sequence is static, so on one GPU it is captured into CUDA graphs and replayed; per-call
+    # event timing (for the roofline) cannot be taken inside a replay and uses a separate un-captured pass below.
+    graphed = args.graph != "off" and world == 1 and hasattr(wl, "capture")
+    launches_per_step = None
+    if graphed:
+        c0 = b.dp_debug_launch_count()
+        wl.run(0)
+        launches_per_step = b.dp_debug_launch_count() - c0
+        torch.cuda.synchronize()
+        wl.capture()
+        for i in range(3):
+            wl.run_graphed(i)
+        barrier()
     rec = CallTimer(torch, len(wl.call_names))
     launches0 = b.dp_debug_launch_count()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for i in range(steps):
-        wl.run(warmup + i, rec)
+        if graphed:
+            wl.run_graphed(warmup + i)
+        else:
+            wl.run(warmup + i, rec)
     t_end.record()
     barrier()
-    launches = b.dp_debug_launch_count() - launches0
+    launches = (launches_per_step * steps) if graphed else (b.dp_debug_launch_count() - launches0)
     clocks = sampler.stop() if rank == 0 else None
     ms = t_start.elapsed_time(t_end)
+    if graphed:
+        for i in range(min(steps, args.profile_steps)):
+            wl.run(warmup + i, rec)
+        barrier()
     if dist:
         t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = t.item()
     value = wl.examples_per_step * steps * world / (ms / 1e3)
@@ -472,7 +522,7 @@ def run_ours(args):
                 "avg_ms_per_launch": round(avg_ms, 5), "traffic": None,
                 "shares": {n: round(t / sum(totals), 4) for n, t in zip(wl.call_names, totals)}}
     if hasattr(wl, "roofline"):
-        own = wl.roofline(dom, totals[dom] / (steps * wl.G), peaks)
+        own = wl.roofline(dom, totals[dom] / (max(1, counts[4]) * wl.G), peaks)
         if own:
             roofline.update(own)
 
@@ -487,7 +537,7 @@ def run_ours(args):
             "dtype": getattr(wl, "dtype_name", "f32"), "data": "synthetic", "config": dict(wl.describe(), parallelism=("single GPU" if world == 1 else f"batch sharded over {world} GPUs, one all-reduce of the accumulator per step")),
             "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
-            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
+            "gpu_launches": int(launches), "launch_mode": ("CUDA graph replay" if graphed else "stream launches"), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
@@ -598,6 +648,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS) + ["sweep", "sweep_all"])
     ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"], help="replay the step from CUDA graphs (single GPU)")
+    ap.add_argument("--profile-steps", type=int, default=20, help="un-captured steps timed per call for the roofline")
     ap.add_argument("--layers", default="", help="sweep workloads: comma-separated layer indices")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

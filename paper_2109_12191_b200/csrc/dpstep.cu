@@ -52,7 +52,7 @@ static bool has_bias_tensor(const dp_layer_desc *d) { return d->kind == DP_LAYER
 static int groups_of(const dp_layer_desc *d) { return (d->bias_separate && has_bias_tensor(d)) ? 2 : 1; }
 
 struct WgradPlan {
-    bool use_tc;
+    bool use_tc, use_thin;
     int slots, w_slots;
     size_t status_off, partial_off, factor_off, db_off, chunk_off, dg_off, tc_off, total;
 };
@@ -61,13 +61,14 @@ static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
     const ConvGeom g = geom_of(d);
     const size_t B = (size_t)d->B;
     pl.use_tc = false;
-    if (d->kind == DP_LAYER_CONV2D && d->impl != DP_IMPL_CUDA_CORE) pl.use_tc = tc_eligible(d->dtype, g, epi);
+    pl.use_thin = d->kind == DP_LAYER_CONV2D && d->impl == DP_IMPL_AUTO && epi != DP_EPI_CLIP_ACCUM && thin_conv_eligible(g);
+    if (d->kind == DP_LAYER_CONV2D && d->impl != DP_IMPL_CUDA_CORE && !pl.use_thin) pl.use_tc = tc_eligible(d->dtype, g, epi);
     size_t off = 0;
     pl.status_off = off; off += 256;
     if (d->kind == DP_LAYER_CONV2D) {
-        const int tiles = pl.use_tc ? tc_norm_slots(d->dtype, g, epi) : fma_tiles_m(g) * fma_tiles_n(g);
+        const int tiles = pl.use_thin ? 1 : (pl.use_tc ? tc_norm_slots(d->dtype, g, epi) : fma_tiles_m(g) * fma_tiles_n(g));
         pl.w_slots = tiles;
-        pl.slots = tiles + (d->has_bias ? bias_blocks(g) : 0);
+        pl.slots = tiles + (d->has_bias ? (pl.use_thin ? 1 : bias_blocks(g)) : 0);
     } else {
         pl.w_slots = 1; pl.slots = 2;
     }
@@ -147,6 +148,11 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
 
     if (d->kind == DP_LAYER_CONV2D) {
         float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;
+        if (pl.use_thin) {
+            rc = launch_conv_thin(d->dtype, X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, partial, pl.slots, d->has_bias, st);
+            if (rc != DP_OK) return rc;
+            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
+        }
         if (d->has_bias) {
             rc = launch_bias(d->dtype, dY, g, db, partial, pl.slots, pl.w_slots, st);
             if (rc != DP_OK) return rc;

@@ -127,6 +127,162 @@ conv_wgrad_fma_kernel(const T *__restrict__ X, const T *__restrict__ dY, const C
     }
 }
 
+// Thin convolutions (R*S*Cin <= 32 columns, e.g. a 3x3 conv on RGB): one block per example.  The zero-padded
+// input of the example sits in shared memory; thread = (pixel group, output channel lane) keeps one gradient row
+// (all columns) per owned output channel in registers and walks its share of the pixels, reading dY coalesced and
+// the input patch by shared-memory broadcast.  The eight pixel groups are folded in order; the bias gradient and
+// both squared norms come out of the same pass.
+// RT x SCT > 0 fixes the filter rows and the run length S*Cin at compile time (3 x 9 for a 3x3 conv on RGB), which
+// turns every patch read into a shared-memory load with an immediate offset; RT = 0 is the any-shape version.
+template <typename T, int KPT, int RT, int SCT>
+__global__ void __launch_bounds__(256)
+conv_wgrad_thin_kernel(const T *__restrict__ X, const T *__restrict__ dY, const ConvGeom g, float *__restrict__ G_w,
+                       float *__restrict__ db, float *__restrict__ partial, int slots, int has_bias) {
+    extern __shared__ float thin_smem[];
+    __shared__ float scratch[32];
+    const int Hp = g.H + 2 * g.pad, Wp = g.W + 2 * g.pad;
+    const int xs_count = Hp * Wp * g.Cin;
+    float *xs = thin_smem;                                   // [Hp][Wp][Cin], zero border
+    float *red = thin_smem + ((xs_count + 3) & ~3);          // [8][Kout*N] then [8][Kout]
+    const int n = blockIdx.x, lane = threadIdx.x & 31, pg = threadIdx.x >> 5;
+    {
+        const int row_in = g.W * g.Cin, row_p = Wp * g.Cin;
+        for (int i = threadIdx.x; i < xs_count; i += 256) xs[i] = 0.f;
+        __syncthreads();
+        const T *Xn = X + (long long)n * g.H * row_in;
+        for (int i = threadIdx.x; i < g.H * row_in; i += 256) {
+            const int h = i / row_in, rest = i - h * row_in;
+            xs[(h + g.pad) * row_p + g.pad * g.Cin + rest] = to_float(Xn[i]);
+        }
+    }
+    int off[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int jj = j < g.N ? j : 0;
+        const int c = jj % g.Cin, rs = jj / g.Cin;
+        off[j] = ((rs / g.S) * Wp + rs % g.S) * g.Cin + c;
+    }
+    float acc[KPT][32], bsum[KPT];
+#pragma unroll
+    for (int kk = 0; kk < KPT; ++kk) {
+        bsum[kk] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[kk][j] = 0.f;
+    }
+    __syncthreads();
+    int oh = pg / g.OW, ow = pg - oh * g.OW;
+    const T *dYn = dY + (long long)n * g.K * g.Kout;
+    // four pixels per trip: their dY loads are issued together so the memory latency is paid once per trip
+    for (int pix = pg; pix < g.K; pix += 32) {
+        float gy[4][KPT];
+        int base[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int pu = pix + 8 * u;
+            base[u] = (oh * g.stride * Wp + ow * g.stride) * g.Cin;
+#pragma unroll
+            for (int kk = 0; kk < KPT; ++kk)
+                gy[u][kk] = pu < g.K ? to_float(dYn[(long long)pu * g.Kout + lane + 32 * kk]) : 0.f;
+            if (pu >= g.K) base[u] = 0;
+            ow += 8;
+            while (ow >= g.OW) { ow -= g.OW; ++oh; }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int kk = 0; kk < KPT; ++kk) bsum[kk] += gy[u][kk];
+            if constexpr (RT > 0) {
+                const float *patch = xs + base[u];
+                const int row_p = Wp * g.Cin;
+#pragma unroll
+                for (int r = 0; r < RT; ++r) {
+#pragma unroll
+                    for (int t = 0; t < SCT; ++t) {
+                        const float x = patch[r * row_p + t];
+#pragma unroll
+                        for (int kk = 0; kk < KPT; ++kk) acc[kk][r * SCT + t] = fmaf(gy[u][kk], x, acc[kk][r * SCT + t]);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (j < g.N) {
+                        const float x = xs[base[u] + off[j]];
+#pragma unroll
+                        for (int kk = 0; kk < KPT; ++kk) acc[kk][j] = fmaf(gy[u][kk], x, acc[kk][j]);
+                    }
+                }
+            }
+        }
+    }
+    const int MN = g.Kout * g.N;
+    float *bred = red + 8 * MN;
+#pragma unroll
+    for (int kk = 0; kk < KPT; ++kk) {
+        const int k = lane + 32 * kk;
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (j < g.N) red[pg * MN + k * g.N + j] = acc[kk][j];
+        bred[pg * g.Kout + k] = bsum[kk];
+    }
+    __syncthreads();
+    float sq = 0.f, sqb = 0.f;
+    for (int t = threadIdx.x; t < MN; t += 256) {
+        float v = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v += red[q * MN + t];
+        if (G_w) G_w[(long long)n * MN + t] = v;
+        sq = fmaf(v, v, sq);
+    }
+    if (has_bias) {
+        for (int k = threadIdx.x; k < g.Kout; k += 256) {
+            float v = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v += bred[q * g.Kout + k];
+            db[(long long)n * g.Kout + k] = v;
+            sqb = fmaf(v, v, sqb);
+        }
+    }
+    sq = block_sum(sq, scratch);
+    sqb = block_sum(sqb, scratch);
+    if (threadIdx.x == 0) {
+        partial[(long long)n * slots] = sq;
+        if (has_bias) partial[(long long)n * slots + 1] = sqb;
+    }
+}
+
+static size_t thin_smem_bytes(const ConvGeom &g) {
+    const size_t xs = ((size_t)(g.H + 2 * g.pad) * (g.W + 2 * g.pad) * g.Cin + 3) & ~(size_t)3;
+    return sizeof(float) * (xs + 8 * (size_t)g.Kout * g.N + 8 * (size_t)g.Kout);
+}
+
+bool thin_conv_eligible(const ConvGeom &g) {
+    return g.N <= 32 && (g.Kout == 32 || g.Kout == 64) && g.K >= 8 && thin_smem_bytes(g) <= 47 * 1024 && g.B <= 0x7fffffff;
+}
+
+template <typename T, int KPT>
+static void thin_launch_t(const T *X, const T *dY, const ConvGeom &g, float *G_w, float *db, float *partial, int slots,
+                          int has_bias, size_t smem, cudaStream_t st) {
+    if (g.R == 3 && g.S * g.Cin == 9)
+        conv_wgrad_thin_kernel<T, KPT, 3, 9><<<g.B, 256, smem, st>>>(X, dY, g, G_w, db, partial, slots, has_bias);
+    else
+        conv_wgrad_thin_kernel<T, KPT, 0, 0><<<g.B, 256, smem, st>>>(X, dY, g, G_w, db, partial, slots, has_bias);
+}
+
+dp_status launch_conv_thin(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
+                           float *partial, int slots, int has_bias, cudaStream_t st) {
+    const size_t smem = thin_smem_bytes(g);
+    if (dtype == DP_F32) {
+        if (g.Kout == 32) thin_launch_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), g, G_w, db, partial, slots, has_bias, smem, st);
+        else thin_launch_t<float, 2>(static_cast<const float *>(X), static_cast<const float *>(dY), g, G_w, db, partial, slots, has_bias, smem, st);
+    } else {
+        if (g.Kout == 32) thin_launch_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), g, G_w, db, partial, slots, has_bias, smem, st);
+        else thin_launch_t<__nv_bfloat16, 2>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), g, G_w, db, partial, slots, has_bias, smem, st);
+    }
+    DP_LAUNCH_CHECK("conv_wgrad_thin_kernel");
+    return DP_OK;
+}
+
 // db[n, k] = sum over pixels of dY[n, pix, k]; 64 channels x 4 pixel lanes per block, lanes folded in order.
 template <typename T>
 __global__ void __launch_bounds__(256)

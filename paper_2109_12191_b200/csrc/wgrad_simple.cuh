@@ -26,6 +26,11 @@ int fma_clip_splits(const ConvGeom &g);
 dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, const ConvGeom &g, float *G_w,
                           float *partial, int slots, const float *factor, float *acc_w, float *sum_ws,
                           cudaStream_t stream);
+// Thin convolutions (at most 32 gradient columns, 32 or 64 output channels, input of one example fits shared memory):
+// gradient (G_w may be null), bias gradient and both squared norms in one launch; partial slot 0 = weights, 1 = bias.
+bool thin_conv_eligible(const ConvGeom &g);
+dp_status launch_conv_thin(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
+                           float *partial, int slots, int has_bias, cudaStream_t stream);
 // db[n,k] = sum over pixels of dY; also sum_k db^2 per block into partial[n*slots + slot0 + block]
 dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
                       cudaStream_t stream);

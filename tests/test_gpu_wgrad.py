@@ -78,6 +78,21 @@ def test_conv_cuda_core(case, dtype):
     check_layer(layer, 5, dtype, CUDA_CORE, (930, sum(case[:6])), spread=True)
 
 
+THIN_CONVS = [(3, 32, 3, 1, 1, 32, True), (3, 64, 3, 2, 1, 17, False), (2, 32, 3, 1, 0, 9, True), (1, 32, 5, 1, 2, 12, True),
+              (3, 32, 3, 1, 1, 3, False)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", THIN_CONVS)
+def test_conv_thin_inputs_default_route(case, dtype):
+    """Few-column convolutions (RGB inputs) under DP_IMPL_AUTO: the one-block-per-example kernel for
+    STORE / NORM, the general kernels for the fused clip."""
+    Cin, Kout, R, stride, pad, H, bias = case
+    layer = synth.conv(Cin, Kout, R, stride, pad, H, bias, name=str(case))
+    check_layer(layer, 6, dtype, AUTO, (945, sum(case[:6])), spread=True)
+    check_layer(layer, 3, dtype, AUTO, (946, sum(case[:6])), bias_separate=1, spread=True)
+
+
 def test_conv_non_square_image_and_filter():
     layer = synth.Layer("conv", 6, 9, R=3, S=5, stride=2, pad=1, H=11, W=14, bias=True, name="3x5")
     check_layer(layer, 3, "f32", CUDA_CORE, (931,), spread=True)
