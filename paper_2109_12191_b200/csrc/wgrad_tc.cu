@@ -15,7 +15,7 @@
 // Every wait is bounded: on expiry the CTA sets a status word, drains and returns.
 //
 // fp32 inputs run as split tf32: the tensor core truncates fp32 to tf32, which biases every norm by about
-// 1e-3, so four more warps split each landed stage into hi = x with the low 13 mantissa bits cleared (kept
+// 1e-3, so eight more warps split each landed stage into hi = x with the low 13 mantissa bits cleared (kept
 // in place) and lo = x - hi (a second buffer of the same layout), and the issuer accumulates
 // hi*hi + lo*hi + hi*lo per step.  What is dropped (lo*lo and the truncation of lo) is below 2^-20 relative.
 #include "wgrad_tc.cuh"
@@ -120,17 +120,22 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], fp32 accumulate, issued by one thread; TF32 selects kind::tf32 (fp32 inputs)
+// D[tmem] (+)= A[smem] * B[smem], fp32 accumulate, issued by one thread; TF32 selects kind::tf32 (fp32 inputs).
+// The operand descriptors arrive as (low word, high word): only the low word (start address) changes from step to
+// step, which keeps the issuing thread's work per instruction to one 32-bit add.
 template <bool TF32>
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                     uint32_t accumulate) {
     if (TF32)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                     "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %4, p;\n\t}"
+                     ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
     else
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                     ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -164,7 +169,7 @@ __device__ __forceinline__ uint32_t instr_desc(int n_cols, uint32_t fmt) {
 }
 
 template <bool TF32, bool CLIP>
-__global__ void __launch_bounds__(TF32 ? 320 : 192, 1)
+__global__ void __launch_bounds__(TF32 ? 448 : 192, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], ready_bar[kMaxStages], tmem_full[2], tmem_empty[2];
@@ -181,7 +186,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 4);
+            mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 8);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -252,9 +257,10 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             uint32_t acc_phase = 0;  // bit b: phase of accumulator buffer b
             int buf = 0;
             bool live = true;
-            const uint64_t desc_hi = operand_desc_base<TF32>((uint32_t)slab_bytes);
+            const uint64_t desc_base = operand_desc_base<TF32>((uint32_t)slab_bytes);
+            const uint32_t desc_lo = (uint32_t)desc_base, desc_hi32 = (uint32_t)(desc_base >> 32);
             const int ksteps = p.Kt / p.krows;
-            const uint32_t kadvance = (uint32_t)(p.krows * kRowBytes) >> 4;     // descriptor start-address units of 16 B
+            constexpr uint32_t kadvance = (uint32_t)((TF32 ? 8 : 16) * kRowBytes) >> 4;   // start-address units of 16 B per MMA step
             for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
               const Item it = decode_item(p, item);
               const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - it.nt * b_slabs_tile);
@@ -268,22 +274,25 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     if (!mbar_wait(smem_u32(TF32 ? &ready_bar[stage] : &full_bar[stage]), phase, abort_p)) { live = false; break; }
                     tc_fence_after();
                     const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
-                    uint64_t ad = desc_hi | (uint64_t)((a_src & 0x3FFFFu) >> 4);
-                    uint64_t bd = desc_hi | (uint64_t)(((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
+                    // descriptor low words: start address >> 4 in bits 0-13, slab stride >> 4 in bits 16-29
+                    uint32_t ad = desc_lo | ((a_src & 0x3FFFFu) >> 4);
+                    uint32_t bd = desc_lo | (((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
                     // rows of the A tile past the operand's extent hold whatever the stage held before:
                     // they only feed rows of D that the epilogue never reads
                     if (TF32) {
-                        const uint64_t lo = (uint64_t)((uint32_t)p.lo_offset >> 4);
+                        const uint32_t lo = (uint32_t)p.lo_offset >> 4;
+#pragma unroll 2
                         for (int ks = 0; ks < ksteps; ++ks) {
-                            umma<TF32>(d_tmem, ad + lo, bd, idesc, accumulate);      // lo(A) * hi(B)
-                            umma<TF32>(d_tmem, ad, bd + lo, idesc, 1u);              // hi(A) * lo(B)
-                            umma<TF32>(d_tmem, ad, bd, idesc, 1u);                   // hi(A) * hi(B)
+                            umma<TF32>(d_tmem, ad + lo, bd, desc_hi32, idesc, accumulate);      // lo(A) * hi(B)
+                            umma<TF32>(d_tmem, ad, bd + lo, desc_hi32, idesc, 1u);              // hi(A) * lo(B)
+                            umma<TF32>(d_tmem, ad, bd, desc_hi32, idesc, 1u);                   // hi(A) * hi(B)
                             accumulate = 1;
                             ad += kadvance; bd += kadvance;
                         }
                     } else {
+#pragma unroll 4
                         for (int ks = 0; ks < ksteps; ++ks) {
-                            umma<TF32>(d_tmem, ad, bd, idesc, accumulate);
+                            umma<TF32>(d_tmem, ad, bd, desc_hi32, idesc, accumulate);
                             accumulate = 1;
                             ad += kadvance; bd += kadvance;
                         }
@@ -315,16 +324,30 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p);
                 if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
                 uint8_t *base = tiles + (size_t)stage * p.stage_bytes;
-                for (int i = tid; i < chunks; i += 128) {
-                    uint8_t *ptr = (i < a_chunks) ? base + ((size_t)i << 4) : base + p.a_bytes + ((size_t)(i - a_chunks) << 4);
-                    const float4 x = *reinterpret_cast<const float4 *>(ptr);
-                    float4 hi, lo;
-                    hi.x = __uint_as_float(__float_as_uint(x.x) & 0xFFFFE000u); lo.x = x.x - hi.x;
-                    hi.y = __uint_as_float(__float_as_uint(x.y) & 0xFFFFE000u); lo.y = x.y - hi.y;
-                    hi.z = __uint_as_float(__float_as_uint(x.z) & 0xFFFFE000u); lo.z = x.z - hi.z;
-                    hi.w = __uint_as_float(__float_as_uint(x.w) & 0xFFFFE000u); lo.w = x.w - hi.w;
-                    *reinterpret_cast<float4 *>(ptr) = hi;
-                    *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;
+                // eight warps (the issue rate of the split is what bounds fp32 layers); four 16-byte groups per
+                // thread and trip with all loads first, A region and B region in turn
+                for (int region = 0; region < 2; ++region) {
+                    uint8_t *rbase = region ? base + p.a_bytes : base;
+                    const int rchunks = region ? chunks - a_chunks : a_chunks;
+                    for (int i0 = tid; i0 < rchunks; i0 += 1024) {
+                        float4 x[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (i0 + 256 * u < rchunks) x[u] = *reinterpret_cast<const float4 *>(rbase + ((size_t)(i0 + 256 * u) << 4));
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (i0 + 256 * u < rchunks) {
+                                uint8_t *ptr = rbase + ((size_t)(i0 + 256 * u) << 4);
+                                float4 hi, lo;
+                                hi.x = __uint_as_float(__float_as_uint(x[u].x) & 0xFFFFE000u); lo.x = x[u].x - hi.x;
+                                hi.y = __uint_as_float(__float_as_uint(x[u].y) & 0xFFFFE000u); lo.y = x[u].y - hi.y;
+                                hi.z = __uint_as_float(__float_as_uint(x[u].z) & 0xFFFFE000u); lo.z = x[u].z - hi.z;
+                                hi.w = __uint_as_float(__float_as_uint(x[u].w) & 0xFFFFE000u); lo.w = x[u].w - hi.w;
+                                *reinterpret_cast<float4 *>(ptr) = hi;
+                                *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;
+                            }
+                        }
+                    }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
                 __syncwarp();
@@ -833,8 +856,8 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
         if (clip) conv_wgrad_tc_kernel<false, true><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
         else conv_wgrad_tc_kernel<false, false><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
     } else {
-        if (clip) conv_wgrad_tc_kernel<true, true><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
-        else conv_wgrad_tc_kernel<true, false><<<grid, 320, pl.smem, stream>>>(tmX, tmY, p);
+        if (clip) conv_wgrad_tc_kernel<true, true><<<grid, 448, pl.smem, stream>>>(tmX, tmY, p);
+        else conv_wgrad_tc_kernel<true, false><<<grid, 448, pl.smem, stream>>>(tmX, tmY, p);
     }
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
     if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g0.M * g0.N, acc_w, stream);
