@@ -144,14 +144,18 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
     const ConvGeom g = geom_of(d);
     const int clip = (epi == DP_EPI_CLIP_ACCUM);
     dp_status rc;
-    DP_CUDA_TRY(cudaMemsetAsync(ws + pl.status_off, 0, 16, st));
+    // Tensor-core launches may set the status word (bounded waits), so it is cleared before them; every other
+    // path has no waits and lets its last small kernel write "ok" instead of paying for a memset node.
+    int *status_word = reinterpret_cast<int *>(ws + pl.status_off);
+    int *reset = pl.use_tc ? nullptr : status_word;
+    if (pl.use_tc) DP_CUDA_TRY(cudaMemsetAsync(ws + pl.status_off, 0, 16, st));
 
     if (d->kind == DP_LAYER_CONV2D) {
         float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;
         if (pl.use_thin) {
             rc = launch_conv_thin(d->dtype, X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, partial, pl.slots, d->has_bias, st);
             if (rc != DP_OK) return rc;
-            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
+            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
         }
         if (d->has_bias) {
             rc = launch_bias(d->dtype, dY, g, db, partial, pl.slots, pl.w_slots, st);
@@ -161,13 +165,13 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             if (pl.use_tc) rc = launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
             else rc = launch_conv_fma(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, nullptr, st);
             if (rc != DP_OK) return rc;
-            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
+            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
         }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
         else rc = launch_conv_fma(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
         if (rc != DP_OK) return rc;
-        rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st);
+        rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st, reset);
         if (rc != DP_OK) return rc;
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true);
         else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
@@ -184,7 +188,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         rc = launch_dense_norm(d->dtype, X, dY, d->B, d->C_in, d->K_out, d->has_bias, partial,
                                (clip && d->has_bias) ? db_ws : nullptr, st);
         if (rc != DP_OK) return rc;
-        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st);
+        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st, reset);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
         rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, 2, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
@@ -200,7 +204,10 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         float *dbt = (epi == DP_EPI_STORE_NORM) ? G_b : reinterpret_cast<float *>(ws + pl.dg_off) + (size_t)d->B * d->C_in;
         rc = launch_norm_affine(d->dtype, X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
         if (rc != DP_OK) return rc;
-        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st);
+        if (clip)
+            return launch_affine_clip_accum(partial, d->B, C_l, groups == 2, sqnorm, sqnorm_stride, clip_out, dg, dbt, d->C_in,
+                                            acc_w, acc_b, st, reset);
+        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st, reset);
         if (rc != DP_OK || !clip) return rc;
         return launch_affine_accum(dg, dbt, d->B, d->C_in, factor, acc_w, acc_b, st);
     }

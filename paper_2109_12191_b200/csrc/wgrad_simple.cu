@@ -349,9 +349,10 @@ bias_vec_kernel(const T *__restrict__ dY, int K, int Kout, float *__restrict__ d
 // One block per example: weight slots [0, w_slots) and bias slots [w_slots, slots) summed in index order.
 __global__ void __launch_bounds__(128)
 finalize_norm_kernel(const float *__restrict__ partial, int slots, int w_slots, int separate, float *__restrict__ sqnorm,
-                     long long sq_stride, int clip, float C_l, float *__restrict__ factor, float *clip_out) {
+                     long long sq_stride, int clip, float C_l, float *__restrict__ factor, float *clip_out, int *status_reset) {
     __shared__ double scratch[32];
     const int n = blockIdx.x;
+    if (status_reset && n == 0 && threadIdx.x == 0) *status_reset = 0;   // paths without bounded waits report "ok"
     const float *p = partial + (long long)n * slots;
     double sw = 0.0, sb = 0.0;
     for (int i = threadIdx.x; i < w_slots; i += 128) sw += (double)p[i];
@@ -453,21 +454,42 @@ norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, in
     for (int v = 0; v < VEC; ++v) { sg[v] = 0.f; sb[v] = 0.f; }
     const int p_end = min(HW, (chunk + 1) * kNormPix);
     if (live) {
-        for (int p = chunk * kNormPix + prow; p < p_end; p += rows) {
-            const long long off = ((long long)n * HW + p) * C + c0;
-            T xv[VEC], gv[VEC];
-            if (VEC * sizeof(T) == 16) {
-                *reinterpret_cast<uint4 *>(xv) = __ldcs(reinterpret_cast<const uint4 *>(X + off));
-                *reinterpret_cast<uint4 *>(gv) = __ldcs(reinterpret_cast<const uint4 *>(dY + off));
-            } else {
+        if (VEC * sizeof(T) == 16) {
+            // four pixels per trip, all eight 16-byte loads issued before any arithmetic
+            for (int p = chunk * kNormPix + prow; p < p_end; p += 4 * rows) {
+                uint4 xr[4], gr[4];
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) { xv[v] = X[off + v]; gv[v] = dY[off + v]; }
+                for (int u = 0; u < 4; ++u) {
+                    const int pu = p + u * rows;
+                    if (pu < p_end) {
+                        const long long off = ((long long)n * HW + pu) * C + c0;
+                        xr[u] = __ldcs(reinterpret_cast<const uint4 *>(X + off));
+                        gr[u] = __ldcs(reinterpret_cast<const uint4 *>(dY + off));
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (p + u * rows < p_end) {
+                        const T *xv = reinterpret_cast<const T *>(&xr[u]);
+                        const T *gv = reinterpret_cast<const T *>(&gr[u]);
+#pragma unroll
+                        for (int v = 0; v < VEC; ++v) {
+                            const float gg = to_float(gv[v]);
+                            sg[v] = fmaf(gg, to_float(xv[v]), sg[v]);
+                            sb[v] += gg;
+                        }
+                    }
+                }
             }
+        } else {
+            for (int p = chunk * kNormPix + prow; p < p_end; p += rows) {
+                const long long off = ((long long)n * HW + p) * C + c0;
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) {
-                const float gg = to_float(gv[v]);
-                sg[v] = fmaf(gg, to_float(xv[v]), sg[v]);
-                sb[v] += gg;
+                for (int v = 0; v < VEC; ++v) {
+                    const float gg = to_float(dY[off + v]);
+                    sg[v] = fmaf(gg, to_float(X[off + v]), sg[v]);
+                    sb[v] += gg;
+                }
             }
         }
     }
@@ -531,6 +553,60 @@ __global__ void affine_accum_kernel(const float *__restrict__ dgamma, const floa
     }
     acc_w[c] += a;
     acc_b[c] += b;
+}
+
+// Normalisation layers, fused clip: every block works out the factors of all examples from the two squared norms
+// (cheap and identical in every block), block 0 publishes norms and factors, then each thread owns one channel and
+// adds sum_n f_n dgamma[n, c] / dbeta[n, c] to the accumulators.
+__global__ void __launch_bounds__(128)
+affine_clip_accum_kernel(const float *__restrict__ partial2, int B, float C_l, int separate, float *__restrict__ sqnorm,
+                         long long sq_stride, float *clip_out, const float *__restrict__ dgamma,
+                         const float *__restrict__ dbeta, int C, float *__restrict__ acc_w, float *__restrict__ acc_b,
+                         int *status_reset) {
+    __shared__ float fw[512], fb[512];
+    if (status_reset && blockIdx.x == 0 && threadIdx.x == 0) *status_reset = 0;
+    const int c = blockIdx.x * 128 + threadIdx.x;
+    float a = 0.f, b = 0.f;
+    for (int n0 = 0; n0 < B; n0 += 512) {
+        const int nb = min(512, B - n0);
+        __syncthreads();
+        for (int t = threadIdx.x; t < nb; t += 128) {
+            const int n = n0 + t;
+            const double sw = (double)partial2[2 * n], sb = (double)partial2[2 * n + 1];
+            float f0, f1;
+            if (separate) { f0 = clip_factor(sw, C_l); f1 = clip_factor(sb, C_l); }
+            else { f0 = f1 = clip_factor(sw + sb, C_l); }
+            fw[t] = f0; fb[t] = f1;
+            if (blockIdx.x == 0) {
+                if (separate) {
+                    sqnorm[n * sq_stride] = (float)sw; sqnorm[n * sq_stride + 1] = (float)sb;
+                    if (clip_out) { clip_out[2 * n] = f0; clip_out[2 * n + 1] = f1; }
+                } else {
+                    sqnorm[n * sq_stride] = (float)(sw + sb);
+                    if (clip_out) clip_out[n] = f0;
+                }
+            }
+        }
+        __syncthreads();
+        if (c < C) {
+            const float *g = dgamma + (long long)n0 * C + c, *h = dbeta + (long long)n0 * C + c;
+#pragma unroll 8
+            for (int t = 0; t < nb; ++t) {
+                a = fmaf(fw[t], g[(long long)t * C], a);
+                b = fmaf(fb[t], h[(long long)t * C], b);
+            }
+        }
+    }
+    if (c < C) { acc_w[c] += a; acc_b[c] += b; }
+}
+
+dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int separate, float *sqnorm, long long sq_stride,
+                                   float *clip_out, const float *dgamma, const float *dbeta, int C, float *acc_w,
+                                   float *acc_b, cudaStream_t st, int *status_reset) {
+    affine_clip_accum_kernel<<<(C + 127) / 128, 128, 0, st>>>(partial2, B, C_l, separate, sqnorm, sq_stride, clip_out, dgamma,
+                                                            dbeta, C, acc_w, acc_b, status_reset);
+    DP_LAUNCH_CHECK("affine_clip_accum_kernel");
+    return DP_OK;
 }
 
 // ------------------------------------------------------------------ host launchers
@@ -599,8 +675,9 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
 }
 
 dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
-                          long long sq_stride, int clip, float C_l, float *factor, float *clip_out, cudaStream_t st) {
-    finalize_norm_kernel<<<B, 128, 0, st>>>(partial, slots, w_slots, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
+                          long long sq_stride, int clip, float C_l, float *factor, float *clip_out, cudaStream_t st,
+                          int *status_reset) {
+    finalize_norm_kernel<<<B, 128, 0, st>>>(partial, slots, w_slots, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out, status_reset);
     DP_LAUNCH_CHECK("finalize_norm_kernel");
     return DP_OK;
 }

@@ -37,7 +37,7 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
 // folds the partial slots of every example into sqnorm (and clip factors when clip != 0)
 dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
                           long long sq_stride, int clip, float C_l, float *factor, float *clip_out,
-                          cudaStream_t stream);
+                          cudaStream_t stream, int *status_reset = nullptr);
 // acc_b[k] += sum_n factor[n*2+1] * db[n,k]
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream);
 
@@ -53,6 +53,11 @@ dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, in
 // acc_w[c] += sum_n factor[n*2] dgamma[n,c]; acc_b[c] += sum_n factor[n*2+1] dbeta[n,c]
 dp_status launch_affine_accum(const float *dgamma, const float *dbeta, int B, int C, const float *factor,
                               float *acc_w, float *acc_b, cudaStream_t stream);
+
+// fused: factors from partial2 (two squared norms per example), publish norms / factors, accumulate both tensors
+dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int separate, float *sqnorm, long long sq_stride,
+                                   float *clip_out, const float *dgamma, const float *dbeta, int C, float *acc_w,
+                                   float *acc_b, cudaStream_t stream, int *status_reset = nullptr);
 
 inline int norm_chunks(int HW) { return (HW + kNormPix - 1) / kNormPix; }
 
