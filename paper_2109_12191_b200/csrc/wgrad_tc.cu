@@ -15,9 +15,9 @@
 // Every wait is bounded: on expiry the CTA sets a status word, drains and returns.
 //
 // fp32 inputs run as split tf32: the tensor core truncates fp32 to tf32, which biases every norm by about
-// 1e-3, so eight more warps split each landed stage into hi = x with the low 13 mantissa bits cleared (kept
-// in place) and lo = x - hi (a second buffer of the same layout), and the issuer accumulates
-// hi*hi + lo*hi + hi*lo per step.  What is dropped (lo*lo and the truncation of lo) is below 2^-20 relative.
+// 1e-3, so eight more warps write lo = x - hi (hi = x with the low 13 mantissa bits cleared) of each landed
+// stage into a second buffer of the same layout; x itself stays in place, where the tensor core's own truncation
+// turns it into hi, and the issuer accumulates lo*hi + hi*lo + hi*hi per step.  What is dropped (lo*lo and the truncation of lo) is below 2^-20 relative.
 #include "wgrad_tc.cuh"
 #include <cuda.h>
 #include <mutex>
@@ -175,6 +175,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], ready_bar[kMaxStages], tmem_full[2], tmem_empty[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ float xpose[4][32][33];      // per epilogue warp: 32 x 32 transpose buffer for coalesced row stores
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -343,8 +344,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                 hi.y = __uint_as_float(__float_as_uint(x[u].y) & 0xFFFFE000u); lo.y = x[u].y - hi.y;
                                 hi.z = __uint_as_float(__float_as_uint(x[u].z) & 0xFFFFE000u); lo.z = x[u].z - hi.z;
                                 hi.w = __uint_as_float(__float_as_uint(x[u].w) & 0xFFFFE000u); lo.w = x[u].w - hi.w;
-                                *reinterpret_cast<float4 *>(ptr) = hi;
-                                *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;
+                                *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;     // x stays: truncated by the MMA itself, it is hi
                             }
                         }
                     }
@@ -410,19 +410,24 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                     float *dst = Gn + (long long)b_idx * p.Ng + a_idx;
 #pragma unroll
                                     for (int i = 0; i < 32; ++i) __stcs(dst + (long long)i * p.Ng, __uint_as_float(v[i]));
-                                } else if (!p.n_pad_cols) {   // row = output channel k, tile columns = 32 consecutive j
-                                    float4 *dst = reinterpret_cast<float4 *>(Gn + (long long)a_idx * p.Ng + b_idx);
-#pragma unroll
-                                    for (int i = 0; i < 8; ++i)
-                                        __stcs(dst + i, make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                                                    __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
-                                } else {             // padded columns: rows are not 16-byte aligned, and j stops at Ng
-                                    float *dst = Gn + (long long)a_idx * p.Ng + b_idx;
-#pragma unroll
-                                    for (int i = 0; i < 32; ++i)
-                                        if (b_idx + i < p.Ng) dst[i] = __uint_as_float(v[i]);
                                 }
                             }
+                        }
+                        if (p.mode == 0 && !p.a_is_x) {
+                            // row = output channel k, tile columns = 32 consecutive j: each lane holds one row, so the
+                            // warp transposes its 32 x 32 block through shared memory and every store instruction then
+                            // writes one 128-byte row segment (scattered 16-byte pieces ran at a fraction of the rate)
+                            float (*xp)[33] = xpose[warp - 2];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) xp[lane][i] = __uint_as_float(v[i]);
+                            __syncwarp();
+                            const int col = nt * p.NT + cc + lane;
+                            const int rows_here = min(32, a_rows - q * 32);
+                            if (col < p.Ng) {
+                                float *dst = Gn + (long long)(mt * 128 + q * 32) * p.Ng + col;
+                                for (int r = 0; r < rows_here; ++r) __stcs(dst + (long long)r * p.Ng, xp[r][lane]);
+                            }
+                            __syncwarp();
                         }
                     }
                     tc_fence_before();
@@ -635,30 +640,39 @@ static TcProblem tc_problem(int dtype, const ConvGeom &g) {
     return pr;
 }
 
-// cycles of one MMA step (one instruction): tensor pipe (N/2) against shared-memory operand reads (4 KB of A + N*32 B of B at 128 B/clk)
-static int step_cycles(int n_cols) {
-    const int pipe = n_cols / 2, smem = 32 + n_cols / 4;
-    return pipe > smem ? pipe : smem;
+// Cycle model of one MMA step (16 bf16 / 8 tf32 reduction rows) for the tiling search.  Measured on B200: an
+// instruction occupies the tensor pipe for N/2 cycles, and shared memory moves 128 B per cycle in total, shared by
+// the tensor core's operand reads (always 128 rows of A plus N rows of B, 32 B per row and step), the TMA fill of the
+// stage and, for split tf32, the split warps (they read every landed byte once and write the lo copy).
+static double step_cycles(bool bf16, int n_cols, double a_slabs_loaded, double b_slabs) {
+    if (bf16) {
+        const double smem = 4096.0 + 32.0 * n_cols + 2048.0 * (a_slabs_loaded + b_slabs);
+        return std::max(n_cols / 2.0, smem / 128.0);
+    }
+    const double smem = 3.0 * (4096.0 + 32.0 * n_cols) + 1024.0 * (a_slabs_loaded + b_slabs) * 3.0;
+    return std::max(3.0 * n_cols / 2.0, smem / 128.0);
 }
 
-static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt);
+static TcPlan search_plan(int dtype, const ConvGeom &g, int mode);
 
 // The tiling search is pure; its results are memoised per layer geometry (host side only).
-static TcPlan make_plan(int dtype, const ConvGeom &g, int max_nt = 256) {
+// mode: 0 gradients are stored, 1 norms only, 2 clipped sum (running sum in registers: at most 128 columns per tile)
+static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
     static std::mutex mu;
     static std::map<std::array<int, 11>, TcPlan> memo;
-    const std::array<int, 11> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, max_nt};
+    const std::array<int, 11> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, mode};
     std::lock_guard<std::mutex> lock(mu);
     auto it = memo.find(key);
     if (it != memo.end()) return it->second;
-    const TcPlan pl = search_plan(dtype, g, max_nt);
+    const TcPlan pl = search_plan(dtype, g, mode);
     memo.emplace(key, pl);
     return pl;
 }
 
 // max_nt = 128 plans the clipped-sum mode: its running sum lives in registers (128 columns per thread) and the
 // work items are (example range, tile) pairs, so the wave count no longer depends on the batch size
-static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
+static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
+    const int max_nt = (mode == 2) ? 128 : 256;
     TcPlan best; best.ok = false;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
@@ -667,7 +681,6 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
     const int sms = sm_count();
     const int a_slabs_tile = 128 / slab_ch;
     const int copies = (dtype == DP_BF16) ? 1 : 2;      // split tf32 keeps a hi and a lo copy of every stage
-    const int mma_per_step = (dtype == DP_BF16) ? 1 : 3;
     double best_cost = 1e300;
     for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
         const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
@@ -679,8 +692,14 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
             const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
             if (total_tiles > 0x7fffffffLL) continue;
             // per-CTA share of (example, tile) units: whole waves of tiles, or in clipped-sum mode an even share of the examples
-            const double waves = (max_nt == 256) ? (double)((total_tiles + sms - 1) / sms)
-                                                 : std::max(1.0, (double)total_tiles / sms);
+            const double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
+                                             : std::max(1.0, (double)total_tiles / sms);
+            const double a_loaded = (double)(a_ext / slab_ch) / m_tiles, b_loaded = (double)(b_ext / slab_ch) / n_tiles;
+            const double step = step_cycles(dtype == DP_BF16, NT, a_loaded, b_loaded);
+            // the epilogue of a tile overlaps the main loop of the next; what it costs depends on what it does with
+            // the 128 x NT accumulator: stores run at about 16 B/clk per SM when lanes write consecutive addresses
+            // (rows of D are gradient columns) and about 7 B/clk otherwise; reading TMEM alone is cheap
+            const double epilogue = (mode == 0) ? 128.0 * NT * 4.0 / (a_is_x ? 16.0 : 7.0) : (mode == 1 ? 6.0 * NT : 10.0 * NT);
             for (int OHt = 1; OHt <= g.OH; ++OHt) {
                 if (OHt * g.stride > 256 || OHt * g.stride > g.H) break;
                 for (int OWt = 1; OWt <= g.OW; ++OWt) {
@@ -692,11 +711,11 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
                     if (stages < 2) continue;
                     if (stages > kMaxStages) stages = kMaxStages;
                     const int tw = (g.OW + OWt - 1) / OWt, th = (g.OH + OHt - 1) / OHt;
-                    // a stage costs the larger of its tensor time and the fixed hand-over work of the issuing threads
-                    const double stage_cost = std::max((double)(Kt / krows) * step_cycles(NT) * mma_per_step, 450.0);
-                    double tile_cost = stage_cost * tw * th + 600.0;
-                    if (stages < 3) tile_cost *= 1.3;
-                    const double cost = tile_cost * waves;
+                    // a stage: its MMA steps plus the hand-over (barrier wait, commit) of the issuing thread
+                    const double stage_cost = (double)(Kt / krows) * step + 250.0;
+                    double mainloop = stage_cost * tw * th;
+                    if (stages < 3) mainloop *= 1.15;
+                    const double cost = (std::max(mainloop, epilogue) + 300.0) * waves;
                     if (cost < best_cost) {
                         best_cost = cost;
                         best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
@@ -715,8 +734,8 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int max_nt) {
 
 bool tc_eligible(int dtype, const ConvGeom &g0, int epilogue) {
     const TcProblem pr = tc_problem(dtype, g0);
-    if (!pr.ok || !encode_fn() || !make_plan(dtype, pr.eff).ok) return false;
-    return epilogue != DP_EPI_CLIP_ACCUM || make_plan(dtype, pr.eff, 128).ok;
+    if (!pr.ok || !encode_fn() || !make_plan(dtype, pr.eff, epilogue == DP_EPI_STORE_NORM ? 0 : 1).ok) return false;
+    return epilogue != DP_EPI_CLIP_ACCUM || make_plan(dtype, pr.eff, 2).ok;
 }
 
 // clipped-sum mode: how many example ranges each tile is cut into so that every SM has an item
@@ -729,10 +748,10 @@ static void clip_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &pe
     splits = (g.B + per_split - 1) / per_split;
 }
 
-int tc_norm_slots(int dtype, const ConvGeom &g0, int) {
+int tc_norm_slots(int dtype, const ConvGeom &g0, int epilogue) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
-    const TcPlan pl = make_plan(dtype, pr.eff);
+    const TcPlan pl = make_plan(dtype, pr.eff, epilogue == DP_EPI_STORE_NORM ? 0 : 1);
     return pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
 }
 
@@ -747,7 +766,7 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
     if (!pr.ok) return 0;
     size_t bytes = unfold_bytes(dtype, g0, pr);
     if (epilogue == DP_EPI_CLIP_ACCUM) {
-        const TcPlan pl = make_plan(dtype, pr.eff, 128);
+        const TcPlan pl = make_plan(dtype, pr.eff, 2);
         if (!pl.ok) return 0;
         int splits, per;
         clip_split(pr.eff, pl, splits, per);
@@ -759,7 +778,7 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
 int tc_describe_plan(int dtype, const ConvGeom &g0, int *out, int n) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
-    const TcPlan pl = make_plan(dtype, pr.eff);
+    const TcPlan pl = make_plan(dtype, pr.eff, 0);
     if (!pl.ok) return 0;
     const int v[12] = {pl.a_is_x, pl.a_ext, pl.b_ext, pl.m_tiles, pl.n_tiles, pl.NT, pl.OWt, pl.OHt, pl.Kt, pl.k_tiles,
                        pl.stages, pl.stage_bytes};
@@ -790,7 +809,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok || !encode_fn()) return DP_ERR_UNSUPPORTED;
     const ConvGeom &g = pr.eff;
-    const TcPlan pl = make_plan(dtype, g, clip ? 128 : 256);
+    const TcPlan pl = make_plan(dtype, g, clip ? 2 : (epilogue == DP_EPI_STORE_NORM ? 0 : 1));
     if (!pl.ok) return DP_ERR_UNSUPPORTED;
     char *ws_bytes = static_cast<char *>(tc_workspace);
     if (pr.unfold) {
