@@ -502,17 +502,17 @@ norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, in
         }
     }
     __syncthreads();
-    if (prow == 0 && c0 < C) {
+    // every thread folds one output column over the pixel rows, in row order
+    {
         float *out = chunk_partial + (((long long)n * chunks + chunk) * 2) * C;
-#pragma unroll
-        for (int v = 0; v < VEC; ++v) {
-            float a = 0.f, b = 0.f;
-            for (int rr = 0; rr < rows; ++rr) {
-                a += red[rr * width + cvi * VEC + v];
-                b += red[rr * width + tcv * VEC + cvi * VEC + v];
-            }
-            out[c0 + v] = a;
-            out[C + c0 + v] = b;
+        const int half = tcv * VEC;
+        for (int e = threadIdx.x; e < 2 * half; e += 256) {
+            const int is_beta = e >= half;
+            const int c = blockIdx.x * half + (is_beta ? e - half : e);
+            if (c >= C) continue;
+            float a = 0.f;
+            for (int rr = 0; rr < rows; ++rr) a += red[rr * width + e];
+            out[is_beta ? C + c : c] = a;
         }
     }
 }
