@@ -211,6 +211,8 @@ class FlatGrad:
         self.torch, self.synth, self.dist, self.world = torch, synth, dist, world
         self.cfg = synth.resnet50_flat()
         self.P, self.B, self.G = self.cfg["P"], self.cfg["B"], self.cfg["G"]
+        if os.environ.get("DPSTEP_FLAT_PARAMS"):          # reduced P for profiler captures (same kernels, fewer bytes held)
+            self.P = int(os.environ["DPSTEP_FLAT_PARAMS"])
         self.step_obj = FlatClipStep(self.P, self.B, self.cfg["C"], self.cfg["sigma"])
         self.examples_per_step = self.B * self.G
         g = torch.Generator(device="cuda"); g.manual_seed(2000 + rank)
@@ -222,7 +224,7 @@ class FlatGrad:
         self.call_names = ["clip_accumulate(norms computed)", "noise_average"]
 
     def describe(self):
-        return {"workload": "flat: ResNet-50 (GroupNorm) flattened per-example gradients, P=25,557,032 fp32 ~N(0,1e-6), "
+        return {"workload": f"flat: ResNet-50 (GroupNorm) flattened per-example gradients, P={self.P:,} fp32 ~N(0,1e-6), "
                             "B=64 per chunk x 16 chunks = |B| 1024, global clip C=1.0, sigma=1.0; norms computed by the library",
                 "examples_per_step": self.examples_per_step, "params": self.P,
                 "l2": "each chunk is 6.54 GB, far larger than L2; two resident chunks alternate"}
