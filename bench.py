@@ -41,6 +41,30 @@ def measured_peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+def source_fingerprint():
+    """sha1 over the CUDA sources: ncu traffic figures are only quoted while the kernels they were taken on are unchanged."""
+    import glob
+    import hashlib
+    h = hashlib.sha1()
+    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2109_12191_b200", "csrc", "*.cu*"))):
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(workload, call_name):
+    """DRAM bytes (read + write) per launch of `call_name` from the committed ncu capture, or None when there is no
+    capture for it or the sources have changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", f"traffic_{workload}.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f)
+    if rec.get("source_sha1") != source_fingerprint():
+        return None
+    return rec.get("dram_bytes_per_launch", {}).get(call_name)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -521,7 +545,8 @@ def run_ours(args):
     achieved = wl.algorithmic_bytes(dom) / (avg_ms / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": wl.call_names[dom], "achieved": round(achieved, 1), "peak": peaks["hbm"],
                 "peak_source": peaks["source"], "unit": "GB/s", "frac": round(achieved / peaks["hbm"], 4),
-                "avg_ms_per_launch": round(avg_ms, 5), "traffic": None,
+                "avg_ms_per_launch": round(avg_ms, 5), "algorithmic_bytes": wl.algorithmic_bytes(dom),
+                "traffic": recorded_traffic(wl.name, wl.call_names[dom]),
                 "shares": {n: round(t / sum(totals), 4) for n, t in zip(wl.call_names, totals)}}
     if hasattr(wl, "roofline"):
         own = wl.roofline(dom, totals[dom] / (max(1, counts[4]) * wl.G), peaks)

@@ -185,10 +185,9 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             rc = launch_dense_store(d->dtype, X, dY, d->B, d->C_in, d->K_out, G_w, d->has_bias ? G_b : nullptr, st);
             if (rc != DP_OK) return rc;
         }
-        rc = launch_dense_norm(d->dtype, X, dY, d->B, d->C_in, d->K_out, d->has_bias, partial,
-                               (clip && d->has_bias) ? db_ws : nullptr, st);
-        if (rc != DP_OK) return rc;
-        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st, reset);
+        float *db_dst = !d->has_bias ? nullptr : (epi == DP_EPI_STORE_NORM ? G_b : (clip ? db_ws : nullptr));
+        rc = launch_dense_norm(d->dtype, X, dY, d->B, d->C_in, d->K_out, d->has_bias, db_dst, groups == 2, sqnorm,
+                               sqnorm_stride, clip, C_l, factor, clip_out, reset, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
         rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, 2, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);

@@ -194,13 +194,33 @@ conv_wgrad_thin_kernel(const T *__restrict__ X, const T *__restrict__ dY, const 
             if constexpr (RT > 0) {
                 const float *patch = xs + base[u];
                 const int row_p = Wp * g.Cin;
+                // the whole warp reads the same patch (broadcast); 64-bit loads halve the shared-memory instructions,
+                // with the pairing chosen by the parity of the patch start (the same for every lane and every row)
+                const bool pairs = ((row_p | SCT) & 1) != 0 ? ((row_p & 1) == 0) : true;
+                const int lead = (base[u] & 1);          // 1: element 0 is unaligned, pairs start at element 1
 #pragma unroll
                 for (int r = 0; r < RT; ++r) {
+                    float x[SCT];
+                    const float *row = patch + r * row_p;
+                    if (pairs && (row_p & 1) == 0) {
+                        if (lead == 0) {
+#pragma unroll
+                            for (int t = 0; t + 1 < SCT; t += 2) { const float2 v = *reinterpret_cast<const float2 *>(row + t); x[t] = v.x; x[t + 1] = v.y; }
+                            if (SCT & 1) x[SCT - 1] = row[SCT - 1];
+                        } else {
+                            x[0] = row[0];
+#pragma unroll
+                            for (int t = 1; t + 1 < SCT; t += 2) { const float2 v = *reinterpret_cast<const float2 *>(row + t); x[t] = v.x; x[t + 1] = v.y; }
+                            if (!(SCT & 1)) x[SCT - 1] = row[SCT - 1];
+                        }
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < SCT; ++t) x[t] = row[t];
+                    }
 #pragma unroll
                     for (int t = 0; t < SCT; ++t) {
-                        const float x = patch[r * row_p + t];
 #pragma unroll
-                        for (int kk = 0; kk < KPT; ++kk) acc[kk][r * SCT + t] = fmaf(gy[u][kk], x, acc[kk][r * SCT + t]);
+                        for (int kk = 0; kk < KPT; ++kk) acc[kk][r * SCT + t] = fmaf(gy[u][kk], x[t], acc[kk][r * SCT + t]);
                     }
                 }
             } else {
@@ -419,21 +439,43 @@ __global__ void widen_kernel(const T *__restrict__ src, long long count, float *
     if (i < count) dst[i] = to_float(src[i]);
 }
 
-// rank-1 closed form: |dY_n^T X_n|_F^2 = |dY_n|^2 |X_n|^2, bias part |dY_n|^2
+// Dense layer, everything but the outer-product store, one block per example: the rank-1 closed form of the squared
+// norm (|dY_n^T X_n|_F^2 = |dY_n|^2 |X_n|^2, bias part |dY_n|^2), the bias gradient db_n = dY_n widened to fp32 (when
+// a destination is given), and the same publishing of norms / clip factors the convolution paths do in a kernel of its own.
 template <typename T>
 __global__ void __launch_bounds__(256)
-dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, int Kout, int has_bias,
-                  float *__restrict__ partial) {
+dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, int Kout, int has_bias, float *__restrict__ db,
+                  int separate, float *__restrict__ sqnorm, long long sq_stride, int clip, float C_l,
+                  float *__restrict__ factor, float *clip_out, int *status_reset) {
     __shared__ double scratch[32];
     const int n = blockIdx.x;
+    if (status_reset && n == 0 && threadIdx.x == 0) *status_reset = 0;
     double sx = 0.0, sy = 0.0;
     for (int i = threadIdx.x; i < Cin; i += 256) { const double v = to_float(X[(long long)n * Cin + i]); sx += v * v; }
-    for (int i = threadIdx.x; i < Kout; i += 256) { const double v = to_float(dY[(long long)n * Kout + i]); sy += v * v; }
+    for (int i = threadIdx.x; i < Kout; i += 256) {
+        const float g = to_float(dY[(long long)n * Kout + i]);
+        if (db) db[(long long)n * Kout + i] = g;
+        sy += (double)g * g;
+    }
     sx = block_sum(sx, scratch);
     sy = block_sum(sy, scratch);
-    if (threadIdx.x == 0) {
-        partial[2 * n] = (float)(sx * sy);
-        partial[2 * n + 1] = has_bias ? (float)sy : 0.f;
+    if (threadIdx.x != 0) return;
+    const double sw = sx * sy, sb = has_bias ? sy : 0.0;
+    if (separate) {
+        sqnorm[n * sq_stride] = (float)sw;
+        sqnorm[n * sq_stride + 1] = (float)sb;
+        if (clip) {
+            const float fw = clip_factor(sw, C_l), fb = clip_factor(sb, C_l);
+            factor[2 * n] = fw; factor[2 * n + 1] = fb;
+            if (clip_out) { clip_out[2 * n] = fw; clip_out[2 * n + 1] = fb; }
+        }
+    } else {
+        sqnorm[n * sq_stride] = (float)(sw + sb);
+        if (clip) {
+            const float f = clip_factor(sw + sb, C_l);
+            factor[2 * n] = f; factor[2 * n + 1] = f;
+            if (clip_out) clip_out[n] = f;
+        }
     }
 }
 
@@ -699,11 +741,7 @@ static dp_status dense_store_t(const T *X, const T *dY, int B, int Cin, int Kout
     if (vec) dense_store_kernel<T, true><<<(unsigned)blocks, 256, 0, st>>>(X, dY, Cin, Kout, per_block, rows, G_w);
     else dense_store_kernel<T, false><<<(unsigned)blocks, 256, 0, st>>>(X, dY, Cin, Kout, per_block, rows, G_w);
     DP_LAUNCH_CHECK("dense_store_kernel");
-    if (G_b) {
-        const long long cnt = (long long)B * Kout;
-        widen_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(dY, cnt, G_b);
-        DP_LAUNCH_CHECK("widen_kernel");
-    }
+    (void)G_b;      // the bias gradient is written by the norm kernel that every dense call runs
     return DP_OK;
 }
 
@@ -713,18 +751,16 @@ dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, in
     return dense_store_t(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, Cin, Kout, G_w, G_b, st);
 }
 
-dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias,
-                            float *partial, float *db, cudaStream_t st) {
-    const long long cnt = (long long)B * Kout;
-    if (dtype == DP_F32) {
-        dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), Cin, Kout, has_bias, partial);
-        DP_LAUNCH_CHECK("dense_norm_kernel");
-        if (db) { widen_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(static_cast<const float *>(dY), cnt, db); DP_LAUNCH_CHECK("widen_kernel"); }
-    } else {
-        dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), Cin, Kout, has_bias, partial);
-        DP_LAUNCH_CHECK("dense_norm_kernel");
-        if (db) { widen_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), cnt, db); DP_LAUNCH_CHECK("widen_kernel"); }
-    }
+dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias, float *db,
+                            int separate, float *sqnorm, long long sq_stride, int clip, float C_l, float *factor,
+                            float *clip_out, int *status_reset, cudaStream_t st) {
+    if (dtype == DP_F32)
+        dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), Cin, Kout, has_bias, db,
+                                             separate, sqnorm, sq_stride, clip, C_l, factor, clip_out, status_reset);
+    else
+        dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), Cin, Kout,
+                                             has_bias, db, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out, status_reset);
+    DP_LAUNCH_CHECK("dense_norm_kernel");
     return DP_OK;
 }
 

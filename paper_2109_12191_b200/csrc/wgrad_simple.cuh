@@ -43,9 +43,10 @@ dp_status launch_bias_accum(const float *db, int B, int Kout, const float *facto
 
 dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, float *G_w,
                              float *G_b, cudaStream_t stream);
-// writes partial[n*2+0] = |dY_n|^2 |X_n|^2 and partial[n*2+1] = |dY_n|^2 (0 without bias); db (optional) = dY as fp32
-dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias,
-                            float *partial, float *db, cudaStream_t stream);
+// closed-form squared norms (|dY_n|^2 |X_n|^2 and |dY_n|^2), db = dY as fp32 (optional), norms and clip factors published
+dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias, float *db,
+                            int separate, float *sqnorm, long long sq_stride, int clip, float C_l, float *factor,
+                            float *clip_out, int *status_reset, cudaStream_t stream);
 
 // stage 1: per pixel-chunk partial sums; stage 2: fold, store, squared norms into partial2[n*2 + {0,1}]
 dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
