@@ -144,11 +144,10 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
     const ConvGeom g = geom_of(d);
     const int clip = (epi == DP_EPI_CLIP_ACCUM);
     dp_status rc;
-    // Tensor-core launches may set the status word (bounded waits), so it is cleared before them; every other
-    // path has no waits and lets its last small kernel write "ok" instead of paying for a memset node.
+    // Tensor-core launches may set the status word (bounded waits): the first of them clears it on entry.  Every
+    // other path has no waits and lets its last small kernel write "ok".  Neither pays for a memset node.
     int *status_word = reinterpret_cast<int *>(ws + pl.status_off);
     int *reset = pl.use_tc ? nullptr : status_word;
-    if (pl.use_tc) DP_CUDA_TRY(cudaMemsetAsync(ws + pl.status_off, 0, 16, st));
 
     if (d->kind == DP_LAYER_CONV2D) {
         float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;

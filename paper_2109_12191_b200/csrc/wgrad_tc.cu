@@ -55,6 +55,7 @@ struct TcParams {
     float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
     int slots;
     int *status;
+    int reset_status;           // 1: this launch is the first of its call and clears the status word itself
     int total_tiles;            // work items: (example, tile) pairs, or (example range, tile) pairs in mode 2
     // mode 2: item = (split, tile); the CTA walks examples [split*per_split, ...) and keeps sum_n f_n D_n in registers
     int splits, per_split;
@@ -182,6 +183,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const uint32_t tiles_u32 = smem_u32(tiles);
 
     if (threadIdx.x == 0) {
+        // a wait can only expire seconds from now, long after this store, so clearing here cannot hide a time-out
+        if (blockIdx.x == 0 && p.reset_status) *p.status = 0;
         // pull both tensor maps into the TMA descriptor cache before the first copy needs them
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
@@ -803,7 +806,7 @@ static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, in
 
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g_in, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace, int *status,
-                         cudaStream_t stream, bool skip_unfold) {
+                         cudaStream_t stream, bool second_pass) {
     const bool clip = epilogue == DP_EPI_CLIP_ACCUM;
     const ConvGeom &g0 = g_in;
     const TcProblem pr = tc_problem(dtype, g0);
@@ -815,7 +818,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     if (pr.unfold) {
         // in a fused clip call this function runs twice (norm pass, then clipped-sum pass): the unfolded input is
         // rebuilt only by the first of them
-        if (!(clip && skip_unfold)) {
+        if (!(clip && second_pass)) {
             const int vec = (dtype == DP_BF16) ? 8 : 4;
             const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / vec);
             const unsigned blocks = (unsigned)((total + 255) / 256);
@@ -852,6 +855,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.lo_offset = pl.stage_bytes / 2;
     p.mode = clip ? 2 : (epilogue == DP_EPI_STORE_NORM ? 0 : 1);
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
+    p.reset_status = second_pass ? 0 : 1;       // the second launch of a fused clip call must keep the first one's verdict
     p.splits = 1; p.per_split = g.B; p.factor = factor; p.sum_out = acc_w;
     if (clip) {
         clip_split(g, pl, p.splits, p.per_split);

@@ -16,6 +16,6 @@ int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n);
 // epilogue as dp_epilogue; factor[n*2] scales example n (CLIP_ACCUM); status: device word set to nonzero on a timed-out wait
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace,
-                         int *status, cudaStream_t stream, bool skip_unfold = false);
+                         int *status, cudaStream_t stream, bool second_pass = false);
 
 }  // namespace dp
