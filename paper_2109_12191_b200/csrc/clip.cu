@@ -285,12 +285,11 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
     // tensors go to the kernels in tables of at most kMaxSeg entries
     // few wide blocks and many rows: use the row-split kernel (needs aligned rows everywhere)
     long long wide_blocks = 0;
-    bool all_vec = true;
-    for (int l = 0; l < L; ++l) {
-        wide_blocks += (P_l[l] + kAccCols - 1) / kAccCols;
-        if ((P_l[l] & 3) || !aligned(G[l], 16) || !aligned(acc[l], 16)) all_vec = false;
-    }
-    const bool row_split = all_vec && B >= 16 && wide_blocks < 4 * 148;
+    for (int l = 0; l < L; ++l) wide_blocks += (P_l[l] + kAccCols - 1) / kAccCols;
+    const bool row_split = false;    // kept for reference measurements; the deep-unroll kernel below is faster
+    // A small model gives few blocks, and each thread then walks all B rows in B/UNROLL dependent trips of one
+    // memory latency each: with many rows, 32 rows in flight per thread instead of 8 quarters that chain.
+    const bool deep = B >= 64 && wide_blocks < 8 * 148;
     const int acc_cols = row_split ? 256 : kAccCols;
 
     auto fill = [&](int l0, SegTable &t, bool norm_blocks, long long &part_cursor) {
@@ -338,6 +337,7 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
             const int blocks = fill(l0, t, false, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
             if (row_split) scale_accumulate_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
+            else if (deep) scale_accumulate_kernel<32><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             else scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             DP_LAUNCH_CHECK("scale_accumulate_kernel");
             l0 += t.nseg;

@@ -190,7 +190,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 8);
+            mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 4);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -315,8 +315,12 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         // ------------------------------------------------------------ split warps (fp32 inputs only)
         // hi stays where TMA put it, lo goes to the same offset of the stage's second half; both keep the
         // swizzled layout because the split is element-wise on identical relative addresses.
-        const int tid = threadIdx.x - 192;
+        // The eight warps work as two groups of four that take alternate stages, so the proxy fence that ends one
+        // group's stage (it waits for that group's stores to drain) overlaps the other group's loads and stores.
+        const int group = (warp - 6) >> 2;
+        const int tid = (threadIdx.x - 192) & 127;
         int stage = 0; uint32_t phase = 0;
+        int turn = 0;                       // global stage counter modulo 2: whose stage is it
         bool live = true;
         for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
             const Item it = decode_item(p, item);
@@ -325,36 +329,38 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const int a_chunks = a_slabs * (slab_bytes >> 4), chunks = a_chunks + b_slabs * (slab_bytes >> 4);
             const int stage_count = (it.n_hi - it.n_lo) * p.k_tiles;
             for (int kt = 0; kt < stage_count; ++kt) {
-                const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p);
-                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
-                uint8_t *base = tiles + (size_t)stage * p.stage_bytes;
-                // eight warps (the issue rate of the split is what bounds fp32 layers); four 16-byte groups per
-                // thread and trip with all loads first, A region and B region in turn
-                for (int region = 0; region < 2; ++region) {
-                    uint8_t *rbase = region ? base + p.a_bytes : base;
-                    const int rchunks = region ? chunks - a_chunks : a_chunks;
-                    for (int i0 = tid; i0 < rchunks; i0 += 1024) {
-                        float4 x[4];
+                if (turn == group) {
+                    const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p);
+                    if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+                    uint8_t *base = tiles + (size_t)stage * p.stage_bytes;
+                    // four 16-byte groups per thread and trip with all loads first, A region and B region in turn
+                    for (int region = 0; region < 2; ++region) {
+                        uint8_t *rbase = region ? base + p.a_bytes : base;
+                        const int rchunks = region ? chunks - a_chunks : a_chunks;
+                        for (int i0 = tid; i0 < rchunks; i0 += 512) {
+                            float4 x[4];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (i0 + 256 * u < rchunks) x[u] = *reinterpret_cast<const float4 *>(rbase + ((size_t)(i0 + 256 * u) << 4));
+                            for (int u = 0; u < 4; ++u)
+                                if (i0 + 128 * u < rchunks) x[u] = *reinterpret_cast<const float4 *>(rbase + ((size_t)(i0 + 128 * u) << 4));
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (i0 + 256 * u < rchunks) {
-                                uint8_t *ptr = rbase + ((size_t)(i0 + 256 * u) << 4);
-                                float4 hi, lo;
-                                hi.x = __uint_as_float(__float_as_uint(x[u].x) & 0xFFFFE000u); lo.x = x[u].x - hi.x;
-                                hi.y = __uint_as_float(__float_as_uint(x[u].y) & 0xFFFFE000u); lo.y = x[u].y - hi.y;
-                                hi.z = __uint_as_float(__float_as_uint(x[u].z) & 0xFFFFE000u); lo.z = x[u].z - hi.z;
-                                hi.w = __uint_as_float(__float_as_uint(x[u].w) & 0xFFFFE000u); lo.w = x[u].w - hi.w;
-                                *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;     // x stays: truncated by the MMA itself, it is hi
+                            for (int u = 0; u < 4; ++u) {
+                                if (i0 + 128 * u < rchunks) {
+                                    uint8_t *ptr = rbase + ((size_t)(i0 + 128 * u) << 4);
+                                    float4 hi, lo;
+                                    hi.x = __uint_as_float(__float_as_uint(x[u].x) & 0xFFFFE000u); lo.x = x[u].x - hi.x;
+                                    hi.y = __uint_as_float(__float_as_uint(x[u].y) & 0xFFFFE000u); lo.y = x[u].y - hi.y;
+                                    hi.z = __uint_as_float(__float_as_uint(x[u].z) & 0xFFFFE000u); lo.z = x[u].z - hi.z;
+                                    hi.w = __uint_as_float(__float_as_uint(x[u].w) & 0xFFFFE000u); lo.w = x[u].w - hi.w;
+                                    *reinterpret_cast<float4 *>(ptr + p.lo_offset) = lo;     // x stays: truncated by the MMA itself, it is hi
+                                }
                             }
                         }
                     }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ready_bar[stage]));
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ready_bar[stage]));
+                turn ^= 1;
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
@@ -715,7 +721,11 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
                     if (stages > kMaxStages) stages = kMaxStages;
                     const int tw = (g.OW + OWt - 1) / OWt, th = (g.OH + OHt - 1) / OHt;
                     // a stage: its MMA steps plus the hand-over (barrier wait, commit) of the issuing thread
-                    const double stage_cost = (double)(Kt / krows) * step + 250.0;
+                    double stage_cost = (double)(Kt / krows) * step + 250.0;
+                    // the TMA warp: barrier wait + expect_tx, then one copy per slab, all latency-bound on one warp
+                    stage_cost = std::max(stage_cost, 350.0 + 110.0 * (a_loaded + b_loaded));
+                    if (dtype != DP_BF16)   // split warps, two groups in turn: a fixed fence/hand-over plus their share of the bytes
+                        stage_cost = std::max(stage_cost, 0.5 * (1000.0 + (a_loaded + b_loaded) * Kt * 2.5));
                     double mainloop = stage_cost * tw * th;
                     if (stages < 3) mainloop *= 1.15;
                     const double cost = (std::max(mainloop, epilogue) + 300.0) * waves;
