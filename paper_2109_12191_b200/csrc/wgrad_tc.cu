@@ -9,7 +9,7 @@
 // 128 bytes with the 128-byte swizzle, which is exactly the canonical MN-major operand slab; the tap
 // shift and the zero padding come from the box start coordinate and TMA's out-of-bounds zero fill.
 //
-// Roles (192 threads): warp 0 issues TMA loads, warp 1 allocates TMEM and issues tcgen05.mma,
+// Roles (224 threads): warps 0 and 6 issue TMA loads (A and B slabs), warp 1 allocates TMEM and issues tcgen05.mma,
 // warps 2-5 read accumulators back with tcgen05.ld, square-sum them (the per-example norm) and store.
 // Two accumulator buffers in TMEM let the epilogue of one tile overlap the main loop of the next.
 // Every wait is bounded: on expiry the CTA sets a status word, drains and returns.
@@ -170,7 +170,7 @@ __device__ __forceinline__ uint32_t instr_desc(int n_cols, uint32_t fmt) {
 }
 
 template <bool TF32, bool CLIP>
-__global__ void __launch_bounds__(TF32 ? 448 : 192, 1)
+__global__ void __launch_bounds__(TF32 ? 480 : 224, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], ready_bar[kMaxStages], tmem_full[2], tmem_empty[2];
@@ -190,7 +190,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 4);
+            mbar_init(smem_u32(&full_bar[s]), 2); mbar_init(smem_u32(&empty_bar[s]), 1); mbar_init(smem_u32(&ready_bar[s]), 4);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -205,10 +205,12 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const int slab_bytes = p.Kt * kRowBytes;
     const int a_slabs_tile = 128 / p.slab_ch, b_slabs_tile = p.NT / p.slab_ch;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        // Lane L owns slab L of the stage (A slabs first, then B slabs): it works out its tap shift and channel
-        // offset once per tile and then only adds the pixel-tile origin, so no division sits in the stage loop.
+    if (warp == 0 || warp == 6) {
+        // ------------------------------------------------------------ TMA producers
+        // Two warps, because issuing a copy costs the issuing warp ~100 cycles: warp 0 loads the A slabs of every
+        // stage, warp 6 the B slabs; each announces its own bytes on the stage's full barrier (two arrivals).
+        // Lane L owns slab L: it works out its tap shift and channel offset once per tile and then only adds the
+        // pixel-tile origin, so no division sits in the stage loop.
         int stage = 0; uint32_t phase = 0;
         bool live = true;
         for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
@@ -216,8 +218,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const int mt = it.mt, nt = it.nt;
             const int a_slab0 = mt * a_slabs_tile, a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - a_slab0);
             const int b_slab0 = nt * b_slabs_tile, b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - b_slab0);
-            const bool is_a = lane < a_slabs_tile;
-            const int local = is_a ? lane : lane - a_slabs_tile;
+            const bool is_a = warp == 0;
+            const int local = lane;
             const bool active = is_a ? (local < a_slabs) : (local < b_slabs);
             const bool is_x = is_a ? (p.a_is_x != 0) : (p.a_is_x == 0);
             const int slab = (is_a ? a_slab0 : b_slab0) + local;
@@ -235,7 +237,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             }
             const CUtensorMap *map = is_x ? &tmX : &tmY;
             const uint32_t dst_off = (is_a ? 0u : (uint32_t)p.a_bytes) + (uint32_t)(local * slab_bytes);
-            const uint32_t tx_bytes = (uint32_t)((a_slabs + b_slabs) * slab_bytes);
+            const uint32_t tx_bytes = (uint32_t)((is_a ? a_slabs : b_slabs) * slab_bytes);
             for (int n = it.n_lo; n < it.n_hi && live; ++n) {
                 int ow0 = 0, oh0 = 0, tw = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
@@ -311,14 +313,14 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
               }
             }
         }
-    } else if (TF32 && warp >= 6) {
+    } else if (TF32 && warp >= 7) {
         // ------------------------------------------------------------ split warps (fp32 inputs only)
         // hi stays where TMA put it, lo goes to the same offset of the stage's second half; both keep the
         // swizzled layout because the split is element-wise on identical relative addresses.
         // The eight warps work as two groups of four that take alternate stages, so the proxy fence that ends one
         // group's stage (it waits for that group's stores to drain) overlaps the other group's loads and stores.
-        const int group = (warp - 6) >> 2;
-        const int tid = (threadIdx.x - 192) & 127;
+        const int group = (warp - 7) >> 2;
+        const int tid = (threadIdx.x - 224) & 127;
         int stage = 0; uint32_t phase = 0;
         int turn = 0;                       // global stage counter modulo 2: whose stage is it
         bool live = true;
@@ -364,7 +366,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
-    } else {
+    } else if (warp >= 2 && warp <= 5) {
         // ------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
         const int q = warp & 3;
         const int row = q * 32 + lane;
@@ -722,8 +724,8 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
                     const int tw = (g.OW + OWt - 1) / OWt, th = (g.OH + OHt - 1) / OHt;
                     // a stage: its MMA steps plus the hand-over (barrier wait, commit) of the issuing thread
                     double stage_cost = (double)(Kt / krows) * step + 250.0;
-                    // the TMA warp: barrier wait + expect_tx, then one copy per slab, all latency-bound on one warp
-                    stage_cost = std::max(stage_cost, 350.0 + 110.0 * (a_loaded + b_loaded));
+                    // a TMA warp: barrier wait + expect_tx, then one copy per slab it owns (A or B), all latency-bound on that warp
+                    stage_cost = std::max(stage_cost, 350.0 + 110.0 * std::max(a_loaded, b_loaded));
                     if (dtype != DP_BF16)   // split warps, two groups in turn: a fixed fence/hand-over plus their share of the bytes
                         stage_cost = std::max(stage_cost, 0.5 * (1000.0 + (a_loaded + b_loaded) * Kt * 2.5));
                     double mainloop = stage_cost * tw * th;
@@ -886,11 +888,11 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
     const unsigned grid = (unsigned)std::min(p.total_tiles, sm_count());
     if (dtype == DP_BF16) {
-        if (clip) conv_wgrad_tc_kernel<false, true><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
-        else conv_wgrad_tc_kernel<false, false><<<grid, 192, pl.smem, stream>>>(tmX, tmY, p);
+        if (clip) conv_wgrad_tc_kernel<false, true><<<grid, 224, pl.smem, stream>>>(tmX, tmY, p);
+        else conv_wgrad_tc_kernel<false, false><<<grid, 224, pl.smem, stream>>>(tmX, tmY, p);
     } else {
-        if (clip) conv_wgrad_tc_kernel<true, true><<<grid, 448, pl.smem, stream>>>(tmX, tmY, p);
-        else conv_wgrad_tc_kernel<true, false><<<grid, 448, pl.smem, stream>>>(tmX, tmY, p);
+        if (clip) conv_wgrad_tc_kernel<true, true><<<grid, 480, pl.smem, stream>>>(tmX, tmY, p);
+        else conv_wgrad_tc_kernel<true, false><<<grid, 480, pl.smem, stream>>>(tmX, tmY, p);
     }
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
     if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g0.M * g0.N, acc_w, stream);
