@@ -170,6 +170,11 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
         else rc = launch_conv_fma(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
         if (rc != DP_OK) return rc;
+        if (pl.use_tc && !d->has_bias) {
+            // no bias: the clipped-sum pass finalises the norms itself
+            const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
+            return launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, nullptr, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true, &ic);
+        }
         rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st, reset);
         if (rc != DP_OK) return rc;
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true);

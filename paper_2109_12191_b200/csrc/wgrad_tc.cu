@@ -59,7 +59,12 @@ struct TcParams {
     int total_tiles;            // work items: (example, tile) pairs, or (example range, tile) pairs in mode 2
     // mode 2: item = (split, tile); the CTA walks examples [split*per_split, ...) and keeps sum_n f_n D_n in registers
     int splits, per_split;
-    const float *factor;        // [B][2], element 0 = weight factor
+    const float *factor;        // [B][2], element 0 = weight factor (used when inline_factor == 0)
+    // inline_factor: the clipped-sum pass works the factor out itself from the norm pass's partial sums (partial,
+    // slots) and publishes the squared norm and the factor, which saves the separate finalising launch
+    int inline_factor;
+    float C_l;
+    float *sqnorm; long long sq_stride; float *clip_out;
     float *sum_out;             // splits == 1: the accumulator (added to); else partial sums [splits][Kout*Ng]
 };
 
@@ -392,7 +397,21 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 tc_fence_after();
                 const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256) + ((uint32_t)(q * 32) << 16);
                 if (CLIP) {
-                    const float f = p.factor[2 * n];
+                    float f;
+                    if (p.inline_factor) {
+                        // same summation order in every warp of every CTA, so all of them apply the identical factor
+                        double sn = 0.0;
+                        const float *pn = p.partial + (long long)n * p.slots;
+                        for (int i = lane; i < p.slots; i += 32) sn += (double)pn[i];
+                        sn = warp_sum(sn);
+                        f = clip_factor(sn, p.C_l);
+                        if (mt == 0 && nt == 0 && q == 0 && lane == 0) {
+                            p.sqnorm[n * p.sq_stride] = (float)sn;
+                            if (p.clip_out) p.clip_out[n] = f;
+                        }
+                    } else {
+                        f = p.factor[2 * n];
+                    }
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4) {
                         if (c4 * 32 < n_cols) {
@@ -818,7 +837,7 @@ static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, in
 
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g_in, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace, int *status,
-                         cudaStream_t stream, bool second_pass) {
+                         cudaStream_t stream, bool second_pass, const TcInlineClip *inline_clip) {
     const bool clip = epilogue == DP_EPI_CLIP_ACCUM;
     const ConvGeom &g0 = g_in;
     const TcProblem pr = tc_problem(dtype, g0);
@@ -869,6 +888,11 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
     p.reset_status = second_pass ? 0 : 1;       // the second launch of a fused clip call must keep the first one's verdict
     p.splits = 1; p.per_split = g.B; p.factor = factor; p.sum_out = acc_w;
+    p.inline_factor = (clip && inline_clip) ? 1 : 0;
+    p.C_l = inline_clip ? inline_clip->C_l : 0.f;
+    p.sqnorm = inline_clip ? inline_clip->sqnorm : nullptr;
+    p.sq_stride = inline_clip ? inline_clip->sq_stride : 0;
+    p.clip_out = inline_clip ? inline_clip->clip_out : nullptr;
     if (clip) {
         clip_split(g, pl, p.splits, p.per_split);
         if (p.splits > 1) p.sum_out = part_ws;

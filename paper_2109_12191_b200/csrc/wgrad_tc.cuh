@@ -13,9 +13,14 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g, int epilogue);
 // acc[i] += sum_s part[s][i] in index order of s (P a multiple of 4)
 dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream);
 int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n);
+// When given to a CLIP_ACCUM launch, the kernel derives each example's factor from the norm pass's partial sums
+// itself (threshold C_l) and writes sqnorm[n*sq_stride] and clip_out[n] (optional), so no finalising launch is needed.
+struct TcInlineClip { float C_l; float *sqnorm; long long sq_stride; float *clip_out; };
+
 // epilogue as dp_epilogue; factor[n*2] scales example n (CLIP_ACCUM); status: device word set to nonzero on a timed-out wait
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace,
-                         int *status, cudaStream_t stream, bool second_pass = false);
+                         int *status, cudaStream_t stream, bool second_pass = false,
+                         const TcInlineClip *inline_clip = nullptr);
 
 }  // namespace dp
