@@ -484,7 +484,8 @@ dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, in
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
 norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, int HW, int C, int tcv,
-                           float *__restrict__ chunk_partial, int chunks) {
+                           float *__restrict__ chunk_partial, int chunks, float *__restrict__ dgamma,
+                           float *__restrict__ dbeta, float *__restrict__ partial2) {
     extern __shared__ float red[];                       // [rows][tcv*VEC*2]
     const int n = blockIdx.z, chunk = blockIdx.y;
     const int rows = 256 / tcv;
@@ -544,17 +545,32 @@ norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, in
         }
     }
     __syncthreads();
-    // every thread folds one output column over the pixel rows, in row order
+    // every thread folds one output column over the pixel rows, in row order.  When this block holds the whole
+    // example (one pixel chunk, all channels) the sums are final: it writes the gradients and both squared norms
+    // itself and the separate folding launch is skipped (dgamma != nullptr says so).
     {
+        __shared__ double scratch[32];
+        const bool whole = dgamma != nullptr;
         float *out = chunk_partial + (((long long)n * chunks + chunk) * 2) * C;
         const int half = tcv * VEC;
+        double qg = 0.0, qb = 0.0;
         for (int e = threadIdx.x; e < 2 * half; e += 256) {
             const int is_beta = e >= half;
             const int c = blockIdx.x * half + (is_beta ? e - half : e);
             if (c >= C) continue;
             float a = 0.f;
             for (int rr = 0; rr < rows; ++rr) a += red[rr * width + e];
-            out[is_beta ? C + c : c] = a;
+            if (whole) {
+                (is_beta ? dbeta : dgamma)[(long long)n * C + c] = a;
+                if (is_beta) qb += (double)a * a; else qg += (double)a * a;
+            } else {
+                out[is_beta ? C + c : c] = a;
+            }
+        }
+        if (whole) {
+            qg = block_sum(qg, scratch);
+            qb = block_sum(qb, scratch);
+            if (threadIdx.x == 0) { partial2[2 * n] = (float)qg; partial2[2 * n + 1] = (float)qb; }
         }
     }
 }
@@ -765,14 +781,17 @@ dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int
 }
 
 template <typename T, int VEC>
-static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, float *chunk_partial, cudaStream_t st) {
+static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, float *chunk_partial, float *dgamma,
+                               float *dbeta, float *partial2, bool &folded, cudaStream_t st) {
     const int cv = (C + VEC - 1) / VEC;
     const int tcv = cv < 256 ? cv : 256;
     const int chunks = norm_chunks(HW);
     const dim3 grid((cv + tcv - 1) / tcv, chunks, B);
     if (grid.y > 65535 || grid.z > 65535) return DP_ERR_UNSUPPORTED;
     const size_t smem = sizeof(float) * (size_t)(256 / tcv) * tcv * VEC * 2;
-    norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, chunk_partial, chunks);
+    folded = grid.x == 1 && chunks == 1;      // one block sees the whole example: it finishes the job itself
+    norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, chunk_partial, chunks,
+                                                               folded ? dgamma : nullptr, dbeta, partial2);
     DP_LAUNCH_CHECK("norm_affine_partial_kernel");
     return DP_OK;
 }
@@ -780,14 +799,15 @@ static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, fl
 dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
                              float *dgamma, float *dbeta, float *partial2, cudaStream_t st) {
     dp_status rc;
+    bool folded = false;
     if (dtype == DP_F32) {
-        if ((C & 3) == 0) rc = norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, st);
-        else rc = norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, st);
+        if ((C & 3) == 0) rc = norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        else rc = norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
     } else {
-        if ((C & 7) == 0) rc = norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, st);
-        else rc = norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, st);
+        if ((C & 7) == 0) rc = norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        else rc = norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
     }
-    if (rc != DP_OK) return rc;
+    if (rc != DP_OK || folded) return rc;
     norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, norm_chunks(HW), C, dgamma, dbeta, partial2);
     DP_LAUNCH_CHECK("norm_affine_fold_kernel");
     return DP_OK;
