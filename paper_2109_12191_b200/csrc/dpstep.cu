@@ -78,7 +78,7 @@ static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
     if (d->kind != DP_LAYER_NORM_AFFINE && d->has_bias) off = round_up(off + sizeof(float) * B * d->K_out, 256);
     pl.chunk_off = off; pl.dg_off = off;
     if (d->kind == DP_LAYER_NORM_AFFINE) {
-        off = round_up(off + sizeof(float) * B * norm_chunks(d->H * d->W) * 2 * d->C_in, 256);
+        off = round_up(off + sizeof(float) * B * norm_chunks(d->dtype, d->B, d->H * d->W, d->C_in) * 2 * d->C_in, 256);
         pl.dg_off = off;
         off = round_up(off + sizeof(float) * B * 2 * d->C_in, 256);
     }

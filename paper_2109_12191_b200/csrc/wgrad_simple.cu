@@ -483,7 +483,7 @@ dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, in
 // stage 1: block = (channel-vector block, pixel chunk, example); thread = (pixel row, channel vector).
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
-norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, int HW, int C, int tcv,
+norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, int HW, int C, int tcv, int pix,
                            float *__restrict__ chunk_partial, int chunks, float *__restrict__ dgamma,
                            float *__restrict__ dbeta, float *__restrict__ partial2) {
     extern __shared__ float red[];                       // [rows][tcv*VEC*2]
@@ -495,11 +495,11 @@ norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, in
     float sg[VEC], sb[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) { sg[v] = 0.f; sb[v] = 0.f; }
-    const int p_end = min(HW, (chunk + 1) * kNormPix);
+    const int p_end = min(HW, (chunk + 1) * pix);
     if (live) {
         if (VEC * sizeof(T) == 16) {
             // four pixels per trip, all eight 16-byte loads issued before any arithmetic
-            for (int p = chunk * kNormPix + prow; p < p_end; p += 4 * rows) {
+            for (int p = chunk * pix + prow; p < p_end; p += 4 * rows) {
                 uint4 xr[4], gr[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -525,7 +525,7 @@ norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, in
                 }
             }
         } else {
-            for (int p = chunk * kNormPix + prow; p < p_end; p += rows) {
+            for (int p = chunk * pix + prow; p < p_end; p += rows) {
                 const long long off = ((long long)n * HW + p) * C + c0;
 #pragma unroll
                 for (int v = 0; v < VEC; ++v) {
@@ -781,16 +781,15 @@ dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int
 }
 
 template <typename T, int VEC>
-static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, float *chunk_partial, float *dgamma,
-                               float *dbeta, float *partial2, bool &folded, cudaStream_t st) {
+static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, int tcv, int pix, float *chunk_partial,
+                               float *dgamma, float *dbeta, float *partial2, bool &folded, cudaStream_t st) {
     const int cv = (C + VEC - 1) / VEC;
-    const int tcv = cv < 256 ? cv : 256;
-    const int chunks = norm_chunks(HW);
+    const int chunks = (HW + pix - 1) / pix;
     const dim3 grid((cv + tcv - 1) / tcv, chunks, B);
     if (grid.y > 65535 || grid.z > 65535) return DP_ERR_UNSUPPORTED;
     const size_t smem = sizeof(float) * (size_t)(256 / tcv) * tcv * VEC * 2;
     folded = grid.x == 1 && chunks == 1;      // one block sees the whole example: it finishes the job itself
-    norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, chunk_partial, chunks,
+    norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, pix, chunk_partial, chunks,
                                                                folded ? dgamma : nullptr, dbeta, partial2);
     DP_LAUNCH_CHECK("norm_affine_partial_kernel");
     return DP_OK;
@@ -800,15 +799,17 @@ dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, in
                              float *dgamma, float *dbeta, float *partial2, cudaStream_t st) {
     dp_status rc;
     bool folded = false;
+    int vec, tcv, pix;
+    norm_shape(dtype, B, HW, C, vec, tcv, pix);
     if (dtype == DP_F32) {
-        if ((C & 3) == 0) rc = norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
-        else rc = norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        if ((C & 3) == 0) rc = norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        else rc = norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
     } else {
-        if ((C & 7) == 0) rc = norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
-        else rc = norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        if ((C & 7) == 0) rc = norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        else rc = norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
     }
     if (rc != DP_OK || folded) return rc;
-    norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, norm_chunks(HW), C, dgamma, dbeta, partial2);
+    norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, (HW + pix - 1) / pix, C, dgamma, dbeta, partial2);
     DP_LAUNCH_CHECK("norm_affine_fold_kernel");
     return DP_OK;
 }

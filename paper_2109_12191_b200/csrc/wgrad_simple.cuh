@@ -13,7 +13,6 @@ struct ConvGeom {
 
 constexpr int kFmaTile = 64;          // output tile edge of the CUDA-core kernel
 constexpr int kBiasCols = 64;         // output channels per bias-reduction block
-constexpr int kNormPix = 256;         // pixels per block in the norm-affine reduction
 
 inline int fma_tiles_m(const ConvGeom &g) { return (g.M + kFmaTile - 1) / kFmaTile; }
 inline int fma_tiles_n(const ConvGeom &g) { return (g.N + kFmaTile - 1) / kFmaTile; }
@@ -60,6 +59,22 @@ dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int 
                                    float *clip_out, const float *dgamma, const float *dbeta, int C, float *acc_w,
                                    float *acc_b, cudaStream_t stream, int *status_reset = nullptr);
 
-inline int norm_chunks(int HW) { return (HW + kNormPix - 1) / kNormPix; }
+// Shape of the norm-affine reduction: channel vectors per block (tcv) and pixels per block (pix).  Starts from whole
+// channel rows and 256 pixels and narrows both until the grid has a couple of blocks per SM, so that layers with
+// many channels on few pixels (2048 x 7 x 7) do not run on a handful of blocks.
+inline void norm_shape(int dtype, int B, int HW, int C, int &vec, int &tcv, int &pix) {
+    vec = (dtype == DP_F32) ? ((C & 3) ? 1 : 4) : ((C & 7) ? 1 : 8);
+    const int cv = (C + vec - 1) / vec;
+    tcv = cv < 256 ? cv : 256;
+    pix = 256;
+    auto blocks = [&]() { return (long long)((cv + tcv - 1) / tcv) * ((HW + pix - 1) / pix) * B; };
+    if (blocks() < 296 && tcv > 32) tcv = 32;
+    while (blocks() < 296 && pix > 32) pix /= 2;
+}
+inline int norm_chunks(int dtype, int B, int HW, int C) {
+    int vec, tcv, pix;
+    norm_shape(dtype, B, HW, C, vec, tcv, pix);
+    return (HW + pix - 1) / pix;
+}
 
 }  // namespace dp
