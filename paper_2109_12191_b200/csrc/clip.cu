@@ -178,60 +178,6 @@ scale_accumulate_kernel(const __grid_constant__ SegTable tab, const float *__res
     }
 }
 
-// Row-split variant for many examples and few parameters (too few 1024-column blocks to fill the GPU):
-// the block covers 256 columns; its 256 threads are 64 column owners (four columns each) x 4 row groups, row
-// group r takes examples n = r, r+4, ...; the four partial sums are folded in group order through shared memory.
-// Requires every row start to be 16-byte aligned (vector path only).
-__global__ void __launch_bounds__(256)
-scale_accumulate_rows_kernel(const __grid_constant__ SegTable tab, const float *__restrict__ factor, int B, int L,
-                             int per_layer) {
-    __shared__ float f_sh[1024];
-    __shared__ float4 part[3][64];
-    const int seg = find_seg(tab, blockIdx.x);
-    const long long P = tab.P[seg];
-    const int col_thread = threadIdx.x & 63, rg = threadIdx.x >> 6;
-    const long long i = (long long)(blockIdx.x - tab.blk_start[seg]) * 256 + 4 * col_thread;
-    const float *G = tab.G[seg];
-    const int f_stride = per_layer ? L : 1, f_off = per_layer ? tab.col[seg] : 0;
-    const bool live = i < P;
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int n0 = 0; n0 < B; n0 += 1024) {
-        const int nb = min(1024, B - n0);
-        __syncthreads();
-        for (int t = threadIdx.x; t < nb; t += 256) f_sh[t] = factor[(long long)(n0 + t) * f_stride + f_off];
-        __syncthreads();
-        if (live) {
-            const float *g = G + (long long)n0 * P + i;
-            int n = rg;
-            for (; n + 12 < nb; n += 16) {
-                float4 v[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) v[u] = __ldcs(reinterpret_cast<const float4 *>(g + (long long)(n + 4 * u) * P));
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float f = f_sh[n + 4 * u];
-                    s.x = fmaf(f, v[u].x, s.x); s.y = fmaf(f, v[u].y, s.y); s.z = fmaf(f, v[u].z, s.z); s.w = fmaf(f, v[u].w, s.w);
-                }
-            }
-            for (; n < nb; n += 4) {
-                const float4 v = __ldcs(reinterpret_cast<const float4 *>(g + (long long)n * P));
-                const float f = f_sh[n];
-                s.x = fmaf(f, v.x, s.x); s.y = fmaf(f, v.y, s.y); s.z = fmaf(f, v.z, s.z); s.w = fmaf(f, v.w, s.w);
-            }
-        }
-    }
-    if (rg > 0) part[rg - 1][col_thread] = s;
-    __syncthreads();
-    if (rg == 0 && live) {
-        float *acc = tab.acc[seg];
-        float4 a = *reinterpret_cast<const float4 *>(acc + i);
-#pragma unroll
-        for (int r = 0; r < 3; ++r) { const float4 q = part[r][col_thread]; s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w; }
-        a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
-        *reinterpret_cast<float4 *>(acc + i) = a;
-    }
-}
-
 struct ClipPlan {
     size_t partial_off, sq_off, factor_off, total;
     long long parts_per_example;
@@ -283,14 +229,12 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
     const int per_layer = (mode == DP_CLIP_PER_LAYER);
 
     // tensors go to the kernels in tables of at most kMaxSeg entries
-    // few wide blocks and many rows: use the row-split kernel (needs aligned rows everywhere)
     long long wide_blocks = 0;
     for (int l = 0; l < L; ++l) wide_blocks += (P_l[l] + kAccCols - 1) / kAccCols;
-    const bool row_split = false;    // kept for reference measurements; the deep-unroll kernel below is faster
     // A small model gives few blocks, and each thread then walks all B rows in B/UNROLL dependent trips of one
     // memory latency each: with many rows, 32 rows in flight per thread instead of 8 quarters that chain.
     const bool deep = B >= 64 && wide_blocks < 8 * 148;
-    const int acc_cols = row_split ? 256 : kAccCols;
+    const int acc_cols = kAccCols;
 
     auto fill = [&](int l0, SegTable &t, bool norm_blocks, long long &part_cursor) {
         t.nseg = 0;
@@ -336,8 +280,7 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
             SegTable t;
             const int blocks = fill(l0, t, false, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
-            if (row_split) scale_accumulate_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
-            else if (deep) scale_accumulate_kernel<32><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
+            if (deep) scale_accumulate_kernel<32><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             else scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             DP_LAUNCH_CHECK("scale_accumulate_kernel");
             l0 += t.nseg;

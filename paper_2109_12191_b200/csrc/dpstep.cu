@@ -210,9 +210,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         if (clip)
             return launch_affine_clip_accum(partial, d->B, C_l, groups == 2, sqnorm, sqnorm_stride, clip_out, dg, dbt, d->C_in,
                                             acc_w, acc_b, st, reset);
-        rc = launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, clip, C_l, factor, clip_out, st, reset);
-        if (rc != DP_OK || !clip) return rc;
-        return launch_affine_accum(dg, dbt, d->B, d->C_in, factor, acc_w, acc_b, st);
+        return launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
     }
 }
 

@@ -433,11 +433,6 @@ dense_store_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, i
     }
 }
 
-template <typename T>
-__global__ void widen_kernel(const T *__restrict__ src, long long count, float *__restrict__ dst) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < count) dst[i] = to_float(src[i]);
-}
 
 // Dense layer, everything but the outer-product store, one block per example: the rank-1 closed form of the squared
 // norm (|dY_n^T X_n|_F^2 = |dY_n|^2 |X_n|^2, bias part |dY_n|^2), the bias gradient db_n = dY_n widened to fp32 (when
@@ -599,19 +594,6 @@ norm_affine_fold_kernel(const float *__restrict__ chunk_partial, int chunks, int
     if (threadIdx.x == 0) { partial2[2 * n] = (float)qg; partial2[2 * n + 1] = (float)qb; }
 }
 
-__global__ void affine_accum_kernel(const float *__restrict__ dgamma, const float *__restrict__ dbeta, int B, int C,
-                                    const float *__restrict__ factor, float *__restrict__ acc_w,
-                                    float *__restrict__ acc_b) {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= C) return;
-    float a = 0.f, b = 0.f;
-    for (int n = 0; n < B; ++n) {
-        a = fmaf(factor[2 * n], dgamma[(long long)n * C + c], a);
-        b = fmaf(factor[2 * n + 1], dbeta[(long long)n * C + c], b);
-    }
-    acc_w[c] += a;
-    acc_b[c] += b;
-}
 
 // Normalisation layers, fused clip: every block works out the factors of all examples from the two squared norms
 // (cheap and identical in every block), block 0 publishes norms and factors, then each thread owns one channel and
@@ -814,11 +796,5 @@ dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, in
     return DP_OK;
 }
 
-dp_status launch_affine_accum(const float *dgamma, const float *dbeta, int B, int C, const float *factor, float *acc_w,
-                              float *acc_b, cudaStream_t st) {
-    affine_accum_kernel<<<(C + 127) / 128, 128, 0, st>>>(dgamma, dbeta, B, C, factor, acc_w, acc_b);
-    DP_LAUNCH_CHECK("affine_accum_kernel");
-    return DP_OK;
-}
 
 }  // namespace dp

@@ -50,9 +50,6 @@ dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int
 // stage 1: per pixel-chunk partial sums; stage 2: fold, store, squared norms into partial2[n*2 + {0,1}]
 dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
                              float *dgamma, float *dbeta, float *partial2, cudaStream_t stream);
-// acc_w[c] += sum_n factor[n*2] dgamma[n,c]; acc_b[c] += sum_n factor[n*2+1] dbeta[n,c]
-dp_status launch_affine_accum(const float *dgamma, const float *dbeta, int B, int C, const float *factor,
-                              float *acc_w, float *acc_b, cudaStream_t stream);
 
 // fused: factors from partial2 (two squared norms per example), publish norms / factors, accumulate both tensors
 dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int separate, float *sqnorm, long long sq_stride,

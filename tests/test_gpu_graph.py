@@ -1,0 +1,72 @@
+"""The launch configuration the benchmark times: the step captured into a CUDA graph and replayed.
+A replay must give the bits of the plain stream launches, and full-size per-layer calls must match the oracle."""
+import math
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2109_12191_b200 import synth
+from paper_2109_12191_b200.step import GlobalClipStep, PerLayerClipStep
+from gpu_util import dev_inputs, oracle_layer, rel_l2, TOL_NORM, TOL_ACC_BF16
+
+pytestmark = pytest.mark.gpu
+
+
+def test_graph_replay_equals_stream_launches():
+    layers = [synth.conv(3, 32, 3, 1, 1, 16, True, "c1"), synth.conv(32, 64, 3, 2, 1, 16, True, "c2"),
+              synth.dense(64 * 64, 10, True, "fc")]
+    Bn = 16
+    st = GlobalClipStep(layers, Bn, "f32", 0.5, 1.0)
+    ins = [dev_inputs(synth.layer_inputs(l, Bn, "f32", 960, li), "f32") for li, l in enumerate(layers)]
+
+    def step():
+        st.begin()
+        st.chunk(ins)
+        return st.finish(seed=2, step=5)
+
+    direct = step().clone()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        out = step()
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, direct)
+
+
+@pytest.mark.parametrize("which", ["s0b0.c2", "s3b2.c3", "s2b0.gn2", "stem"])
+def test_per_layer_workload_full_size_layers(which):
+    """Layers of the per-layer ResNet-50 workload at full size (B = 32, threshold C/sqrt(161)), run from a replayed
+    CUDA graph as the benchmark does; the oracle checks every example's factor and the whole clipped sum."""
+    layer = next(l for l in synth.resnet50_gn_layers() if l.name == which)
+    Bn, C_l = 32, 1.0 / math.sqrt(synth.RESNET50_GN_TENSORS)
+    inp = synth.layer_inputs(layer, Bn, "bf16", 4, 7, 0)
+    # norms of N(0,1) inputs are far above the threshold; scale so that they straddle it
+    s = (np.logspace(-0.5, 0.5, Bn) * C_l / math.sqrt(layer.flops() / 2)).astype(np.float32)
+    dY = inp["dY"] * s.reshape((Bn,) + (1,) * (inp["dY"].ndim - 1))
+    inp["dY_bits"], inp["dY"] = synth.round_to_bf16(dY)
+    st = PerLayerClipStep([layer], Bn, "bf16", 1.0, 1.0)
+    st.C_l = C_l                                           # the threshold of the 161-tensor model, not of this one layer
+    X, dYd = dev_inputs(inp, "bf16")
+    st.begin()
+    st.wgrad(0, X, dYd)                                    # warm-up launch (sets kernel attributes before capture)
+    torch.cuda.synchronize()
+    st.begin()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        st.wgrad(0, X, dYd)
+    g.replay()
+    torch.cuda.synchronize()
+    dW, db = oracle_layer(layer, inp)
+    groups = [dW] + ([db] if db is not None else [])
+    sq = st.sq.cpu().numpy()
+    for gi, grad in enumerate(groups):
+        ref_sq = oracle.sqnorm(grad)
+        np.testing.assert_allclose(sq[:, gi], ref_sq, rtol=TOL_NORM)
+        f = oracle.clip_factor(ref_sq, C_l)
+        assert (f == 1.0).any() and (f < 1.0).any()
+        got = (st.acc_w[0] if gi == 0 else st.acc_b[0]).cpu().numpy()
+        # capturing records without running: the accumulator holds the single replay's contribution
+        assert rel_l2(got, np.einsum("n,np->p", f, grad)) <= TOL_ACC_BF16
