@@ -105,8 +105,12 @@ DP_API size_t dp_workspace_bytes(const dp_layer_desc *desc, int epilogue);
  *   acc_w/b    [P_w], [P_b] fp32, read-modify-write; DP_EPI_CLIP_ACCUM only:
  *              acc += sum_n min(1, C_l/||g_n||) * g_n  (section 3.5, one group = this layer).
  *   clip_out   optional [B, groups] fp32: the factors that were applied (DP_EPI_CLIP_ACCUM).
- *   workspace  at least dp_workspace_bytes(desc, epilogue) bytes, 256-byte aligned.
+ *   workspace  at least dp_workspace_bytes(desc, epilogue) bytes, 256-byte aligned.  Usually a few hundred KB; layers
+ *              with very few input channels (C_in <= 8) that run on tensor cores keep an unfolded copy of X there
+ *              (B*OH*OW*pad(R*S*C_in) elements), and the fused clip keeps partial sums when it splits the batch.
  *
+ * The first tensor-core call of a process raises a kernel attribute (shared-memory size); make one call of each
+ * kind before capturing calls into a CUDA graph.
  * Results are bit-reproducible from run to run (fixed reduction orders, no float atomics).
  * Errors: DP_ERR_INVALID_ARG, DP_ERR_UNSUPPORTED, DP_ERR_WORKSPACE, DP_ERR_CUDA. */
 DP_API dp_status dp_per_example_wgrad(const dp_layer_desc *desc, const void *X, const void *dY,
