@@ -183,6 +183,20 @@ DP_API dp_status dp_noise_average(const float *acc, long long P, long long param
                            unsigned long long seed, unsigned long long step,
                            float *out, void *cuda_stream);
 
+/* dp_noise_average fused with the parameter update that consumes its result (section 2: the noised, averaged
+ * gradient is "used to update the parameters via SGD"; the CIFAR experiments use momentum 0.9):
+ *     g_i = (acc[i] + sigma*C*z_{param_offset+i}) / total_batch
+ *     m_i <- momentum * m_i + g_i      (only when momentum_buf is given; heavy ball, no dampening, no Nesterov)
+ *     theta_i <- theta_i - lr * m_i    (or - lr * g_i without a momentum buffer)
+ * One pass over the parameters instead of two.  theta [P] and momentum_buf [P] (optional) are fp32, read-modify-write;
+ * g_out [P] is optional and receives g.  Noise stream, argument rules and errors as for dp_noise_average; lr and
+ * momentum must be finite, momentum >= 0. */
+DP_API dp_status dp_noise_average_sgd(const float *acc, long long P, long long param_offset,
+                               float sigma, float C, long long total_batch,
+                               unsigned long long seed, unsigned long long step,
+                               float lr, float momentum, float *theta, float *momentum_buf, float *g_out,
+                               void *cuda_stream);
+
 /* Test hook: the raw Philox words of blocks first_block .. first_block+n_blocks-1 of the
  * (seed, step) stream described above, out4 = [n_blocks, 4] uint32 on the device. */
 DP_API dp_status dp_debug_philox_raw(unsigned int *out4, long long n_blocks, long long first_block,

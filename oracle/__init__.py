@@ -220,6 +220,20 @@ def noise_average(acc, param_offset, sigma, C, total_batch, seed, step):
     return out
 
 
+def sgd_update(g, lr, mu, theta, m=None):
+    """theta, m (float64, updated in place): m <- mu*m + g; theta <- theta - lr*m.  m=None is plain SGD."""
+    lib = _load()
+    g, gp = _f64(g)
+    assert theta.dtype == np.float64 and theta.flags.c_contiguous and theta.size == g.size
+    mp = None
+    if m is not None:
+        assert m.dtype == np.float64 and m.flags.c_contiguous and m.size == g.size
+        mp = m.ctypes.data_as(_f64p)
+    lib.oracle_sgd_update(gp, ctypes.c_size_t(g.size), ctypes.c_double(lr), ctypes.c_double(mu),
+                          theta.ctypes.data_as(_f64p), mp)
+    return theta
+
+
 def privatise(chunks, C, sigma, mode, seed, step):
     """The whole step.  chunks: iterable of lists of L per-example gradient arrays [B, ...].
 

@@ -237,6 +237,18 @@ void oracle_noise_average(const double *acc, size_t P, uint64_t param_offset, do
     }
 }
 
+/* Parameter update that consumes g_t (section 2: "gradients are then used to update the parameters via SGD"; the
+ * CIFAR experiments add momentum 0.9).  Heavy-ball form, no dampening, no Nesterov:
+ *     m <- mu * m + g        theta <- theta - lr * m        (mu = 0: plain SGD, m is then just g) */
+void oracle_sgd_update(const double *g, size_t P, double lr, double mu, double *theta, double *m)
+{
+    for (size_t i = 0; i < P; ++i) {
+        const double v = (m ? mu * m[i] : 0.0) + g[i];
+        if (m) m[i] = v;
+        theta[i] -= lr * v;
+    }
+}
+
 /* The paper's own variant: every clipped example gets its own noise of
  * variance sigma^2 C^2 / |B| before accumulation (equal in distribution).
  * Stream keyed by (seed, step) with the example folded into the high counter

@@ -28,7 +28,7 @@ EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_
            "dp_clip_accumulate", "dp_noise_average", "dp_debug_philox_raw", "dp_debug_noise_z",
            "dp_wgrad_check", "dp_wgrad_uses_tensor_cores", "dp_status_string", "dp_last_cuda_error",
            "dp_debug_launch_count", "dp_debug_wgrad_plan", "dp_clip_accumulate_static",
-           "dp_clip_static_scratch_bytes"]
+           "dp_clip_static_scratch_bytes", "dp_noise_average_sgd"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -65,6 +65,8 @@ _lib.dp_clip_accumulate_static.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctyp
 _lib.dp_clip_accumulate_static.restype = _i
 _lib.dp_clip_static_scratch_bytes.argtypes = []; _lib.dp_clip_static_scratch_bytes.restype = _sz
 _lib.dp_noise_average.argtypes = [_vp, _ll, _ll, _f, _f, _ll, _ull, _ull, _vp, _vp]; _lib.dp_noise_average.restype = _i
+_lib.dp_noise_average_sgd.argtypes = [_vp, _ll, _ll, _f, _f, _ll, _ull, _ull, _f, _f, _vp, _vp, _vp, _vp]
+_lib.dp_noise_average_sgd.restype = _i
 _lib.dp_debug_philox_raw.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_philox_raw.restype = _i
 _lib.dp_debug_noise_z.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_noise_z.restype = _i
 _lib.dp_wgrad_check.argtypes = [_vp, _vp]; _lib.dp_wgrad_check.restype = _i
@@ -153,6 +155,12 @@ def dp_clip_static_scratch_bytes():
 
 def dp_noise_average(acc, P, param_offset, sigma, C, total_batch, seed, step, out, stream=None):
     return _lib.dp_noise_average(_ptr(acc), P, param_offset, sigma, C, total_batch, seed, step, _ptr(out), _stream(stream))
+
+
+def dp_noise_average_sgd(acc, P, param_offset, sigma, C, total_batch, seed, step, lr, momentum, theta, momentum_buf=None,
+                         g_out=None, stream=None):
+    return _lib.dp_noise_average_sgd(_ptr(acc), P, param_offset, sigma, C, total_batch, seed, step, lr, momentum,
+                                     _ptr(theta), _ptr(momentum_buf), _ptr(g_out), _stream(stream))
 
 
 def dp_debug_philox_raw(out4, n_blocks, first_block, seed, step, stream=None):

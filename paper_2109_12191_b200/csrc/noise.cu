@@ -77,6 +77,30 @@ noise_average_kernel(const float *acc, float *out, long long P,   // out may ali
     }
 }
 
+// Noise, average and the parameter update in one pass: g = (acc + std*z) / |B|;  m <- mu*m + g (when a momentum
+// buffer is given);  theta <- theta - lr*m (or - lr*g).  Same thread-to-Philox-block mapping as above.
+__global__ void __launch_bounds__(256)
+noise_average_sgd_kernel(const float *acc, long long P, unsigned long long param_offset, unsigned long long n_blocks,
+                         float noise_std, float inv_batch, unsigned long long seed, unsigned long long step, float lr,
+                         float mu, float *theta, float *mom, float *g_out) {
+    const unsigned long long t = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_blocks) return;
+    const unsigned long long block = (param_offset >> 2) + t;
+    float z[4] = {0.f, 0.f, 0.f, 0.f};
+    if (noise_std != 0.0f) normals4(seed, step, block, z);
+    const long long i0 = (long long)(4ull * block - param_offset);
+#pragma unroll
+    for (int lane = 0; lane < 4; ++lane) {
+        const long long i = i0 + lane;
+        if (i < 0 || i >= P) continue;
+        const float g = (acc[i] + noise_std * z[lane]) * inv_batch;
+        float v = g;
+        if (mom) { v = fmaf(mu, mom[i], g); mom[i] = v; }
+        theta[i] = fmaf(-lr, v, theta[i]);
+        if (g_out) g_out[i] = g;
+    }
+}
+
 __global__ void philox_raw_kernel(uint32_t *out4, long long n_blocks, unsigned long long first_block,
                                   unsigned long long seed, unsigned long long step) {
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -124,6 +148,27 @@ extern "C" dp_status dp_noise_average(const float *acc, long long P, long long p
         dp::noise_average_kernel<false><<<(unsigned)grid, 256, 0, stream>>>(acc, out, P, off, n_blocks, noise_std,
                                                                            inv_batch, seed, step);
     DP_LAUNCH_CHECK("noise_average_kernel");
+    return DP_OK;
+}
+
+extern "C" dp_status dp_noise_average_sgd(const float *acc, long long P, long long param_offset, float sigma, float C,
+                                          long long total_batch, unsigned long long seed, unsigned long long step,
+                                          float lr, float momentum, float *theta, float *momentum_buf, float *g_out,
+                                          void *cuda_stream) {
+    if (!acc || !theta || P <= 0 || param_offset < 0 || total_batch <= 0) return DP_ERR_INVALID_ARG;
+    if (!(sigma >= 0.0f) || !(C > 0.0f) || isinf(sigma) || (sigma > 0.0f && isinf(C))) return DP_ERR_INVALID_ARG;
+    if (!(lr == lr) || isinf(lr) || !(momentum >= 0.0f) || isinf(momentum)) return DP_ERR_INVALID_ARG;
+    if (!dp::aligned(acc, 4) || !dp::aligned(theta, 4) || (momentum_buf && !dp::aligned(momentum_buf, 4)) ||
+        (g_out && !dp::aligned(g_out, 4)))
+        return DP_ERR_INVALID_ARG;
+    const unsigned long long off = (unsigned long long)param_offset;
+    const unsigned long long n_blocks = ((off & 3ull) + (unsigned long long)P + 3ull) >> 2;
+    const unsigned long long grid = (n_blocks + 255) / 256;
+    if (grid > 0x7fffffffull) return DP_ERR_UNSUPPORTED;
+    dp::noise_average_sgd_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        acc, P, off, n_blocks, (sigma == 0.0f) ? 0.0f : sigma * C, 1.0f / (float)total_batch, seed, step, lr, momentum,
+        theta, momentum_buf, g_out);
+    DP_LAUNCH_CHECK("noise_average_sgd_kernel");
     return DP_OK;
 }
 

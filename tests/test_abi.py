@@ -129,6 +129,12 @@ def test_noise_rejects_bad_arguments(b):
     assert call(C=float("inf")) == b.DP_ERR_INVALID_ARG       # infinite C with sigma > 0 has no finite noise scale
     assert call(tb=0) == b.DP_ERR_INVALID_ARG
     assert call(acc=A + 4) == b.DP_ERR_INVALID_ARG
+    sgd = lambda acc=A, theta=A, lr=0.1, mu=0.9, sigma=1.0, C=1.0: b.dp_noise_average_sgd(acc, 16, 0, sigma, C, 8, 0, 0, lr, mu, theta, None, None, stream=0)
+    assert sgd(acc=None) == b.DP_ERR_INVALID_ARG
+    assert sgd(theta=None) == b.DP_ERR_INVALID_ARG
+    assert sgd(lr=float("nan")) == b.DP_ERR_INVALID_ARG
+    assert sgd(mu=-0.1) == b.DP_ERR_INVALID_ARG
+    assert sgd(C=float("inf")) == b.DP_ERR_INVALID_ARG
     assert b.dp_debug_philox_raw(None, 4, 0, 0, 0, stream=0) == b.DP_ERR_INVALID_ARG
     assert b.dp_debug_philox_raw(A, 0, 0, 0, 0, stream=0) == b.DP_ERR_INVALID_ARG
     assert b.dp_debug_noise_z(None, 4, 0, 0, 0, stream=0) == b.DP_ERR_INVALID_ARG

@@ -87,3 +87,29 @@ def test_statistics_at_full_model_size():
     idx = np.random.default_rng(0).integers(0, P, 2000)
     ref = np.array([oracle.noise_z(0, 0, int(i), 1)[0] for i in idx])
     assert np.max(np.abs(acc[torch.from_numpy(idx).cuda()].cpu().numpy() - ref)) <= 1e-5
+
+
+@pytest.mark.parametrize("P,off,mu", [(4099, 0, 0.9), (1000, 3, 0.0), (37, 6, 0.5)])
+def test_fused_sgd_update_matches_oracle_over_several_steps(P, off, mu):
+    """noise + average + (momentum) SGD in one pass against the oracle's noise_average followed by sgd_update."""
+    b = B()
+    sigma, C, total, lr = 0.8, 1.2, 16, 0.05
+    rng = np.random.default_rng(P)
+    theta0 = rng.standard_normal(P).astype(np.float32)
+    theta, mom = dev(theta0), torch.zeros(P, device="cuda")
+    g_out = torch.full((P,), float("nan"), device="cuda")
+    ref_theta, ref_m = theta0.astype(np.float64), np.zeros(P)
+    for step in range(3):
+        acc = (rng.standard_normal(P) * 4).astype(np.float32)
+        b.check(b.dp_noise_average_sgd(dev(acc), P, off, sigma, C, total, 21, step, lr, mu, theta,
+                                       mom if mu > 0 else None, g_out))
+        g = oracle.noise_average(acc.astype(np.float64), off, sigma, C, total, 21, step)
+        oracle.sgd_update(g, lr, mu, ref_theta, ref_m if mu > 0 else None)
+        assert np.max(np.abs(g_out.cpu().numpy() - g)) <= 1e-5 * sigma * C / total + 1e-6 * np.max(np.abs(g))
+    assert np.max(np.abs(theta.cpu().numpy() - ref_theta)) <= 1e-5
+    if mu > 0:
+        assert np.max(np.abs(mom.cpu().numpy() - ref_m)) <= 1e-5
+    # the same gradient as the unfused entry point, bit for bit
+    out = torch.empty(P, device="cuda")
+    b.check(b.dp_noise_average(dev(acc), P, off, sigma, C, total, 21, 2, out))
+    np.testing.assert_array_equal(out.cpu().numpy(), g_out.cpu().numpy())

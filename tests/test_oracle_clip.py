@@ -142,3 +142,24 @@ def test_noise_std_uses_the_global_C_in_per_layer_mode():
     out, _, _ = oracle.privatise(chunks, 2.0, 0.5, "per_layer", seed=9, step=1)
     z = oracle.noise_z(9, 1, 0, 16)
     np.testing.assert_allclose(np.concatenate(out), 0.5 * 2.0 * z / 2.0, rtol=1e-15)
+
+
+def test_sgd_update_plain_and_momentum_closed_form():
+    """theta after k steps of a constant gradient g: theta_0 - lr*g*sum_{j=1..k} (1-mu^j)/(1-mu)."""
+    P, lr, mu, k = 7, 0.1, 0.9, 5
+    g = np.linspace(-1.0, 2.0, P)
+    theta = np.ones(P)
+    oracle.sgd_update(g, lr, 0.0, theta)                      # no momentum buffer: theta - lr*g
+    np.testing.assert_allclose(theta, 1.0 - lr * g, rtol=1e-15)
+    theta, m = np.zeros(P), np.zeros(P)
+    for _ in range(k):
+        oracle.sgd_update(g, lr, mu, theta, m)
+    np.testing.assert_allclose(m, g * (1 - mu ** k) / (1 - mu), rtol=1e-13)
+    np.testing.assert_allclose(theta, -lr * g * sum((1 - mu ** j) / (1 - mu) for j in range(1, k + 1)), rtol=1e-13)
+    # against torch.optim.SGD (momentum, no dampening, no Nesterov)
+    w = torch.zeros(P, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([w], lr=lr, momentum=mu)
+    for _ in range(k):
+        w.grad = torch.from_numpy(g.copy())
+        opt.step()
+    np.testing.assert_allclose(theta, w.detach().numpy(), rtol=1e-13)
