@@ -220,6 +220,28 @@ def noise_average(acc, param_offset, sigma, C, total_batch, seed, step):
     return out
 
 
+def example_noise_z(seed, step, example, first_index, count):
+    """Standard normals of example `example`'s own stream for global parameter indices first_index .. +count-1."""
+    lib = _load()
+    z = np.empty(count, dtype=np.float64)
+    lib.oracle_example_noise_z(ctypes.c_uint64(seed), ctypes.c_uint64(step), ctypes.c_uint32(example),
+                               ctypes.c_uint64(first_index), ctypes.c_size_t(count), z.ctypes.data_as(_f64p))
+    return z
+
+
+def clip_accumulate_noised(G, factor, acc, sd, seed, step, example0, param_offset):
+    """acc[P] += sum_n (factor[n]*G[n,:] + sd*z_{example0+n}); G float32 [B, P], acc float64 updated in place."""
+    lib = _load()
+    G, gp = _f32(G)
+    B, P = G.shape[0], int(np.prod(G.shape[1:]))
+    factor, fp = _f64(factor)
+    assert acc.dtype == np.float64 and acc.size == P and acc.flags.c_contiguous and factor.size == B
+    lib.oracle_clip_accumulate_noised_f32(gp, B, ctypes.c_size_t(P), fp, ctypes.c_double(sd), ctypes.c_uint64(seed),
+                                          ctypes.c_uint64(step), ctypes.c_uint32(example0), ctypes.c_uint64(param_offset),
+                                          acc.ctypes.data_as(_f64p))
+    return acc
+
+
 def sgd_update(g, lr, mu, theta, m=None):
     """theta, m (float64, updated in place): m <- mu*m + g; theta <- theta - lr*m.  m=None is plain SGD."""
     lib = _load()

@@ -249,21 +249,39 @@ void oracle_sgd_update(const double *g, size_t P, double lr, double mu, double *
     }
 }
 
-/* The paper's own variant: every clipped example gets its own noise of
- * variance sigma^2 C^2 / |B| before accumulation (equal in distribution).
- * Stream keyed by (seed, step) with the example folded into the high counter
- * bits is NOT defined here; this helper only states the arithmetic for a
- * caller-supplied standard-normal array zn[n,i]. */
-void oracle_per_example_noised_sum(const double *G, int B, size_t P, const double *factor,
-                                   const double *zn, double sigma, double C, double total_batch,
-                                   double *acc)
+/* The paper's own variant (section 2, the align block after the equation for g_t): every clipped example gets
+ * its own noise of variance sigma^2 C^2 / |B| before accumulation, which is equal in distribution to one draw of
+ * variance sigma^2 C^2 on the sum.  Example e of the step draws from its own stream: the Philox counter carries
+ * (lo32(g/4), 0x80000000 | e, step lo, step hi) for global parameter index g, same key, same Box-Muller lanes. */
+static double example_noise_z_one(uint64_t seed, uint64_t step, uint32_t example, uint64_t g)
 {
-    const double sd = sigma * C / sqrt(total_batch);
+    const double two_pi = 6.283185307179586476925286766559;
+    const uint32_t ctr[4] = {(uint32_t)(g >> 2), 0x80000000u | example, (uint32_t)step, (uint32_t)(step >> 32)};
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t w[4];
+    oracle_philox4x32_10(ctr, key, w);
+    const int lane = (int)(g & 3);
+    double u1, u2;
+    uniforms(w[lane & 2], w[(lane & 2) + 1], &u1, &u2);
+    const double radius = sqrt(-2.0 * log(u1));
+    return (lane & 1) ? radius * sin(two_pi * u2) : radius * cos(two_pi * u2);
+}
+
+void oracle_example_noise_z(uint64_t seed, uint64_t step, uint32_t example, uint64_t first_index, size_t count, double *z)
+{
+    for (size_t t = 0; t < count; ++t) z[t] = example_noise_z_one(seed, step, example, first_index + t);
+}
+
+/* acc[i] += sum_n ( factor[n] * G[n,i] + sd * z_{example0+n}(param_offset + i) ),  sd = sigma*C/sqrt(|B|) */
+void oracle_clip_accumulate_noised_f32(const float *G, int B, size_t P, const double *factor, double sd, uint64_t seed,
+                                       uint64_t step, uint32_t example0, uint64_t param_offset, double *acc)
+{
 #pragma omp parallel for
     for (size_t i = 0; i < P; ++i) {
         double a = 0.0;
         for (int n = 0; n < B; ++n)
-            a += factor[n] * G[(size_t)n * P + i] + sd * zn[(size_t)n * P + i];
+            a += factor[n] * (double)G[(size_t)n * P + i] +
+                 (sd == 0.0 ? 0.0 : sd * example_noise_z_one(seed, step, example0 + (uint32_t)n, param_offset + i));
         acc[i] += a;
     }
 }

@@ -119,3 +119,34 @@ def test_scaled_noise_has_std_sigma_C_and_per_example_form_has_the_same_variance
     assert abs(out.std() * Bt - sigma * C) < 5 * sigma * C / math.sqrt(2 * P)
     per_example = sum(oracle.noise_z(100 + n, 0, 0, P) for n in range(Bt)) * (sigma * C / math.sqrt(Bt))
     assert abs(per_example.std() - sigma * C) < 5 * sigma * C / math.sqrt(2 * P)
+
+
+def test_example_stream_layout_and_independence():
+    """Per-example noise (section 2, the paper's own variant): counter word 1 carries 0x80000000 | example."""
+    seed, step, e, g0 = 77, 5, 9, 40
+    w = _philox_python([g0 // 4, 0x80000000 | e, step, 0], [seed, 0])
+    z = oracle.example_noise_z(seed, step, e, g0, 4)
+    for pair in range(2):
+        u1 = ((w[2 * pair] >> 9) + 0.5) / 2 ** 23
+        u2 = (w[2 * pair + 1] >> 8) / 2 ** 24
+        r = math.sqrt(-2.0 * math.log(u1))
+        assert abs(z[2 * pair] - r * math.cos(2 * math.pi * u2)) < 1e-14
+        assert abs(z[2 * pair + 1] - r * math.sin(2 * math.pi * u2)) < 1e-14
+    n = 200_000
+    a, b, c = oracle.example_noise_z(1, 0, 0, 0, n), oracle.example_noise_z(1, 0, 1, 0, n), oracle.noise_z(1, 0, 0, n)
+    for x, y in [(a, b), (a, c), (b, c)]:
+        assert abs(np.corrcoef(x, y)[0, 1]) < 5 / math.sqrt(n)
+    assert abs(a.var() - 1.0) < 0.02 and abs(a.mean()) < 0.02
+
+
+def test_per_example_noised_sum_is_the_clipped_sum_plus_the_example_draws():
+    B, P, sd = 5, 64, 0.3
+    G = np.random.default_rng(3).standard_normal((B, P)).astype(np.float32)
+    f = np.linspace(0.2, 1.0, B)
+    acc = oracle.clip_accumulate_noised(G, f, np.zeros(P), sd, 8, 2, 10, 100)
+    want = np.einsum("n,np->p", f, G.astype(np.float64)) + sd * sum(oracle.example_noise_z(8, 2, 10 + n, 100, P) for n in range(B))
+    np.testing.assert_allclose(acc, want, rtol=1e-13, atol=1e-13)
+    # sd = sigma*C/sqrt(|B|) over |B| examples gives total variance (sigma*C)^2
+    Bt, Pn = 16, 100_000
+    tot = sum(oracle.example_noise_z(4, 0, e, 0, Pn) for e in range(Bt)) * (1.3 * 0.7 / math.sqrt(Bt))
+    assert abs(tot.std() - 1.3 * 0.7) < 5 * 1.3 * 0.7 / math.sqrt(2 * Pn)
