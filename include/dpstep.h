@@ -143,6 +143,35 @@ DP_API dp_status dp_clip_accumulate(int mode, int B, int L, const float *const *
                              float *norms_out, float *clip_out,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* dp_clip_accumulate with the noise added per example, before the sum (section 2, the block after the equation for
+ * g_t: each clipped example receives its own draw of variance sigma^2 C^2 / |B|, which is equal in distribution to one
+ * draw of variance sigma^2 C^2 on the sum; this is the form the paper's own implementation uses):
+ *     acc_l[i] += sum_n ( f_n * G_l[n,i] + sd * z_{example0+n}(param_offset_l[l] + i) ),   sd = sigma*C/sqrt(total_batch)
+ * with f_n as in dp_clip_accumulate (both modes).  After the last chunk the step ends with dp_noise_average(sigma = 0),
+ * the plain division by |B|.
+ * z_e(g) is example e's own stream: Philox4x32-10 with counter (lo32(g/4), 0x80000000 | e, lo32(step), hi32(step)),
+ * key (lo32(seed), hi32(seed)), and the Box-Muller lanes of dp_noise_average; it depends only on
+ * (seed, step, e, g), never on chunking or launch shape, and never meets the per-parameter stream of dp_noise_average.
+ *
+ *   param_offset_l  host array of L global indices: where each tensor starts in the model's parameter vector (>= 0,
+ *                   offset + P_l <= 2^34).  Multiples of four take the fast path.
+ *   sigma, C        sigma >= 0 (0 adds nothing); with sigma > 0, C must be finite.  C is always the whole-gradient
+ *                   bound, also in PER_LAYER mode.
+ *   total_batch     |B| of the whole step (all chunks, all ranks), > 0.
+ *   example0        index within the step of this chunk's first example (>= 0, example0 + B <= 2^31); chunks of one
+ *                   step must use disjoint ranges, or two examples would share a draw.
+ * Everything else, and the errors, as for dp_clip_accumulate.  The work is B*P normals per chunk: arithmetic-bound,
+ * where the once-per-step form costs P normals per step. */
+DP_API dp_status dp_clip_accumulate_noised(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                           const long long *param_offset_l, const float *sqnorm, float C, float sigma,
+                                           long long total_batch, unsigned long long seed, unsigned long long step,
+                                           long long example0, float *const *acc, float *norms_out, float *clip_out,
+                                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Test hook: the standard normals of example `example`'s stream for global indices first_index .. +count-1. */
+DP_API dp_status dp_debug_example_noise_z(float *z, long long count, long long first_index, long long example,
+                                          unsigned long long seed, unsigned long long step, void *cuda_stream);
+
 /* dp_clip_accumulate for callers that cannot allocate device memory.  (The paper has no counterpart;
  * this exists for deployment reasons only.)
  *

@@ -8,6 +8,7 @@
 //   3. every thread owns four neighbouring parameters, streams the B example rows through
 //      registers with 128-bit loads, and touches the accumulator once.
 #include "common.cuh"
+#include "philox.cuh"
 #include <math.h>
 #include <mutex>
 
@@ -24,7 +25,16 @@ struct SegTable {
     int blk_start[kMaxSeg + 1];      // first block of each tensor within this launch
     int col[kMaxSeg];                // index l of the tensor in the [B, L] norm / factor tables
     long long part_start[kMaxSeg];   // first partial slot of each tensor within one example's row of partials
+    long long goff[kMaxSeg];         // global index of the tensor's first parameter (per-example noise only)
     int nseg;
+};
+
+// Per-example noise (the paper's own implementation, section 2, the block after the equation for g_t):
+// example e of the step adds sd * z_e(g), sd = sigma*C/sqrt(|B|), to its clipped gradient before the sum.
+struct ExampleNoise {
+    float sd;
+    unsigned long long seed, step;
+    uint32_t example0;               // index within the step of this chunk's first example
 };
 
 __device__ __forceinline__ int find_seg(const SegTable &t, int blk) {
@@ -178,6 +188,95 @@ scale_accumulate_kernel(const __grid_constant__ SegTable tab, const float *__res
     }
 }
 
+// stage 3 with per-example noise: acc[i] += sum_n ( factor * G[n, i] + sd * z_{example0+n}(goff + i) ).
+// Every thread owns the four parameters of one Philox block when the tensor starts on a multiple of four global
+// indices; otherwise each parameter draws its own block and keeps one lane.  Bound by the integer and
+// transcendental work of B*P normals, not by memory.
+__global__ void __launch_bounds__(256)
+scale_accumulate_noised_kernel(const __grid_constant__ SegTable tab, const float *__restrict__ factor, int B, int L,
+                               int per_layer, const ExampleNoise nz) {
+    __shared__ float f_sh[256];
+    const int seg = find_seg(tab, blockIdx.x);
+    const long long P = tab.P[seg];
+    const long long c0 = (long long)(blockIdx.x - tab.blk_start[seg]) * kAccCols;
+    const float *G = tab.G[seg];
+    float *acc = tab.acc[seg];
+    const long long goff = tab.goff[seg];
+    const int f_stride = per_layer ? L : 1;
+    const int f_off = per_layer ? tab.col[seg] : 0;
+    const bool vec = ((P & 3) == 0) && ((goff & 3) == 0) && ((reinterpret_cast<uintptr_t>(G) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(acc) & 15) == 0);
+    if (vec) {
+        const long long i = c0 + 4 * threadIdx.x;
+        const bool live = i < P;
+        const uint32_t block = (uint32_t)((unsigned long long)(goff + i) >> 2);
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int n0 = 0; n0 < B; n0 += 256) {
+            const int nb = min(256, B - n0);
+            __syncthreads();
+            if (threadIdx.x < nb) f_sh[threadIdx.x] = factor[(long long)(n0 + threadIdx.x) * f_stride + f_off];
+            __syncthreads();
+            if (live) {
+                const float *g = G + (long long)n0 * P + i;
+                int n = 0;
+                for (; n + 4 <= nb; n += 4) {
+                    float4 v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v[u] = __ldcs(reinterpret_cast<const float4 *>(g + (long long)(n + u) * P));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        float z[4];
+                        example_normals4(nz.seed, nz.step, nz.example0 + (uint32_t)(n0 + n + u), block, z);
+                        const float f = f_sh[n + u];
+                        s.x += fmaf(f, v[u].x, nz.sd * z[0]); s.y += fmaf(f, v[u].y, nz.sd * z[1]);
+                        s.z += fmaf(f, v[u].z, nz.sd * z[2]); s.w += fmaf(f, v[u].w, nz.sd * z[3]);
+                    }
+                }
+                for (; n < nb; ++n) {
+                    const float4 v = __ldcs(reinterpret_cast<const float4 *>(g + (long long)n * P));
+                    float z[4];
+                    example_normals4(nz.seed, nz.step, nz.example0 + (uint32_t)(n0 + n), block, z);
+                    const float f = f_sh[n];
+                    s.x += fmaf(f, v.x, nz.sd * z[0]); s.y += fmaf(f, v.y, nz.sd * z[1]);
+                    s.z += fmaf(f, v.z, nz.sd * z[2]); s.w += fmaf(f, v.w, nz.sd * z[3]);
+                }
+            }
+        }
+        if (live) {
+            float4 a = *reinterpret_cast<const float4 *>(acc + i);
+            a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
+            *reinterpret_cast<float4 *>(acc + i) = a;
+        }
+    } else {
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int n0 = 0; n0 < B; n0 += 256) {
+            const int nb = min(256, B - n0);
+            __syncthreads();
+            if (threadIdx.x < nb) f_sh[threadIdx.x] = factor[(long long)(n0 + threadIdx.x) * f_stride + f_off];
+            __syncthreads();
+            for (int n = 0; n < nb; ++n) {
+                const float f = f_sh[n];
+                const float *g = G + (long long)(n0 + n) * P + c0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const long long i = threadIdx.x + 256 * q;
+                    if (c0 + i < P) {
+                        const unsigned long long gi = (unsigned long long)(goff + c0 + i);
+                        float z[4];
+                        example_normals4(nz.seed, nz.step, nz.example0 + (uint32_t)(n0 + n), (uint32_t)(gi >> 2), z);
+                        s[q] += fmaf(f, g[i], nz.sd * z[gi & 3]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const long long i = c0 + threadIdx.x + 256 * q;
+            if (i < P) acc[i] += s[q];
+        }
+    }
+}
+
 struct ClipPlan {
     size_t partial_off, sq_off, factor_off, total;
     long long parts_per_example;
@@ -206,10 +305,13 @@ extern "C" size_t dp_clip_workspace_bytes(int B, int L, const long long *P_l) {
     return pl.total;
 }
 
-extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *const *G, const long long *P_l,
-                                        const float *sqnorm, float C, float *const *acc, float *norms_out,
-                                        float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
-    using namespace dp;
+namespace dp {
+// Host side of dp_clip_accumulate; with `noise` (and the tensors' global offsets) stage 3 also adds each example's
+// own noise draw.
+static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                      const float *sqnorm, float C, float *const *acc, float *norms_out,
+                                      float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream,
+                                      const ExampleNoise *noise, const long long *goff_l) {
     if (mode != DP_CLIP_GLOBAL && mode != DP_CLIP_PER_LAYER) return DP_ERR_INVALID_ARG;
     if (B <= 0 || L <= 0 || !G || !P_l || !acc || !(C > 0.0f)) return DP_ERR_INVALID_ARG;
     if (B > 65535) return DP_ERR_UNSUPPORTED;
@@ -242,6 +344,7 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
         for (int l = l0; l < L && t.nseg < kMaxSeg; ++l) {
             const int s = t.nseg++;
             t.G[s] = G[l]; t.acc[s] = acc[l]; t.P[s] = P_l[l]; t.col[s] = l;
+            t.goff[s] = goff_l ? goff_l[l] : 0;
             t.blk_start[s] = blk;
             t.part_start[s] = part_cursor;
             const long long nparts = (P_l[l] + kNormChunk - 1) / kNormChunk;
@@ -280,13 +383,46 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
             SegTable t;
             const int blocks = fill(l0, t, false, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
-            if (deep) scale_accumulate_kernel<32><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
+            if (noise) scale_accumulate_noised_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer, *noise);
+            else if (deep) scale_accumulate_kernel<32><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             else scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             DP_LAUNCH_CHECK("scale_accumulate_kernel");
             l0 += t.nseg;
         }
     }
     return DP_OK;
+}
+}  // namespace dp
+
+extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                        const float *sqnorm, float C, float *const *acc, float *norms_out,
+                                        float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace, workspace_bytes,
+                                    cuda_stream, nullptr, nullptr);
+}
+
+extern "C" dp_status dp_clip_accumulate_noised(int mode, int B, int L, const float *const *G, const long long *P_l,
+                                               const long long *param_offset_l, const float *sqnorm, float C,
+                                               float sigma, long long total_batch, unsigned long long seed,
+                                               unsigned long long step, long long example0, float *const *acc,
+                                               float *norms_out, float *clip_out, void *workspace,
+                                               size_t workspace_bytes, void *cuda_stream) {
+    if (!param_offset_l || L <= 0 || B <= 0 || !P_l) return DP_ERR_INVALID_ARG;
+    if (!(sigma >= 0.0f) || isinf(sigma) || total_batch <= 0 || example0 < 0) return DP_ERR_INVALID_ARG;
+    if (sigma > 0.0f && (isinf(C) || !(C > 0.0f))) return DP_ERR_INVALID_ARG;
+    if (example0 + (long long)B > 0x80000000ll) return DP_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l) {
+        if (param_offset_l[l] < 0 || P_l[l] <= 0) return DP_ERR_INVALID_ARG;
+        if (((unsigned long long)param_offset_l[l] + (unsigned long long)P_l[l]) > (1ull << 34)) return DP_ERR_UNSUPPORTED;
+    }
+    if (sigma == 0.0f)
+        return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace,
+                                        workspace_bytes, cuda_stream, nullptr, nullptr);
+    dp::ExampleNoise nz;
+    nz.sd = (float)((double)sigma * (double)C / sqrt((double)total_batch));
+    nz.seed = seed; nz.step = step; nz.example0 = (uint32_t)example0;
+    return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace, workspace_bytes,
+                                    cuda_stream, &nz, param_offset_l);
 }
 
 // ----------------------------------------------------------------------------------------------------

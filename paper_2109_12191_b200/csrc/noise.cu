@@ -83,6 +83,23 @@ __global__ void noise_z_kernel(float *z, long long count, unsigned long long fir
     }
 }
 
+// z[t] = normal of example `example`'s stream at global index first_index + t (one thread per Philox block)
+__global__ void example_noise_z_kernel(float *z, long long count, unsigned long long first_index,
+                                       unsigned long long n_blocks, uint32_t example, unsigned long long seed,
+                                       unsigned long long step) {
+    const unsigned long long t = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_blocks) return;
+    const unsigned long long block = (first_index >> 2) + t;
+    float v[4];
+    example_normals4(seed, step, example, (uint32_t)block, v);
+    const long long i0 = (long long)(4ull * block - first_index);
+#pragma unroll
+    for (int lane = 0; lane < 4; ++lane) {
+        const long long i = i0 + lane;
+        if (i >= 0 && i < count) z[i] = v[lane];
+    }
+}
+
 }  // namespace dp
 
 extern "C" dp_status dp_noise_average(const float *acc, long long P, long long param_offset, float sigma, float C,
@@ -152,5 +169,19 @@ extern "C" dp_status dp_debug_noise_z(float *z, long long count, long long first
     dp::noise_z_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(z, count, off, n_blocks,
                                                                                          seed, step);
     DP_LAUNCH_CHECK("noise_z_kernel");
+    return DP_OK;
+}
+
+extern "C" dp_status dp_debug_example_noise_z(float *z, long long count, long long first_index, long long example,
+                                              unsigned long long seed, unsigned long long step, void *cuda_stream) {
+    if (!z || count <= 0 || first_index < 0 || example < 0 || example >= 0x80000000ll) return DP_ERR_INVALID_ARG;
+    const unsigned long long off = (unsigned long long)first_index;
+    if (off + (unsigned long long)count > (1ull << 34)) return DP_ERR_UNSUPPORTED;
+    const unsigned long long n_blocks = ((off & 3ull) + (unsigned long long)count + 3ull) >> 2;
+    const unsigned long long grid = (n_blocks + 255) / 256;
+    if (grid > 0x7fffffffull) return DP_ERR_UNSUPPORTED;
+    dp::example_noise_z_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        z, count, off, n_blocks, (uint32_t)example, seed, step);
+    DP_LAUNCH_CHECK("example_noise_z_kernel");
     return DP_OK;
 }

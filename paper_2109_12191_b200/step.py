@@ -31,12 +31,30 @@ def _tensors_of(layers):
     return out
 
 
+class _NoiseKey:
+    """Where the noise enters: once per step in finish() (default), or per example inside every chunk call, in which
+    case the chunk calls need the step's total batch and key and finish() only divides."""
+
+    def __init__(self, per_example, total_batch, seed, step, example0):
+        if per_example and not total_batch:
+            raise ValueError("per-example noise needs begin(total_batch=...)")
+        self.per_example, self.total_batch, self.seed, self.step, self.example0 = per_example, total_batch, seed, step, example0
+
+    def finish_sigma(self, sigma, total):
+        if not self.per_example:
+            return sigma
+        if total != self.total_batch:
+            raise ValueError(f"step saw {total} examples but its noise was scaled for {self.total_batch}")
+        return 0.0
+
+
 class GlobalClipStep:
     """Whole-model clipping: per-example gradients are materialised per layer (STORE+NORM epilogue),
     one dp_clip_accumulate call per chunk consumes them with the norms the epilogues produced."""
 
-    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda"):
+    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda", per_example_noise=False):
         self.layers, self.B, self.dtype, self.C, self.sigma = list(layers), B, dtype, float(C), float(sigma)
+        self.per_example_noise = bool(per_example_noise)
         self.tensors = _tensors_of(self.layers)
         self.L = len(self.tensors)
         self.P_l = [t[2] for t in self.tensors]
@@ -64,9 +82,11 @@ class GlobalClipStep:
             col += 2 if l.n_bias else 1
         self.chunks_done = 0
 
-    def begin(self):
+    def begin(self, total_batch=None, seed=0, step=0, example0=0):
+        """Per-example noise needs the step's total batch, its (seed, step) and this rank's first example index up front."""
         self.acc.zero_()
         self.chunks_done = 0
+        self._noise = _NoiseKey(self.per_example_noise, total_batch, seed, step, example0)
 
     def wgrad(self, li, X, dY):
         col = self._col[li]
@@ -76,8 +96,16 @@ class GlobalClipStep:
                                        b.DP_EPI_STORE_NORM, 0.0, None, None, None, self.ws), "dp_per_example_wgrad")
 
     def clip_accumulate(self, use_epilogue_norms=True):
-        b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, self.G, self.P_l, self.sq if use_epilogue_norms else None,
-                                     self.C, self.acc_views, self.norms, self.clip, self.clip_ws), "dp_clip_accumulate")
+        sq = self.sq if use_epilogue_norms else None
+        if self.per_example_noise:
+            k = self._noise
+            b.check(b.dp_clip_accumulate_noised(b.DP_CLIP_GLOBAL, self.B, self.G, self.P_l, self.offsets, sq, self.C,
+                                                self.sigma, k.total_batch, k.seed, k.step,
+                                                k.example0 + self.B * self.chunks_done, self.acc_views, self.norms,
+                                                self.clip, self.clip_ws), "dp_clip_accumulate_noised")
+        else:
+            b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, self.G, self.P_l, sq, self.C, self.acc_views, self.norms,
+                                         self.clip, self.clip_ws), "dp_clip_accumulate")
         self.chunks_done += 1
 
     def chunk(self, inputs):
@@ -89,15 +117,17 @@ class GlobalClipStep:
     def finish(self, seed=0, step=0, world=1):
         """world > 1: `acc` already holds the sum over all ranks (see sharding.allreduce_accumulator)."""
         total = self.B * self.chunks_done * world
-        b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, total, seed, step, self.out), "dp_noise_average")
+        sigma = self._noise.finish_sigma(self.sigma, total)
+        b.check(b.dp_noise_average(self.acc, self.P, 0, sigma, self.C, total, seed, step, self.out), "dp_noise_average")
         return self.out
 
 
 class FlatClipStep:
     """Flattened per-example gradients [B, P] handed in directly (no weight-gradient stage)."""
 
-    def __init__(self, P, B, C, sigma, device="cuda"):
+    def __init__(self, P, B, C, sigma, device="cuda", per_example_noise=False):
         self.P, self.B, self.C, self.sigma = P, B, float(C), float(sigma)
+        self.per_example_noise = bool(per_example_noise)
         self.acc = torch.zeros(P, dtype=torch.float32, device=device)
         self.out = torch.empty(P, dtype=torch.float32, device=device)
         self.norms = torch.empty(B, dtype=torch.float32, device=device)
@@ -105,18 +135,26 @@ class FlatClipStep:
         self.ws = torch.empty(max(b.dp_clip_workspace_bytes(B, [P]), 256), dtype=torch.uint8, device=device)
         self.chunks_done = 0
 
-    def begin(self):
+    def begin(self, total_batch=None, seed=0, step=0, example0=0):
         self.acc.zero_()
         self.chunks_done = 0
+        self._noise = _NoiseKey(self.per_example_noise, total_batch, seed, step, example0)
 
     def chunk(self, G, sqnorm=None):
-        b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, [G], [self.P], sqnorm, self.C, [self.acc], self.norms,
-                                     self.clip, self.ws), "dp_clip_accumulate")
+        if self.per_example_noise:
+            k = self._noise
+            b.check(b.dp_clip_accumulate_noised(b.DP_CLIP_GLOBAL, self.B, [G], [self.P], [0], sqnorm, self.C, self.sigma,
+                                                k.total_batch, k.seed, k.step, k.example0 + self.B * self.chunks_done,
+                                                [self.acc], self.norms, self.clip, self.ws), "dp_clip_accumulate_noised")
+        else:
+            b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, [G], [self.P], sqnorm, self.C, [self.acc], self.norms,
+                                         self.clip, self.ws), "dp_clip_accumulate")
         self.chunks_done += 1
 
     def finish(self, seed=0, step=0, world=1):
-        b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, self.B * self.chunks_done * world, seed, step,
-                                   self.out), "dp_noise_average")
+        total = self.B * self.chunks_done * world
+        sigma = self._noise.finish_sigma(self.sigma, total)
+        b.check(b.dp_noise_average(self.acc, self.P, 0, sigma, self.C, total, seed, step, self.out), "dp_noise_average")
         return self.out
 
 

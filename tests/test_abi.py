@@ -116,6 +116,28 @@ def test_clip_rejects_bad_arguments(b):
     assert call(workspace_bytes=ws - 1) == b.DP_ERR_WORKSPACE
 
 
+def test_noised_clip_rejects_bad_arguments(b):
+    A = 4096
+    P = [100, 8]
+    ws = b.dp_clip_workspace_bytes(4, P)
+    ok = dict(mode=0, B=4, G=[A, A], P_l=P, param_offset_l=[0, 100], sqnorm=None, C=1.0, sigma=1.0, total_batch=16, seed=1,
+              step=2, example0=4, acc=[A, A], norms_out=None, clip_out=None, workspace=A, workspace_bytes=ws, stream=0)
+    call = lambda **kw: b.dp_clip_accumulate_noised(**{**ok, **kw})
+    assert call(param_offset_l=None) == b.DP_ERR_INVALID_ARG
+    assert call(param_offset_l=[0, -1]) == b.DP_ERR_INVALID_ARG
+    assert call(param_offset_l=[0, 2**34]) == b.DP_ERR_UNSUPPORTED     # global index beyond the stream's counter word
+    assert call(sigma=-1.0) == b.DP_ERR_INVALID_ARG
+    assert call(sigma=float("nan")) == b.DP_ERR_INVALID_ARG
+    assert call(C=float("inf")) == b.DP_ERR_INVALID_ARG                # no finite noise scale
+    assert call(total_batch=0) == b.DP_ERR_INVALID_ARG
+    assert call(example0=-1) == b.DP_ERR_INVALID_ARG
+    assert call(example0=2**31 - 3) == b.DP_ERR_INVALID_ARG            # example index leaves its 31 bits
+    assert call(G=[A, None]) == b.DP_ERR_INVALID_ARG                   # the shared checks of dp_clip_accumulate
+    assert call(workspace=None) == b.DP_ERR_WORKSPACE
+    assert b.dp_debug_example_noise_z(None, 4, 0, 0, 0, 0, stream=0) == b.DP_ERR_INVALID_ARG
+    assert b.dp_debug_example_noise_z(A, 4, 0, 2**31, 0, 0, stream=0) == b.DP_ERR_INVALID_ARG
+
+
 def test_noise_rejects_bad_arguments(b):
     A = 4096
     call = lambda acc=A, P=16, off=0, sigma=1.0, C=1.0, tb=8, out=A: b.dp_noise_average(acc, P, off, sigma, C, tb, 0, 0, out, stream=0)
