@@ -310,7 +310,8 @@ class PerLayer:
         self.torch, self.synth, self.dist, self.world, self.b = torch, synth, dist, world, binding
         self.cfg = synth.resnet50_per_layer()
         self.layers, self.B, self.G = self.cfg["layers"], self.cfg["B"], self.cfg["G"]
-        self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"])
+        self.lanes = int(os.environ.get("DP_BENCH_LANES", "4")) if world == 1 else 1
+        self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"], lanes=self.lanes)
         self.examples_per_step = self.B * self.G
         g = torch.Generator(device="cuda"); g.manual_seed(4000 + rank)
         self.inputs = []
@@ -334,17 +335,23 @@ class PerLayer:
                             "weight + bias), bf16 X/dY ~N(0,1), B=32 per chunk x 32 chunks = |B| 1024, C=1.0 (C_l = C/sqrt(161)), "
                             "sigma=1.0; clip + accumulate fused into dp_per_example_wgrad",
                 "examples_per_step": self.examples_per_step, "params": self.step_obj.P,
-                "l2": f"one chunk of inputs is {self.in_bytes / 1e9:.2f} GB, far larger than L2"}
+                "l2": f"one chunk of inputs is {self.in_bytes / 1e9:.2f} GB, far larger than L2",
+                "streams": self.lanes}
 
     def run(self, i, rec=None):
+        """With a recorder the calls run one after the other on one stream so that each can be timed; otherwise the
+        chunk's calls are spread over the step object's lanes."""
         st = self.step_obj
         st.begin()
         for c in range(self.G):
-            for li, (X, dY) in enumerate(self.inputs):
-                k = self.kind_of[li]
-                if rec: rec.start(k)
-                st.wgrad(li, X, dY)
-                if rec: rec.stop(k)
+            if rec is None:
+                st.chunk_calls(self.inputs)
+            else:
+                for li, (X, dY) in enumerate(self.inputs):
+                    k = self.kind_of[li]
+                    rec.start(k)
+                    st.wgrad(li, X, dY)
+                    rec.stop(k)
             st.chunks_done += 1
         if rec: rec.start(4)
         st.finish(seed=0, step=i)
@@ -355,8 +362,7 @@ class PerLayer:
         t, st = self.torch, self.step_obj
         self.chunk_graph = t.cuda.CUDAGraph()
         with t.cuda.graph(self.chunk_graph):
-            for li, (X, dY) in enumerate(self.inputs):
-                st.wgrad(li, X, dY)
+            st.chunk_calls(self.inputs)
 
     def run_graphed(self, i):
         st = self.step_obj

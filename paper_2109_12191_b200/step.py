@@ -162,7 +162,10 @@ class PerLayerClipStep:
     """Per-layer clipping (threshold C/sqrt(L) per parameter tensor) fused into the weight-gradient call:
     no per-example gradient is written to memory."""
 
-    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda"):
+    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda", lanes=1):
+        """lanes > 1: chunk() spreads the layer calls over that many CUDA streams (each with a workspace of its own).
+        The calls of one chunk touch disjoint outputs, so they may overlap; a chunk of few examples leaves most of
+        the GPU idle inside any single call."""
         self.layers, self.B, self.dtype, self.C, self.sigma = list(layers), B, dtype, float(C), float(sigma)
         self.tensors = _tensors_of(self.layers)
         self.L = len(self.tensors)
@@ -172,13 +175,23 @@ class PerLayerClipStep:
         self.acc_b = [torch.zeros(l.n_bias, dtype=torch.float32, device=device) if l.n_bias else None for l in self.layers]
         self.sq = torch.zeros((B, self.L), dtype=torch.float32, device=device)
         ws = max([b.dp_workspace_bytes(d, b.DP_EPI_CLIP_ACCUM) for d in self.descs] + [256])
-        self.ws = torch.empty(ws, dtype=torch.uint8, device=device)
+        self.lanes = max(1, int(lanes))
+        self.ws_lane = [torch.empty(ws, dtype=torch.uint8, device=device) for _ in range(self.lanes)]
+        self.ws = self.ws_lane[0]
         self._col, col = [], 0
         for l in self.layers:
             self._col.append(col)
             col += 2 if l.n_bias else 1
         self.P = sum(t[2] for t in self.tensors)
         self.chunks_done = 0
+        self._side = [torch.cuda.Stream(device=device) for _ in range(self.lanes - 1)] if self.lanes > 1 else []
+        # layer -> lane: each call goes to the lane with the least work so far (a rough per-call cost is enough)
+        load, self._lane_of = [0.0] * self.lanes, []
+        for l in self.layers:
+            cost = 12.0 + (l.flops() * B / 2.0e8 if l.kind == "conv" else 6.0)
+            k = min(range(self.lanes), key=lambda q: load[q])
+            load[k] += cost
+            self._lane_of.append(k)
 
     def begin(self):
         for a in self.acc_w:
@@ -188,15 +201,39 @@ class PerLayerClipStep:
                 a.zero_()
         self.chunks_done = 0
 
-    def wgrad(self, li, X, dY):
+    def wgrad(self, li, X, dY, lane=0, stream=None):
         b.check(b.dp_per_example_wgrad(self.descs[li], X, dY, None, None, self.sq.data_ptr() + 4 * self._col[li], self.L,
-                                       b.DP_EPI_CLIP_ACCUM, self.C_l, self.acc_w[li], self.acc_b[li], None, self.ws),
-                "dp_per_example_wgrad")
+                                       b.DP_EPI_CLIP_ACCUM, self.C_l, self.acc_w[li], self.acc_b[li], None,
+                                       self.ws_lane[lane], stream=stream), "dp_per_example_wgrad")
+
+    def chunk_calls(self, inputs):
+        """The layer calls of one chunk: in order on the current stream, or forked over the lanes and joined again."""
+        if self.lanes == 1:
+            for li, (X, dY) in enumerate(inputs):
+                self.wgrad(li, X, dY)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        streams = [main] + self._side
+        for s in self._side:
+            s.wait_event(fork)
+        for li, (X, dY) in enumerate(inputs):
+            k = self._lane_of[li]
+            self.wgrad(li, X, dY, lane=k, stream=streams[k])
+        for s in self._side:
+            done = torch.cuda.Event()
+            done.record(s)
+            main.wait_event(done)
 
     def chunk(self, inputs):
-        for li, (X, dY) in enumerate(inputs):
-            self.wgrad(li, X, dY)
+        self.chunk_calls(inputs)
         self.chunks_done += 1
+
+    def check(self):
+        """Status words of the tensor-core launches of every lane (synchronises)."""
+        for w in self.ws_lane:
+            b.check(b.dp_wgrad_check(w), "dp_wgrad_check")
 
     def finish(self, seed=0, step=0):
         """Noise uses the whole-gradient bound C (the per-tensor thresholds keep the sensitivity at C)."""

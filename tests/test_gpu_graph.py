@@ -70,3 +70,35 @@ def test_per_layer_workload_full_size_layers(which):
         got = (st.acc_w[0] if gi == 0 else st.acc_b[0]).cpu().numpy()
         # capturing records without running: the accumulator holds the single replay's contribution
         assert rel_l2(got, np.einsum("n,np->p", f, grad)) <= TOL_ACC_BF16
+
+
+def test_layer_calls_spread_over_streams_give_the_same_bits():
+    """The per-layer step may fork its layer calls over several streams (one workspace each) and join them again; the
+    calls write disjoint outputs, so the result must equal the single-stream one bit for bit, also from a replayed graph."""
+    layers = [synth.conv(64, 64, 3, 1, 1, 14, name="a"), synth.norm(64, 14, "gn_a"), synth.conv(64, 128, 1, 1, 0, 14, name="b"),
+              synth.norm(128, 14, "gn_b"), synth.conv(128, 128, 3, 2, 1, 14, name="c"), synth.norm(128, 7, "gn_c"),
+              synth.dense(128, 10, True, "fc")]
+    Bn = 8
+    ins = [dev_inputs(synth.layer_inputs(l, Bn, "bf16", 961, li), "bf16") for li, l in enumerate(layers)]
+
+    def result(st):
+        return torch.cat([t for pair in zip(st.acc_w, st.acc_b) for t in pair if t is not None]).clone()
+
+    one = PerLayerClipStep(layers, Bn, "bf16", 50.0, 1.0)
+    one.begin(); one.chunk(ins); one.chunk(ins)
+    torch.cuda.synchronize()
+    many = PerLayerClipStep(layers, Bn, "bf16", 50.0, 1.0, lanes=3)
+    assert len(set(many._lane_of)) == 3
+    many.begin(); many.chunk(ins); many.chunk(ins)
+    torch.cuda.synchronize()
+    many.check()
+    assert torch.equal(result(many), result(one))
+    assert torch.equal(many.sq, one.sq)
+    many.begin()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        many.chunk_calls(ins)
+    g.replay(); g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(result(many), result(one))
