@@ -188,6 +188,85 @@ scale_accumulate_kernel(const __grid_constant__ SegTable tab, const float *__res
     }
 }
 
+// stage 3 for small models with many examples: too few 1024-parameter blocks exist to fill the GPU, so a block takes
+// only 128 parameters and splits the example rows over its eight warps (warp w owns rows w, w+8, ...), sixteen rows in
+// flight per thread; the eight partial sums are folded in warp order through shared memory.
+constexpr int kSplitCols = 128;
+__global__ void __launch_bounds__(256)
+scale_accumulate_rowsplit_kernel(const __grid_constant__ SegTable tab, const float *__restrict__ factor, int B, int L,
+                                 int per_layer) {
+    __shared__ float f_sh[256];
+    __shared__ float4 part[8][32];
+    const int seg = find_seg(tab, blockIdx.x);
+    const long long P = tab.P[seg];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const long long i = (long long)(blockIdx.x - tab.blk_start[seg]) * kSplitCols + 4 * lane;
+    const float *G = tab.G[seg];
+    float *acc = tab.acc[seg];
+    const int f_stride = per_layer ? L : 1;
+    const int f_off = per_layer ? tab.col[seg] : 0;
+    const bool vec = ((P & 3) == 0) && ((reinterpret_cast<uintptr_t>(G) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(acc) & 15) == 0);
+    const int live = i >= P ? 0 : (int)min(4ll, P - i);           // parameters this thread owns (vec: 0 or 4)
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int n0 = 0; n0 < B; n0 += 256) {
+        const int nb = min(256, B - n0);
+        __syncthreads();
+        if (threadIdx.x < nb) f_sh[threadIdx.x] = factor[(long long)(n0 + threadIdx.x) * f_stride + f_off];
+        __syncthreads();
+        if (live == 0) continue;
+        const float *g = G + (long long)n0 * P + i;
+        if (vec) {
+            int n = w;
+            for (; n + 8 * 15 < nb; n += 8 * 16) {
+                float4 v[16];
+#pragma unroll
+                for (int u = 0; u < 16; ++u) v[u] = __ldcs(reinterpret_cast<const float4 *>(g + (long long)(n + 8 * u) * P));
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const float f = f_sh[n + 8 * u];
+                    s.x = fmaf(f, v[u].x, s.x); s.y = fmaf(f, v[u].y, s.y);
+                    s.z = fmaf(f, v[u].z, s.z); s.w = fmaf(f, v[u].w, s.w);
+                }
+            }
+            for (; n < nb; n += 8) {
+                const float4 v = __ldcs(reinterpret_cast<const float4 *>(g + (long long)n * P));
+                const float f = f_sh[n];
+                s.x = fmaf(f, v.x, s.x); s.y = fmaf(f, v.y, s.y); s.z = fmaf(f, v.z, s.z); s.w = fmaf(f, v.w, s.w);
+            }
+        } else {
+            for (int n = w; n < nb; n += 8) {
+                const float *row = g + (long long)n * P;
+                const float f = f_sh[n];
+                s.x = fmaf(f, row[0], s.x);
+                if (live > 1) s.y = fmaf(f, row[1], s.y);
+                if (live > 2) s.z = fmaf(f, row[2], s.z);
+                if (live > 3) s.w = fmaf(f, row[3], s.w);
+            }
+        }
+    }
+    part[w][lane] = s;
+    __syncthreads();
+    if (w == 0 && live > 0) {
+        float4 t = part[0][lane];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) {
+            const float4 v = part[q][lane];
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        if (vec) {
+            float4 a = *reinterpret_cast<const float4 *>(acc + i);
+            a.x += t.x; a.y += t.y; a.z += t.z; a.w += t.w;
+            *reinterpret_cast<float4 *>(acc + i) = a;
+        } else {
+            acc[i] += t.x;
+            if (live > 1) acc[i + 1] += t.y;
+            if (live > 2) acc[i + 2] += t.z;
+            if (live > 3) acc[i + 3] += t.w;
+        }
+    }
+}
+
 // stage 3 with per-example noise: acc[i] += sum_n ( factor * G[n, i] + sd * z_{example0+n}(goff + i) ).
 // Every thread owns the four parameters of one Philox block when the tensor starts on a multiple of four global
 // indices; otherwise each parameter draws its own block and keeps one lane.  Bound by the integer and
@@ -319,7 +398,7 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
     if (!plan(B, L, P_l, pl)) return DP_ERR_INVALID_ARG;
     for (int l = 0; l < L; ++l) {
         if (!G[l] || !acc[l] || !aligned(G[l], 4) || !aligned(acc[l], 4)) return DP_ERR_INVALID_ARG;
-        if ((P_l[l] + kAccCols - 1) / kAccCols > 0x3fffffffll) return DP_ERR_UNSUPPORTED;
+        if ((P_l[l] + kSplitCols - 1) / kSplitCols > 0x3fffffffll) return DP_ERR_UNSUPPORTED;
     }
     if (sqnorm && !aligned(sqnorm, 4)) return DP_ERR_INVALID_ARG;
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < pl.total) return DP_ERR_WORKSPACE;
@@ -333,10 +412,10 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
     // tensors go to the kernels in tables of at most kMaxSeg entries
     long long wide_blocks = 0;
     for (int l = 0; l < L; ++l) wide_blocks += (P_l[l] + kAccCols - 1) / kAccCols;
-    // A small model gives few blocks, and each thread then walks all B rows in B/UNROLL dependent trips of one
-    // memory latency each: with many rows, 32 rows in flight per thread instead of 8 quarters that chain.
-    const bool deep = B >= 64 && wide_blocks < 8 * 148;
-    const int acc_cols = kAccCols;
+    // A small model gives few blocks, and each thread would walk all B rows alone: with many rows the block narrows
+    // to 128 parameters and its warps share the rows.
+    const bool split = B >= 64 && wide_blocks < 8 * 148;
+    const int acc_cols = (split && !noise) ? kSplitCols : kAccCols;
 
     auto fill = [&](int l0, SegTable &t, bool norm_blocks, long long &part_cursor) {
         t.nseg = 0;
@@ -384,7 +463,7 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
             const int blocks = fill(l0, t, false, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
             if (noise) scale_accumulate_noised_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer, *noise);
-            else if (deep) scale_accumulate_kernel<32><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
+            else if (split) scale_accumulate_rowsplit_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             else scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             DP_LAUNCH_CHECK("scale_accumulate_kernel");
             l0 += t.nseg;

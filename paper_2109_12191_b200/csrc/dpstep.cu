@@ -151,6 +151,9 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
 
     if (d->kind == DP_LAYER_CONV2D) {
         float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;
+        if (pl.use_thin && rgb3_conv_eligible(g))
+            return launch_conv_rgb3(d->dtype, X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, d->has_bias, groups == 2,
+                                    sqnorm, sqnorm_stride, reset, st);
         if (pl.use_thin) {
             rc = launch_conv_thin(d->dtype, X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, partial, pl.slots, d->has_bias, st);
             if (rc != DP_OK) return rc;

@@ -172,23 +172,28 @@ conv_wgrad_thin_kernel(const T *__restrict__ X, const T *__restrict__ dY, const 
     __syncthreads();
     int oh = pg / g.OW, ow = pg - oh * g.OW;
     const T *dYn = dY + (long long)n * g.K * g.Kout;
-    // four pixels per trip: their dY loads are issued together so the memory latency is paid once per trip
-    for (int pix = pg; pix < g.K; pix += 32) {
-        float gy[4][KPT];
-        int base[4];
+    // U pixels per trip, and the next trip's dY loads are issued before this trip's arithmetic: a warp always has
+    // U (then 2U) 128-byte rows in flight, which is what hides the memory latency at one or two blocks per SM.
+    constexpr int U = 8;
+    float gy[U][KPT], gyn[U][KPT];
+    int base[U], basen[U];
+    auto load_trip = [&](int pix, float (&y)[U][KPT], int (&b)[U]) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int pu = pix + 8 * u;
-            base[u] = (oh * g.stride * Wp + ow * g.stride) * g.Cin;
+            b[u] = pu < g.K ? (oh * g.stride * Wp + ow * g.stride) * g.Cin : 0;
 #pragma unroll
             for (int kk = 0; kk < KPT; ++kk)
-                gy[u][kk] = pu < g.K ? to_float(dYn[(long long)pu * g.Kout + lane + 32 * kk]) : 0.f;
-            if (pu >= g.K) base[u] = 0;
+                y[u][kk] = pu < g.K ? to_float(dYn[(long long)pu * g.Kout + lane + 32 * kk]) : 0.f;
             ow += 8;
             while (ow >= g.OW) { ow -= g.OW; ++oh; }
         }
+    };
+    load_trip(pg, gy, base);
+    for (int pix = pg; pix < g.K; pix += 8 * U) {
+        if (pix + 8 * U < g.K) load_trip(pix + 8 * U, gyn, basen);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
 #pragma unroll
             for (int kk = 0; kk < KPT; ++kk) bsum[kk] += gy[u][kk];
             if constexpr (RT > 0) {
@@ -233,6 +238,12 @@ conv_wgrad_thin_kernel(const T *__restrict__ X, const T *__restrict__ dY, const 
                     }
                 }
             }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            base[u] = basen[u];
+#pragma unroll
+            for (int kk = 0; kk < KPT; ++kk) gy[u][kk] = gyn[u][kk];
         }
     }
     const int MN = g.Kout * g.N;
@@ -300,6 +311,192 @@ dp_status launch_conv_thin(int dtype, const void *X, const void *dY, const ConvG
         else thin_launch_t<__nv_bfloat16, 2>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), g, G_w, db, partial, slots, has_bias, smem, st);
     }
     DP_LAUNCH_CHECK("conv_wgrad_thin_kernel");
+    return DP_OK;
+}
+
+// 3x3 convolutions on three input channels (image stems), output channels a multiple of 32: one block per example,
+// the zero-padded image in shared memory.  Lane = output pixel (32 consecutive pixels per trip), warp w owns output
+// channels 4w .. 4w+3 of the current group of 32, so a thread keeps a 4 x 27 block of the gradient in registers, every
+// shared-memory word it reads feeds four FMAs, and the 32 lanes read 32 different words (3 floats apart: no bank
+// conflict) instead of one broadcast word.  A trip is short (a few hundred cycles) against the memory latency, so dY
+// streams through a ring of kRgbStages stages of 64 pixels x 32 channels, filled by coalesced asynchronous copies
+// (cp.async, each thread two pieces of four channels per stage) three stages ahead of the arithmetic, one barrier per
+// stage.  Inside a stage the piece of (pixel l, channel quad c) sits at quad position c ^ (l & 7) of its pixel row, so
+// that the 32 lanes of a warp, which read the same quad of 32 different pixels, hit different banks.  The 32 pixel
+// lanes are folded by two shuffle steps and then, in lane order, through shared memory; gradient, bias gradient and
+// the example's squared norms leave from the same pass.
+constexpr int kRgbRed = 113;      // floats per (warp, lane group) in the fold buffer: 4 x 27 weights + 4 bias sums (+1: odd stride)
+constexpr int kRgbStages = 4;     // stages of dY in the ring
+constexpr int kRgbStagePix = 64;  // pixels per stage (two trips)
+constexpr int kRgbStageFloats = kRgbStagePix * 32;   // ring stride in 4-byte words (bf16 stages use half of it)
+
+template <int BYTES>
+__device__ __forceinline__ void cp_async_zfill(void *smem_dst, const void *src, bool valid) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    const int n = valid ? BYTES : 0;                          // 0 source bytes: the destination is zero-filled
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;\n" ::"r"(dst), "l"(src), "n"(BYTES), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+template <typename T>
+__global__ void __launch_bounds__(256, 1)
+conv_wgrad_rgb3_kernel(const T *__restrict__ X, const T *__restrict__ dY, const ConvGeom g, float *__restrict__ G_w,
+                       float *__restrict__ db, int has_bias, int separate, float *__restrict__ sqnorm,
+                       long long sq_stride, int *status_reset) {
+    extern __shared__ __align__(16) float rgb_smem[];
+    __shared__ double scratch[32];
+    constexpr int kQuad = 4 * (int)sizeof(T);                // bytes of four output channels of dY
+    const int Hp = g.H + 2 * g.pad, Wp = g.W + 2 * g.pad, row_p = Wp * 3;
+    const int xs_count = Hp * row_p;
+    char *ring = reinterpret_cast<char *>(rgb_smem);         // [kRgbStages][64 pixels][8 quads]; afterwards the fold
+    float *red = rgb_smem;                                   //   buffer [8 warps][8 lane groups][kRgbRed]
+    float *xs = rgb_smem + kRgbStages * kRgbStageFloats;     // [Hp][Wp][3], zero border
+    const int n = blockIdx.x, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (status_reset && n == 0 && threadIdx.x == 0) *status_reset = 0;
+    {
+        const int row_in = g.W * 3;
+        for (int i = threadIdx.x; i < xs_count; i += 256) xs[i] = 0.f;
+        __syncthreads();
+        const T *Xn = X + (long long)n * g.H * row_in;
+        for (int i = threadIdx.x; i < g.H * row_in; i += 256) {
+            const int h = i / row_in, rest = i - h * row_in;
+            xs[(h + g.pad) * row_p + g.pad * 3 + rest] = to_float(Xn[i]);
+        }
+    }
+    float sq = 0.f, sqb = 0.f;
+    const int stages = (g.K + kRgbStagePix - 1) / kRgbStagePix;
+    // copies of this thread: quad cq of pixels cl and cl + 32 of a stage; reads: quad w of pixel lane (+32 on the second trip)
+    const int cl = threadIdx.x >> 3, cq = threadIdx.x & 7;
+    const int copy_off = cl * 8 * kQuad + ((cq ^ (cl & 7)) * kQuad);        // (cl + 32) & 7 == cl & 7
+    const int read_off = lane * 8 * kQuad + ((w ^ (lane & 7)) * kQuad);
+    for (int kg = 0; kg < g.Kout / 32; ++kg) {
+        const T *dyp = dY + (long long)n * g.K * g.Kout + kg * 32;
+        auto fetch = [&](int stage) {                        // one commit group per stage, also past the end
+            char *dst = ring + (stage % kRgbStages) * (kRgbStageFloats * 4) + copy_off;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int p = stage * kRgbStagePix + cl + 32 * h;
+                const bool valid = stage < stages && p < g.K;
+                cp_async_zfill<kQuad>(dst + h * 32 * 8 * kQuad, dyp + (long long)(valid ? p : 0) * g.Kout + 4 * cq, valid);
+            }
+            cp_async_commit();
+        };
+        float acc[4][27], bs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+            for (int j = 0; j < 27; ++j) acc[kk][j] = 0.f;
+        for (int t = 0; t < kRgbStages - 1; ++t) fetch(t);
+        int oh = lane / g.OW, ow = lane - oh * g.OW;         // pixel of this lane in the current trip
+        for (int st = 0; st < stages; ++st) {
+            cp_async_wait<kRgbStages - 2>();                 // this thread's pieces of stage st have landed
+            __syncthreads();                                 // ... and everyone's; stage st-1 is no longer read
+            fetch(st + kRgbStages - 1);                      // refills the slot of stage st-1
+            const char *src = ring + (st % kRgbStages) * (kRgbStageFloats * 4) + read_off;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float gy[4];
+                if constexpr (sizeof(T) == 4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(src + h * 32 * 8 * kQuad);
+                    gy[0] = v.x; gy[1] = v.y; gy[2] = v.z; gy[3] = v.w;
+                } else {
+                    const uint2 v = *reinterpret_cast<const uint2 *>(src + h * 32 * 8 * kQuad);
+                    gy[0] = __uint_as_float(v.x << 16); gy[1] = __uint_as_float(v.x & 0xffff0000u);
+                    gy[2] = __uint_as_float(v.y << 16); gy[3] = __uint_as_float(v.y & 0xffff0000u);
+                }
+                // lanes past the last pixel carry zeros of dY; their patch address is clamped to pixel 0
+                const bool live = st * kRgbStagePix + 32 * h + lane < g.K;
+                const float *patch = xs + (live ? (oh * g.stride * Wp + ow * g.stride) * 3 : 0);
+#pragma unroll
+                for (int r = 0; r < 3; ++r) {
+                    float x[9];
+#pragma unroll
+                    for (int q = 0; q < 9; ++q) x[q] = patch[r * row_p + q];
+#pragma unroll
+                    for (int q = 0; q < 9; ++q)
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) acc[kk][r * 9 + q] = fmaf(gy[kk], x[q], acc[kk][r * 9 + q]);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) bs[kk] += gy[kk];
+                ow += 32;
+                while (ow >= g.OW) { ow -= g.OW; ++oh; }
+            }
+        }
+        cp_async_wait<0>();
+        __syncthreads();                                     // every thread is done with the ring: it becomes the fold buffer
+        // fold the 32 pixel lanes: two butterfly steps leave eight partial sums (lanes 0..7), added in lane order below
+        float *mine = red + (w * 8 + (lane & 7)) * kRgbRed;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+            for (int j = 0; j < 27; ++j) {
+                float v = acc[kk][j];
+                v += __shfl_xor_sync(0xffffffffu, v, 16);
+                v += __shfl_xor_sync(0xffffffffu, v, 8);
+                if (lane < 8) mine[kk * 27 + j] = v;
+            }
+            float v = bs[kk];
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            if (lane < 8) mine[108 + kk] = v;
+        }
+        __syncthreads();
+        // entry o of this group of 32 channels is (warp o/108, register o%108) and sits at G_w[n][kg*864 + o]
+        for (int o = threadIdx.x; o < 864; o += 256) {
+            const float *src = red + (o / 108) * 8 * kRgbRed + (o % 108);
+            float v = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v += src[q * kRgbRed];
+            if (G_w) G_w[(long long)n * g.Kout * 27 + kg * 864 + o] = v;
+            sq = fmaf(v, v, sq);
+        }
+        if (has_bias && threadIdx.x < 32) {
+            const float *src = red + (threadIdx.x >> 2) * 8 * kRgbRed + 108 + (threadIdx.x & 3);
+            float v = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v += src[q * kRgbRed];
+            db[(long long)n * g.Kout + kg * 32 + threadIdx.x] = v;
+            sqb = fmaf(v, v, sqb);
+        }
+        __syncthreads();
+    }
+    const double sw = block_sum((double)sq, scratch);
+    const double sb = block_sum((double)sqb, scratch);
+    if (threadIdx.x == 0) {
+        if (separate) {
+            sqnorm[n * sq_stride] = (float)sw;
+            sqnorm[n * sq_stride + 1] = (float)sb;
+        } else {
+            sqnorm[n * sq_stride] = (float)(sw + sb);
+        }
+    }
+}
+
+static size_t rgb3_smem_bytes(const ConvGeom &g) {
+    static_assert(kRgbStages * kRgbStageFloats >= 8 * 8 * kRgbRed, "the fold buffer reuses the dY ring");
+    const size_t xs = ((size_t)(g.H + 2 * g.pad) * (g.W + 2 * g.pad) * 3 + 3) & ~(size_t)3;
+    return sizeof(float) * (xs + (size_t)kRgbStages * kRgbStageFloats);
+}
+
+bool rgb3_conv_eligible(const ConvGeom &g) {
+    return g.R == 3 && g.S == 3 && g.Cin == 3 && g.Kout % 32 == 0 && g.Kout <= 256 && rgb3_smem_bytes(g) <= 47 * 1024;
+}
+
+dp_status launch_conv_rgb3(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
+                           int has_bias, int separate, float *sqnorm, long long sq_stride, int *status_reset,
+                           cudaStream_t st) {
+    const size_t smem = rgb3_smem_bytes(g);
+    if (dtype == DP_F32)
+        conv_wgrad_rgb3_kernel<float><<<g.B, 256, smem, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), g,
+                                                              G_w, db, has_bias, separate, sqnorm, sq_stride, status_reset);
+    else
+        conv_wgrad_rgb3_kernel<__nv_bfloat16><<<g.B, 256, smem, st>>>(static_cast<const __nv_bfloat16 *>(X),
+                                                                      static_cast<const __nv_bfloat16 *>(dY), g, G_w, db,
+                                                                      has_bias, separate, sqnorm, sq_stride, status_reset);
+    DP_LAUNCH_CHECK("conv_wgrad_rgb3_kernel");
     return DP_OK;
 }
 

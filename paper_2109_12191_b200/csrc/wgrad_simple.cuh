@@ -30,6 +30,12 @@ dp_status launch_conv_fma(int dtype, int mode, const void *X, const void *dY, co
 bool thin_conv_eligible(const ConvGeom &g);
 dp_status launch_conv_thin(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
                            float *partial, int slots, int has_bias, cudaStream_t stream);
+// 3x3 convolutions on three input channels with a multiple of 32 output channels: gradient (G_w may be null), bias
+// gradient and the published squared norms (sqnorm[n*sq_stride + {0,1}] when `separate`, else their sum) in one launch.
+bool rgb3_conv_eligible(const ConvGeom &g);
+dp_status launch_conv_rgb3(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
+                           int has_bias, int separate, float *sqnorm, long long sq_stride, int *status_reset,
+                           cudaStream_t stream);
 // db[n,k] = sum over pixels of dY; also sum_k db^2 per block into partial[n*slots + slot0 + block]
 dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
                       cudaStream_t stream);

@@ -52,7 +52,9 @@ class GlobalClipStep:
     """Whole-model clipping: per-example gradients are materialised per layer (STORE+NORM epilogue),
     one dp_clip_accumulate call per chunk consumes them with the norms the epilogues produced."""
 
-    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda", per_example_noise=False):
+    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda", per_example_noise=False, lanes=1):
+        """lanes > 1: chunk() spreads the layers' weight-gradient calls over that many CUDA streams (a workspace each)
+        and joins them before the clip: the calls write disjoint buffers, so they may overlap."""
         self.layers, self.B, self.dtype, self.C, self.sigma = list(layers), B, dtype, float(C), float(sigma)
         self.per_example_noise = bool(per_example_noise)
         self.tensors = _tensors_of(self.layers)
@@ -73,7 +75,10 @@ class GlobalClipStep:
         self.norms = torch.empty(B, dtype=torch.float32, device=device)
         self.clip = torch.empty(B, dtype=torch.float32, device=device)
         ws = max([b.dp_workspace_bytes(d, b.DP_EPI_STORE_NORM) for d in self.descs] + [256])
-        self.ws = torch.empty(ws, dtype=torch.uint8, device=device)
+        self.lanes = max(1, min(int(lanes), len(self.layers)))
+        self.ws_lane = [torch.empty(ws, dtype=torch.uint8, device=device) for _ in range(self.lanes)]
+        self.ws = self.ws_lane[0]
+        self._side = [torch.cuda.Stream(device=device) for _ in range(self.lanes - 1)] if self.lanes > 1 else []
         self.clip_ws = torch.empty(max(b.dp_clip_workspace_bytes(B, self.P_l), 256), dtype=torch.uint8, device=device)
         # column of each layer's first tensor in the [B, L] norm table, and its G buffers
         self._col, col = [], 0
@@ -88,12 +93,33 @@ class GlobalClipStep:
         self.chunks_done = 0
         self._noise = _NoiseKey(self.per_example_noise, total_batch, seed, step, example0)
 
-    def wgrad(self, li, X, dY):
+    def wgrad(self, li, X, dY, lane=0, stream=None):
         col = self._col[li]
         G_w = self.G[col]
         G_b = self.G[col + 1] if self.layers[li].n_bias else None
         b.check(b.dp_per_example_wgrad(self.descs[li], X, dY, G_w, G_b, self.sq.data_ptr() + 4 * col, self.L,
-                                       b.DP_EPI_STORE_NORM, 0.0, None, None, None, self.ws), "dp_per_example_wgrad")
+                                       b.DP_EPI_STORE_NORM, 0.0, None, None, None, self.ws_lane[lane], stream=stream),
+                "dp_per_example_wgrad")
+
+    def wgrad_all(self, inputs):
+        """Every layer's weight-gradient call: in order on the current stream, or forked over the lanes and joined."""
+        if self.lanes == 1:
+            for li, (X, dY) in enumerate(inputs):
+                self.wgrad(li, X, dY)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        streams = [main] + self._side
+        for s in self._side:
+            s.wait_event(fork)
+        for li, (X, dY) in enumerate(inputs):
+            k = li % self.lanes
+            self.wgrad(li, X, dY, lane=k, stream=streams[k])
+        for s in self._side:
+            done = torch.cuda.Event()
+            done.record(s)
+            main.wait_event(done)
 
     def clip_accumulate(self, use_epilogue_norms=True):
         sq = self.sq if use_epilogue_norms else None
@@ -110,8 +136,7 @@ class GlobalClipStep:
 
     def chunk(self, inputs):
         """inputs: list of (X, dY) device tensors, one pair per layer."""
-        for li, (X, dY) in enumerate(inputs):
-            self.wgrad(li, X, dY)
+        self.wgrad_all(inputs)
         self.clip_accumulate()
 
     def finish(self, seed=0, step=0, world=1):

@@ -79,7 +79,7 @@ def test_conv_cuda_core(case, dtype):
 
 
 THIN_CONVS = [(3, 32, 3, 1, 1, 32, True), (3, 64, 3, 2, 1, 17, False), (2, 32, 3, 1, 0, 9, True), (1, 32, 5, 1, 2, 12, True),
-              (3, 32, 3, 1, 1, 3, False)]
+              (3, 32, 3, 1, 1, 3, False), (3, 64, 3, 1, 1, 13, True)]
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
