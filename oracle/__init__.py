@@ -178,6 +178,36 @@ def clipped_sum(groups, C, mode, acc=None):
     return acc, sq, factor
 
 
+def clipped_sum_grouped(groups, group_of, C, acc=None):
+    """Section 3.5 with M groups of parameter tensors (the paper's pipeline stages): group m holds the tensors l with
+    group_of[l] == m, its per-example norm is taken over all of them, and it is clipped to C/sqrt(M).
+    Returns (acc, sq [B, M], factor [B, M])."""
+    L, B = len(groups), groups[0].shape[0]
+    group_of = [int(m) for m in group_of]
+    M = max(group_of) + 1
+    assert len(group_of) == L and sorted(set(group_of)) == list(range(M))
+    sq = np.zeros((B, M), dtype=np.float64)
+    for g, m in zip(groups, group_of):
+        sq[:, m] += sqnorm(g)
+    factor = clip_factor(sq, C / np.sqrt(M)).reshape(B, M)
+    if acc is None:
+        acc = [np.zeros(int(np.prod(g.shape[1:])), dtype=np.float64) for g in groups]
+    for g, m, a in zip(groups, group_of, acc):
+        clip_accumulate(g, np.ascontiguousarray(factor[:, m]), a)
+    return acc, sq, factor
+
+
+def clipped_sum_micro(groups, C, micro, acc=None):
+    """Micro-batch clipping (the TFDP option of the paper's Table 1): consecutive runs of `micro` examples are
+    averaged first, the average is clipped to C over the whole model, and the clipped averages are summed.
+    Returns (acc, sq [B/micro] of the averages, factor [B/micro])."""
+    B = groups[0].shape[0]
+    assert micro >= 1 and B % micro == 0
+    means = [g.reshape(B // micro, micro, -1).astype(np.float64).mean(axis=1) for g in groups]
+    acc, sq, factor = clipped_sum(means, C, "global", acc)
+    return acc, sq.sum(axis=1), factor
+
+
 # ----------------------------------------------------------------------------- noise
 def philox4x32_10(ctr, key):
     """Raw Philox4x32-10: 4 counter words, 2 key words -> 4 output words."""

@@ -163,3 +163,71 @@ def test_sgd_update_plain_and_momentum_closed_form():
         w.grad = torch.from_numpy(g.copy())
         opt.step()
     np.testing.assert_allclose(theta, w.detach().numpy(), rtol=1e-13)
+
+
+def test_grouped_clipping_special_cases_and_bound():
+    """Section 3.5 with M groups of tensors: one tensor per group is per-layer clipping, one group is whole-model
+    clipping, and in between every group keeps norm <= C/sqrt(M), hence the whole vector norm <= C."""
+    B, sizes, C = 10, [10, 200, 3, 64, 17], 0.8
+    groups = _groups(B, sizes, 20)
+    scale = np.logspace(-2.5, 0.5, B).astype(np.float32)
+    groups = [g * scale[:, None] for g in groups]
+    acc_a, _, f_a = oracle.clipped_sum_grouped(groups, [0, 1, 2, 3, 4], C)
+    acc_b, _, f_b = oracle.clipped_sum(groups, C, "per_layer")
+    np.testing.assert_array_equal(f_a, f_b)
+    for a, b in zip(acc_a, acc_b):
+        np.testing.assert_array_equal(a, b)
+    acc_a, _, f_a = oracle.clipped_sum_grouped(groups, [0] * 5, C)
+    acc_b, _, f_b = oracle.clipped_sum(groups, C, "global")
+    np.testing.assert_array_equal(f_a[:, 0], f_b)
+    for a, b in zip(acc_a, acc_b):
+        np.testing.assert_array_equal(a, b)
+    # two stages, tensors interleaved; brute force with numpy on the concatenated stage vectors
+    group_of = [1, 0, 1, 0, 0]
+    acc, sq, f = oracle.clipped_sum_grouped(groups, group_of, C)
+    thr = C / math.sqrt(2)
+    total = np.zeros(B)
+    for m in range(2):
+        flat = np.concatenate([g.astype(np.float64) for g, mm in zip(groups, group_of) if mm == m], axis=1)
+        norms = np.linalg.norm(flat, axis=1)
+        np.testing.assert_allclose(np.sqrt(sq[:, m]), norms, rtol=1e-13)
+        np.testing.assert_allclose(f[:, m], np.minimum(1.0, thr / norms), rtol=1e-14)
+        clipped = np.linalg.norm(flat * f[:, m:m + 1], axis=1)
+        assert np.all(clipped <= thr * (1 + 1e-14))
+        total += clipped ** 2
+    assert np.all(np.sqrt(total) <= C * (1 + 1e-14))
+    assert (f == 1.0).any() and (f < 1.0).any()
+    for g, m, a in zip(groups, group_of, acc):
+        np.testing.assert_allclose(a, np.einsum("n,np->p", f[:, m], g.astype(np.float64)), rtol=1e-13, atol=1e-18)
+
+
+def test_micro_batch_clipping_special_cases_and_brute_force():
+    """Clipping the mean of each run of `micro` examples: micro = 1 is per-example clipping; with C = inf the sum of the
+    micro-batch means times micro is the plain sum; otherwise a Python loop over micro-batches gives the same."""
+    B, sizes, C = 12, [33, 7], 0.05
+    groups = _groups(B, sizes, 21, scale=0.02)
+    scale = np.logspace(-1.5, 1.0, B).astype(np.float32)
+    groups = [g * scale[:, None] for g in groups]
+    acc_a, sq_a, f_a = oracle.clipped_sum_micro(groups, C, 1)
+    acc_b, sq_b, f_b = oracle.clipped_sum(groups, C, "global")
+    np.testing.assert_allclose(f_a, f_b, rtol=1e-15)
+    for a, b in zip(acc_a, acc_b):
+        np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-18)
+    acc, _, f = oracle.clipped_sum_micro(groups, math.inf, 4)
+    assert np.all(f == 1.0)
+    for a, g in zip(acc, groups):
+        np.testing.assert_allclose(4 * a, g.astype(np.float64).sum(0), rtol=1e-12, atol=1e-15)
+    mu = 3
+    acc, sq, f = oracle.clipped_sum_micro(groups, C, mu)
+    want = [np.zeros(p) for p in sizes]
+    for j in range(B // mu):
+        mean = [sum(g[j * mu + i].astype(np.float64) for i in range(mu)) / mu for g in groups]
+        norm = math.sqrt(sum(float(np.dot(m, m)) for m in mean))
+        fac = 1.0 if norm <= C else C / norm
+        assert abs(f[j] - fac) <= 1e-15 and abs(math.sqrt(sq[j]) - norm) <= 1e-13 * norm
+        assert norm * fac <= C * (1 + 1e-14)
+        for w, m in zip(want, mean):
+            w += fac * m
+    assert (f == 1.0).any() and (f < 1.0).any()
+    for a, w in zip(acc, want):
+        np.testing.assert_allclose(a, w, rtol=1e-12, atol=1e-18)
