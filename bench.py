@@ -241,7 +241,11 @@ class FlatGrad:
         self.P, self.B, self.G = self.cfg["P"], self.cfg["B"], self.cfg["G"]
         if os.environ.get("DPSTEP_FLAT_PARAMS"):          # reduced P for profiler captures (same kernels, fewer bytes held)
             self.P = int(os.environ["DPSTEP_FLAT_PARAMS"])
-        self.step_obj = FlatClipStep(self.P, self.B, self.cfg["C"], self.cfg["sigma"])
+        # --variant: "per_example_noise" (the paper's own form of the noise) or "microN" (clip the mean of N examples)
+        self.variant = VARIANT
+        micro = int(self.variant[5:]) if self.variant.startswith("micro") else 1
+        self.step_obj = FlatClipStep(self.P, self.B, self.cfg["C"], self.cfg["sigma"],
+                                     per_example_noise=(self.variant == "per_example_noise"), micro=micro)
         self.examples_per_step = self.B * self.G
         g = torch.Generator(device="cuda"); g.manual_seed(2000 + rank)
         self.bufs = []
@@ -253,13 +257,14 @@ class FlatGrad:
 
     def describe(self):
         return {"workload": f"flat: ResNet-50 (GroupNorm) flattened per-example gradients, P={self.P:,} fp32 ~N(0,1e-6), "
-                            "B=64 per chunk x 16 chunks = |B| 1024, global clip C=1.0, sigma=1.0; norms computed by the library",
+                            "B=64 per chunk x 16 chunks = |B| 1024, global clip C=1.0, sigma=1.0; norms computed by the library"
+                            + ("" if self.variant == "plain" else f"; variant {self.variant}"),
                 "examples_per_step": self.examples_per_step, "params": self.P,
                 "l2": "each chunk is 6.54 GB, far larger than L2; two resident chunks alternate"}
 
     def run(self, i, rec=None):
         st = self.step_obj
-        st.begin()
+        st.begin(total_batch=self.B * self.G * self.world, seed=0, step=i)
         for c in range(self.G):
             if rec: rec.start(0)
             st.chunk(self.bufs[c & 1])
@@ -274,6 +279,17 @@ class FlatGrad:
             return 2 * self.B * self.P * 4 + 2 * self.P * 4   # norm pass + clip pass over the chunk, accumulator r+w
         return 2 * self.P * 4
 
+    def roofline(self, dom, avg_ms_per_chunk, peaks):
+        """Per-example noise draws B*P normals per chunk and is bound by integer and transcendental arithmetic: about
+        45 instructions per normal (a quarter of a ten-round Philox block, half a Box-Muller pair, the scaled add), so
+        the ceiling is SMs x 128 lanes x SM clock / 45 normals per second."""
+        if self.variant != "per_example_noise" or dom != 0:
+            return None
+        peak = 148 * 128 * 1.965e9 / 45.0 / 1e9
+        got = self.B * self.P / (avg_ms_per_chunk / 1e3) / 1e9
+        return {"bound": "alu", "achieved": round(got, 1), "peak": round(peak, 1), "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz / 45 instructions per normal",
+                "unit": "Gnormal/s", "frac": round(got / peak, 4)}
+
     def e2e_prepare(self):
         t = self.torch
         self.host_chunk = t.empty((self.B, self.P), dtype=t.float32).pin_memory()
@@ -283,7 +299,7 @@ class FlatGrad:
 
     def e2e_run(self, i):
         st = self.step_obj
-        st.begin()
+        st.begin(total_batch=self.B * self.G * self.world, seed=0, step=i)
         for c in range(self.G):
             self.bufs[c & 1].copy_(self.host_chunk, non_blocking=True)
             st.chunk(self.bufs[c & 1])
@@ -429,6 +445,7 @@ class PerLayer:
 
 
 WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad, "per_layer": PerLayer}
+VARIANT = "plain"
 
 
 class CallTimer:
@@ -559,7 +576,7 @@ def run_ours(args):
                 "traffic": recorded_traffic(wl.name, wl.call_names[dom]),
                 "shares": {n: round(t / sum(totals), 4) for n, t in zip(wl.call_names, totals)}}
     if hasattr(wl, "roofline"):
-        own = wl.roofline(dom, totals[dom] / (max(1, counts[4]) * wl.G), peaks)
+        own = wl.roofline(dom, totals[dom] / (max(1, counts[-1]) * wl.G), peaks)
         if own:
             roofline.update(own)
 
@@ -689,10 +706,14 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=20, help="un-captured steps timed per call for the roofline")
     ap.add_argument("--layers", default="", help="sweep workloads: comma-separated layer indices")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--variant", default="plain", help="flat workload: plain | per_example_noise | micro2 | micro4 ...")
     args = ap.parse_args()
+    global VARIANT
+    VARIANT = args.variant
     if args.workload in ("sweep", "sweep_all"):
         return run_sweep(args)
-    defaults = {"small_cnn": (400, 10), "flat": (8, 3), "per_layer": (2, 3)}
+    # the small-CNN step lasts ~0.16 ms: 6000 steps give the clock sampler (200 ms period) several readings under load
+    defaults = {"small_cnn": (6000, 10), "flat": (8, 3), "per_layer": (4, 3)}
     if args.steps is None:
         args.steps = defaults[args.workload][0]
     if args.warmup is None:

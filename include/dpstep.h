@@ -172,6 +172,34 @@ DP_API dp_status dp_clip_accumulate_noised(int mode, int B, int L, const float *
 DP_API dp_status dp_debug_example_noise_z(float *z, long long count, long long first_index, long long example,
                                           unsigned long long seed, unsigned long long step, void *cuda_stream);
 
+/* dp_clip_accumulate with the parameter tensors gathered into M groups, each clipped on its own to C/sqrt(M)
+ * (section 3.5: the groups are the paper's pipeline stages; no stage needs another stage's norm, and the bound on the
+ * whole gradient stays C because the squares of the M bounds add up to C^2):
+ *     s_{n,m} = sum over tensors l of group m of ||G_l[n]||^2,   f_{n,m} = min(1, (C/sqrt(M)) / sqrt(s_{n,m})),
+ *     acc_l += sum_n f_{n,group_of[l]} * G_l[n].
+ * One tensor per group is DP_CLIP_PER_LAYER, a single group is DP_CLIP_GLOBAL.
+ *   group_of   host array of L group indices in [0, M); every group must own at least one tensor.  L <= 1024.
+ *   sqnorm     device [B, L] per-tensor squared norms or NULL (computed here), as for dp_clip_accumulate.
+ *   norms_out, clip_out   optional device [B, M]: the groups' L2 norms and factors.
+ * Everything else, and the errors, as for dp_clip_accumulate. */
+DP_API dp_status dp_clip_accumulate_grouped(int B, int L, int M, const int *group_of, const float *const *G,
+                                            const long long *P_l, const float *sqnorm, float C, float *const *acc,
+                                            float *norms_out, float *clip_out, void *workspace, size_t workspace_bytes,
+                                            void *cuda_stream);
+
+/* Micro-batch clipping (the option of the paper's first table, which the paper advises against: it trades accuracy for
+ * speed): the B examples of the chunk form B/micro runs of `micro` consecutive examples; each run is averaged, the
+ * average is clipped to C over the whole model and the clipped averages are added:
+ *     gbar_j = (1/micro) sum_{n in run j} g_n,   f_j = min(1, C/||gbar_j||),   acc += sum_j f_j * gbar_j.
+ * The unit that is clipped is the run, so the step ends with dp_noise_average(total_batch = number of runs).
+ *   micro      >= 1, must divide B (1 is plain whole-model clipping).
+ *   norms_out, clip_out   optional device [B/micro].
+ * The norms are always computed here (a run's norm does not follow from its examples' norms): two passes over G.
+ * Everything else, and the errors, as for dp_clip_accumulate in DP_CLIP_GLOBAL mode. */
+DP_API dp_status dp_clip_accumulate_micro(int B, int L, int micro, const float *const *G, const long long *P_l, float C,
+                                          float *const *acc, float *norms_out, float *clip_out, void *workspace,
+                                          size_t workspace_bytes, void *cuda_stream);
+
 /* dp_clip_accumulate for callers that cannot allocate device memory.  (The paper has no counterpart;
  * this exists for deployment reasons only.)
  *

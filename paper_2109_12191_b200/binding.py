@@ -29,7 +29,7 @@ EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_
            "dp_wgrad_check", "dp_wgrad_uses_tensor_cores", "dp_status_string", "dp_last_cuda_error",
            "dp_debug_launch_count", "dp_debug_wgrad_plan", "dp_clip_accumulate_static",
            "dp_clip_static_scratch_bytes", "dp_noise_average_sgd", "dp_clip_accumulate_noised",
-           "dp_debug_example_noise_z"]
+           "dp_debug_example_noise_z", "dp_clip_accumulate_grouped", "dp_clip_accumulate_micro"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -65,6 +65,12 @@ _lib.dp_clip_accumulate_noised.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctyp
                                            _f, _f, _ll, _ull, _ull, _ll, ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
 _lib.dp_clip_accumulate_noised.restype = _i
 _lib.dp_debug_example_noise_z.argtypes = [_vp, _ll, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_example_noise_z.restype = _i
+_lib.dp_clip_accumulate_grouped.argtypes = [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_vp), ctypes.POINTER(_ll), _vp, _f,
+                                            ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
+_lib.dp_clip_accumulate_grouped.restype = _i
+_lib.dp_clip_accumulate_micro.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctypes.POINTER(_ll), _f, ctypes.POINTER(_vp), _vp,
+                                          _vp, _vp, _sz, _vp]
+_lib.dp_clip_accumulate_micro.restype = _i
 _lib.dp_clip_accumulate_static.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctypes.POINTER(_ll), _vp, _f,
                                            ctypes.POINTER(_vp), _vp, _vp, _vp]
 _lib.dp_clip_accumulate_static.restype = _i
@@ -161,6 +167,30 @@ def dp_clip_accumulate_noised(mode, B, G, P_l, param_offset_l, sqnorm, C, sigma,
 
 def dp_debug_example_noise_z(z, count, first_index, example, seed, step, stream=None):
     return _lib.dp_debug_example_noise_z(_ptr(z), count, first_index, example, seed, step, _stream(stream))
+
+
+def dp_clip_accumulate_grouped(B, M, group_of, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace, workspace_bytes=None,
+                               stream=None):
+    """dp_clip_accumulate over M groups of tensors, each clipped to C/sqrt(M)."""
+    L = len(P_l)
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else _nbytes(workspace)
+    Gp = (_vp * L)(*[_ptr(g) for g in G]) if G is not None else None
+    Ap = (_vp * L)(*[_ptr(a) for a in acc]) if acc is not None else None
+    go = (_i * L)(*group_of) if group_of is not None else None
+    return _lib.dp_clip_accumulate_grouped(B, L, M, go, Gp, (_ll * L)(*P_l), _ptr(sqnorm), C, Ap, _ptr(norms_out),
+                                           _ptr(clip_out), _ptr(workspace), workspace_bytes, _stream(stream))
+
+
+def dp_clip_accumulate_micro(B, micro, G, P_l, C, acc, norms_out, clip_out, workspace, workspace_bytes=None, stream=None):
+    """Whole-model clipping of the means of runs of `micro` consecutive examples."""
+    L = len(P_l)
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else _nbytes(workspace)
+    Gp = (_vp * L)(*[_ptr(g) for g in G]) if G is not None else None
+    Ap = (_vp * L)(*[_ptr(a) for a in acc]) if acc is not None else None
+    return _lib.dp_clip_accumulate_micro(B, L, micro, Gp, (_ll * L)(*P_l), C, Ap, _ptr(norms_out), _ptr(clip_out),
+                                         _ptr(workspace), workspace_bytes, _stream(stream))
 
 
 def dp_clip_accumulate_static(mode, B, G, P_l, sqnorm, C, acc, norms_out, clip_out, stream=None):

@@ -111,6 +111,90 @@ __global__ void clip_factor_kernel(const float *__restrict__ sq, int B, int L, i
     }
 }
 
+// stage 1a for micro-batch clipping: row j of the partials belongs to the MEAN of examples j*micro .. j*micro+micro-1
+// (the unit that is clipped), so the rows are added before they are squared.
+__global__ void __launch_bounds__(256)
+sqnorm_partial_micro_kernel(const __grid_constant__ SegTable tab, float *__restrict__ partial,
+                            long long parts_per_example, int micro) {
+    __shared__ float scratch[32];
+    const int seg = find_seg(tab, blockIdx.x);
+    const int j = blockIdx.x - tab.blk_start[seg];
+    const long long P = tab.P[seg];
+    const long long c0 = (long long)j * kNormChunk;
+    const int len = (int)min((long long)kNormChunk, P - c0);
+    const float *row = tab.G[seg] + (long long)blockIdx.y * micro * P + c0;
+    const float inv = 1.0f / (float)micro;
+    float a = 0.f;
+    if (((reinterpret_cast<uintptr_t>(row) | (uintptr_t)(P * 4)) & 15) == 0) {
+        const int n4 = len >> 2;
+        for (int i = threadIdx.x; i < n4; i += 256) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r = 0; r < micro; ++r) {
+                const float4 x = __ldg(reinterpret_cast<const float4 *>(row + (long long)r * P) + i);
+                v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+            }
+            v.x *= inv; v.y *= inv; v.z *= inv; v.w *= inv;
+            a = fmaf(v.x, v.x, a); a = fmaf(v.y, v.y, a); a = fmaf(v.z, v.z, a); a = fmaf(v.w, v.w, a);
+        }
+        for (int i = (n4 << 2) + threadIdx.x; i < len; i += 256) {
+            float v = 0.f;
+            for (int r = 0; r < micro; ++r) v += row[(long long)r * P + i];
+            v *= inv;
+            a = fmaf(v, v, a);
+        }
+    } else {
+        for (int i = threadIdx.x; i < len; i += 256) {
+            float v = 0.f;
+            for (int r = 0; r < micro; ++r) v += row[(long long)r * P + i];
+            v *= inv;
+            a = fmaf(v, v, a);
+        }
+    }
+    a = block_sum(a, scratch);
+    if (threadIdx.x == 0) partial[(long long)blockIdx.y * parts_per_example + tab.part_start[seg] + j] = a;
+}
+
+// stage 2 for micro-batch clipping: one factor per micro-batch from the norm of its mean; every example of the
+// micro-batch then carries factor / micro, so that stage 3 adds factor * mean.
+__global__ void clip_factor_micro_kernel(const float *__restrict__ sq, int n_micro, int L, int micro, float C,
+                                         float *__restrict__ factor, float *norms_out, float *clip_out) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n_micro) return;
+    double s = 0.0;
+    for (int l = 0; l < L; ++l) s += (double)sq[(long long)j * L + l];
+    const float f = clip_factor(s, C);
+    const float each = f / (float)micro;
+    for (int i = 0; i < micro; ++i) factor[(long long)j * micro + i] = each;
+    if (norms_out) norms_out[j] = (float)sqrt(s);
+    if (clip_out) clip_out[j] = f;
+}
+
+// stage 2 for groups of tensors (section 3.5: M pipeline stages, each clipped to C/sqrt(M)): one block per example
+// sums the squared norms of each group's tensors in tensor order, then every tensor gets its group's factor.
+constexpr int kMaxGroupedTensors = 1024;
+struct GroupTable {
+    int M;
+    unsigned short of[kMaxGroupedTensors];   // group of tensor l
+};
+__global__ void __launch_bounds__(128)
+clip_factor_grouped_kernel(const float *__restrict__ sq, int L, const __grid_constant__ GroupTable gt, float C,
+                           float *__restrict__ factor, float *norms_out, float *clip_out) {
+    __shared__ float f_sh[kMaxGroupedTensors];
+    const int n = blockIdx.x;
+    const float thr = (float)((double)C / sqrt((double)gt.M));
+    for (int m = threadIdx.x; m < gt.M; m += 128) {
+        double s = 0.0;
+        for (int l = 0; l < L; ++l)
+            if (gt.of[l] == m) s += (double)sq[(long long)n * L + l];
+        const float f = clip_factor(s, thr);
+        f_sh[m] = f;
+        if (norms_out) norms_out[(long long)n * gt.M + m] = (float)sqrt(s);
+        if (clip_out) clip_out[(long long)n * gt.M + m] = f;
+    }
+    __syncthreads();
+    for (int l = threadIdx.x; l < L; l += 128) factor[(long long)n * L + l] = f_sh[gt.of[l]];
+}
+
 // stage 3: acc[i] += sum_n factor * G[n, i].  factor index: GLOBAL n, PER_LAYER n*L + col.
 template <int UNROLL>
 __global__ void __launch_bounds__(256)
@@ -385,12 +469,22 @@ extern "C" size_t dp_clip_workspace_bytes(int B, int L, const long long *P_l) {
 }
 
 namespace dp {
-// Host side of dp_clip_accumulate; with `noise` (and the tensors' global offsets) stage 3 also adds each example's
-// own noise draw.
+// What differs from plain dp_clip_accumulate in the other entry points.
+struct ClipVariant {
+    const ExampleNoise *noise = nullptr;   // stage 3 also adds each example's own noise draw ...
+    const long long *goff_l = nullptr;     // ... addressed by the tensors' global offsets
+    const GroupTable *groups = nullptr;    // factors per (example, group of tensors) instead of per tensor
+    int micro = 1;                         // examples averaged before clipping
+};
+
+// Host side of dp_clip_accumulate and its variants.
 static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const *G, const long long *P_l,
                                       const float *sqnorm, float C, float *const *acc, float *norms_out,
                                       float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream,
-                                      const ExampleNoise *noise, const long long *goff_l) {
+                                      const ClipVariant &var = ClipVariant()) {
+    const ExampleNoise *noise = var.noise;
+    const long long *goff_l = var.goff_l;
+    const int micro = var.micro;
     if (mode != DP_CLIP_GLOBAL && mode != DP_CLIP_PER_LAYER) return DP_ERR_INVALID_ARG;
     if (B <= 0 || L <= 0 || !G || !P_l || !acc || !(C > 0.0f)) return DP_ERR_INVALID_ARG;
     if (B > 65535) return DP_ERR_UNSUPPORTED;
@@ -443,9 +537,12 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
             SegTable t;
             const int blocks = fill(l0, t, true, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
-            sqnorm_partial_kernel<<<dim3((unsigned)blocks, (unsigned)B), 256, 0, stream>>>(t, partial, pl.parts_per_example);
+            if (micro > 1)
+                sqnorm_partial_micro_kernel<<<dim3((unsigned)blocks, (unsigned)(B / micro)), 256, 0, stream>>>(t, partial, pl.parts_per_example, micro);
+            else
+                sqnorm_partial_kernel<<<dim3((unsigned)blocks, (unsigned)B), 256, 0, stream>>>(t, partial, pl.parts_per_example);
             DP_LAUNCH_CHECK("sqnorm_partial_kernel");
-            sqnorm_fold_kernel<<<dim3((unsigned)t.nseg, (unsigned)B), 128, 0, stream>>>(t, partial, pl.parts_per_example, sq_ws, L);
+            sqnorm_fold_kernel<<<dim3((unsigned)t.nseg, (unsigned)(B / micro)), 128, 0, stream>>>(t, partial, pl.parts_per_example, sq_ws, L);
             DP_LAUNCH_CHECK("sqnorm_fold_kernel");
             l0 += t.nseg;
         }
@@ -453,7 +550,12 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
     }
     {
         const long long count = per_layer ? (long long)B * L : B;
-        clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, stream>>>(sq, B, L, per_layer, C, factor, norms_out, clip_out);
+        if (var.groups)
+            clip_factor_grouped_kernel<<<(unsigned)B, 128, 0, stream>>>(sq, L, *var.groups, C, factor, norms_out, clip_out);
+        else if (micro > 1)
+            clip_factor_micro_kernel<<<(unsigned)((B / micro + 127) / 128), 128, 0, stream>>>(sq, B / micro, L, micro, C, factor, norms_out, clip_out);
+        else
+            clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, stream>>>(sq, B, L, per_layer, C, factor, norms_out, clip_out);
         DP_LAUNCH_CHECK("clip_factor_kernel");
     }
     {
@@ -477,7 +579,39 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
                                         const float *sqnorm, float C, float *const *acc, float *norms_out,
                                         float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace, workspace_bytes,
-                                    cuda_stream, nullptr, nullptr);
+                                    cuda_stream);
+}
+
+extern "C" dp_status dp_clip_accumulate_grouped(int B, int L, int M, const int *group_of, const float *const *G,
+                                                const long long *P_l, const float *sqnorm, float C, float *const *acc,
+                                                float *norms_out, float *clip_out, void *workspace,
+                                                size_t workspace_bytes, void *cuda_stream) {
+    if (L <= 0 || M <= 0 || M > L || !group_of) return DP_ERR_INVALID_ARG;
+    if (L > dp::kMaxGroupedTensors) return DP_ERR_UNSUPPORTED;
+    dp::GroupTable gt;
+    gt.M = M;
+    unsigned char used[dp::kMaxGroupedTensors] = {0};
+    for (int l = 0; l < L; ++l) {
+        if (group_of[l] < 0 || group_of[l] >= M) return DP_ERR_INVALID_ARG;
+        gt.of[l] = (unsigned short)group_of[l];
+        used[group_of[l]] = 1;
+    }
+    for (int m = 0; m < M; ++m)
+        if (!used[m]) return DP_ERR_INVALID_ARG;                 // an empty group would still count in C/sqrt(M)
+    dp::ClipVariant var;
+    var.groups = &gt;
+    return dp::clip_accumulate_impl(DP_CLIP_PER_LAYER, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace,
+                                    workspace_bytes, cuda_stream, var);
+}
+
+extern "C" dp_status dp_clip_accumulate_micro(int B, int L, int micro, const float *const *G, const long long *P_l,
+                                              float C, float *const *acc, float *norms_out, float *clip_out,
+                                              void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (micro <= 0 || B <= 0 || B % micro != 0) return DP_ERR_INVALID_ARG;
+    dp::ClipVariant var;
+    var.micro = micro;
+    return dp::clip_accumulate_impl(DP_CLIP_GLOBAL, B, L, G, P_l, nullptr, C, acc, norms_out, clip_out, workspace,
+                                    workspace_bytes, cuda_stream, var);
 }
 
 extern "C" dp_status dp_clip_accumulate_noised(int mode, int B, int L, const float *const *G, const long long *P_l,
@@ -496,12 +630,15 @@ extern "C" dp_status dp_clip_accumulate_noised(int mode, int B, int L, const flo
     }
     if (sigma == 0.0f)
         return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace,
-                                        workspace_bytes, cuda_stream, nullptr, nullptr);
+                                        workspace_bytes, cuda_stream);
     dp::ExampleNoise nz;
     nz.sd = (float)((double)sigma * (double)C / sqrt((double)total_batch));
     nz.seed = seed; nz.step = step; nz.example0 = (uint32_t)example0;
+    dp::ClipVariant var;
+    var.noise = &nz;
+    var.goff_l = param_offset_l;
     return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace, workspace_bytes,
-                                    cuda_stream, &nz, param_offset_l);
+                                    cuda_stream, var);
 }
 
 // ----------------------------------------------------------------------------------------------------

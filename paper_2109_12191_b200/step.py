@@ -150,9 +150,13 @@ class GlobalClipStep:
 class FlatClipStep:
     """Flattened per-example gradients [B, P] handed in directly (no weight-gradient stage)."""
 
-    def __init__(self, P, B, C, sigma, device="cuda", per_example_noise=False):
+    def __init__(self, P, B, C, sigma, device="cuda", per_example_noise=False, micro=1):
+        """micro > 1: runs of `micro` consecutive examples are averaged before clipping (the clipped unit is the run)."""
         self.P, self.B, self.C, self.sigma = P, B, float(C), float(sigma)
         self.per_example_noise = bool(per_example_noise)
+        self.micro = int(micro)
+        if self.micro < 1 or B % self.micro or (self.micro > 1 and per_example_noise):
+            raise ValueError("micro must divide B, and per-example noise is defined for single examples")
         self.acc = torch.zeros(P, dtype=torch.float32, device=device)
         self.out = torch.empty(P, dtype=torch.float32, device=device)
         self.norms = torch.empty(B, dtype=torch.float32, device=device)
@@ -166,7 +170,10 @@ class FlatClipStep:
         self._noise = _NoiseKey(self.per_example_noise, total_batch, seed, step, example0)
 
     def chunk(self, G, sqnorm=None):
-        if self.per_example_noise:
+        if self.micro > 1:
+            b.check(b.dp_clip_accumulate_micro(self.B, self.micro, [G], [self.P], self.C, [self.acc], self.norms, self.clip,
+                                               self.ws), "dp_clip_accumulate_micro")
+        elif self.per_example_noise:
             k = self._noise
             b.check(b.dp_clip_accumulate_noised(b.DP_CLIP_GLOBAL, self.B, [G], [self.P], [0], sqnorm, self.C, self.sigma,
                                                 k.total_batch, k.seed, k.step, k.example0 + self.B * self.chunks_done,
@@ -179,7 +186,8 @@ class FlatClipStep:
     def finish(self, seed=0, step=0, world=1):
         total = self.B * self.chunks_done * world
         sigma = self._noise.finish_sigma(self.sigma, total)
-        b.check(b.dp_noise_average(self.acc, self.P, 0, sigma, self.C, total, seed, step, self.out), "dp_noise_average")
+        b.check(b.dp_noise_average(self.acc, self.P, 0, sigma, self.C, total // self.micro, seed, step, self.out),
+                "dp_noise_average")
         return self.out
 
 

@@ -138,6 +138,29 @@ def test_noised_clip_rejects_bad_arguments(b):
     assert b.dp_debug_example_noise_z(A, 4, 0, 2**31, 0, 0, stream=0) == b.DP_ERR_INVALID_ARG
 
 
+def test_grouped_and_micro_clip_reject_bad_arguments(b):
+    A = 4096
+    P = [100, 8, 16]
+    ws = b.dp_clip_workspace_bytes(4, P)
+    grouped = lambda **kw: b.dp_clip_accumulate_grouped(**{**dict(B=4, M=2, group_of=[0, 1, 1], G=[A, A, A], P_l=P, sqnorm=None,
+                                                                  C=1.0, acc=[A, A, A], norms_out=None, clip_out=None,
+                                                                  workspace=A, workspace_bytes=ws, stream=0), **kw})
+    assert grouped(group_of=None) == b.DP_ERR_INVALID_ARG
+    assert grouped(group_of=[0, 0, 0]) == b.DP_ERR_INVALID_ARG          # group 1 owns no tensor
+    assert grouped(group_of=[0, 1, 2]) == b.DP_ERR_INVALID_ARG          # index outside [0, M)
+    assert grouped(M=0) == b.DP_ERR_INVALID_ARG
+    assert grouped(M=4, group_of=[0, 1, 2]) == b.DP_ERR_INVALID_ARG     # more groups than tensors
+    assert grouped(C=0.0) == b.DP_ERR_INVALID_ARG
+    assert grouped(workspace=None) == b.DP_ERR_WORKSPACE
+    micro = lambda **kw: b.dp_clip_accumulate_micro(**{**dict(B=4, micro=2, G=[A, A, A], P_l=P, C=1.0, acc=[A, A, A],
+                                                              norms_out=None, clip_out=None, workspace=A, workspace_bytes=ws,
+                                                              stream=0), **kw})
+    assert micro(micro=0) == b.DP_ERR_INVALID_ARG
+    assert micro(micro=3) == b.DP_ERR_INVALID_ARG                       # does not divide B
+    assert micro(G=[A, None, A]) == b.DP_ERR_INVALID_ARG
+    assert micro(workspace_bytes=ws - 1) == b.DP_ERR_WORKSPACE
+
+
 def test_noise_rejects_bad_arguments(b):
     A = 4096
     call = lambda acc=A, P=16, off=0, sigma=1.0, C=1.0, tb=8, out=A: b.dp_noise_average(acc, P, off, sigma, C, tb, 0, 0, out, stream=0)
