@@ -118,6 +118,23 @@ DP_API dp_status dp_per_example_wgrad(const dp_layer_desc *desc, const void *X, 
                                int epilogue, float C_l, float *acc_w, float *acc_b, float *clip_out,
                                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The clipped sum of one layer with the factors already known: acc_w += sum_n factor_w[n*factor_stride] * g_w,n and
+ * acc_b += sum_n factor_b[n*factor_stride] * g_b,n, the per-example gradients formed on the fly and never written
+ * (section 2: the sum over the batch of clip(g_j, C), whose factor min(1, C/||g_j||) needs every layer's norm first).
+ * Together with DP_EPI_NORM_ONLY and dp_clip_factors this gives whole-model clipping without materialising a layer's
+ * per-example gradients: the layer's inputs are read twice instead of its B gradients being written and read back,
+ * which is cheaper whenever a gradient is larger than the inputs it comes from (late convolutions, dense layers).
+ *
+ *   factor_w, factor_b   device fp32, one value per example at stride factor_stride (>= 1).  factor_b = NULL uses
+ *                        factor_w for the bias-like tensor too (whole-model clipping: one factor per example).
+ *   acc_w, acc_b         [P_w], [P_b] fp32, read-modify-write (acc_b only when the layer has a bias-like tensor).
+ *   workspace            at least dp_workspace_bytes(desc, DP_EPI_CLIP_ACCUM) bytes, 256-byte aligned.
+ * Errors as for dp_per_example_wgrad. */
+DP_API dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *desc, const void *X, const void *dY,
+                                             const float *factor_w, const float *factor_b, long long factor_stride,
+                                             float *acc_w, float *acc_b, void *workspace, size_t workspace_bytes,
+                                             void *cuda_stream);
+
 /* Bytes of device scratch dp_clip_accumulate needs (per-block partial norms and factors). */
 DP_API size_t dp_clip_workspace_bytes(int B, int L, const long long *P_l /* host, [L] */);
 
@@ -171,6 +188,19 @@ DP_API dp_status dp_clip_accumulate_noised(int mode, int B, int L, const float *
 /* Test hook: the standard normals of example `example`'s stream for global indices first_index .. +count-1. */
 DP_API dp_status dp_debug_example_noise_z(float *z, long long count, long long first_index, long long example,
                                           unsigned long long seed, unsigned long long step, void *cuda_stream);
+
+/* The two halves of dp_clip_accumulate on their own, for steps that keep only some tensors' per-example gradients in
+ * memory and form the others' clipped sums with dp_per_example_wgrad_scaled.
+ *
+ * dp_clip_factors: the factors from a table of squared norms (section 2 / 3.5, as in dp_clip_accumulate):
+ *   sqnorm       device [B, L] fp32: per-tensor squared norms of every example (all L tensors of the model).
+ *   factors_out  device fp32: GLOBAL [B], PER_LAYER [B, L].   norms_out  optional, same shape: the L2 norms.
+ * dp_scale_accumulate: acc_l += sum_n f * G_l[n] with f = factor[n] (per_tensor = 0) or factor[n*L + l] (per_tensor = 1);
+ *   G, P_l, acc as for dp_clip_accumulate.  Neither call needs a workspace. */
+DP_API dp_status dp_clip_factors(int mode, int B, int L, const float *sqnorm, float C, float *norms_out,
+                                 float *factors_out, void *cuda_stream);
+DP_API dp_status dp_scale_accumulate(int B, int L, const float *const *G, const long long *P_l, const float *factor,
+                                     int per_tensor, float *const *acc, void *cuda_stream);
 
 /* dp_clip_accumulate with the parameter tensors gathered into M groups, each clipped on its own to C/sqrt(M)
  * (section 3.5: the groups are the paper's pipeline stages; no stage needs another stage's norm, and the bound on the

@@ -29,7 +29,8 @@ EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_
            "dp_wgrad_check", "dp_wgrad_uses_tensor_cores", "dp_status_string", "dp_last_cuda_error",
            "dp_debug_launch_count", "dp_debug_wgrad_plan", "dp_clip_accumulate_static",
            "dp_clip_static_scratch_bytes", "dp_noise_average_sgd", "dp_clip_accumulate_noised",
-           "dp_debug_example_noise_z", "dp_clip_accumulate_grouped", "dp_clip_accumulate_micro"]
+           "dp_debug_example_noise_z", "dp_clip_accumulate_grouped", "dp_clip_accumulate_micro",
+           "dp_per_example_wgrad_scaled", "dp_clip_factors", "dp_scale_accumulate"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -57,6 +58,11 @@ _lib.dp_workspace_bytes.argtypes = [_dp, _i]; _lib.dp_workspace_bytes.restype = 
 _lib.dp_wgrad_uses_tensor_cores.argtypes = [_dp, _i]; _lib.dp_wgrad_uses_tensor_cores.restype = _i
 _lib.dp_per_example_wgrad.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _ll, _i, _f, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.dp_per_example_wgrad.restype = _i
+_lib.dp_per_example_wgrad_scaled.argtypes = [_dp, _vp, _vp, _vp, _vp, _ll, _vp, _vp, _vp, _sz, _vp]
+_lib.dp_per_example_wgrad_scaled.restype = _i
+_lib.dp_clip_factors.argtypes = [_i, _i, _i, _vp, _f, _vp, _vp, _vp]; _lib.dp_clip_factors.restype = _i
+_lib.dp_scale_accumulate.argtypes = [_i, _i, ctypes.POINTER(_vp), ctypes.POINTER(_ll), _vp, _i, ctypes.POINTER(_vp), _vp]
+_lib.dp_scale_accumulate.restype = _i
 _lib.dp_clip_workspace_bytes.argtypes = [_i, _i, ctypes.POINTER(_ll)]; _lib.dp_clip_workspace_bytes.restype = _sz
 _lib.dp_clip_accumulate.argtypes = [_i, _i, _i, ctypes.POINTER(_vp), ctypes.POINTER(_ll), _vp, _f,
                                     ctypes.POINTER(_vp), _vp, _vp, _vp, _sz, _vp]
@@ -133,6 +139,26 @@ def dp_per_example_wgrad(desc, X, dY, G_w, G_b, sqnorm, sqnorm_stride, epilogue,
     return _lib.dp_per_example_wgrad(ctypes.byref(desc) if desc is not None else None, _ptr(X), _ptr(dY), _ptr(G_w),
                                      _ptr(G_b), _ptr(sqnorm), sqnorm_stride, epilogue, C_l, _ptr(acc_w), _ptr(acc_b),
                                      _ptr(clip_out), _ptr(workspace), workspace_bytes, _stream(stream))
+
+
+def dp_per_example_wgrad_scaled(desc, X, dY, factor_w, factor_b, factor_stride, acc_w, acc_b, workspace, workspace_bytes=None,
+                                stream=None):
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else _nbytes(workspace)
+    return _lib.dp_per_example_wgrad_scaled(ctypes.byref(desc) if desc is not None else None, _ptr(X), _ptr(dY), _ptr(factor_w),
+                                            _ptr(factor_b), factor_stride, _ptr(acc_w), _ptr(acc_b), _ptr(workspace),
+                                            workspace_bytes, _stream(stream))
+
+
+def dp_clip_factors(mode, B, L, sqnorm, C, norms_out, factors_out, stream=None):
+    return _lib.dp_clip_factors(mode, B, L, _ptr(sqnorm), C, _ptr(norms_out), _ptr(factors_out), _stream(stream))
+
+
+def dp_scale_accumulate(B, G, P_l, factor, per_tensor, acc, stream=None):
+    L = len(P_l)
+    Gp = (_vp * L)(*[_ptr(g) for g in G]) if G is not None else None
+    Ap = (_vp * L)(*[_ptr(a) for a in acc]) if acc is not None else None
+    return _lib.dp_scale_accumulate(B, L, Gp, (_ll * L)(*P_l), _ptr(factor), per_tensor, Ap, _stream(stream))
 
 
 def dp_clip_workspace_bytes(B, P_l):

@@ -475,6 +475,7 @@ struct ClipVariant {
     const long long *goff_l = nullptr;     // ... addressed by the tensors' global offsets
     const GroupTable *groups = nullptr;    // factors per (example, group of tensors) instead of per tensor
     int micro = 1;                         // examples averaged before clipping
+    const float *given_factor = nullptr;   // stage 3 only, with the caller's factors ([B] or [B, L]); no workspace
 };
 
 // Host side of dp_clip_accumulate and its variants.
@@ -488,6 +489,7 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
     if (mode != DP_CLIP_GLOBAL && mode != DP_CLIP_PER_LAYER) return DP_ERR_INVALID_ARG;
     if (B <= 0 || L <= 0 || !G || !P_l || !acc || !(C > 0.0f)) return DP_ERR_INVALID_ARG;
     if (B > 65535) return DP_ERR_UNSUPPORTED;
+    const bool stage3_only = var.given_factor != nullptr;
     ClipPlan pl;
     if (!plan(B, L, P_l, pl)) return DP_ERR_INVALID_ARG;
     for (int l = 0; l < L; ++l) {
@@ -495,12 +497,13 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
         if ((P_l[l] + kSplitCols - 1) / kSplitCols > 0x3fffffffll) return DP_ERR_UNSUPPORTED;
     }
     if (sqnorm && !aligned(sqnorm, 4)) return DP_ERR_INVALID_ARG;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < pl.total) return DP_ERR_WORKSPACE;
+    if (!stage3_only && (!workspace || !aligned(workspace, 256) || workspace_bytes < pl.total)) return DP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char *ws = static_cast<char *>(workspace);
-    float *partial = reinterpret_cast<float *>(ws + pl.partial_off);
-    float *sq_ws = reinterpret_cast<float *>(ws + pl.sq_off);
-    float *factor = reinterpret_cast<float *>(ws + pl.factor_off);
+    float *partial = stage3_only ? nullptr : reinterpret_cast<float *>(ws + pl.partial_off);
+    float *sq_ws = stage3_only ? nullptr : reinterpret_cast<float *>(ws + pl.sq_off);
+    const float *factor = stage3_only ? var.given_factor : reinterpret_cast<float *>(ws + pl.factor_off);
+    float *factor_ws = stage3_only ? nullptr : reinterpret_cast<float *>(ws + pl.factor_off);
     const int per_layer = (mode == DP_CLIP_PER_LAYER);
 
     // tensors go to the kernels in tables of at most kMaxSeg entries
@@ -531,7 +534,7 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
     };
 
     const float *sq = sqnorm;
-    if (!sq) {
+    if (!sq && !stage3_only) {
         long long cursor = 0;
         for (int l0 = 0; l0 < L;) {
             SegTable t;
@@ -548,14 +551,14 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
         }
         sq = sq_ws;
     }
-    {
+    if (!stage3_only) {
         const long long count = per_layer ? (long long)B * L : B;
         if (var.groups)
-            clip_factor_grouped_kernel<<<(unsigned)B, 128, 0, stream>>>(sq, L, *var.groups, C, factor, norms_out, clip_out);
+            clip_factor_grouped_kernel<<<(unsigned)B, 128, 0, stream>>>(sq, L, *var.groups, C, factor_ws, norms_out, clip_out);
         else if (micro > 1)
-            clip_factor_micro_kernel<<<(unsigned)((B / micro + 127) / 128), 128, 0, stream>>>(sq, B / micro, L, micro, C, factor, norms_out, clip_out);
+            clip_factor_micro_kernel<<<(unsigned)((B / micro + 127) / 128), 128, 0, stream>>>(sq, B / micro, L, micro, C, factor_ws, norms_out, clip_out);
         else
-            clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, stream>>>(sq, B, L, per_layer, C, factor, norms_out, clip_out);
+            clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, stream>>>(sq, B, L, per_layer, C, factor_ws, norms_out, clip_out);
         DP_LAUNCH_CHECK("clip_factor_kernel");
     }
     {
@@ -580,6 +583,28 @@ extern "C" dp_status dp_clip_accumulate(int mode, int B, int L, const float *con
                                         float *clip_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     return dp::clip_accumulate_impl(mode, B, L, G, P_l, sqnorm, C, acc, norms_out, clip_out, workspace, workspace_bytes,
                                     cuda_stream);
+}
+
+extern "C" dp_status dp_clip_factors(int mode, int B, int L, const float *sqnorm, float C, float *norms_out,
+                                     float *factors_out, void *cuda_stream) {
+    if (mode != DP_CLIP_GLOBAL && mode != DP_CLIP_PER_LAYER) return DP_ERR_INVALID_ARG;
+    if (B <= 0 || L <= 0 || !sqnorm || !factors_out || !(C > 0.0f)) return DP_ERR_INVALID_ARG;
+    if (!dp::aligned(sqnorm, 4) || !dp::aligned(factors_out, 4) || (norms_out && !dp::aligned(norms_out, 4))) return DP_ERR_INVALID_ARG;
+    const int per_layer = (mode == DP_CLIP_PER_LAYER);
+    const long long count = per_layer ? (long long)B * L : B;
+    dp::clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        sqnorm, B, L, per_layer, C, factors_out, norms_out, nullptr);
+    DP_LAUNCH_CHECK("clip_factor_kernel");
+    return DP_OK;
+}
+
+extern "C" dp_status dp_scale_accumulate(int B, int L, const float *const *G, const long long *P_l, const float *factor,
+                                         int per_tensor, float *const *acc, void *cuda_stream) {
+    if (!factor || !dp::aligned(factor, 4) || (per_tensor != 0 && per_tensor != 1)) return DP_ERR_INVALID_ARG;
+    dp::ClipVariant var;
+    var.given_factor = factor;
+    return dp::clip_accumulate_impl(per_tensor ? DP_CLIP_PER_LAYER : DP_CLIP_GLOBAL, B, L, G, P_l, nullptr, 1.0f, acc,
+                                    nullptr, nullptr, nullptr, 0, cuda_stream, var);
 }
 
 extern "C" dp_status dp_clip_accumulate_grouped(int B, int L, int M, const int *group_of, const float *const *G,

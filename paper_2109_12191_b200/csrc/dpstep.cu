@@ -197,7 +197,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
                                sqnorm_stride, clip, C_l, factor, clip_out, reset, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
-        rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, 2, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
+        rc = launch_dense_scaled_sum(d->dtype, X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
@@ -214,6 +214,62 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             return launch_affine_clip_accum(partial, d->B, C_l, groups == 2, sqnorm, sqnorm_stride, clip_out, dg, dbt, d->C_in,
                                             acc_w, acc_b, st, reset);
         return launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
+    }
+}
+
+extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const void *X, const void *dY,
+                                                 const float *factor_w, const float *factor_b, long long factor_stride,
+                                                 float *acc_w, float *acc_b, void *workspace, size_t workspace_bytes,
+                                                 void *cuda_stream) {
+    if (!valid_desc(d)) return DP_ERR_INVALID_ARG;
+    if (!X || !dY || !aligned(X, 16) || !aligned(dY, 16)) return DP_ERR_INVALID_ARG;
+    if (!factor_w || !aligned(factor_w, 4) || (factor_b && !aligned(factor_b, 4)) || factor_stride < 1) return DP_ERR_INVALID_ARG;
+    const bool bias = has_bias_tensor(d);
+    if (!acc_w || !aligned(acc_w, 16) || (bias && (!acc_b || !aligned(acc_b, 16)))) return DP_ERR_INVALID_ARG;
+    if (!factor_b) factor_b = factor_w;
+    WgradPlan pl;
+    make_plan(d, DP_EPI_CLIP_ACCUM, pl);
+    if (d->impl == DP_IMPL_TENSOR_CORE && !pl.use_tc) return DP_ERR_UNSUPPORTED;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < pl.total) return DP_ERR_WORKSPACE;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    float *partial = reinterpret_cast<float *>(ws + pl.partial_off);
+    float *factor = reinterpret_cast<float *>(ws + pl.factor_off);
+    float *db_ws = reinterpret_cast<float *>(ws + pl.db_off);
+    const ConvGeom g = geom_of(d);
+    int *status_word = reinterpret_cast<int *>(ws + pl.status_off);
+    // the clipped-sum kernels read one (weight, bias) pair of factors per example
+    dp_status rc = launch_expand_factor(factor_w, factor_b, factor_stride, d->B, factor, pl.use_tc ? nullptr : status_word, st);
+    if (rc != DP_OK) return rc;
+
+    if (d->kind == DP_LAYER_CONV2D) {
+        if (d->has_bias) {
+            rc = launch_bias(d->dtype, dY, g, db_ws, partial, pl.slots, pl.w_slots, st);
+            if (rc != DP_OK) return rc;
+        }
+        if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, status_word, st);
+        else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
+        if (rc != DP_OK) return rc;
+        if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
+        return DP_OK;
+    }
+    if (d->kind == DP_LAYER_DENSE) {
+        // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis; the bias gradient is dY itself
+        rc = launch_dense_scaled_sum(d->dtype, X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
+        if (rc != DP_OK) return rc;
+        if (d->has_bias) return launch_dense_bias_accum(d->dtype, dY, d->B, d->K_out, factor, acc_b, st);
+        return DP_OK;
+    }
+    {
+        float *chunk_partial = reinterpret_cast<float *>(ws + pl.chunk_off);
+        float *dg = reinterpret_cast<float *>(ws + pl.dg_off);
+        float *dbt = dg + (size_t)d->B * d->C_in;
+        rc = launch_norm_affine(d->dtype, X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
+        if (rc != DP_OK) return rc;
+        rc = launch_bias_accum(dg, d->B, d->C_in, factor, acc_w, st, 0);
+        if (rc != DP_OK) return rc;
+        return launch_bias_accum(dbt, d->B, d->C_in, factor, acc_b, st, 1);
     }
 }
 

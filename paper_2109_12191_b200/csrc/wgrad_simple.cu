@@ -596,13 +596,89 @@ finalize_norm_kernel(const float *__restrict__ partial, int slots, int w_slots, 
     }
 }
 
-__global__ void bias_accum_kernel(const float *__restrict__ db, int B, int Kout, const float *__restrict__ factor,
-                                  float *__restrict__ acc_b) {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= Kout) return;
+// acc[k] += sum_n factor[2n + which] * v[n, k]   (which = 1: the bias-like tensor's factor, 0: the weight's).
+// Block = 32 channels x 8 example groups (group q owns examples q, q+8, ...), groups folded in order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bias_accum_kernel(const T *__restrict__ db, int B, int Kout, const float *__restrict__ factor, int which,
+                  float *__restrict__ acc_b) {
+    __shared__ float part[8][32];
+    const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
     float a = 0.f;
-    for (int n = 0; n < B; ++n) a = fmaf(factor[2 * n + 1], db[(long long)n * Kout + k], a);
-    acc_b[k] += a;
+    if (k < Kout)
+        for (int n = q; n < B; n += 8) a = fmaf(factor[2 * n + which], to_float(db[(long long)n * Kout + k]), a);
+    part[q][lane] = a;
+    __syncthreads();
+    if (q == 0 && k < Kout) {
+        float t = part[0][lane];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) t += part[i][lane];
+        acc_b[k] += t;
+    }
+}
+
+// Dense layer, clipped sum with known factors: acc[o, i] += sum_n (f_n dY[n, o]) X[n, i], a matrix product with the
+// batch as the reduction axis and a tiny output.  Block = 32 input columns x 16 outputs; its eight warps share the
+// examples (warp q owns q, q+8, ...), the scaled dY rows sit in shared memory, and the eight partial tiles are folded
+// in warp order.  Bound by latency and by the accumulator's read-modify-write, not by arithmetic.
+constexpr int kDenseOT = 16;
+template <typename T>
+__global__ void __launch_bounds__(256)
+dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const float *__restrict__ factor, int B,
+                        int Cin, int Kout, float *__restrict__ acc) {
+    __shared__ __align__(16) float fy[256][kDenseOT];        // f_n * dY[n, o0 .. o0+15] for a run of 256 examples
+    __shared__ float part[8][kDenseOT][32];
+    const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
+    const int i = blockIdx.x * 32 + lane, o0 = blockIdx.y * kDenseOT;
+    float a[kDenseOT];
+#pragma unroll
+    for (int o = 0; o < kDenseOT; ++o) a[o] = 0.f;
+    for (int n0 = 0; n0 < B; n0 += 256) {
+        const int nb = min(256, B - n0);
+        __syncthreads();
+        for (int t = threadIdx.x; t < nb * kDenseOT; t += 256) {
+            const int n = t / kDenseOT, o = t - n * kDenseOT;
+            fy[n][o] = (o0 + o < Kout) ? factor[2 * (n0 + n)] * to_float(dY[(long long)(n0 + n) * Kout + o0 + o]) : 0.f;
+        }
+        __syncthreads();
+        if (i < Cin) {
+#pragma unroll 4
+            for (int n = q; n < nb; n += 8) {
+                const float x = to_float(X[(long long)(n0 + n) * Cin + i]);
+                const float4 *row = reinterpret_cast<const float4 *>(fy[n]);
+#pragma unroll
+                for (int v = 0; v < kDenseOT / 4; ++v) {
+                    const float4 y = row[v];
+                    a[4 * v] = fmaf(y.x, x, a[4 * v]); a[4 * v + 1] = fmaf(y.y, x, a[4 * v + 1]);
+                    a[4 * v + 2] = fmaf(y.z, x, a[4 * v + 2]); a[4 * v + 3] = fmaf(y.w, x, a[4 * v + 3]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 0; o < kDenseOT; ++o) part[q][o][lane] = a[o];
+    __syncthreads();
+    // 512 tile entries, two per thread: entry e = (output e / 32, column e % 32)
+    for (int e = threadIdx.x; e < kDenseOT * 32; e += 256) {
+        const int o = e >> 5, c = e & 31;
+        if (o0 + o < Kout && blockIdx.x * 32 + c < Cin) {
+            float t = part[0][o][c];
+#pragma unroll
+            for (int w = 1; w < 8; ++w) t += part[w][o][c];
+            acc[(long long)(o0 + o) * Cin + blockIdx.x * 32 + c] += t;
+        }
+    }
+}
+
+// factor2[n] = (factor_w[n*stride], factor_b[n*stride]): caller-supplied factors in the layout the clipped-sum kernels read
+__global__ void expand_factor_kernel(const float *__restrict__ factor_w, const float *__restrict__ factor_b,
+                                     long long stride, int B, float *__restrict__ factor2, int *status_reset) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (status_reset && n == 0) *status_reset = 0;
+    if (n >= B) return;
+    factor2[2 * n] = factor_w[n * stride];
+    factor2[2 * n + 1] = factor_b[n * stride];
 }
 
 // ------------------------------------------------------------------ dense layer
@@ -919,9 +995,37 @@ dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, i
     return DP_OK;
 }
 
-dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st) {
-    bias_accum_kernel<<<(Kout + 127) / 128, 128, 0, st>>>(db, B, Kout, factor, acc_b);
+dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st, int which) {
+    bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(db, B, Kout, factor, which, acc_b);
     DP_LAUNCH_CHECK("bias_accum_kernel");
+    return DP_OK;
+}
+
+dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st) {
+    if (dtype == DP_F32)
+        bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const float *>(dY), B, Kout, factor, 1, acc_b);
+    else
+        bias_accum_kernel<__nv_bfloat16><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), B, Kout, factor, 1, acc_b);
+    DP_LAUNCH_CHECK("bias_accum_kernel");
+    return DP_OK;
+}
+
+dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, int B, int Cin, int Kout,
+                                  float *acc_w, cudaStream_t st) {
+    const dim3 grid((unsigned)((Cin + 31) / 32), (unsigned)((Kout + kDenseOT - 1) / kDenseOT));
+    if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
+    if (dtype == DP_F32)
+        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, B, Cin, Kout, acc_w);
+    else
+        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, B, Cin, Kout, acc_w);
+    DP_LAUNCH_CHECK("dense_scaled_sum_kernel");
+    return DP_OK;
+}
+
+dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2,
+                               int *status_reset, cudaStream_t st) {
+    expand_factor_kernel<<<(B + 127) / 128, 128, 0, st>>>(factor_w, factor_b, stride, B, factor2, status_reset);
+    DP_LAUNCH_CHECK("expand_factor_kernel");
     return DP_OK;
 }
 

@@ -43,8 +43,18 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
 dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
                           long long sq_stride, int clip, float C_l, float *factor, float *clip_out,
                           cudaStream_t stream, int *status_reset = nullptr);
-// acc_b[k] += sum_n factor[n*2+1] * db[n,k]
-dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream);
+// acc_b[k] += sum_n factor[n*2+which] * db[n,k]
+dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream,
+                            int which = 1);
+// dense layer, db = dY: acc_b[k] += sum_n factor[n*2+1] * dY[n,k]
+dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *factor, float *acc_b,
+                                  cudaStream_t stream);
+// dense layer: acc_w[o, i] += sum_n factor[n*2] * dY[n, o] * X[n, i]
+dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, int B, int Cin, int Kout,
+                                  float *acc_w, cudaStream_t stream);
+// factor2[n] = (factor_w[n*stride], factor_b[n*stride]); optionally clears a status word
+dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2,
+                               int *status_reset, cudaStream_t stream);
 
 dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, float *G_w,
                              float *G_b, cudaStream_t stream);

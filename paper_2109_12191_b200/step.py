@@ -49,12 +49,15 @@ class _NoiseKey:
 
 
 class GlobalClipStep:
-    """Whole-model clipping: per-example gradients are materialised per layer (STORE+NORM epilogue),
-    one dp_clip_accumulate call per chunk consumes them with the norms the epilogues produced."""
+    """Whole-model clipping.  A layer's per-example gradients are either materialised (STORE+NORM epilogue, consumed by
+    the clipped sum over memory) or, when `recompute` names the layer, never written: its norms come from a NORM_ONLY
+    call and its clipped sum from dp_per_example_wgrad_scaled once every layer's norm is known.  "auto" recomputes the
+    dense layers whose gradients are larger than the inputs they come from; a list of layer indices names any layers."""
 
-    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda", per_example_noise=False, lanes=1):
-        """lanes > 1: chunk() spreads the layers' weight-gradient calls over that many CUDA streams (a workspace each)
-        and joins them before the clip: the calls write disjoint buffers, so they may overlap."""
+    def __init__(self, layers, B, dtype, C, sigma, impl=b.DP_IMPL_AUTO, device="cuda", per_example_noise=False, lanes=1,
+                 recompute="none"):
+        """lanes > 1: chunk() spreads the layers' calls over that many CUDA streams (a workspace each) and joins them
+        around the factor computation: the calls write disjoint buffers, so they may overlap."""
         self.layers, self.B, self.dtype, self.C, self.sigma = list(layers), B, dtype, float(C), float(sigma)
         self.per_example_noise = bool(per_example_noise)
         self.tensors = _tensors_of(self.layers)
@@ -62,7 +65,6 @@ class GlobalClipStep:
         self.P_l = [t[2] for t in self.tensors]
         self.P = sum(self.P_l)
         self.descs = [layer_desc(l, B, dtype, impl, 1) for l in self.layers]
-        self.G = [torch.empty((B, p), dtype=torch.float32, device=device) for p in self.P_l]
         self.sq = torch.zeros((B, self.L), dtype=torch.float32, device=device)
         self.acc = torch.zeros(self.P, dtype=torch.float32, device=device)
         self.out = torch.empty(self.P, dtype=torch.float32, device=device)
@@ -72,20 +74,47 @@ class GlobalClipStep:
             o += p
         self.offsets = offs
         self.acc_views = [self.acc[o:o + p] for o, p in zip(offs, self.P_l)]
+        # column of each layer's first tensor in the [B, L] norm table
+        self._col, col = [], 0
+        for l in self.layers:
+            self._col.append(col)
+            col += 2 if l.n_bias else 1
+        self.recompute = self._recompute_set(recompute)
+        if self.recompute and self.per_example_noise:
+            raise ValueError("per-example noise is added by the clipped sum over materialised gradients")
+        kept = [t[0] not in self.recompute for t in self.tensors]
+        self.G = [torch.empty((B, p), dtype=torch.float32, device=device) if k else None for p, k in zip(self.P_l, kept)]
+        self._kept = [i for i, k in enumerate(kept) if k]
         self.norms = torch.empty(B, dtype=torch.float32, device=device)
         self.clip = torch.empty(B, dtype=torch.float32, device=device)
-        ws = max([b.dp_workspace_bytes(d, b.DP_EPI_STORE_NORM) for d in self.descs] + [256])
+        ws = max([b.dp_workspace_bytes(d, e) for d in self.descs for e in (b.DP_EPI_STORE_NORM, b.DP_EPI_CLIP_ACCUM)] + [256])
         self.lanes = max(1, min(int(lanes), len(self.layers)))
         self.ws_lane = [torch.empty(ws, dtype=torch.uint8, device=device) for _ in range(self.lanes)]
         self.ws = self.ws_lane[0]
         self._side = [torch.cuda.Stream(device=device) for _ in range(self.lanes - 1)] if self.lanes > 1 else []
         self.clip_ws = torch.empty(max(b.dp_clip_workspace_bytes(B, self.P_l), 256), dtype=torch.uint8, device=device)
-        # column of each layer's first tensor in the [B, L] norm table, and its G buffers
-        self._col, col = [], 0
-        for l in self.layers:
-            self._col.append(col)
-            col += 2 if l.n_bias else 1
         self.chunks_done = 0
+
+    def _recompute_set(self, recompute):
+        if recompute == "none" or not recompute:
+            return set()
+        if recompute != "auto":
+            return set(int(i) for i in recompute)
+        out = set()
+        esize = 2 if self.dtype == "bf16" else 4
+        for li, (l, d) in enumerate(zip(self.layers, self.descs)):
+            if l.kind == "norm":
+                continue
+            inputs = (math.prod(l.x_shape(self.B)) + math.prod(l.dy_shape(self.B))) * esize
+            grads = (l.n_weight + l.n_bias) * self.B * 4
+            # a dense layer's gradient is a rank-1 product: its second pass costs next to nothing.  A convolution's
+            # second pass runs the whole contraction again, which only pays when the layer is bound by its stores.
+            fast = l.kind == "dense"
+            col = self._col[li]
+            views = self.acc_views[col:col + (2 if l.n_bias else 1)]
+            if grads > inputs and fast and all(v.data_ptr() % 16 == 0 for v in views):
+                out.add(li)
+        return out
 
     def begin(self, total_batch=None, seed=0, step=0, example0=0):
         """Per-example noise needs the step's total batch, its (seed, step) and this rank's first example index up front."""
@@ -94,34 +123,59 @@ class GlobalClipStep:
         self._noise = _NoiseKey(self.per_example_noise, total_batch, seed, step, example0)
 
     def wgrad(self, li, X, dY, lane=0, stream=None):
+        """First pass of layer li: its norms, and its per-example gradients unless the layer is recomputed."""
         col = self._col[li]
+        keep = li not in self.recompute
         G_w = self.G[col]
         G_b = self.G[col + 1] if self.layers[li].n_bias else None
         b.check(b.dp_per_example_wgrad(self.descs[li], X, dY, G_w, G_b, self.sq.data_ptr() + 4 * col, self.L,
-                                       b.DP_EPI_STORE_NORM, 0.0, None, None, None, self.ws_lane[lane], stream=stream),
-                "dp_per_example_wgrad")
+                                       b.DP_EPI_STORE_NORM if keep else b.DP_EPI_NORM_ONLY, 0.0, None, None, None,
+                                       self.ws_lane[lane], stream=stream), "dp_per_example_wgrad")
 
-    def wgrad_all(self, inputs):
-        """Every layer's weight-gradient call: in order on the current stream, or forked over the lanes and joined."""
-        if self.lanes == 1:
-            for li, (X, dY) in enumerate(inputs):
-                self.wgrad(li, X, dY)
+    def wgrad_scaled(self, li, X, dY, lane=0, stream=None):
+        """Second pass of a recomputed layer: its clipped sum with the factors in self.clip."""
+        col = self._col[li]
+        acc_b = self.acc_views[col + 1] if self.layers[li].n_bias else None
+        b.check(b.dp_per_example_wgrad_scaled(self.descs[li], X, dY, self.clip, None, 1, self.acc_views[col], acc_b,
+                                              self.ws_lane[lane], stream=stream), "dp_per_example_wgrad_scaled")
+
+    def clip_factors(self):
+        """One factor per example from the norm table every layer's first pass has filled."""
+        b.check(b.dp_clip_factors(b.DP_CLIP_GLOBAL, self.B, self.L, self.sq, self.C, self.norms, self.clip), "dp_clip_factors")
+
+    def scale_kept(self, stream=None):
+        """Clipped sum of the tensors whose per-example gradients are in memory, with the factors in self.clip."""
+        b.check(b.dp_scale_accumulate(self.B, [self.G[i] for i in self._kept], [self.P_l[i] for i in self._kept], self.clip, 0,
+                                      [self.acc_views[i] for i in self._kept], stream=stream), "dp_scale_accumulate")
+
+    def _forked(self, calls):
+        """Runs calls[k](lane, stream) spread over the lanes, joined again on the current stream."""
+        if self.lanes == 1 or len(calls) <= 1:
+            for c in calls:
+                c(0, None)
             return
         main = torch.cuda.current_stream()
         fork = torch.cuda.Event()
         fork.record(main)
         streams = [main] + self._side
-        for s in self._side:
+        used = min(self.lanes, len(calls))
+        for s in streams[1:used]:
             s.wait_event(fork)
-        for li, (X, dY) in enumerate(inputs):
-            k = li % self.lanes
-            self.wgrad(li, X, dY, lane=k, stream=streams[k])
-        for s in self._side:
+        for i, c in enumerate(calls):
+            c(i % used, streams[i % used])
+        for s in streams[1:used]:
             done = torch.cuda.Event()
             done.record(s)
             main.wait_event(done)
 
-    def clip_accumulate(self, use_epilogue_norms=True):
+    def wgrad_all(self, inputs):
+        """Every layer's first-pass call: in order on the current stream, or forked over the lanes and joined."""
+        self._forked([(lambda lane, stream, li=li, X=X, dY=dY: self.wgrad(li, X, dY, lane, stream))
+                      for li, (X, dY) in enumerate(inputs)])
+
+    def clip_accumulate(self, use_epilogue_norms=True, inputs=None):
+        """Factors from the norm table, then the clipped sums: over memory for the kept tensors, by a second pass over
+        `inputs` for the recomputed layers."""
         sq = self.sq if use_epilogue_norms else None
         if self.per_example_noise:
             k = self._noise
@@ -129,15 +183,31 @@ class GlobalClipStep:
                                                 self.sigma, k.total_batch, k.seed, k.step,
                                                 k.example0 + self.B * self.chunks_done, self.acc_views, self.norms,
                                                 self.clip, self.clip_ws), "dp_clip_accumulate_noised")
-        else:
+        elif not self.recompute:
             b.check(b.dp_clip_accumulate(b.DP_CLIP_GLOBAL, self.B, self.G, self.P_l, sq, self.C, self.acc_views, self.norms,
                                          self.clip, self.clip_ws), "dp_clip_accumulate")
+        else:
+            if inputs is None:
+                raise ValueError("recomputed layers need the chunk's inputs for their second pass")
+            self.clip_factors()
+            calls = []
+            if self._kept:
+                calls.append(lambda lane, stream: self.scale_kept(stream))
+            for li in sorted(self.recompute):
+                X, dY = inputs[li]
+                calls.append(lambda lane, stream, li=li, X=X, dY=dY: self.wgrad_scaled(li, X, dY, lane, stream))
+            self._forked(calls)
         self.chunks_done += 1
 
     def chunk(self, inputs):
         """inputs: list of (X, dY) device tensors, one pair per layer."""
         self.wgrad_all(inputs)
-        self.clip_accumulate()
+        self.clip_accumulate(inputs=inputs)
+
+    def check(self):
+        """Status words of the tensor-core launches of every lane (synchronises)."""
+        for w in self.ws_lane:
+            b.check(b.dp_wgrad_check(w), "dp_wgrad_check")
 
     def finish(self, seed=0, step=0, world=1):
         """world > 1: `acc` already holds the sum over all ranks (see sharding.allreduce_accumulator)."""
