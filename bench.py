@@ -343,7 +343,7 @@ class PerLayer:
         from paper_2109_12191_b200 import synth, binding
         from paper_2109_12191_b200.step import PerLayerClipStep
         self.torch, self.synth, self.dist, self.world, self.b = torch, synth, dist, world, binding
-        self.cfg = synth.resnet50_per_layer()
+        self.cfg = self.config(synth)
         self.layers, self.B, self.G = self.cfg["layers"], self.cfg["B"], self.cfg["G"]
         self.lanes = int(os.environ.get("DP_BENCH_LANES", "4")) if world == 1 else 1
         self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"], lanes=self.lanes)
@@ -365,10 +365,18 @@ class PerLayer:
         self.flops_tc = sum(l.flops() for l, k in zip(self.layers, self.kind_of) if k == 0) * self.B
         self.bytes_kind = [sum((x.numel() + y.numel()) * 2 for (x, y), k in zip(self.inputs, self.kind_of) if k == kk) for kk in range(4)]
 
+    model = "ResNet-50"
+
+    @staticmethod
+    def config(synth):
+        return synth.resnet50_per_layer()
+
     def describe(self):
-        return {"workload": "per_layer: ResNet-50 (GroupNorm 32) at 224x224, all 161 parameter tensors (53 conv, 53x2 norm, fc "
-                            "weight + bias), bf16 X/dY ~N(0,1), B=32 per chunk x 32 chunks = |B| 1024, C=1.0 (C_l = C/sqrt(161)), "
-                            "sigma=1.0; clip + accumulate fused into dp_per_example_wgrad",
+        n_conv = sum(l.kind == "conv" for l in self.layers)
+        L = self.step_obj.L
+        return {"workload": f"{self.name}: {self.model} (GroupNorm 32) at 224x224, all {L} parameter tensors ({n_conv} conv, "
+                            f"{n_conv}x2 norm, fc weight + bias), bf16 X/dY ~N(0,1), B=32 per chunk x 32 chunks = |B| 1024, "
+                            f"C=1.0 (C_l = C/sqrt({L})), sigma=1.0; clip + accumulate fused into dp_per_example_wgrad",
                 "examples_per_step": self.examples_per_step, "params": self.step_obj.P,
                 "l2": f"one chunk of inputs is {self.in_bytes / 1e9:.2f} GB, far larger than L2",
                 "streams": self.lanes}
@@ -459,7 +467,17 @@ class PerLayer:
                                       f"{total / 1e9:.2f} Gflop by the flop ratio")
 
 
-WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad, "per_layer": PerLayer}
+class PerLayer101(PerLayer):
+    """The same path on ResNet-101 (GroupNorm), the second model of the paper's throughput comparison: 314 tensors."""
+    name = "per_layer_r101"
+    model = "ResNet-101"
+
+    @staticmethod
+    def config(synth):
+        return synth.resnet101_per_layer()
+
+
+WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad, "per_layer": PerLayer, "per_layer_r101": PerLayer101}
 VARIANT = "plain"
 
 
@@ -662,10 +680,11 @@ def run_sweep(args):
     from paper_2109_12191_b200 import binding as b, synth
     from paper_2109_12191_b200.step import layer_desc
     peaks = measured_peaks()
-    cfg = synth.resnet50_sweep() if args.workload == "sweep" else None
-    layers = cfg["layers"]
+    layers = synth.resnet50_sweep()["layers"]
     if args.workload == "sweep_all":
         layers = [l for l in synth.resnet50_gn_layers() if l.kind != "norm"]
+    if args.workload == "sweep_all_r101":
+        layers = [l for l in synth.resnet101_gn_layers() if l.kind != "norm"]
     if args.layers:
         layers = [layers[int(i)] for i in args.layers.split(",")]
     Bn, dtype = 32, "bf16"
@@ -716,7 +735,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS) + ["sweep", "sweep_all"])
+    ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS) + ["sweep", "sweep_all", "sweep_all_r101"])
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"], help="replay the step from CUDA graphs (single GPU)")
     ap.add_argument("--profile-steps", type=int, default=20, help="un-captured steps timed per call for the roofline")
@@ -726,10 +745,10 @@ def main():
     args = ap.parse_args()
     global VARIANT
     VARIANT = args.variant
-    if args.workload in ("sweep", "sweep_all"):
+    if args.workload.startswith("sweep"):
         return run_sweep(args)
     # the small-CNN step lasts ~0.16 ms: 6000 steps give the clock sampler (200 ms period) several readings under load
-    defaults = {"small_cnn": (6000, 10), "flat": (8, 3), "per_layer": (4, 3)}
+    defaults = {"small_cnn": (6000, 10), "flat": (8, 3), "per_layer": (4, 3), "per_layer_r101": (3, 3)}
     if args.steps is None:
         args.steps = defaults[args.workload][0]
     if args.warmup is None:

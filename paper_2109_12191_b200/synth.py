@@ -129,13 +129,12 @@ def resnet50_sweep():
     return dict(layers=layers, B=32, G=1, dtype="bf16", C=1.0, sigma=1.0, seed=0, step=0, mode="global")
 
 
-def resnet50_gn_layers(separate_fc_bias=True):
-    """All parameter tensors of a bottleneck ResNet-50 [3,4,6,3] with a group norm after
-    every convolution, stride on the 3x3 of the first block of stages 2-4 and a 1x1
-    projection shortcut: 53 convs + 53 norm layers (scale and shift) + classifier."""
+def resnet_gn_layers(blocks):
+    """All parameter tensors of a bottleneck ResNet with `blocks` blocks per stage and a group norm after every
+    convolution, stride on the 3x3 of the first block of stages 2-4 and a 1x1 projection shortcut."""
     layers = [conv(3, 64, 7, 2, 3, 224, name="stem"), norm(64, 112, "stem.gn")]
     H, inpl = 56, 64
-    for si, (w, nb) in enumerate(zip([64, 128, 256, 512], [3, 4, 6, 3])):
+    for si, (w, nb) in enumerate(zip([64, 128, 256, 512], blocks)):
         for b in range(nb):
             s = 2 if (b == 0 and si > 0) else 1
             Ho = (H + 2 - 3) // s + 1
@@ -150,8 +149,21 @@ def resnet50_gn_layers(separate_fc_bias=True):
     return layers
 
 
+def resnet50_gn_layers():
+    """ResNet-50 [3,4,6,3]: 53 convs + 53 norm layers (scale and shift) + classifier."""
+    return resnet_gn_layers([3, 4, 6, 3])
+
+
+def resnet101_gn_layers():
+    """ResNet-101 [3,4,23,3], the second model of the paper's throughput comparison: 104 convs + 104 norm layers +
+    classifier.  Its layer shapes are those of ResNet-50; only the third stage is longer."""
+    return resnet_gn_layers([3, 4, 23, 3])
+
+
 RESNET50_GN_PARAMS = 25_557_032   # sum of n_weight + n_bias over resnet50_gn_layers()
 RESNET50_GN_TENSORS = 161         # 53 conv weights + 53*2 norm tensors + fc weight + fc bias
+RESNET101_GN_PARAMS = 44_549_160
+RESNET101_GN_TENSORS = 314        # 104 conv weights + 104*2 norm tensors + fc weight + fc bias
 
 
 def resnet50_flat():
@@ -164,6 +176,12 @@ def resnet50_per_layer():
     """Per-layer clipping over all 161 tensors, B=32 per chunk, 32 chunks, bf16 inputs."""
     return dict(layers=resnet50_gn_layers(), B=32, G=32, dtype="bf16", C=1.0, sigma=1.0,
                 seed=0, step=0, mode="per_layer", L=RESNET50_GN_TENSORS)
+
+
+def resnet101_per_layer():
+    """Per-layer clipping over all 314 tensors of ResNet-101, B=32 per chunk, 32 chunks, bf16 inputs."""
+    return dict(layers=resnet101_gn_layers(), B=32, G=32, dtype="bf16", C=1.0, sigma=1.0,
+                seed=0, step=0, mode="per_layer", L=RESNET101_GN_TENSORS)
 
 
 def layer_inputs(layer: Layer, B: int, dtype: str, *key: int):

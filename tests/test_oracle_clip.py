@@ -231,3 +231,13 @@ def test_micro_batch_clipping_special_cases_and_brute_force():
     assert (f == 1.0).any() and (f < 1.0).any()
     for a, w in zip(acc, want):
         np.testing.assert_allclose(a, w, rtol=1e-12, atol=1e-18)
+
+
+def test_synthetic_model_inventories():
+    """Tensor and parameter counts of the two ResNets whose layer shapes the workloads use (the counts of the public
+    architectures: 25,557,032 and 44,549,160 parameters)."""
+    for layers, tensors, params in ((synth.resnet50_gn_layers(), synth.RESNET50_GN_TENSORS, synth.RESNET50_GN_PARAMS),
+                                    (synth.resnet101_gn_layers(), synth.RESNET101_GN_TENSORS, synth.RESNET101_GN_PARAMS)):
+        assert sum(1 + (l.n_bias > 0) for l in layers) == tensors
+        assert sum(l.n_weight + l.n_bias for l in layers) == params
+    assert synth.RESNET50_GN_PARAMS == 25_557_032 and synth.RESNET101_GN_PARAMS == 44_549_160
