@@ -125,7 +125,11 @@ class SmallCnn:
         self.lanes = int(os.environ.get("DP_BENCH_LANES", "4")) if world == 1 else 1
         # layers whose per-example gradients outweigh their inputs (conv3, the classifier) are not materialised
         self.recompute = os.environ.get("DP_BENCH_RECOMPUTE", "auto")
-        self.step_obj = GlobalClipStep(self.layers, self.B, "f32", self.cfg["C"], self.cfg["sigma"], lanes=self.lanes,
+        # fp32 inputs; tensor-core layers take them as tf32 (one pass, the precision class the accuracy bounds name)
+        # or, with --precision f32, as three products of a hi/lo split
+        self.precision = PRECISION
+        self.dtype_name = "tf32" if PRECISION == "tf32" else "f32 (3 x tf32 on tensor cores)"
+        self.step_obj = GlobalClipStep(self.layers, self.B, PRECISION, self.cfg["C"], self.cfg["sigma"], lanes=self.lanes,
                                        recompute=self.recompute)
         self.examples_per_step = self.B
         # inputs rotate over several sets so that consecutive steps never find their inputs in L2
@@ -140,7 +144,9 @@ class SmallCnn:
 
     def describe(self):
         return {"workload": "small_cnn: conv3x3 3->32 s1, 32->64 s2, 64->128 s2, dense 8192->10 (all with bias) on 32x32x3, "
-                            "B=256 fp32, global clip C=1.5, sigma=1.0, |B|=256",
+                            "B=256 fp32 inputs, global clip C=1.5, sigma=1.0, |B|=256",
+                "precision": ("tensor-core layers round the fp32 inputs to tf32 (nearest even), one pass" if self.precision == "tf32"
+                              else "tensor-core layers run three split-tf32 passes"),
                 "examples_per_step": self.B, "params": self.step_obj.P,
                 "l2": f"inputs rotate over {self.n_sets} resident sets ({self.n_sets * self.in_bytes / 1e6:.0f} MB) and "
                       f"{sum(self.step_obj.P_l[i] for i in self.step_obj._kept) * self.B * 4 / 1e6:.0f} MB of per-example gradients are written and re-read per step",
@@ -479,6 +485,7 @@ class PerLayer101(PerLayer):
 
 WORKLOADS = {"small_cnn": SmallCnn, "flat": FlatGrad, "per_layer": PerLayer, "per_layer_r101": PerLayer101}
 VARIANT = "plain"
+PRECISION = "tf32"
 
 
 class CallTimer:
@@ -741,10 +748,13 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=20, help="un-captured steps timed per call for the roofline")
     ap.add_argument("--layers", default="", help="sweep workloads: comma-separated layer indices")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--precision", default="tf32", choices=["tf32", "f32"],
+                    help="small_cnn: how tensor-core layers take the fp32 inputs (one tf32 pass | three split-tf32 passes)")
     ap.add_argument("--variant", default="plain", help="flat workload: plain | per_example_noise | micro2 | micro4 ...")
     args = ap.parse_args()
-    global VARIANT
+    global VARIANT, PRECISION
     VARIANT = args.variant
+    PRECISION = args.precision
     if args.workload.startswith("sweep"):
         return run_sweep(args)
     # the small-CNN step lasts ~0.16 ms: 6000 steps give the clock sampler (200 ms period) several readings under load

@@ -48,7 +48,15 @@ typedef enum {
     DP_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up (reported through dp_wgrad_check) */
 } dp_status;
 
-typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;            /* type of X and dY; every output is fp32 */
+typedef enum {
+    DP_F32 = 0,               /* X and dY are fp32; tensor-core layers run them as three tf32 products of a hi/lo split
+                                 (error about 4e-6 relative), everything else in plain fp32 */
+    DP_BF16 = 1,              /* X and dY are bf16, products exact in fp32 */
+    DP_TF32 = 2               /* X and dY are fp32; tensor-core layers round them to tf32 (nearest even) and run ONE
+                                 product: per-example norms stay within 1e-4, gradients within 2e-3 relative L2, at
+                                 two thirds of the shared-memory traffic and a third of the tensor work of DP_F32.
+                                 Layers that do not run on tensor cores behave exactly as under DP_F32. */
+} dp_dtype;                   /* every output is fp32 */
 typedef enum { DP_LAYER_DENSE = 0, DP_LAYER_CONV2D = 1, DP_LAYER_NORM_AFFINE = 2 } dp_layer_kind;
 typedef enum { DP_CLIP_GLOBAL = 0, DP_CLIP_PER_LAYER = 1 } dp_clip_mode;
 typedef enum {

@@ -18,7 +18,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 # enums of dpstep.h
 DP_OK, DP_ERR_INVALID_ARG, DP_ERR_UNSUPPORTED, DP_ERR_WORKSPACE, DP_ERR_CUDA, DP_ERR_TIMEOUT = range(6)
-DP_F32, DP_BF16 = 0, 1
+DP_F32, DP_BF16, DP_TF32 = 0, 1, 2
 DP_LAYER_DENSE, DP_LAYER_CONV2D, DP_LAYER_NORM_AFFINE = 0, 1, 2
 DP_CLIP_GLOBAL, DP_CLIP_PER_LAYER = 0, 1
 DP_EPI_STORE_NORM, DP_EPI_NORM_ONLY, DP_EPI_CLIP_ACCUM = 0, 1, 2

@@ -24,7 +24,7 @@ void note_error(const char *message) { snprintf(g_last_error, sizeof(g_last_erro
 static bool valid_desc(const dp_layer_desc *d) {
     if (!d) return false;
     if (d->kind != DP_LAYER_DENSE && d->kind != DP_LAYER_CONV2D && d->kind != DP_LAYER_NORM_AFFINE) return false;
-    if (d->dtype != DP_F32 && d->dtype != DP_BF16) return false;
+    if (d->dtype != DP_F32 && d->dtype != DP_BF16 && d->dtype != DP_TF32) return false;
     if (d->impl != DP_IMPL_AUTO && d->impl != DP_IMPL_CUDA_CORE && d->impl != DP_IMPL_TENSOR_CORE) return false;
     if (d->B <= 0 || d->C_in <= 0 || d->K_out <= 0 || d->H <= 0 || d->W <= 0) return false;
     if (d->kind == DP_LAYER_CONV2D) {
@@ -47,6 +47,9 @@ static ConvGeom geom_of(const dp_layer_desc *d) {
     g.M = d->K_out; g.N = d->R * d->S * d->C_in; g.K = g.OH * g.OW;
     return g;
 }
+
+// Element type of X and dY in memory: DP_TF32 only changes the arithmetic of the tensor-core kernel.
+static int storage_type(const dp_layer_desc *d) { return d->dtype == DP_TF32 ? DP_F32 : d->dtype; }
 
 static bool has_bias_tensor(const dp_layer_desc *d) { return d->kind == DP_LAYER_NORM_AFFINE || d->has_bias != 0; }
 static int groups_of(const dp_layer_desc *d) { return (d->bias_separate && has_bias_tensor(d)) ? 2 : 1; }
@@ -78,7 +81,7 @@ static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
     if (d->kind != DP_LAYER_NORM_AFFINE && d->has_bias) off = round_up(off + sizeof(float) * B * d->K_out, 256);
     pl.chunk_off = off; pl.dg_off = off;
     if (d->kind == DP_LAYER_NORM_AFFINE) {
-        off = round_up(off + sizeof(float) * B * norm_chunks(d->dtype, d->B, d->H * d->W, d->C_in) * 2 * d->C_in, 256);
+        off = round_up(off + sizeof(float) * B * norm_chunks(storage_type(d), d->B, d->H * d->W, d->C_in) * 2 * d->C_in, 256);
         pl.dg_off = off;
         off = round_up(off + sizeof(float) * B * 2 * d->C_in, 256);
     }
@@ -152,26 +155,26 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
     if (d->kind == DP_LAYER_CONV2D) {
         float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;
         if (pl.use_thin && rgb3_conv_eligible(g))
-            return launch_conv_rgb3(d->dtype, X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, d->has_bias, groups == 2,
+            return launch_conv_rgb3(storage_type(d), X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, d->has_bias, groups == 2,
                                     sqnorm, sqnorm_stride, reset, st);
         if (pl.use_thin) {
-            rc = launch_conv_thin(d->dtype, X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, partial, pl.slots, d->has_bias, st);
+            rc = launch_conv_thin(storage_type(d), X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, partial, pl.slots, d->has_bias, st);
             if (rc != DP_OK) return rc;
             return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
         }
         if (d->has_bias) {
-            rc = launch_bias(d->dtype, dY, g, db, partial, pl.slots, pl.w_slots, st);
+            rc = launch_bias(storage_type(d), dY, g, db, partial, pl.slots, pl.w_slots, st);
             if (rc != DP_OK) return rc;
         }
         if (epi != DP_EPI_CLIP_ACCUM) {
             if (pl.use_tc) rc = launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
-            else rc = launch_conv_fma(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, nullptr, st);
+            else rc = launch_conv_fma(storage_type(d), epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, nullptr, st);
             if (rc != DP_OK) return rc;
             return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
         }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
-        else rc = launch_conv_fma(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
+        else rc = launch_conv_fma(storage_type(d), DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
         if (rc != DP_OK) return rc;
         if (pl.use_tc && !d->has_bias) {
             // no bias: the clipped-sum pass finalises the norms itself
@@ -181,7 +184,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st, reset);
         if (rc != DP_OK) return rc;
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true);
-        else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
+        else rc = launch_conv_fma(storage_type(d), DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
@@ -189,15 +192,15 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
 
     if (d->kind == DP_LAYER_DENSE) {
         if (epi == DP_EPI_STORE_NORM) {
-            rc = launch_dense_store(d->dtype, X, dY, d->B, d->C_in, d->K_out, G_w, d->has_bias ? G_b : nullptr, st);
+            rc = launch_dense_store(storage_type(d), X, dY, d->B, d->C_in, d->K_out, G_w, d->has_bias ? G_b : nullptr, st);
             if (rc != DP_OK) return rc;
         }
         float *db_dst = !d->has_bias ? nullptr : (epi == DP_EPI_STORE_NORM ? G_b : (clip ? db_ws : nullptr));
-        rc = launch_dense_norm(d->dtype, X, dY, d->B, d->C_in, d->K_out, d->has_bias, db_dst, groups == 2, sqnorm,
+        rc = launch_dense_norm(storage_type(d), X, dY, d->B, d->C_in, d->K_out, d->has_bias, db_dst, groups == 2, sqnorm,
                                sqnorm_stride, clip, C_l, factor, clip_out, reset, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
-        rc = launch_dense_scaled_sum(d->dtype, X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
+        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
@@ -208,7 +211,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         float *chunk_partial = reinterpret_cast<float *>(ws + pl.chunk_off);
         float *dg = (epi == DP_EPI_STORE_NORM) ? G_w : reinterpret_cast<float *>(ws + pl.dg_off);
         float *dbt = (epi == DP_EPI_STORE_NORM) ? G_b : reinterpret_cast<float *>(ws + pl.dg_off) + (size_t)d->B * d->C_in;
-        rc = launch_norm_affine(d->dtype, X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
+        rc = launch_norm_affine(storage_type(d), X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
         if (rc != DP_OK) return rc;
         if (clip)
             return launch_affine_clip_accum(partial, d->B, C_l, groups == 2, sqnorm, sqnorm_stride, clip_out, dg, dbt, d->C_in,
@@ -245,27 +248,27 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
 
     if (d->kind == DP_LAYER_CONV2D) {
         if (d->has_bias) {
-            rc = launch_bias(d->dtype, dY, g, db_ws, partial, pl.slots, pl.w_slots, st);
+            rc = launch_bias(storage_type(d), dY, g, db_ws, partial, pl.slots, pl.w_slots, st);
             if (rc != DP_OK) return rc;
         }
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, status_word, st);
-        else rc = launch_conv_fma(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
+        else rc = launch_conv_fma(storage_type(d), DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
     }
     if (d->kind == DP_LAYER_DENSE) {
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis; the bias gradient is dY itself
-        rc = launch_dense_scaled_sum(d->dtype, X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
+        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
         if (rc != DP_OK) return rc;
-        if (d->has_bias) return launch_dense_bias_accum(d->dtype, dY, d->B, d->K_out, factor, acc_b, st);
+        if (d->has_bias) return launch_dense_bias_accum(storage_type(d), dY, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
     }
     {
         float *chunk_partial = reinterpret_cast<float *>(ws + pl.chunk_off);
         float *dg = reinterpret_cast<float *>(ws + pl.dg_off);
         float *dbt = dg + (size_t)d->B * d->C_in;
-        rc = launch_norm_affine(d->dtype, X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
+        rc = launch_norm_affine(storage_type(d), X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
         if (rc != DP_OK) return rc;
         rc = launch_bias_accum(dg, d->B, d->C_in, factor, acc_w, st, 0);
         if (rc != DP_OK) return rc;

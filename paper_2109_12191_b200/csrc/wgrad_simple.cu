@@ -341,7 +341,7 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
 template <typename T>
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(256, 2)
 conv_wgrad_rgb3_kernel(const T *__restrict__ X, const T *__restrict__ dY, const ConvGeom g, float *__restrict__ G_w,
                        float *__restrict__ db, int has_bias, int separate, float *__restrict__ sqnorm,
                        long long sq_stride, int *status_reset) {

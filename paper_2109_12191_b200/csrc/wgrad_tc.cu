@@ -50,6 +50,7 @@ struct TcParams {
     int a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT;
     int OWt, OHt, tiles_w, Kt, k_tiles, stages, stage_bytes, a_bytes;
     int lo_offset;              // split tf32: byte offset of the lo copy inside a stage
+    int single_pass;            // fp32 inputs rounded to tf32 (nearest even) in place, one MMA per step, no lo copy
     int mode;                   // 0 store + norm, 1 norm only, 2 clipped sum over a range of examples
     float *G_w;
     float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
@@ -290,7 +291,14 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     uint32_t bd = desc_lo | (((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
                     // rows of the A tile past the operand's extent hold whatever the stage held before:
                     // they only feed rows of D that the epilogue never reads
-                    if (TF32) {
+                    if (TF32 && p.single_pass) {
+#pragma unroll 4
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            umma<TF32>(d_tmem, ad, bd, desc_hi32, idesc, accumulate);
+                            accumulate = 1;
+                            ad += kadvance; bd += kadvance;
+                        }
+                    } else if (TF32) {
                         const uint32_t lo = (uint32_t)p.lo_offset >> 4;
 #pragma unroll 2
                         for (int ks = 0; ks < ksteps; ++ks) {
@@ -351,7 +359,15 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                 if (i0 + 128 * u < rchunks) x[u] = *reinterpret_cast<const float4 *>(rbase + ((size_t)(i0 + 128 * u) << 4));
 #pragma unroll
                             for (int u = 0; u < 4; ++u) {
-                                if (i0 + 128 * u < rchunks) {
+                                if (i0 + 128 * u < rchunks && p.single_pass) {
+                                    // round to tf32, nearest even, in place: the tensor core's own truncation then changes nothing
+                                    uint4 b = *reinterpret_cast<const uint4 *>(&x[u]);
+                                    b.x = (b.x + 0xFFFu + ((b.x >> 13) & 1u)) & 0xFFFFE000u;
+                                    b.y = (b.y + 0xFFFu + ((b.y >> 13) & 1u)) & 0xFFFFE000u;
+                                    b.z = (b.z + 0xFFFu + ((b.z >> 13) & 1u)) & 0xFFFFE000u;
+                                    b.w = (b.w + 0xFFFu + ((b.w >> 13) & 1u)) & 0xFFFFE000u;
+                                    *reinterpret_cast<uint4 *>(rbase + ((size_t)(i0 + 128 * u) << 4)) = b;
+                                } else if (i0 + 128 * u < rchunks) {
                                     uint8_t *ptr = rbase + ((size_t)(i0 + 128 * u) << 4);
                                     float4 hi, lo;
                                     hi.x = __uint_as_float(__float_as_uint(x[u].x) & 0xFFFFE000u); lo.x = x[u].x - hi.x;
@@ -674,9 +690,13 @@ static TcProblem tc_problem(int dtype, const ConvGeom &g) {
 // instruction occupies the tensor pipe for N/2 cycles, and shared memory moves 128 B per cycle in total, shared by
 // the tensor core's operand reads (always 128 rows of A plus N rows of B, 32 B per row and step), the TMA fill of the
 // stage and, for split tf32, the split warps (they read every landed byte once and write the lo copy).
-static double step_cycles(bool bf16, int n_cols, double a_slabs_loaded, double b_slabs) {
-    if (bf16) {
+static double step_cycles(int dtype, int n_cols, double a_slabs_loaded, double b_slabs) {
+    if (dtype == DP_BF16) {
         const double smem = 4096.0 + 32.0 * n_cols + 2048.0 * (a_slabs_loaded + b_slabs);
+        return std::max(n_cols / 2.0, smem / 128.0);
+    }
+    if (dtype == DP_TF32) {   // one MMA per step; the stage is filled once, read once and written back once by the rounding warps
+        const double smem = 4096.0 + 32.0 * n_cols + 1024.0 * (a_slabs_loaded + b_slabs) * 3.0;
         return std::max(n_cols / 2.0, smem / 128.0);
     }
     const double smem = 3.0 * (4096.0 + 32.0 * n_cols) + 1024.0 * (a_slabs_loaded + b_slabs) * 3.0;
@@ -710,7 +730,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
     if (g.stride > 8 || g.K < 1 || g.OH > 65535) return best;
     const int sms = sm_count();
     const int a_slabs_tile = 128 / slab_ch;
-    const int copies = (dtype == DP_BF16) ? 1 : 2;      // split tf32 keeps a hi and a lo copy of every stage
+    const int copies = (dtype == DP_F32) ? 2 : 1;       // split tf32 keeps a hi and a lo copy of every stage
     double best_cost = 1e300;
     for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
         const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
@@ -725,7 +745,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             const double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
                                              : std::max(1.0, (double)total_tiles / sms);
             const double a_loaded = (double)(a_ext / slab_ch) / m_tiles, b_loaded = (double)(b_ext / slab_ch) / n_tiles;
-            const double step = step_cycles(dtype == DP_BF16, NT, a_loaded, b_loaded);
+            const double step = step_cycles(dtype, NT, a_loaded, b_loaded);
             // the epilogue of a tile overlaps the main loop of the next; what it costs depends on what it does with
             // the 128 x NT accumulator: stores run at about 16 B/clk per SM when lanes write consecutive addresses
             // (rows of D are gradient columns) and about 7 B/clk otherwise; reading TMEM alone is cheap
@@ -884,6 +904,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
     p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
     p.lo_offset = pl.stage_bytes / 2;
+    p.single_pass = (dtype == DP_TF32) ? 1 : 0;
     p.mode = clip ? 2 : (epilogue == DP_EPI_STORE_NORM ? 0 : 1);
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
     p.reset_status = second_pass ? 0 : 1;       // the second launch of a fused clip call must keep the first one's verdict

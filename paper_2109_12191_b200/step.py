@@ -16,8 +16,11 @@ from .synth import Layer
 _KIND = {"conv": b.DP_LAYER_CONV2D, "dense": b.DP_LAYER_DENSE, "norm": b.DP_LAYER_NORM_AFFINE}
 
 
+_DTYPE = {"f32": b.DP_F32, "bf16": b.DP_BF16, "tf32": b.DP_TF32}   # "tf32": fp32 in memory, one tf32 pass on tensor cores
+
+
 def layer_desc(layer: Layer, B: int, dtype: str, impl=b.DP_IMPL_AUTO, bias_separate=1):
-    return b.make_desc(_KIND[layer.kind], b.DP_BF16 if dtype == "bf16" else b.DP_F32, B, layer.Cin, layer.Kout,
+    return b.make_desc(_KIND[layer.kind], _DTYPE[dtype], B, layer.Cin, layer.Kout,
                        layer.H, layer.W, layer.R, layer.S, layer.stride, layer.pad, int(layer.bias), bias_separate, impl)
 
 

@@ -43,7 +43,8 @@ def dev_inputs(inp, dtype):
 def make_desc(layer, Bn, dtype, impl=0, bias_separate=0):
     b = B()
     kind = {"conv": b.DP_LAYER_CONV2D, "dense": b.DP_LAYER_DENSE, "norm": b.DP_LAYER_NORM_AFFINE}[layer.kind]
-    return b.make_desc(kind, b.DP_BF16 if dtype == "bf16" else b.DP_F32, Bn, layer.Cin, layer.Kout, layer.H, layer.W,
+    code = {"f32": b.DP_F32, "bf16": b.DP_BF16, "tf32": b.DP_TF32}[dtype]
+    return b.make_desc(kind, code, Bn, layer.Cin, layer.Kout, layer.H, layer.W,
                        layer.R, layer.S, layer.stride, layer.pad, int(layer.bias), bias_separate, impl)
 
 

@@ -60,8 +60,11 @@ def test_single_dense_layer_workload():
     assert np.all(f < 1.0)                                   # norms are about 128, every example is clipped
 
 
-def test_small_cnn_workload_full_batch():
-    f = run_global_step(synth.small_cnn())
+@pytest.mark.parametrize("dtype", ["f32", "tf32"])
+def test_small_cnn_workload_full_batch(dtype):
+    """fp32 inputs as three split-tf32 products, and in the benchmark's mode: rounded to tf32, one product."""
+    cfg = dict(synth.small_cnn()); cfg["dtype"] = dtype
+    f = run_global_step(cfg)
     assert np.all(f < 1.0)
 
 
