@@ -200,7 +200,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
                                sqnorm_stride, clip, C_l, factor, clip_out, reset, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
-        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
+        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, 2, d->B, d->C_in, d->K_out, acc_w, nullptr, st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
@@ -242,8 +242,17 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
     float *db_ws = reinterpret_cast<float *>(ws + pl.db_off);
     const ConvGeom g = geom_of(d);
     int *status_word = reinterpret_cast<int *>(ws + pl.status_off);
+    dp_status rc;
+    if (d->kind == DP_LAYER_DENSE) {
+        // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis; the bias gradient is dY itself.
+        // Both kernels read the caller's factors in place.
+        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor_w, factor_stride, d->B, d->C_in, d->K_out, acc_w, status_word, st);
+        if (rc != DP_OK) return rc;
+        if (d->has_bias) rc = launch_dense_bias_accum(storage_type(d), dY, d->B, d->K_out, factor_b, factor_stride, acc_b, st);
+        return rc;
+    }
     // the clipped-sum kernels read one (weight, bias) pair of factors per example
-    dp_status rc = launch_expand_factor(factor_w, factor_b, factor_stride, d->B, factor, pl.use_tc ? nullptr : status_word, st);
+    rc = launch_expand_factor(factor_w, factor_b, factor_stride, d->B, factor, pl.use_tc ? nullptr : status_word, st);
     if (rc != DP_OK) return rc;
 
     if (d->kind == DP_LAYER_CONV2D) {
@@ -255,13 +264,6 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
         else rc = launch_conv_fma(storage_type(d), DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
-        return DP_OK;
-    }
-    if (d->kind == DP_LAYER_DENSE) {
-        // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis; the bias gradient is dY itself
-        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, d->B, d->C_in, d->K_out, acc_w, st);
-        if (rc != DP_OK) return rc;
-        if (d->has_bias) return launch_dense_bias_accum(storage_type(d), dY, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
     }
     {

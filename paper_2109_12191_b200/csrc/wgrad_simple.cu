@@ -596,18 +596,20 @@ finalize_norm_kernel(const float *__restrict__ partial, int slots, int w_slots, 
     }
 }
 
-// acc[k] += sum_n factor[2n + which] * v[n, k]   (which = 1: the bias-like tensor's factor, 0: the weight's).
-// Block = 32 channels x 8 example groups (group q owns examples q, q+8, ...), groups folded in order.
+// acc[k] += sum_n f[n * f_stride] * v[n, k].  Block = 32 channels x 8 example groups (group q owns examples
+// q, q+8, ...), groups folded in order.
 template <typename T>
 __global__ void __launch_bounds__(256)
-bias_accum_kernel(const T *__restrict__ db, int B, int Kout, const float *__restrict__ factor, int which,
+bias_accum_kernel(const T *__restrict__ db, int B, int Kout, const float *__restrict__ f, long long f_stride,
                   float *__restrict__ acc_b) {
     __shared__ float part[8][32];
     const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
     const int k = blockIdx.x * 32 + lane;
     float a = 0.f;
-    if (k < Kout)
-        for (int n = q; n < B; n += 8) a = fmaf(factor[2 * n + which], to_float(db[(long long)n * Kout + k]), a);
+    if (k < Kout) {
+#pragma unroll 8
+        for (int n = q; n < B; n += 8) a = fmaf(f[n * f_stride], to_float(db[(long long)n * Kout + k]), a);
+    }
     part[q][lane] = a;
     __syncthreads();
     if (q == 0 && k < Kout) {
@@ -625,9 +627,10 @@ bias_accum_kernel(const T *__restrict__ db, int B, int Kout, const float *__rest
 constexpr int kDenseOT = 16;
 template <typename T>
 __global__ void __launch_bounds__(256)
-dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const float *__restrict__ factor, int B,
-                        int Cin, int Kout, float *__restrict__ acc) {
-    __shared__ __align__(16) float fy[256][kDenseOT];        // f_n * dY[n, o0 .. o0+15] for a run of 256 examples
+dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const float *__restrict__ factor,
+                        long long f_stride, int B, int Cin, int Kout, float *__restrict__ acc, int *status_reset) {
+    __shared__ __align__(16) float fy[256][kDenseOT];
+    if (status_reset && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status_reset = 0;   // no waits on this path        // f_n * dY[n, o0 .. o0+15] for a run of 256 examples
     __shared__ float part[8][kDenseOT][32];
     const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
     const int i = blockIdx.x * 32 + lane, o0 = blockIdx.y * kDenseOT;
@@ -639,11 +642,11 @@ dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const
         __syncthreads();
         for (int t = threadIdx.x; t < nb * kDenseOT; t += 256) {
             const int n = t / kDenseOT, o = t - n * kDenseOT;
-            fy[n][o] = (o0 + o < Kout) ? factor[2 * (n0 + n)] * to_float(dY[(long long)(n0 + n) * Kout + o0 + o]) : 0.f;
+            fy[n][o] = (o0 + o < Kout) ? factor[(n0 + n) * f_stride] * to_float(dY[(long long)(n0 + n) * Kout + o0 + o]) : 0.f;
         }
         __syncthreads();
         if (i < Cin) {
-#pragma unroll 4
+#pragma unroll 8
             for (int n = q; n < nb; n += 8) {
                 const float x = to_float(X[(long long)(n0 + n) * Cin + i]);
                 const float4 *row = reinterpret_cast<const float4 *>(fy[n]);
@@ -996,28 +999,29 @@ dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, i
 }
 
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st, int which) {
-    bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(db, B, Kout, factor, which, acc_b);
+    bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(db, B, Kout, factor + which, 2, acc_b);
     DP_LAUNCH_CHECK("bias_accum_kernel");
     return DP_OK;
 }
 
-dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st) {
+dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *f, long long f_stride, float *acc_b,
+                                  cudaStream_t st) {
     if (dtype == DP_F32)
-        bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const float *>(dY), B, Kout, factor, 1, acc_b);
+        bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const float *>(dY), B, Kout, f, f_stride, acc_b);
     else
-        bias_accum_kernel<__nv_bfloat16><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), B, Kout, factor, 1, acc_b);
+        bias_accum_kernel<__nv_bfloat16><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), B, Kout, f, f_stride, acc_b);
     DP_LAUNCH_CHECK("bias_accum_kernel");
     return DP_OK;
 }
 
-dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, int B, int Cin, int Kout,
-                                  float *acc_w, cudaStream_t st) {
+dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, long long f_stride, int B,
+                                  int Cin, int Kout, float *acc_w, int *status_reset, cudaStream_t st) {
     const dim3 grid((unsigned)((Cin + 31) / 32), (unsigned)((Kout + kDenseOT - 1) / kDenseOT));
     if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
     if (dtype == DP_F32)
-        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, B, Cin, Kout, acc_w);
+        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, f_stride, B, Cin, Kout, acc_w, status_reset);
     else
-        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, B, Cin, Kout, acc_w);
+        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, f_stride, B, Cin, Kout, acc_w, status_reset);
     DP_LAUNCH_CHECK("dense_scaled_sum_kernel");
     return DP_OK;
 }

@@ -46,12 +46,12 @@ dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, i
 // acc_b[k] += sum_n factor[n*2+which] * db[n,k]
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream,
                             int which = 1);
-// dense layer, db = dY: acc_b[k] += sum_n factor[n*2+1] * dY[n,k]
-dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *factor, float *acc_b,
+// dense layer, db = dY: acc_b[k] += sum_n f[n*f_stride] * dY[n,k]
+dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *f, long long f_stride, float *acc_b,
                                   cudaStream_t stream);
-// dense layer: acc_w[o, i] += sum_n factor[n*2] * dY[n, o] * X[n, i]
-dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, int B, int Cin, int Kout,
-                                  float *acc_w, cudaStream_t stream);
+// dense layer: acc_w[o, i] += sum_n factor[n*f_stride] * dY[n, o] * X[n, i]
+dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, long long f_stride, int B,
+                                  int Cin, int Kout, float *acc_w, int *status_reset, cudaStream_t stream);
 // factor2[n] = (factor_w[n*stride], factor_b[n*stride]); optionally clears a status word
 dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2,
                                int *status_reset, cudaStream_t stream);
