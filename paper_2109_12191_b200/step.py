@@ -90,7 +90,7 @@ class GlobalClipStep:
         self._kept = [i for i, k in enumerate(kept) if k]
         self.norms = torch.empty(B, dtype=torch.float32, device=device)
         self.clip = torch.empty(B, dtype=torch.float32, device=device)
-        ws = max([b.dp_workspace_bytes(d, e) for d in self.descs for e in (b.DP_EPI_STORE_NORM, b.DP_EPI_CLIP_ACCUM)] + [256])
+        ws = max([b.dp_workspace_bytes(d, e) for d in self.descs for e in (b.DP_EPI_STORE_NORM, b.DP_EPI_NORM_ONLY, b.DP_EPI_CLIP_ACCUM)] + [256])
         self.lanes = max(1, min(int(lanes), len(self.layers)))
         self.ws_lane = [torch.empty(ws, dtype=torch.uint8, device=device) for _ in range(self.lanes)]
         self.ws = self.ws_lane[0]

@@ -102,3 +102,41 @@ def test_layer_calls_spread_over_streams_give_the_same_bits():
     g.replay(); g.replay()
     torch.cuda.synchronize()
     assert torch.equal(result(many), result(one))
+
+
+def test_full_resnet50_chunk_in_the_benchmarks_launch_configuration():
+    """One whole 32-example chunk of the per-layer ResNet-50 workload (all 107 layer calls, 2.8 GB of inputs) the way the
+    benchmark times it -- four streams, replayed from a CUDA graph -- against plain launches on one stream: the 161
+    accumulators and the norm table must agree bit for bit.  (Single layers at this size are checked against the oracle
+    above; the oracle cannot run the whole chunk in a test's time.)"""
+    cfg = synth.resnet50_per_layer()
+    layers, Bn = cfg["layers"], cfg["B"]
+    g = torch.Generator(device="cuda"); g.manual_seed(77)
+    ins = [(torch.empty(l.x_shape(Bn), device="cuda", dtype=torch.bfloat16).normal_(generator=g),
+            (torch.empty(l.dy_shape(Bn), device="cuda", dtype=torch.bfloat16).normal_(generator=g) * 1e-3).contiguous())
+           for l in layers]
+
+    def result(st):
+        return torch.cat([t for pair in zip(st.acc_w, st.acc_b) for t in pair if t is not None]).clone()
+
+    one = PerLayerClipStep(layers, Bn, "bf16", cfg["C"], cfg["sigma"])
+    one.begin(); one.chunk(ins)
+    torch.cuda.synchronize()
+    one.check()
+    ref, ref_sq = result(one), one.sq.clone()
+    assert ref.numel() == synth.RESNET50_GN_PARAMS and torch.isfinite(ref).all() and ref.abs().max() > 0
+    f = torch.clamp((cfg["C"] / math.sqrt(one.L)) / ref_sq.sqrt(), max=1.0)
+    assert (f == 1.0).any() and (f < 1.0).any()            # the scaled dY puts examples on both sides of the thresholds
+    del one
+    many = PerLayerClipStep(layers, Bn, "bf16", cfg["C"], cfg["sigma"], lanes=4)
+    many.begin(); many.chunk(ins)                           # warm-up outside the capture
+    torch.cuda.synchronize()
+    many.begin()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        many.chunk_calls(ins)
+    graph.replay()
+    torch.cuda.synchronize()
+    many.check()
+    assert torch.equal(result(many), ref)
+    assert torch.equal(many.sq, ref_sq)
