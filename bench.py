@@ -113,7 +113,7 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------- workloads (device side)
 class SmallCnn:
-    """configs[1]: 3 convs + classifier on 32x32x3, B=256, fp32, whole-model clip C=1.5, sigma=1."""
+    """The small-CNN workload: 3 convs + classifier on 32x32x3, B=256, fp32, whole-model clip C=1.5, sigma=1."""
     name = "small_cnn"
 
     def __init__(self, torch, rank, dist=None, world=1):
@@ -251,7 +251,7 @@ class SmallCnn:
 
 
 class FlatGrad:
-    """configs[3]: flattened ResNet-50 gradients, P=25,557,032, B=64 per chunk, 16 chunks, C=1, sigma=1."""
+    """The flat workload: flattened ResNet-50 gradients, P=25,557,032, B=64 per chunk, 16 chunks, C=1, sigma=1."""
     name = "flat"
 
     def __init__(self, torch, rank, dist=None, world=1):
@@ -340,7 +340,7 @@ class FlatGrad:
 
 
 class PerLayer:
-    """configs[4]: ResNet-50 (GroupNorm) per-layer clipping over all 161 tensors, bf16 inputs, B=32 per chunk,
+    """The per-layer workload: ResNet-50 (GroupNorm) per-layer clipping over all 161 tensors, bf16 inputs, B=32 per chunk,
     32 chunks, C_l = C/sqrt(161), clip + accumulate fused into the weight-gradient call."""
     name = "per_layer"
     dtype_name = "bf16"
@@ -678,7 +678,7 @@ def run_reference(args):
 
 
 def run_sweep(args):
-    """configs[2] / any layer list: time dp_per_example_wgrad per layer with both epilogues.
+    """The layer sweep (or any layer list): time dp_per_example_wgrad per layer with both epilogues.
     L2 is flushed (a 512 MB buffer is overwritten) before every timed launch."""
     import torch
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
