@@ -253,6 +253,7 @@ class SmallCnn:
 class FlatGrad:
     """The flat workload: flattened ResNet-50 gradients, P=25,557,032, B=64 per chunk, 16 chunks, C=1, sigma=1."""
     name = "flat"
+    e2e_cap = 8          # an end-to-end step copies 105 GB from the host: a few of them are enough
 
     def __init__(self, torch, rank, dist=None, world=1):
         from paper_2109_12191_b200 import synth
@@ -262,7 +263,9 @@ class FlatGrad:
         self.P, self.B, self.G = self.cfg["P"], self.cfg["B"], self.cfg["G"]
         if os.environ.get("DPSTEP_FLAT_PARAMS"):          # reduced P for profiler captures (same kernels, fewer bytes held)
             self.P = int(os.environ["DPSTEP_FLAT_PARAMS"])
-        # --variant: "per_example_noise" (the paper's own form of the noise) or "microN" (clip the mean of N examples)
+        # --variant: "per_example_noise" (the paper's own form of the noise), "microN" (clip the mean of N examples) or
+        # "norms_supplied" (the squared norms come in with the gradients, as they do from the weight-gradient
+        # epilogues, so the chunk is read once instead of twice)
         self.variant = VARIANT
         micro = int(self.variant[5:]) if self.variant.startswith("micro") else 1
         self.step_obj = FlatClipStep(self.P, self.B, self.cfg["C"], self.cfg["sigma"],
@@ -274,11 +277,17 @@ class FlatGrad:
             t = torch.empty((self.B, self.P), device="cuda")
             t.normal_(0.0, self.cfg["grad_std"], generator=g)
             self.bufs.append(t)
-        self.call_names = ["clip_accumulate(norms computed)", "noise_average"]
+        self.supplied = None
+        if self.variant == "norms_supplied":                 # set-up, outside every timed region
+            self.supplied = [(t.double() ** 2).sum(1, keepdim=True).float().contiguous() if self.P < 1 << 22
+                             else torch.stack([(row.double() ** 2).sum() for row in t]).float().reshape(self.B, 1).contiguous()
+                             for t in self.bufs]
+        self.call_names = ["clip_accumulate(norms supplied)" if self.supplied else "clip_accumulate(norms computed)", "noise_average"]
 
     def describe(self):
         return {"workload": f"flat: ResNet-50 (GroupNorm) flattened per-example gradients, P={self.P:,} fp32 ~N(0,1e-6), "
-                            "B=64 per chunk x 16 chunks = |B| 1024, global clip C=1.0, sigma=1.0; norms computed by the library"
+                            "B=64 per chunk x 16 chunks = |B| 1024, global clip C=1.0, sigma=1.0; "
+                            + ("squared norms supplied with the gradients" if self.supplied else "norms computed by the library")
                             + ("" if self.variant == "plain" else f"; variant {self.variant}"),
                 "examples_per_step": self.examples_per_step, "params": self.P,
                 "l2": "each chunk is 6.54 GB, far larger than L2; two resident chunks alternate"}
@@ -288,7 +297,7 @@ class FlatGrad:
         st.begin(total_batch=self.B * self.G * self.world, seed=0, step=i)
         for c in range(self.G):
             if rec: rec.start(0)
-            st.chunk(self.bufs[c & 1])
+            st.chunk(self.bufs[c & 1], self.supplied[c & 1] if self.supplied else None)
             if rec: rec.stop(0)
         allreduce_accumulator(st.acc, self.dist)
         if rec: rec.start(1)
@@ -296,8 +305,8 @@ class FlatGrad:
         if rec: rec.stop(1)
 
     def algorithmic_bytes(self, call):
-        if call == 0:
-            return 2 * self.B * self.P * 4 + 2 * self.P * 4   # norm pass + clip pass over the chunk, accumulator r+w
+        if call == 0:                                         # norm pass (unless supplied) + clip pass, accumulator r+w
+            return (1 if self.supplied else 2) * self.B * self.P * 4 + 2 * self.P * 4
         return 2 * self.P * 4
 
     def roofline(self, dom, avg_ms_per_chunk, peaks):
@@ -323,7 +332,7 @@ class FlatGrad:
         st.begin(total_batch=self.B * self.G * self.world, seed=0, step=i)
         for c in range(self.G):
             self.bufs[c & 1].copy_(self.host_chunk, non_blocking=True)
-            st.chunk(self.bufs[c & 1])
+            st.chunk(self.bufs[c & 1], self.supplied[c & 1] if self.supplied else None)
         allreduce_accumulator(st.acc, self.dist)
         self.host_out.copy_(st.finish(seed=0, step=i, world=self.world), non_blocking=True)
 
@@ -584,7 +593,7 @@ def run_ours(args):
 
     # ---- end to end: pinned host inputs -> device, the step, result -> host, every step
     h2d, d2h = wl.e2e_prepare()
-    e2e_steps = max(3, min(steps, args.e2e_steps))
+    e2e_steps = max(3, min(steps, args.e2e_steps, getattr(wl, "e2e_cap", steps)))
     for i in range(2):
         wl.e2e_run(i)
     barrier()
@@ -750,7 +759,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--precision", default="tf32", choices=["tf32", "f32"],
                     help="small_cnn: how tensor-core layers take the fp32 inputs (one tf32 pass | three split-tf32 passes)")
-    ap.add_argument("--variant", default="plain", help="flat workload: plain | per_example_noise | micro2 | micro4 ...")
+    ap.add_argument("--variant", default="plain", help="flat workload: plain | norms_supplied | per_example_noise | micro2 | micro4 ...")
     args = ap.parse_args()
     global VARIANT, PRECISION
     VARIANT = args.variant
@@ -758,7 +767,7 @@ def main():
     if args.workload.startswith("sweep"):
         return run_sweep(args)
     # the small-CNN step lasts ~0.16 ms: 6000 steps give the clock sampler (200 ms period) several readings under load
-    defaults = {"small_cnn": (6000, 10), "flat": (8, 3), "per_layer": (4, 3), "per_layer_r101": (3, 3)}
+    defaults = {"small_cnn": (6000, 10), "flat": (40, 3), "per_layer": (4, 3), "per_layer_r101": (3, 3)}
     if args.steps is None:
         args.steps = defaults[args.workload][0]
     if args.warmup is None:
