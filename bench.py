@@ -3,11 +3,15 @@
 gradients + clip + noise) on synthetic inputs, with the roofline fraction of the dominant kernel
 and the float64 CPU oracle timed beside it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload small_cnn|flat|sweep|per_layer]
-    python bench.py --impl reference ...        # times the CPU oracle on a bounded sample
+    python bench.py [--gpus N] [--steps K] [--warmup W]     # headline: per-layer ResNet-50; other workloads as "legs"
+    python bench.py --workload small_cnn|flat|per_layer|per_layer_r101|sweep|sweep_all ...   # one workload only
+    python bench.py --impl reference ...                    # times the CPU oracle on a bounded sample
 
-One "step" is one pass of the whole path over one batch: for `small_cnn` 256 examples through
-four weight-gradient calls, one clip-accumulate and one noise-average.  Rank 0 prints one JSON line.
+One "step" is one pass of the whole path over one batch: for the headline workload 1024 examples (32 chunks of 32)
+through 107 fused weight-gradient + clip calls per chunk and one noise-average.  Rank 0 prints one JSON line; with
+no --workload it carries the per-layer ResNet-50 workload in `value` / `config` / `roofline` and, on one GPU, the
+flat-gradient (norms computed and norms supplied), small-CNN and layer-sweep workloads under `legs`.  Every timed
+region lasts at least a second: the K steps are repeated `repeats` times when K of them are shorter than that.
 """
 from __future__ import annotations
 
@@ -37,8 +41,8 @@ def measured_peaks():
         with open(path) as f:
             d = json.load(f)
         return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]), bf16_sustained=float(d["bf16_tflops_sustained"]),
-                    source="measured")
-    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+                    sm_max_mhz=float(d.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
 
 
 def source_fingerprint():
@@ -122,7 +126,7 @@ class SmallCnn:
         self.torch, self.synth, self.dist, self.world = torch, synth, dist, world
         self.cfg = synth.small_cnn()
         self.layers, self.B = self.cfg["layers"], self.cfg["B"]
-        self.lanes = int(os.environ.get("DP_BENCH_LANES", "4")) if world == 1 else 1
+        self.lanes = int(os.environ.get("DP_BENCH_LANES", "4"))
         # layers whose per-example gradients outweigh their inputs (conv3, the classifier) are not materialised
         self.recompute = os.environ.get("DP_BENCH_RECOMPUTE", "auto")
         # fp32 inputs; tensor-core layers take them as tf32 (one pass, the precision class the accuracy bounds name)
@@ -171,27 +175,33 @@ class SmallCnn:
                 st.chunks_done += 1
             else:
                 rec.start(k); st.clip_accumulate(); rec.stop(k)
-        allreduce_accumulator(st.acc, self.dist)          # N > 1: the one exchange of the step
-        if rec: rec.start(k + 1)
-        st.finish(seed=0, step=i, world=self.world)
-        if rec: rec.stop(k + 1)
+        self._finish(i, rec, k + 1)
+
+    def _finish(self, i, rec=None, slot=None):
+        allreduce_accumulator(self.step_obj.acc, self.dist)   # N > 1: the one exchange of the step
+        if rec: rec.start(slot)
+        self.step_obj.finish(seed=0, step=i, total_batch=self.B * self.world)
+        if rec: rec.stop(slot)
 
     def parts_of(self, call):
         return 2 if call in self.step_obj.recompute else 1
 
     def capture(self):
-        """One CUDA graph per input set, each holding a whole step (the noise step index is baked in: it does
-        not change the work)."""
-        t = self.torch
+        """One CUDA graph per input set holding the step up to the clipped sum.  The exchange between ranks and the
+        noise call stay outside: a captured noise call would freeze its step index and repeat the same draw."""
+        t, st = self.torch, self.step_obj
         self.graphs = []
         for k in range(self.n_sets):
             g = t.cuda.CUDAGraph()
             with t.cuda.graph(g):
-                self.run(k)
+                st.begin()
+                st.wgrad_all(self.sets[k])
+                st.clip_accumulate(inputs=self.sets[k])
             self.graphs.append(g)
 
     def run_graphed(self, i):
         self.graphs[i % self.n_sets].replay()
+        self._finish(i)
 
     def algorithmic_bytes(self, call):
         """Bytes each call must move per step.  A materialised layer reads its inputs and writes its per-example
@@ -226,7 +236,7 @@ class SmallCnn:
         st.wgrad_all(self.stage)
         st.clip_accumulate(inputs=self.stage)
         allreduce_accumulator(st.acc, self.dist)
-        out = st.finish(seed=0, step=i, world=self.world)
+        out = st.finish(seed=0, step=i, total_batch=self.B * self.world)
         self.host_out.copy_(out, non_blocking=True)
 
     def cpu_sample(self, budget_s):
@@ -301,7 +311,7 @@ class FlatGrad:
             if rec: rec.stop(0)
         allreduce_accumulator(st.acc, self.dist)
         if rec: rec.start(1)
-        st.finish(seed=0, step=i, world=self.world)
+        st.finish(seed=0, step=i, total_batch=self.B * self.G * self.world)
         if rec: rec.stop(1)
 
     def algorithmic_bytes(self, call):
@@ -309,15 +319,19 @@ class FlatGrad:
             return (1 if self.supplied else 2) * self.B * self.P * 4 + 2 * self.P * 4
         return 2 * self.P * 4
 
-    def roofline(self, dom, avg_ms_per_chunk, peaks):
+    def roofline(self, dom, totals, prof_steps, peaks):
         """Per-example noise draws B*P normals per chunk and is bound by integer and transcendental arithmetic: about
         45 instructions per normal (a quarter of a ten-round Philox block, half a Box-Muller pair, the scaled add), so
         the ceiling is SMs x 128 lanes x SM clock / 45 normals per second."""
         if self.variant != "per_example_noise" or dom != 0:
             return None
-        peak = 148 * 128 * 1.965e9 / 45.0 / 1e9
+        avg_ms_per_chunk = totals[0] / (prof_steps * self.G)
+        props = self.torch.cuda.get_device_properties(self.torch.cuda.current_device())
+        sms, ghz = props.multi_processor_count, peaks.get("sm_max_mhz", 1965.0) / 1e3
+        peak = sms * 128 * ghz * 1e9 / 45.0 / 1e9
         got = self.B * self.P / (avg_ms_per_chunk / 1e3) / 1e9
-        return {"bound": "alu", "achieved": round(got, 1), "peak": round(peak, 1), "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz / 45 instructions per normal",
+        return {"bound": "alu", "achieved": round(got, 1), "peak": round(peak, 1),
+                "peak_source": f"derived: {sms} SMs x 128 lanes x {ghz:.3f} GHz / 45 instructions per normal (an estimate of the instruction count)",
                 "unit": "Gnormal/s", "frac": round(got / peak, 4)}
 
     def e2e_prepare(self):
@@ -334,7 +348,7 @@ class FlatGrad:
             self.bufs[c & 1].copy_(self.host_chunk, non_blocking=True)
             st.chunk(self.bufs[c & 1], self.supplied[c & 1] if self.supplied else None)
         allreduce_accumulator(st.acc, self.dist)
-        self.host_out.copy_(st.finish(seed=0, step=i, world=self.world), non_blocking=True)
+        self.host_out.copy_(st.finish(seed=0, step=i, total_batch=self.B * self.G * self.world), non_blocking=True)
 
     def cpu_sample(self, budget_s):
         import numpy as np
@@ -360,7 +374,7 @@ class PerLayer:
         self.torch, self.synth, self.dist, self.world, self.b = torch, synth, dist, world, binding
         self.cfg = self.config(synth)
         self.layers, self.B, self.G = self.cfg["layers"], self.cfg["B"], self.cfg["G"]
-        self.lanes = int(os.environ.get("DP_BENCH_LANES", "4")) if world == 1 else 1
+        self.lanes = int(os.environ.get("DP_BENCH_LANES", "4"))
         self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"], lanes=self.lanes)
         self.examples_per_step = self.B * self.G
         g = torch.Generator(device="cuda"); g.manual_seed(4000 + rank)
@@ -386,12 +400,15 @@ class PerLayer:
     def config(synth):
         return synth.resnet50_per_layer()
 
+    @classmethod
+    def workload_text(cls, layers, L):
+        n_conv = sum(l.kind == "conv" for l in layers)
+        return (f"{cls.name}: {cls.model} (GroupNorm 32) at 224x224, all {L} parameter tensors ({n_conv} conv, "
+                f"{n_conv}x2 norm, fc weight + bias), bf16 X/dY ~N(0,1), B=32 per chunk x 32 chunks = |B| 1024, "
+                f"C=1.0 (C_l = C/sqrt({L})), sigma=1.0; clip + accumulate fused into dp_per_example_wgrad")
+
     def describe(self):
-        n_conv = sum(l.kind == "conv" for l in self.layers)
-        L = self.step_obj.L
-        return {"workload": f"{self.name}: {self.model} (GroupNorm 32) at 224x224, all {L} parameter tensors ({n_conv} conv, "
-                            f"{n_conv}x2 norm, fc weight + bias), bf16 X/dY ~N(0,1), B=32 per chunk x 32 chunks = |B| 1024, "
-                            f"C=1.0 (C_l = C/sqrt({L})), sigma=1.0; clip + accumulate fused into dp_per_example_wgrad",
+        return {"workload": self.workload_text(self.layers, self.step_obj.L),
                 "examples_per_step": self.examples_per_step, "params": self.step_obj.P,
                 "l2": f"one chunk of inputs is {self.in_bytes / 1e9:.2f} GB, far larger than L2",
                 "streams": self.lanes}
@@ -411,8 +428,9 @@ class PerLayer:
                     st.wgrad(li, X, dY)
                     rec.stop(k)
             st.chunks_done += 1
+        allreduce_accumulator(st.acc, self.dist)
         if rec: rec.start(4)
-        st.finish(seed=0, step=i)
+        st.finish(seed=0, step=i, total_batch=self.B * self.G * self.world)
         if rec: rec.stop(4)
 
     def capture(self):
@@ -428,25 +446,40 @@ class PerLayer:
         for c in range(self.G):
             self.chunk_graph.replay()
             st.chunks_done += 1
-        st.finish(seed=0, step=i)
+        allreduce_accumulator(st.acc, self.dist)
+        st.finish(seed=0, step=i, total_batch=self.B * self.G * self.world)
 
     def algorithmic_bytes(self, call):
         return self.bytes_kind[call] if call < 4 else 2 * self.step_obj.P * 4
 
-    def roofline(self, dom, avg_ms_total_per_chunk, peaks):
-        """Tensor-core convs are reported against the bf16 tensor peak (flops counted once although the two-pass
-        scheme executes them twice); everything else against HBM."""
+    def roofline(self, dom, totals, prof_steps, peaks):
+        """Tensor-core convs are reported against the sustained bf16 tensor peak (they are timed inside a long step;
+        flops counted once even where a two-pass scheme executes them twice); the normalisation layers against HBM;
+        and the whole chunk against the sum over layers of max(HBM time, tensor time) at the measured peaks."""
+        per_chunk = [t / (prof_steps * self.G) for t in totals]          # ms per chunk of each call class, one stream
+        gn_gbs = self.bytes_kind[2] / (per_chunk[2] / 1e3) / 1e9 if per_chunk[2] > 0 else 0.0
+        ceiling_ms = 0.0
+        for l, (x, y), k in zip(self.layers, self.inputs, self.kind_of):
+            t_hbm = (x.numel() + y.numel()) * 2 / (peaks["hbm"] * 1e9) * 1e3
+            t_tc = (l.flops() * self.B / (peaks["bf16_sustained"] * 1e12) * 1e3) if k == 0 else 0.0
+            ceiling_ms += max(t_hbm, t_tc)
+        extra = {"norm_affine": {"bound": "hbm", "achieved": round(gn_gbs, 1), "peak": peaks["hbm"], "unit": "GB/s",
+                                 "frac": round(gn_gbs / peaks["hbm"], 4), "algorithmic_bytes": self.bytes_kind[2],
+                                 "avg_ms_per_chunk": round(per_chunk[2], 5)},
+                 "chunk_ceiling": {"ms_at_measured_peaks": round(ceiling_ms, 4), "ms_one_stream": round(sum(per_chunk[:4]), 4),
+                                   "frac": round(ceiling_ms / max(sum(per_chunk[:4]), 1e-9), 4)}}
         if dom != 0:
-            return None
-        tf = self.flops_tc / (avg_ms_total_per_chunk / 1e3) / 1e12
-        return {"bound": "tensor", "achieved": round(tf, 1), "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
-                "frac": round(tf / peaks["bf16_sustained"], 4)}
+            return extra
+        tf = self.flops_tc / (per_chunk[0] / 1e3) / 1e12
+        return dict(extra, bound="tensor", achieved=round(tf, 1), peak=peaks["bf16_sustained"], unit="TFLOP/s",
+                    frac=round(tf / peaks["bf16_sustained"], 4), algorithmic_flops=self.flops_tc,
+                    avg_ms_per_launch=round(per_chunk[0] / max(1, sum(1 for k in self.kind_of if k == 0)), 5))
 
     def e2e_prepare(self):
         t = self.torch
         self.host_inputs = [(x.cpu().pin_memory(), y.cpu().pin_memory()) for x, y in self.inputs]
-        self.host_sum = t.empty(1, dtype=t.float32).pin_memory()
-        return self.in_bytes * self.G, 4 * self.step_obj.P
+        self.host_out = t.empty(self.step_obj.acc.numel(), dtype=t.float32).pin_memory()
+        return self.in_bytes * self.G, 4 * self.step_obj.acc.numel()
 
     def e2e_run(self, i):
         st = self.step_obj
@@ -456,9 +489,9 @@ class PerLayer:
                 X.copy_(hx, non_blocking=True); dY.copy_(hy, non_blocking=True)
                 st.wgrad(li, X, dY)
             st.chunks_done += 1
-        acc_w, acc_b = st.finish(seed=0, step=i)
-        for a in acc_w:
-            a.cpu()
+        allreduce_accumulator(st.acc, self.dist)
+        st.finish(seed=0, step=i, total_batch=self.B * self.G * self.world)
+        self.host_out.copy_(st.acc, non_blocking=True)      # the whole noised, averaged gradient (all 161 tensors)
 
     def cpu_sample(self, budget_s):
         import oracle
@@ -522,98 +555,125 @@ class CallTimer:
         return [len(p) for p in self.pairs]
 
 
-def run_ours(args):
-    import torch
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    import __graft_entry__
-    if rank == 0:
-        __graft_entry__.build()
-    if dist:
-        dist.barrier()
-    from paper_2109_12191_b200 import binding as b
+MIN_TIMED_MS = float(os.environ.get("DP_BENCH_MIN_MS", "1000"))   # every timed region lasts at least this long (profiler captures shorten it)
 
-    wl = WORKLOADS[args.workload](torch, rank, dist, world)
-    steps, warmup = args.steps, max(args.warmup, 3)
 
-    def barrier():
-        if dist:
-            dist.barrier()
-        torch.cuda.synchronize()
+class Env:
+    """What every measurement needs: torch, the binding, the process group (or None) and this rank's place in it."""
 
-    # ---- device-resident timing
+    def __init__(self):
+        import torch
+        self.torch = torch
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+        torch.cuda.set_device(self.local)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+            self.dist = dist
+        import __graft_entry__
+        if self.rank == 0:
+            __graft_entry__.build()
+        self.barrier()
+        from paper_2109_12191_b200 import binding
+        self.b = binding
+
+    def barrier(self):
+        if self.dist:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def max_over_ranks(self, v):
+        if not self.dist:
+            return v
+        t = self.torch.tensor([v], device="cuda", dtype=self.torch.float64)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return t.item()
+
+    def close(self):
+        if self.dist:
+            self.dist.destroy_process_group()
+
+
+def measure(env, wl, steps, warmup, args, want_e2e=True, want_cpu=True):
+    """Times one workload.  Returns the result dict on rank 0 (None elsewhere)."""
+    torch, b = env.torch, env.b
+    warmup = max(warmup, 3)
     for i in range(warmup):
         wl.run(i)
-    barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    # The step's launch sequence is static, so on one GPU it is captured into CUDA graphs and replayed; per-call
-    # event timing (for the roofline) cannot be taken inside a replay and uses a separate un-captured pass below.
-    graphed = args.graph != "off" and world == 1 and hasattr(wl, "capture")
-    launches_per_step = None
+    env.barrier()
+    # The step's launch sequence is static, so it is captured into CUDA graphs and replayed (all ranks alike; the
+    # exchange between ranks and the noise call stay outside the graphs); per-call event timing (for the roofline)
+    # cannot be taken inside a replay and uses a separate un-captured pass below.
+    graphed = args.graph != "off" and hasattr(wl, "capture")
+    c0 = b.dp_debug_launch_count()
+    wl.run(0)
+    launches_per_step = b.dp_debug_launch_count() - c0
+    torch.cuda.synchronize()
     if graphed:
-        c0 = b.dp_debug_launch_count()
-        wl.run(0)
-        launches_per_step = b.dp_debug_launch_count() - c0
-        torch.cuda.synchronize()
         wl.capture()
-        for i in range(3):
-            wl.run_graphed(i)
-        barrier()
-    rec = CallTimer(torch, len(wl.call_names))
-    launches0 = b.dp_debug_launch_count()
+    go = wl.run_graphed if graphed else wl.run
+    for i in range(3):
+        go(i)
+    env.barrier()
+    # how often the K steps must be repeated for the timed region to last a second
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    probe = max(1, min(steps, 3))
+    p0.record()
+    for i in range(probe):
+        go(i)
+    p1.record()
+    env.barrier()
+    est_ms = env.max_over_ranks(p0.elapsed_time(p1) / probe)
+    repeats = max(1, int(math.ceil(MIN_TIMED_MS * 1.1 / max(est_ms * steps, 1e-3))))
+    sampler = ClockSampler(env.local)
+    if env.rank == 0:
+        sampler.start()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    env.barrier()
     t_start.record()
-    for i in range(steps):
-        if graphed:
-            wl.run_graphed(warmup + i)
-        else:
-            wl.run(warmup + i, rec)
+    for i in range(steps * repeats):
+        go(warmup + i)
     t_end.record()
-    barrier()
-    launches = (launches_per_step * steps) if graphed else (b.dp_debug_launch_count() - launches0)
-    clocks = sampler.stop() if rank == 0 else None
-    ms = t_start.elapsed_time(t_end)
-    if graphed:
-        for i in range(min(steps, args.profile_steps)):
-            wl.run(warmup + i, rec)
-        barrier()
-    if dist:
-        t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = t.item()
-    value = wl.examples_per_step * steps * world / (ms / 1e3)
+    env.barrier()
+    clocks = sampler.stop() if env.rank == 0 else None
+    ms = env.max_over_ranks(t_start.elapsed_time(t_end))
+    if hasattr(wl.step_obj, "check"):
+        wl.step_obj.check()                                  # a bounded wait that gave up would invalidate the timing
+    value = wl.examples_per_step * steps * repeats * env.world / (ms / 1e3)
 
-    # ---- end to end: pinned host inputs -> device, the step, result -> host, every step
-    h2d, d2h = wl.e2e_prepare()
-    e2e_steps = max(3, min(steps, args.e2e_steps, getattr(wl, "e2e_cap", steps)))
-    for i in range(2):
-        wl.e2e_run(i)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(e2e_steps):
-        wl.e2e_run(i)
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist:
-        t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = t.item()
-    e2e_value = wl.examples_per_step * e2e_steps * world / (e2e_ms / 1e3)
+    # per-call timing: every call in order on one stream, event pairs around each
+    rec = CallTimer(torch, len(wl.call_names))
+    est_run_ms = est_ms * (1.6 if graphed else 1.0)
+    prof_steps = max(1, min(steps, args.profile_steps, int(math.ceil(300.0 / max(est_run_ms, 1e-3)))))
+    for i in range(prof_steps):
+        wl.run(warmup + i, rec)
+    env.barrier()
 
-    if rank != 0:
-        if dist:
-            dist.destroy_process_group()
-        return
+    e2e = None
+    if want_e2e:
+        # end to end: pinned host inputs -> device, the step, result -> host, every step
+        h2d, d2h = wl.e2e_prepare()
+        e2e_steps = max(2, min(steps, args.e2e_steps, getattr(wl, "e2e_cap", steps)))
+        wl.e2e_run(0)
+        env.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e2e_steps):
+            wl.e2e_run(i)
+        e1.record()
+        env.barrier()
+        e2e_ms = env.max_over_ranks(e0.elapsed_time(e1))
+        e2e = {"value": round(wl.examples_per_step * e2e_steps * env.world / (e2e_ms / 1e3), 1), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+    if env.rank != 0:
+        return None
 
-    # ---- roofline of the dominant call (largest share of device time)
+    # roofline of the dominant call (largest share of device time in the per-call pass)
     peaks = measured_peaks()
     totals, counts = rec.totals_ms(), rec.counts()
     dom = max(range(len(totals)), key=lambda k: totals[k])
@@ -626,25 +686,77 @@ def run_ours(args):
                 "traffic": recorded_traffic(wl.name, wl.call_names[dom]),
                 "shares": {n: round(t / sum(totals), 4) for n, t in zip(wl.call_names, totals)}}
     if hasattr(wl, "roofline"):
-        own = wl.roofline(dom, totals[dom] / (max(1, counts[-1]) * wl.G), peaks)
+        own = wl.roofline(dom, totals, prof_steps, peaks)
         if own:
             roofline.update(own)
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if want_cpu and not args.no_cpu_baseline:
         import oracle
         v, sample = wl.cpu_sample(10.0)
         cpu = {"value": round(v, 3), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample}
 
-    line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": round(ms / steps, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": getattr(wl, "dtype_name", "f32"), "data": "synthetic", "config": dict(wl.describe(), parallelism=("single GPU" if world == 1 else f"batch sharded over {world} GPUs, one all-reduce of the accumulator per step")),
-            "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps},
-            "gpu_launches": int(launches), "launch_mode": ("CUDA graph replay" if graphed else "stream launches"), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
-    print(json.dumps(line))
-    if dist:
-        dist.destroy_process_group()
+    return {"value": round(value, 1), "unit": UNIT, "steps": steps, "repeats": repeats, "warmup": warmup,
+            "ms_per_step": round(ms / (steps * repeats), 5), "timed_ms": round(ms, 2),
+            "dtype": getattr(wl, "dtype_name", "f32"),
+            "config": dict(wl.describe(), parallelism=("single GPU" if env.world == 1 else
+                                                       f"batch sharded over {env.world} GPUs, one all-reduce of the accumulator per step")),
+            "e2e": e2e, "gpu_launches": int(launches_per_step * steps * repeats),
+            "launch_mode": ("CUDA graph replay" if graphed else "stream launches"), "clocks": clocks,
+            "roofline": roofline, "cpu_baseline": cpu}
+
+
+def release(env, wl):
+    del wl
+    import gc
+    gc.collect()
+    env.torch.cuda.empty_cache()
+
+
+def line_of(env, res):
+    """The contract's JSON line from a measure() result."""
+    line = {"metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": env.world, "steps": res["steps"],
+            "warmup": res["warmup"], "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": res["dtype"], "data": "synthetic"}
+    for k in ("config", "e2e", "gpu_launches", "launch_mode", "repeats", "timed_ms", "clocks", "roofline", "cpu_baseline"):
+        line[k] = res[k]
+    return line
+
+
+def run_ours(args):
+    global VARIANT
+    env = Env()
+    names = [args.workload] if args.workload != "all" else ["per_layer"]
+    head = None
+    for name in names:
+        VARIANT = args.variant
+        wl = WORKLOADS[name](env.torch, env.rank, env.dist, env.world)
+        steps = args.steps if args.steps is not None else DEFAULT_STEPS[name][0]
+        warmup = args.warmup if args.warmup is not None else DEFAULT_STEPS[name][1]
+        if args.chunks and hasattr(wl, "G"):
+            wl.G = args.chunks
+            wl.examples_per_step = wl.B * wl.G
+        head = measure(env, wl, steps, warmup, args, want_e2e=not args.no_e2e)
+        release(env, wl)
+    legs = {}
+    if args.workload == "all" and env.world == 1 and args.legs != "off":
+        # the other workloads, device-resident timing only; each with its own clock samples and roofline
+        for key, name, variant in (("flat", "flat", "plain"), ("flat_norms_supplied", "flat", "norms_supplied"),
+                                   ("small_cnn", "small_cnn", "plain")):
+            VARIANT = variant
+            wl = WORKLOADS[name](env.torch, env.rank, env.dist, env.world)
+            st, wu = DEFAULT_STEPS[name]
+            res = measure(env, wl, st, wu, args, want_e2e=False, want_cpu=False)
+            release(env, wl)
+            legs[key] = {k: res[k] for k in ("value", "unit", "ms_per_step", "steps", "repeats", "timed_ms", "dtype",
+                                             "config", "gpu_launches", "launch_mode", "clocks", "roofline")}
+        legs["sweep"] = sweep(env, "sweep", "", reps=150)
+    if env.rank == 0:
+        line = line_of(env, head)
+        if legs:
+            line["legs"] = legs
+        print(json.dumps(line))
+    env.close()
 
 
 def run_reference(args):
@@ -656,19 +768,22 @@ def run_reference(args):
     import oracle
     oracle.build()
 
-    class _NoTorch:
-        pass
-    cls = WORKLOADS[args.workload]
+    name = "per_layer" if args.workload == "all" else args.workload
+    cls = WORKLOADS[name]
     wl = cls.__new__(cls)
     from paper_2109_12191_b200 import synth
     wl.synth = synth
-    if args.workload == "small_cnn":
+    if name == "small_cnn":
         wl.cfg = synth.small_cnn(); wl.layers = wl.cfg["layers"]; wl.B = wl.cfg["B"]
         config = {"workload": "small_cnn (CPU oracle, whole batches)", "examples_per_step": 256}
-    else:
+    elif name == "flat":
         wl.cfg = synth.resnet50_flat(); wl.P, wl.B, wl.G = wl.cfg["P"], wl.cfg["B"], wl.cfg["G"]
         config = {"workload": "flat (CPU oracle on a sample)", "examples_per_step": 8}
-    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
+    else:
+        wl.cfg = cls.config(synth); wl.layers = wl.cfg["layers"]
+        config = {"workload": cls.workload_text(wl.layers, wl.cfg["L"]), "examples_per_step": 1024,
+                  "sampled": "the CPU oracle runs a sample of layers on two examples, scaled to one example by the flop ratio"}
+    steps, warmup = max(1, min(args.steps or 3, 5)), min(args.warmup or 1, 1)
     for _ in range(warmup):
         wl.cpu_sample(1.0)
     vals, sample = [], ""
@@ -686,40 +801,48 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def run_sweep(args):
-    """The layer sweep (or any layer list): time dp_per_example_wgrad per layer with both epilogues.
-    L2 is flushed (a 512 MB buffer is overwritten) before every timed launch."""
-    import torch
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    import __graft_entry__
-    __graft_entry__.build()
-    from paper_2109_12191_b200 import binding as b, synth
+def sweep(env, which, layer_sel, reps):
+    """The layer sweep (or any layer list): dp_per_example_wgrad per layer with the three epilogues, one call per timing.
+    L2 is flushed (a 512 MB buffer is overwritten) before every timed call."""
+    torch, b = env.torch, env.b
+    from paper_2109_12191_b200 import synth
     from paper_2109_12191_b200.step import layer_desc
     peaks = measured_peaks()
     layers = synth.resnet50_sweep()["layers"]
-    if args.workload == "sweep_all":
-        layers = [l for l in synth.resnet50_gn_layers() if l.kind != "norm"]
-    if args.workload == "sweep_all_r101":
-        layers = [l for l in synth.resnet101_gn_layers() if l.kind != "norm"]
-    if args.layers:
-        layers = [layers[int(i)] for i in args.layers.split(",")]
+    if which == "sweep_all":
+        layers = synth.resnet50_gn_layers()
+    if which == "sweep_all_r101":
+        layers = synth.resnet101_gn_layers()
+    if layer_sel:
+        layers = [layers[int(i)] for i in layer_sel.split(",")]
     Bn, dtype = 32, "bf16"
     flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")
-    rows, reps = [], max(3, args.steps or 10)
+    rows = []
     g = torch.Generator(device="cuda"); g.manual_seed(5)
+    sampler = ClockSampler(env.local)
+    sampler.start()
+    t_wall = time.perf_counter()
     for l in layers:
         X = torch.randn(l.x_shape(Bn), device="cuda", generator=g).to(torch.bfloat16)
         dY = torch.randn(l.dy_shape(Bn), device="cuda", generator=g).to(torch.bfloat16)
         G_w = torch.empty((Bn, l.n_weight), device="cuda")
+        G_b = torch.empty((Bn, l.n_bias), device="cuda") if l.n_bias else None
+        acc_w = torch.zeros(l.n_weight, device="cuda")
+        acc_b = torch.zeros(l.n_bias, device="cuda") if l.n_bias else None
         sq = torch.empty((Bn, 1), device="cuda")
-        row = {"layer": l.name, "M": l.Kout, "N": l.R * l.S * l.Cin, "K": l.OH * l.OW}
+        row = {"layer": l.name, "kind": l.kind, "M": l.Kout, "N": l.R * l.S * l.Cin, "K": l.OH * l.OW}
         in_bytes = (X.numel() + dY.numel()) * 2
         flops = l.flops() * Bn
-        for epi, tag, out_bytes in ((b.DP_EPI_STORE_NORM, "store", G_w.numel() * 4), (b.DP_EPI_NORM_ONLY, "norm", 0)):
+        for epi, tag, out_bytes in ((b.DP_EPI_STORE_NORM, "store", G_w.numel() * 4), (b.DP_EPI_NORM_ONLY, "norm", 0),
+                                    (b.DP_EPI_CLIP_ACCUM, "clip", 2 * acc_w.numel() * 4)):
             d = layer_desc(l, Bn, dtype, b.DP_IMPL_AUTO, 0)
             ws = torch.empty(max(b.dp_workspace_bytes(d, epi), 256), dtype=torch.uint8, device="cuda")
-            call = lambda: b.check(b.dp_per_example_wgrad(d, X, dY, G_w, None, sq, 1, epi, 0.0, None, None, None, ws))
-            for _ in range(3):
+            b.check(b.dp_workspace_init(ws))
+            c0 = b.dp_debug_launch_count()
+            call = lambda: b.check(b.dp_per_example_wgrad(d, X, dY, G_w, G_b, sq, 1, epi, 1.0, acc_w, acc_b, None, ws))
+            call()
+            launches = b.dp_debug_launch_count() - c0
+            for _ in range(2):
                 call()
             times = []
             for _ in range(reps):
@@ -732,17 +855,37 @@ def run_sweep(args):
             ms = statistics.median(times)
             t_hbm = (in_bytes + out_bytes) / (peaks["hbm"] * 1e9) * 1e3
             t_tc = flops / (peaks["bf16"] * 1e12) * 1e3
-            row[tag] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1), "gbs": round((in_bytes + out_bytes) / ms / 1e6, 1),
-                        "bound": "hbm" if t_hbm > t_tc else "tensor", "frac_of_bound": round(max(t_hbm, t_tc) / ms, 3),
+            bound = "hbm" if t_hbm > t_tc else "tensor"
+            row[tag] = {"ms": round(ms, 4), "launches": int(launches), "tflops": round(flops / ms / 1e9, 1),
+                        "gbs": round((in_bytes + out_bytes) / ms / 1e6, 1), "bound": bound,
+                        "peak": peaks["hbm"] if bound == "hbm" else peaks["bf16"], "frac": round(max(t_hbm, t_tc) / ms, 3),
+                        "algorithmic_bytes": in_bytes + out_bytes, "algorithmic_flops": flops,
                         "tc": bool(b.dp_wgrad_uses_tensor_cores(d, epi)), "ex_per_s": round(Bn / ms * 1e3, 1)}
         rows.append(row)
         del X, dY, G_w
-    tot_store = sum(r["store"]["ms"] for r in rows)
-    tot_norm = sum(r["norm"]["ms"] for r in rows)
-    print(json.dumps({"metric": METRIC, "unit": UNIT, "workload": args.workload, "B": Bn, "dtype": "bf16", "peaks": peaks,
-                      "store_total_ms": round(tot_store, 3), "norm_total_ms": round(tot_norm, 3),
-                      "store_ex_per_s": round(Bn / tot_store * 1e3, 1), "norm_ex_per_s": round(Bn / tot_norm * 1e3, 1),
-                      "layers": rows}))
+    clocks = sampler.stop()
+    tot = {t: sum(r[t]["ms"] for r in rows) for t in ("store", "norm", "clip")}
+    top = max(rows, key=lambda r: r["norm"]["ms"])
+    return {"value": round(Bn / tot["norm"] * 1e3, 1), "unit": UNIT, "ms_per_step": round(tot["norm"], 4),
+            "what": "examples/s through the listed layers' weight-gradient calls with the fused norm epilogue, one call per "
+                    "timing, median of `reps`; store_ / clip_ give the same with the gradients stored resp. clipped and summed",
+            "store_ex_per_s": round(Bn / tot["store"] * 1e3, 1), "clip_ex_per_s": round(Bn / tot["clip"] * 1e3, 1),
+            "B": Bn, "dtype": "bf16", "reps": reps, "wall_s": round(time.perf_counter() - t_wall, 2),
+            "l2": "a 512 MB buffer is overwritten before every timed call", "clocks": clocks,
+            "roofline": dict(top["norm"], kernel=f"wgrad:{top['layer']} (norm epilogue; the slowest row)", traffic=None,
+                             peak_source=peaks["source"], unit="GB/s" if top["norm"]["bound"] == "hbm" else "TFLOP/s",
+                             achieved=top["norm"]["gbs"] if top["norm"]["bound"] == "hbm" else top["norm"]["tflops"]),
+            "layers": rows}
+
+
+def run_sweep(args):
+    env = Env()
+    out = sweep(env, args.workload, args.layers, max(3, args.steps or 30))
+    print(json.dumps(dict({"metric": METRIC, "workload": args.workload, "peaks": measured_peaks()}, **out)))
+    env.close()
+
+
+DEFAULT_STEPS = {"small_cnn": (6000, 10), "flat": (40, 3), "per_layer": (20, 3), "per_layer_r101": (10, 3)}
 
 
 def main():
@@ -751,12 +894,16 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="small_cnn", choices=sorted(WORKLOADS) + ["sweep", "sweep_all", "sweep_all_r101"])
-    ap.add_argument("--e2e-steps", type=int, default=20)
-    ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"], help="replay the step from CUDA graphs (single GPU)")
-    ap.add_argument("--profile-steps", type=int, default=20, help="un-captured steps timed per call for the roofline")
+    ap.add_argument("--workload", default="all", choices=["all"] + sorted(WORKLOADS) + ["sweep", "sweep_all", "sweep_all_r101"],
+                    help="all: the per-layer ResNet-50 workload as the headline, the others as legs of the same line")
+    ap.add_argument("--legs", default="on", choices=["on", "off"], help="with --workload all on one GPU: also time the other workloads")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"], help="replay the step from CUDA graphs")
+    ap.add_argument("--profile-steps", type=int, default=20, help="un-captured steps timed per call for the roofline (at most)")
     ap.add_argument("--layers", default="", help="sweep workloads: comma-separated layer indices")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end (host buffers) measurement")
+    ap.add_argument("--chunks", type=int, default=0, help="per_layer workloads: chunks per step (profiler captures only; 0 = the workload's 32)")
     ap.add_argument("--precision", default="tf32", choices=["tf32", "f32"],
                     help="small_cnn: how tensor-core layers take the fp32 inputs (one tf32 pass | three split-tf32 passes)")
     ap.add_argument("--variant", default="plain", help="flat workload: plain | norms_supplied | per_example_noise | micro2 | micro4 ...")
@@ -764,18 +911,11 @@ def main():
     global VARIANT, PRECISION
     VARIANT = args.variant
     PRECISION = args.precision
+    if args.impl == "reference":
+        return run_reference(args)
     if args.workload.startswith("sweep"):
         return run_sweep(args)
-    # the small-CNN step lasts ~0.16 ms: 6000 steps give the clock sampler (200 ms period) several readings under load
-    defaults = {"small_cnn": (6000, 10), "flat": (40, 3), "per_layer": (4, 3), "per_layer_r101": (3, 3)}
-    if args.steps is None:
-        args.steps = defaults[args.workload][0]
-    if args.warmup is None:
-        args.warmup = defaults[args.workload][1]
-    if args.impl == "reference":
-        run_reference(args)
-    else:
-        run_ours(args)
+    run_ours(args)
 
 
 if __name__ == "__main__":

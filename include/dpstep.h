@@ -13,6 +13,8 @@
  *   - Every data pointer is a DEVICE pointer unless its comment says "host".  All device
  *     buffers are allocated, owned and freed by the caller; the library allocates no
  *     device memory and keeps no state between calls (scratch comes in as `workspace`).
+ *     One exception, stated at its declaration: dp_clip_accumulate_static works in a fixed
+ *     device array that is part of the library image.
  *   - Device pointers must be 16-byte aligned; tensors are dense, row-major, channels-last:
  *       conv   X [B,H,W,C_in]   dY [B,OH,OW,K_out]   G_w [B,K_out,R,S,C_in]   G_b [B,K_out]
  *       dense  X [B,C_in]       dY [B,K_out]         G_w [B,K_out,C_in]       G_b [B,K_out]
@@ -93,6 +95,15 @@ DP_API int dp_layer_groups(const dp_layer_desc *desc);
  * for some paths, per-example bias gradients or clip factors. */
 DP_API size_t dp_workspace_bytes(const dp_layer_desc *desc, int epilogue);
 
+/* Prepares a freshly allocated (or otherwise overwritten) workspace of dp_per_example_wgrad /
+ * dp_per_example_wgrad_scaled: clears its header, i.e. the status word dp_wgrad_check reports and the ticket
+ * counters with which the last thread block to finish an example finds out that it is the last.  Call it once
+ * per workspace before the first layer call (it enqueues one small memset on `cuda_stream`); the layer calls
+ * leave the counters cleared again, so one workspace serves any number of calls, of any layers, one after the
+ * other.  Between calls the caller must not write to the workspace.
+ * Errors: DP_ERR_WORKSPACE (null, not 256-byte aligned, or smaller than any dp_workspace_bytes() result). */
+DP_API dp_status dp_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Per-example weight gradients of one layer for a chunk of B examples
  * (section 2: "per-example gradients are computed"; the layer formulas are the standard
  * weight gradients given X and dY):
@@ -113,7 +124,8 @@ DP_API size_t dp_workspace_bytes(const dp_layer_desc *desc, int epilogue);
  *   acc_w/b    [P_w], [P_b] fp32, read-modify-write; DP_EPI_CLIP_ACCUM only:
  *              acc += sum_n min(1, C_l/||g_n||) * g_n  (section 3.5, one group = this layer).
  *   clip_out   optional [B, groups] fp32: the factors that were applied (DP_EPI_CLIP_ACCUM).
- *   workspace  at least dp_workspace_bytes(desc, epilogue) bytes, 256-byte aligned.  Usually a few hundred KB; layers
+ *   workspace  at least dp_workspace_bytes(desc, epilogue) bytes, 256-byte aligned, prepared once by
+ *              dp_workspace_init.  Calls that may overlap on the GPU need a workspace each.  Usually a few hundred KB; layers
  *              with very few input channels (C_in <= 8) that run on tensor cores keep an unfolded copy of X there
  *              (B*OH*OW*pad(R*S*C_in) elements), and the fused clip keeps partial sums when it splits the batch.
  *
@@ -250,8 +262,9 @@ DP_API dp_status dp_clip_accumulate_micro(int B, int L, int micro, const float *
  *
  *   - Limit: problems whose dp_clip_workspace_bytes(B, L, P_l) exceeds the array are refused with
  *     DP_ERR_WORKSPACE (dp_last_cuda_error() says why); nothing is launched.
- *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
- *     device current); make that first call outside any stream capture.  No call allocates or frees memory.
+ *   - Every call looks up the array's device address (cudaGetSymbolAddress, with the caller's device current);
+ *     the first look-up on a device loads the library image there, so make that first call outside any stream
+ *     capture.  No call allocates or frees memory, and no address is kept across calls.
  *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to start at
  *     zero (each call writes what it later reads), but two calls whose kernels overlap on the GPU -- different
  *     streams, or different host threads on the same device -- race on it: keep such calls ordered. */
@@ -301,10 +314,17 @@ DP_API dp_status dp_debug_philox_raw(unsigned int *out4, long long n_blocks, lon
 DP_API dp_status dp_debug_noise_z(float *z, long long count, long long first_index,
                            unsigned long long seed, unsigned long long step, void *cuda_stream);
 
-/* Reads (with a synchronising copy) the device status word some tensor-core launches keep at
- * the start of `workspace`: DP_OK, or DP_ERR_TIMEOUT when a bounded wait inside the kernel
- * expired (the kernel then returned early and its outputs are invalid). */
-DP_API dp_status dp_wgrad_check(const void *workspace, void *cuda_stream);
+/* Reads (with a synchronising copy) the status word at the start of `workspace`: DP_OK, or DP_ERR_TIMEOUT when
+ * a bounded wait inside a tensor-core kernel expired in ANY call that used this workspace since the word was last
+ * cleared (that kernel returned early; its outputs, and everything computed from them, are invalid).  The word is
+ * sticky: kernels only ever set it, later calls do not hide it.  Reporting a time-out clears it and re-initialises
+ * the workspace header, as dp_workspace_init does. */
+DP_API dp_status dp_wgrad_check(void *workspace, void *cuda_stream);
+
+/* Test hook: the number of polls (each about a microsecond) after which the bounded waits of the tensor-core kernel
+ * give up; 0 makes every wait give up before anything is copied or multiplied, a negative value restores the
+ * default (about two seconds).  Process-wide; applies to launches enqueued afterwards. */
+DP_API void dp_debug_set_wait_polls(long long polls);
 
 /* 1 if dp_per_example_wgrad would run this layer on the tcgen05 tensor-core kernel under
  * DP_IMPL_AUTO, else 0 (also 0 for an invalid descriptor). */
@@ -315,11 +335,11 @@ DP_API const char *dp_status_string(int status);
 /* Text of the last CUDA error this thread's calls ran into ("" if none). Host memory owned by the library. */
 DP_API const char *dp_last_cuda_error(void);
 
-/* Test / report hook: the tiling the tensor-core kernel would use for a conv layer, as up to 12 ints
+/* Test / report hook: the tiling the tensor-core kernel would use for a conv layer and epilogue, as up to 12 ints
  * {rows-are-input-columns, row extent, column extent, row tiles, column tiles, columns per tile,
  *  pixel-tile width, pixel-tile height, pixels per stage, pixel tiles, pipeline stages, bytes per stage}.
  * Returns the number of values available (0 when the layer is not eligible). `out` is host memory. */
-DP_API int dp_debug_wgrad_plan(const dp_layer_desc *desc, int *out, int n);
+DP_API int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n);
 
 /* Number of kernels this process has launched through the library so far (a host-side counter;
  * benchmarks report the difference over their timed region). */

@@ -30,7 +30,8 @@ EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_
            "dp_debug_launch_count", "dp_debug_wgrad_plan", "dp_clip_accumulate_static",
            "dp_clip_static_scratch_bytes", "dp_noise_average_sgd", "dp_clip_accumulate_noised",
            "dp_debug_example_noise_z", "dp_clip_accumulate_grouped", "dp_clip_accumulate_micro",
-           "dp_per_example_wgrad_scaled", "dp_clip_factors", "dp_scale_accumulate"]
+           "dp_per_example_wgrad_scaled", "dp_clip_factors", "dp_scale_accumulate", "dp_workspace_init",
+           "dp_debug_set_wait_polls"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -87,10 +88,12 @@ _lib.dp_noise_average_sgd.restype = _i
 _lib.dp_debug_philox_raw.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_philox_raw.restype = _i
 _lib.dp_debug_noise_z.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug_noise_z.restype = _i
 _lib.dp_wgrad_check.argtypes = [_vp, _vp]; _lib.dp_wgrad_check.restype = _i
+_lib.dp_workspace_init.argtypes = [_vp, _sz, _vp]; _lib.dp_workspace_init.restype = _i
+_lib.dp_debug_set_wait_polls.argtypes = [_ll]; _lib.dp_debug_set_wait_polls.restype = None
 _lib.dp_status_string.argtypes = [_i]; _lib.dp_status_string.restype = ctypes.c_char_p
 _lib.dp_last_cuda_error.argtypes = []; _lib.dp_last_cuda_error.restype = ctypes.c_char_p
 _lib.dp_debug_launch_count.argtypes = []; _lib.dp_debug_launch_count.restype = _ull
-_lib.dp_debug_wgrad_plan.argtypes = [_dp, ctypes.POINTER(_i), _i]; _lib.dp_debug_wgrad_plan.restype = _i
+_lib.dp_debug_wgrad_plan.argtypes = [_dp, _i, ctypes.POINTER(_i), _i]; _lib.dp_debug_wgrad_plan.restype = _i
 
 
 def _ptr(t):
@@ -250,6 +253,16 @@ def dp_debug_noise_z(z, count, first_index, seed, step, stream=None):
     return _lib.dp_debug_noise_z(_ptr(z), count, first_index, seed, step, _stream(stream))
 
 
+def dp_workspace_init(workspace, workspace_bytes=None, stream=None):
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else _nbytes(workspace)
+    return _lib.dp_workspace_init(_ptr(workspace), workspace_bytes, _stream(stream))
+
+
+def dp_debug_set_wait_polls(polls):
+    _lib.dp_debug_set_wait_polls(polls)
+
+
 def dp_wgrad_check(workspace, stream=None):
     return _lib.dp_wgrad_check(_ptr(workspace), _stream(stream))
 
@@ -269,7 +282,7 @@ def dp_debug_launch_count():
 PLAN_FIELDS = ("a_is_x", "a_ext", "b_ext", "m_tiles", "n_tiles", "NT", "OWt", "OHt", "Kt", "k_tiles", "stages", "stage_bytes")
 
 
-def dp_debug_wgrad_plan(desc):
+def dp_debug_wgrad_plan(desc, epilogue=DP_EPI_STORE_NORM):
     out = (_i * 12)()
-    n = _lib.dp_debug_wgrad_plan(ctypes.byref(desc), out, 12)
+    n = _lib.dp_debug_wgrad_plan(ctypes.byref(desc), epilogue, out, 12)
     return dict(zip(PLAN_FIELDS, list(out)[:n])) if n else None

@@ -511,7 +511,7 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
     for (int l = 0; l < L; ++l) wide_blocks += (P_l[l] + kAccCols - 1) / kAccCols;
     // A small model gives few blocks, and each thread would walk all B rows alone: with many rows the block narrows
     // to 128 parameters and its warps share the rows.
-    const bool split = B >= 64 && wide_blocks < 8 * 148;
+    const bool split = B >= 64 && wide_blocks < 8 * sm_count();
     const int acc_cols = (split && !noise) ? kSplitCols : kAccCols;
 
     auto fill = [&](int l0, SegTable &t, bool norm_blocks, long long &part_cursor) {
@@ -552,6 +552,7 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
         sq = sq_ws;
     }
     if (!stage3_only) {
+        DP_MAX_SHARED_CARVEOUT((clip_factor_kernel));
         const long long count = per_layer ? (long long)B * L : B;
         if (var.groups)
             clip_factor_grouped_kernel<<<(unsigned)B, 128, 0, stream>>>(sq, L, *var.groups, C, factor_ws, norms_out, clip_out);
@@ -567,6 +568,8 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
             SegTable t;
             const int blocks = fill(l0, t, false, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
+            DP_MAX_SHARED_CARVEOUT((scale_accumulate_rowsplit_kernel));
+            DP_MAX_SHARED_CARVEOUT((scale_accumulate_kernel<8>));
             if (noise) scale_accumulate_noised_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer, *noise);
             else if (split) scale_accumulate_rowsplit_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             else scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
@@ -592,6 +595,7 @@ extern "C" dp_status dp_clip_factors(int mode, int B, int L, const float *sqnorm
     if (!dp::aligned(sqnorm, 4) || !dp::aligned(factors_out, 4) || (norms_out && !dp::aligned(norms_out, 4))) return DP_ERR_INVALID_ARG;
     const int per_layer = (mode == DP_CLIP_PER_LAYER);
     const long long count = per_layer ? (long long)B * L : B;
+    DP_MAX_SHARED_CARVEOUT((dp::clip_factor_kernel));
     dp::clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         sqnorm, B, L, per_layer, C, factors_out, norms_out, nullptr);
     DP_LAUNCH_CHECK("clip_factor_kernel");
@@ -674,25 +678,15 @@ namespace dp {
 constexpr size_t kStaticScratchBytes = 2u << 20;   // 2 MiB
 static __device__ __align__(256) unsigned char g_clip_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
-static std::mutex g_scratch_mu;
-static void *g_scratch_addr[kMaxDevices] = {nullptr};
-
 // Device address of g_clip_scratch on the current device.  In host code the array's name is only a
-// stand-in for the symbol, never a usable address, so the address is asked for once per device, with
-// that device current, and remembered.
+// stand-in for the symbol, never a usable address, so the address is asked for with the caller's
+// device current.  It is asked for on every call (after the first one on a device this is a table
+// look-up inside the runtime and allocates nothing), so no address outlives a cudaDeviceReset.
 static dp_status static_scratch(void **out) {
-    int dev = -1;
-    DP_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxDevices) return DP_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lock(g_scratch_mu);
-    if (!g_scratch_addr[dev]) {
-        void *ptr = nullptr;
-        DP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_clip_scratch));
-        if (!ptr) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_clip_scratch)");
-        g_scratch_addr[dev] = ptr;
-    }
-    *out = g_scratch_addr[dev];
+    void *ptr = nullptr;
+    DP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_clip_scratch));
+    if (!ptr) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_clip_scratch)");
+    *out = ptr;
     return DP_OK;
 }
 }  // namespace dp

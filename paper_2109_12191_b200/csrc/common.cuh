@@ -13,6 +13,16 @@ dp_status cuda_fail(cudaError_t e, const char *where);
 // Records a plain message for dp_last_cuda_error() (used where the failure is not a CUDA error code).
 void note_error(const char *message);
 
+// Number of SMs of the current device (cached per device; 148 if the query fails).
+int sm_count();
+
+// Every dp_per_example_wgrad workspace starts with this header, cleared by dp_workspace_init: the sticky status word
+// at byte 0 and, from byte 256, the ticket counters with which the last block to finish a unit of work finds out
+// that it is the last (each kernel leaves its counters at zero again).
+constexpr size_t kWsHeaderBytes = 16384;
+constexpr size_t kWsCounterOffset = 256;
+constexpr int kWsCounters = (int)((kWsHeaderBytes - kWsCounterOffset) / sizeof(int));
+
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -24,6 +34,17 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Host-side count of kernel launches made by this process (read by dp_debug_launch_count).
 void count_launch();
+
+// Before a launch: asks once for the largest shared-memory carve-out for this kernel.  The tensor-core kernel needs
+// nearly all of an SM's shared memory; an SM whose L1 / shared-memory split has to change between two kernels must
+// drain first, which serialises kernels that could otherwise follow or overlap each other.  With every kernel of the
+// library on the same split no such change happens.  (A hint: its failure is ignored.)
+#define DP_MAX_SHARED_CARVEOUT(kern)                                                                              \
+    do {                                                                                                          \
+        static const cudaError_t carve__ = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, \
+                                                                (int)cudaSharedmemCarveoutMaxShared);            \
+        (void)carve__;                                                                                            \
+    } while (0)
 
 // After a kernel launch: picks up launch-configuration errors without synchronising.
 #define DP_LAUNCH_CHECK(name)                                          \

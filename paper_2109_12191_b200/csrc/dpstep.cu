@@ -21,6 +21,17 @@ dp_status cuda_fail(cudaError_t e, const char *where) {
 
 void note_error(const char *message) { snprintf(g_last_error, sizeof(g_last_error), "%s", message); }
 
+int sm_count() {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int v = cached[dev].load(std::memory_order_relaxed);
+    if (v > 0) return v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+    cached[dev].store(v, std::memory_order_relaxed);
+    return v;
+}
+
 static bool valid_desc(const dp_layer_desc *d) {
     if (!d) return false;
     if (d->kind != DP_LAYER_DENSE && d->kind != DP_LAYER_CONV2D && d->kind != DP_LAYER_NORM_AFFINE) return false;
@@ -67,7 +78,7 @@ static bool make_plan(const dp_layer_desc *d, int epi, WgradPlan &pl) {
     pl.use_thin = d->kind == DP_LAYER_CONV2D && d->impl == DP_IMPL_AUTO && epi != DP_EPI_CLIP_ACCUM && thin_conv_eligible(g);
     if (d->kind == DP_LAYER_CONV2D && d->impl != DP_IMPL_CUDA_CORE && !pl.use_thin) pl.use_tc = tc_eligible(d->dtype, g, epi);
     size_t off = 0;
-    pl.status_off = off; off += 256;
+    pl.status_off = off; off += kWsHeaderBytes;      // status word, then the ticket counters
     if (d->kind == DP_LAYER_CONV2D) {
         const int tiles = pl.use_thin ? 1 : (pl.use_tc ? tc_norm_slots(d->dtype, g, epi) : fma_tiles_m(g) * fma_tiles_n(g));
         pl.w_slots = tiles;
@@ -147,30 +158,34 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
     const ConvGeom g = geom_of(d);
     const int clip = (epi == DP_EPI_CLIP_ACCUM);
     dp_status rc;
-    // Tensor-core launches may set the status word (bounded waits): the first of them clears it on entry.  Every
-    // other path has no waits and lets its last small kernel write "ok".  Neither pays for a memset node.
-    int *status_word = reinterpret_cast<int *>(ws + pl.status_off);
-    int *reset = pl.use_tc ? nullptr : status_word;
+    // The status word is sticky: dp_workspace_init clears it, a tensor-core launch whose bounded wait expired sets it,
+    // and only dp_wgrad_check clears it again after reporting it.
 
     if (d->kind == DP_LAYER_CONV2D) {
         float *db = (epi == DP_EPI_STORE_NORM) ? G_b : db_ws;
         if (pl.use_thin && rgb3_conv_eligible(g))
             return launch_conv_rgb3(storage_type(d), X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, d->has_bias, groups == 2,
-                                    sqnorm, sqnorm_stride, reset, st);
+                                    sqnorm, sqnorm_stride, st);
         if (pl.use_thin) {
             rc = launch_conv_thin(storage_type(d), X, dY, g, epi == DP_EPI_STORE_NORM ? G_w : nullptr, db, partial, pl.slots, d->has_bias, st);
             if (rc != DP_OK) return rc;
-            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
+            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
         }
         if (d->has_bias) {
             rc = launch_bias(storage_type(d), dY, g, db, partial, pl.slots, pl.w_slots, st);
             if (rc != DP_OK) return rc;
         }
         if (epi != DP_EPI_CLIP_ACCUM) {
+            if (pl.use_tc) {
+                // one launch: the kernel's last CTA folds the partial norms (a ticket in the workspace header)
+                const TcPublish pub = {reinterpret_cast<int *>(ws + kWsCounterOffset), pl.w_slots, groups == 2, sqnorm, sqnorm_stride};
+                return launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off,
+                                      reinterpret_cast<int *>(ws + pl.status_off), st, false, nullptr, &pub);
+            }
             if (pl.use_tc) rc = launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
             else rc = launch_conv_fma(storage_type(d), epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, nullptr, st);
             if (rc != DP_OK) return rc;
-            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
+            return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
         }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
@@ -181,7 +196,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
             return launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, nullptr, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true, &ic);
         }
-        rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st, reset);
+        rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st);
         if (rc != DP_OK) return rc;
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true);
         else rc = launch_conv_fma(storage_type(d), DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, reinterpret_cast<float *>(ws + pl.tc_off), st);
@@ -197,10 +212,10 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         }
         float *db_dst = !d->has_bias ? nullptr : (epi == DP_EPI_STORE_NORM ? G_b : (clip ? db_ws : nullptr));
         rc = launch_dense_norm(storage_type(d), X, dY, d->B, d->C_in, d->K_out, d->has_bias, db_dst, groups == 2, sqnorm,
-                               sqnorm_stride, clip, C_l, factor, clip_out, reset, st);
+                               sqnorm_stride, clip, C_l, factor, clip_out, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
-        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, 2, d->B, d->C_in, d->K_out, acc_w, nullptr, st);
+        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, 2, d->B, d->C_in, d->K_out, acc_w, st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
         return DP_OK;
@@ -211,12 +226,16 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         float *chunk_partial = reinterpret_cast<float *>(ws + pl.chunk_off);
         float *dg = (epi == DP_EPI_STORE_NORM) ? G_w : reinterpret_cast<float *>(ws + pl.dg_off);
         float *dbt = (epi == DP_EPI_STORE_NORM) ? G_b : reinterpret_cast<float *>(ws + pl.dg_off) + (size_t)d->B * d->C_in;
+        if (affine_fused_eligible(d->B))
+            return launch_norm_affine_fused(storage_type(d), X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, factor,
+                                            reinterpret_cast<int *>(ws + kWsCounterOffset), clip, C_l, groups == 2, sqnorm,
+                                            sqnorm_stride, clip_out, acc_w, acc_b, st);
         rc = launch_norm_affine(storage_type(d), X, dY, d->B, d->H * d->W, d->C_in, chunk_partial, dg, dbt, partial, st);
         if (rc != DP_OK) return rc;
         if (clip)
             return launch_affine_clip_accum(partial, d->B, C_l, groups == 2, sqnorm, sqnorm_stride, clip_out, dg, dbt, d->C_in,
-                                            acc_w, acc_b, st, reset);
-        return launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st, reset);
+                                            acc_w, acc_b, st);
+        return launch_finalize(partial, d->B, 2, 1, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
     }
 }
 
@@ -246,13 +265,13 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
     if (d->kind == DP_LAYER_DENSE) {
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis; the bias gradient is dY itself.
         // Both kernels read the caller's factors in place.
-        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor_w, factor_stride, d->B, d->C_in, d->K_out, acc_w, status_word, st);
+        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor_w, factor_stride, d->B, d->C_in, d->K_out, acc_w, st);
         if (rc != DP_OK) return rc;
         if (d->has_bias) rc = launch_dense_bias_accum(storage_type(d), dY, d->B, d->K_out, factor_b, factor_stride, acc_b, st);
         return rc;
     }
     // the clipped-sum kernels read one (weight, bias) pair of factors per example
-    rc = launch_expand_factor(factor_w, factor_b, factor_stride, d->B, factor, pl.use_tc ? nullptr : status_word, st);
+    rc = launch_expand_factor(factor_w, factor_b, factor_stride, d->B, factor, st);
     if (rc != DP_OK) return rc;
 
     if (d->kind == DP_LAYER_CONV2D) {
@@ -278,18 +297,32 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
     }
 }
 
-extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int *out, int n) {
-    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || !out || n <= 0) return 0;
-    return tc_describe_plan(desc->dtype, geom_of(desc), out, n);
+extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n) {
+    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 2 || !out || n <= 0) return 0;
+    return tc_describe_plan(desc->dtype, geom_of(desc), epilogue, out, n);
 }
 
-extern "C" dp_status dp_wgrad_check(const void *workspace, void *cuda_stream) {
+extern "C" dp_status dp_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < kWsHeaderBytes) return DP_ERR_WORKSPACE;
+    DP_CUDA_TRY(cudaMemsetAsync(workspace, 0, kWsHeaderBytes, static_cast<cudaStream_t>(cuda_stream)));
+    return DP_OK;
+}
+
+extern "C" dp_status dp_wgrad_check(void *workspace, void *cuda_stream) {
     if (!workspace) return DP_ERR_INVALID_ARG;
     int status = 0;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DP_CUDA_TRY(cudaMemcpyAsync(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost, st));
     DP_CUDA_TRY(cudaStreamSynchronize(st));
-    return status == 0 ? DP_OK : DP_ERR_TIMEOUT;
+    if (status == 0) return DP_OK;
+    // reported once: a launch that gave up may also have left ticket counters behind, so the whole header starts over
+    DP_CUDA_TRY(cudaMemsetAsync(workspace, 0, kWsHeaderBytes, st));
+    DP_CUDA_TRY(cudaStreamSynchronize(st));
+    return DP_ERR_TIMEOUT;
+}
+
+extern "C" void dp_debug_set_wait_polls(long long polls) {
+    set_wait_polls(polls < 0 ? default_wait_polls() : (uint32_t)(polls > 0xffffffffll ? 0xffffffffll : polls));
 }
 
 extern "C" const char *dp_status_string(int status) {

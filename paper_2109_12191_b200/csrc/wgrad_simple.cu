@@ -344,7 +344,7 @@ template <typename T>
 __global__ void __launch_bounds__(256, 2)
 conv_wgrad_rgb3_kernel(const T *__restrict__ X, const T *__restrict__ dY, const ConvGeom g, float *__restrict__ G_w,
                        float *__restrict__ db, int has_bias, int separate, float *__restrict__ sqnorm,
-                       long long sq_stride, int *status_reset) {
+                       long long sq_stride) {
     extern __shared__ __align__(16) float rgb_smem[];
     __shared__ double scratch[32];
     constexpr int kQuad = 4 * (int)sizeof(T);                // bytes of four output channels of dY
@@ -354,7 +354,6 @@ conv_wgrad_rgb3_kernel(const T *__restrict__ X, const T *__restrict__ dY, const 
     float *red = rgb_smem;                                   //   buffer [8 warps][8 lane groups][kRgbRed]
     float *xs = rgb_smem + kRgbStages * kRgbStageFloats;     // [Hp][Wp][3], zero border
     const int n = blockIdx.x, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    if (status_reset && n == 0 && threadIdx.x == 0) *status_reset = 0;
     {
         const int row_in = g.W * 3;
         for (int i = threadIdx.x; i < xs_count; i += 256) xs[i] = 0.f;
@@ -486,16 +485,18 @@ bool rgb3_conv_eligible(const ConvGeom &g) {
 }
 
 dp_status launch_conv_rgb3(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
-                           int has_bias, int separate, float *sqnorm, long long sq_stride, int *status_reset,
+                           int has_bias, int separate, float *sqnorm, long long sq_stride,
                            cudaStream_t st) {
     const size_t smem = rgb3_smem_bytes(g);
+    DP_MAX_SHARED_CARVEOUT((conv_wgrad_rgb3_kernel<float>));
+    DP_MAX_SHARED_CARVEOUT((conv_wgrad_rgb3_kernel<__nv_bfloat16>));
     if (dtype == DP_F32)
         conv_wgrad_rgb3_kernel<float><<<g.B, 256, smem, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), g,
-                                                              G_w, db, has_bias, separate, sqnorm, sq_stride, status_reset);
+                                                              G_w, db, has_bias, separate, sqnorm, sq_stride);
     else
         conv_wgrad_rgb3_kernel<__nv_bfloat16><<<g.B, 256, smem, st>>>(static_cast<const __nv_bfloat16 *>(X),
                                                                       static_cast<const __nv_bfloat16 *>(dY), g, G_w, db,
-                                                                      has_bias, separate, sqnorm, sq_stride, status_reset);
+                                                                      has_bias, separate, sqnorm, sq_stride);
     DP_LAUNCH_CHECK("conv_wgrad_rgb3_kernel");
     return DP_OK;
 }
@@ -566,10 +567,9 @@ bias_vec_kernel(const T *__restrict__ dY, int K, int Kout, float *__restrict__ d
 // One block per example: weight slots [0, w_slots) and bias slots [w_slots, slots) summed in index order.
 __global__ void __launch_bounds__(128)
 finalize_norm_kernel(const float *__restrict__ partial, int slots, int w_slots, int separate, float *__restrict__ sqnorm,
-                     long long sq_stride, int clip, float C_l, float *__restrict__ factor, float *clip_out, int *status_reset) {
+                     long long sq_stride, int clip, float C_l, float *__restrict__ factor, float *clip_out) {
     __shared__ double scratch[32];
     const int n = blockIdx.x;
-    if (status_reset && n == 0 && threadIdx.x == 0) *status_reset = 0;   // paths without bounded waits report "ok"
     const float *p = partial + (long long)n * slots;
     double sw = 0.0, sb = 0.0;
     for (int i = threadIdx.x; i < w_slots; i += 128) sw += (double)p[i];
@@ -628,9 +628,8 @@ constexpr int kDenseOT = 16;
 template <typename T>
 __global__ void __launch_bounds__(256)
 dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const float *__restrict__ factor,
-                        long long f_stride, int B, int Cin, int Kout, float *__restrict__ acc, int *status_reset) {
+                        long long f_stride, int B, int Cin, int Kout, float *__restrict__ acc) {
     __shared__ __align__(16) float fy[256][kDenseOT];
-    if (status_reset && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status_reset = 0;   // no waits on this path        // f_n * dY[n, o0 .. o0+15] for a run of 256 examples
     __shared__ float part[8][kDenseOT][32];
     const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
     const int i = blockIdx.x * 32 + lane, o0 = blockIdx.y * kDenseOT;
@@ -676,9 +675,8 @@ dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const
 
 // factor2[n] = (factor_w[n*stride], factor_b[n*stride]): caller-supplied factors in the layout the clipped-sum kernels read
 __global__ void expand_factor_kernel(const float *__restrict__ factor_w, const float *__restrict__ factor_b,
-                                     long long stride, int B, float *__restrict__ factor2, int *status_reset) {
+                                     long long stride, int B, float *__restrict__ factor2) {
     const int n = blockIdx.x * blockDim.x + threadIdx.x;
-    if (status_reset && n == 0) *status_reset = 0;
     if (n >= B) return;
     factor2[2 * n] = factor_w[n * stride];
     factor2[2 * n + 1] = factor_b[n * stride];
@@ -717,10 +715,9 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, int Kout, int has_bias, float *__restrict__ db,
                   int separate, float *__restrict__ sqnorm, long long sq_stride, int clip, float C_l,
-                  float *__restrict__ factor, float *clip_out, int *status_reset) {
+                  float *__restrict__ factor, float *clip_out) {
     __shared__ double scratch[32];
     const int n = blockIdx.x;
-    if (status_reset && n == 0 && threadIdx.x == 0) *status_reset = 0;
     double sx = 0.0, sy = 0.0;
     for (int i = threadIdx.x; i < Cin; i += 256) { const double v = to_float(X[(long long)n * Cin + i]); sx += v * v; }
     for (int i = threadIdx.x; i < Kout; i += 256) {
@@ -751,12 +748,118 @@ dense_norm_kernel(const T *__restrict__ X, const T *__restrict__ dY, int Cin, in
 }
 
 // ------------------------------------------------------------------ normalisation affine
+// What the last thread block to finish an example does in the one-launch form of the layer: fold the example's
+// pixel-chunk partial sums in chunk order, publish its squared norms (and clip factors), and -- when it is also the
+// last block of the whole call and the batch is small enough to walk alone -- add the clipped sum over the examples
+// to the accumulators.  "Last" is found with ticket counters (no block ever waits for another); the arithmetic and
+// its order do not depend on which block turns out to be last, so results stay bit-reproducible.
+struct AffineTail {
+    int *counters;            // [B + 1] tickets: one per example, one for the call; zero on entry, left at zero.  null: off
+    int blocks_per_example;
+    int B;
+    int clip;                 // 1: factors against C_l, clipped sum into acc_w / acc_b;  0: norms only
+    int accumulate_here;      // 1: the last block of the call adds the clipped sum itself; 0: a second launch does
+    int separate;
+    float C_l;
+    float *sqnorm; long long sq_stride; float *clip_out;
+    float *factor;            // [B][2] scratch: (scale factor, shift factor) per example
+    float *dgamma, *dbeta;    // [B][C] finished per-example gradients (scratch, or the caller's G_w / G_b)
+    float *acc_w, *acc_b;
+};
+
+__device__ __forceinline__ void affine_tail(const AffineTail &t, int n, bool whole, const float *chunk_partial, int chunks,
+                                            int C, double qg, double qb, double *scratch) {
+    __shared__ int last_flag;
+    if (!whole) {
+        __threadfence();                                   // this block's chunk partials are visible before its ticket
+        __syncthreads();
+        if (threadIdx.x == 0) last_flag = (atomicAdd(&t.counters[n], 1) == t.blocks_per_example - 1);
+        __syncthreads();
+        if (!last_flag) return;
+        __threadfence();
+        qg = 0.0; qb = 0.0;
+        for (int c = threadIdx.x; c < C; c += 256) {
+            float a = 0.f, b = 0.f;
+            const float *p = chunk_partial + ((long long)n * chunks * 2) * C + c;
+            int k = 0;
+            for (; k + 8 <= chunks; k += 8) {              // eight chunks' loads in flight, added in chunk order
+                float x[8], y[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { x[u] = __ldcg(p + (long long)(k + u) * 2 * C); y[u] = __ldcg(p + (long long)(k + u) * 2 * C + C); }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { a += x[u]; b += y[u]; }
+            }
+            for (; k < chunks; ++k) { a += __ldcg(p + (long long)k * 2 * C); b += __ldcg(p + (long long)k * 2 * C + C); }
+            t.dgamma[(long long)n * C + c] = a;
+            t.dbeta[(long long)n * C + c] = b;
+            qg += (double)a * a;
+            qb += (double)b * b;
+        }
+        qg = block_sum(qg, scratch);
+        qb = block_sum(qb, scratch);
+        if (threadIdx.x == 0) t.counters[n] = 0;
+    }
+    if (threadIdx.x == 0) {
+        float f0 = 1.f, f1 = 1.f;
+        if (t.separate) {
+            t.sqnorm[n * t.sq_stride] = (float)qg; t.sqnorm[n * t.sq_stride + 1] = (float)qb;
+            if (t.clip) { f0 = clip_factor(qg, t.C_l); f1 = clip_factor(qb, t.C_l); }
+            if (t.clip && t.clip_out) { t.clip_out[2 * n] = f0; t.clip_out[2 * n + 1] = f1; }
+        } else {
+            t.sqnorm[n * t.sq_stride] = (float)(qg + qb);
+            if (t.clip) f0 = f1 = clip_factor(qg + qb, t.C_l);
+            if (t.clip && t.clip_out) t.clip_out[n] = f0;
+        }
+        t.factor[2 * n] = f0; t.factor[2 * n + 1] = f1;
+    }
+    if (!t.clip || !t.accumulate_here) return;
+    __threadfence();                                       // this example's gradients and factors before the call's ticket
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        last_flag = (atomicAdd(&t.counters[t.B], 1) == t.B - 1);
+        if (last_flag) t.counters[t.B] = 0;
+    }
+    __syncthreads();
+    if (!last_flag) return;
+    __threadfence();
+    // thread = (channel, tensor); the factors of up to 256 examples at a time sit in shared memory and eight examples'
+    // values are in flight per thread (the walk is latency-bound: everything comes from L2)
+    __shared__ float f_sh[2][256];
+    for (int c0 = 0; c0 < 2 * C; c0 += 256) {
+        const int e = c0 + threadIdx.x;
+        const int which = e >= C, c = which ? e - C : e;
+        const float *v = (which ? t.dbeta : t.dgamma) + c;
+        float a = 0.f;
+        for (int m0 = 0; m0 < t.B; m0 += 256) {
+            const int mb = min(256, t.B - m0);
+            __syncthreads();
+            if (threadIdx.x < mb) {
+                f_sh[0][threadIdx.x] = __ldcg(t.factor + 2 * (m0 + threadIdx.x));
+                f_sh[1][threadIdx.x] = __ldcg(t.factor + 2 * (m0 + threadIdx.x) + 1);
+            }
+            __syncthreads();
+            if (e < 2 * C) {
+                int m = 0;
+                for (; m + 8 <= mb; m += 8) {
+                    float x[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) x[u] = __ldcg(v + (long long)(m0 + m + u) * C);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) a = fmaf(f_sh[which][m + u], x[u], a);
+                }
+                for (; m < mb; ++m) a = fmaf(f_sh[which][m], __ldcg(v + (long long)(m0 + m) * C), a);
+            }
+        }
+        if (e < 2 * C) (which ? t.acc_b : t.acc_w)[c] += a;
+    }
+}
+
 // stage 1: block = (channel-vector block, pixel chunk, example); thread = (pixel row, channel vector).
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
 norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, int HW, int C, int tcv, int pix,
                            float *__restrict__ chunk_partial, int chunks, float *__restrict__ dgamma,
-                           float *__restrict__ dbeta, float *__restrict__ partial2) {
+                           float *__restrict__ dbeta, float *__restrict__ partial2, const AffineTail tail) {
     extern __shared__ float red[];                       // [rows][tcv*VEC*2]
     const int n = blockIdx.z, chunk = blockIdx.y;
     const int rows = 256 / tcv;
@@ -841,8 +944,9 @@ norm_affine_partial_kernel(const T *__restrict__ X, const T *__restrict__ dY, in
         if (whole) {
             qg = block_sum(qg, scratch);
             qb = block_sum(qb, scratch);
-            if (threadIdx.x == 0) { partial2[2 * n] = (float)qg; partial2[2 * n + 1] = (float)qb; }
+            if (threadIdx.x == 0 && !tail.counters) { partial2[2 * n] = (float)qg; partial2[2 * n + 1] = (float)qb; }
         }
+        if (tail.counters) affine_tail(tail, n, whole, chunk_partial, chunks, C, qg, qb, scratch);
     }
 }
 
@@ -877,10 +981,8 @@ norm_affine_fold_kernel(const float *__restrict__ chunk_partial, int chunks, int
 __global__ void __launch_bounds__(128)
 affine_clip_accum_kernel(const float *__restrict__ partial2, int B, float C_l, int separate, float *__restrict__ sqnorm,
                          long long sq_stride, float *clip_out, const float *__restrict__ dgamma,
-                         const float *__restrict__ dbeta, int C, float *__restrict__ acc_w, float *__restrict__ acc_b,
-                         int *status_reset) {
+                         const float *__restrict__ dbeta, int C, float *__restrict__ acc_w, float *__restrict__ acc_b) {
     __shared__ float fw[512], fb[512];
-    if (status_reset && blockIdx.x == 0 && threadIdx.x == 0) *status_reset = 0;
     const int c = blockIdx.x * 128 + threadIdx.x;
     float a = 0.f, b = 0.f;
     for (int n0 = 0; n0 < B; n0 += 512) {
@@ -918,9 +1020,10 @@ affine_clip_accum_kernel(const float *__restrict__ partial2, int B, float C_l, i
 
 dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int separate, float *sqnorm, long long sq_stride,
                                    float *clip_out, const float *dgamma, const float *dbeta, int C, float *acc_w,
-                                   float *acc_b, cudaStream_t st, int *status_reset) {
+                                   float *acc_b, cudaStream_t st) {
+    DP_MAX_SHARED_CARVEOUT((affine_clip_accum_kernel));
     affine_clip_accum_kernel<<<(C + 127) / 128, 128, 0, st>>>(partial2, B, C_l, separate, sqnorm, sq_stride, clip_out, dgamma,
-                                                            dbeta, C, acc_w, acc_b, status_reset);
+                                                            dbeta, C, acc_w, acc_b);
     DP_LAUNCH_CHECK("affine_clip_accum_kernel");
     return DP_OK;
 }
@@ -928,7 +1031,7 @@ dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int 
 // ------------------------------------------------------------------ host launchers
 int fma_clip_splits(const ConvGeom &g) {
     const int tiles = fma_tiles_m(g) * fma_tiles_n(g);
-    int want = (2 * 148) / tiles;
+    int want = (2 * sm_count()) / tiles;
     if (want < 1) want = 1;
     if (want > g.B) want = g.B;
     const int per = (g.B + want - 1) / want;
@@ -957,6 +1060,7 @@ static dp_status conv_fma_t(int mode, const T *X, const T *dY, const ConvGeom &g
     DP_LAUNCH_CHECK("conv_wgrad_fma_kernel");
     if (mode == 2 && splits > 1) {
         const long long P = (long long)g.M * g.N;
+        DP_MAX_SHARED_CARVEOUT((fold_sums_kernel));
         fold_sums_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(sum_ws, splits, P, acc_w);
         DP_LAUNCH_CHECK("fold_sums_kernel");
     }
@@ -975,6 +1079,8 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
     const int vec = (dtype == DP_F32) ? 4 : 8;
     if (g.Kout % vec == 0 && g.Kout / vec <= 256 && bias_blocks(g) <= 256) {
         const size_t smem = sizeof(float) * (size_t)(256 / (g.Kout / vec)) * g.Kout;
+        DP_MAX_SHARED_CARVEOUT((bias_vec_kernel<float, 4>));
+        DP_MAX_SHARED_CARVEOUT((bias_vec_kernel<__nv_bfloat16, 8>));
         if (dtype == DP_F32)
             bias_vec_kernel<float, 4><<<g.B, 256, smem, st>>>(static_cast<const float *>(dY), g.K, g.Kout, db, partial, slots, slot0, bias_blocks(g));
         else
@@ -991,14 +1097,15 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
 }
 
 dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
-                          long long sq_stride, int clip, float C_l, float *factor, float *clip_out, cudaStream_t st,
-                          int *status_reset) {
-    finalize_norm_kernel<<<B, 128, 0, st>>>(partial, slots, w_slots, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out, status_reset);
+                          long long sq_stride, int clip, float C_l, float *factor, float *clip_out, cudaStream_t st) {
+    DP_MAX_SHARED_CARVEOUT((finalize_norm_kernel));
+    finalize_norm_kernel<<<B, 128, 0, st>>>(partial, slots, w_slots, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
     DP_LAUNCH_CHECK("finalize_norm_kernel");
     return DP_OK;
 }
 
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st, int which) {
+    DP_MAX_SHARED_CARVEOUT((bias_accum_kernel<float>));
     bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(db, B, Kout, factor + which, 2, acc_b);
     DP_LAUNCH_CHECK("bias_accum_kernel");
     return DP_OK;
@@ -1015,20 +1122,22 @@ dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, co
 }
 
 dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, long long f_stride, int B,
-                                  int Cin, int Kout, float *acc_w, int *status_reset, cudaStream_t st) {
+                                  int Cin, int Kout, float *acc_w, cudaStream_t st) {
     const dim3 grid((unsigned)((Cin + 31) / 32), (unsigned)((Kout + kDenseOT - 1) / kDenseOT));
     if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
+    DP_MAX_SHARED_CARVEOUT((dense_scaled_sum_kernel<float>));
+    DP_MAX_SHARED_CARVEOUT((dense_scaled_sum_kernel<__nv_bfloat16>));
     if (dtype == DP_F32)
-        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, f_stride, B, Cin, Kout, acc_w, status_reset);
+        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, f_stride, B, Cin, Kout, acc_w);
     else
-        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, f_stride, B, Cin, Kout, acc_w, status_reset);
+        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, f_stride, B, Cin, Kout, acc_w);
     DP_LAUNCH_CHECK("dense_scaled_sum_kernel");
     return DP_OK;
 }
 
-dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2,
-                               int *status_reset, cudaStream_t st) {
-    expand_factor_kernel<<<(B + 127) / 128, 128, 0, st>>>(factor_w, factor_b, stride, B, factor2, status_reset);
+dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2, cudaStream_t st) {
+    DP_MAX_SHARED_CARVEOUT((expand_factor_kernel));
+    expand_factor_kernel<<<(B + 127) / 128, 128, 0, st>>>(factor_w, factor_b, stride, B, factor2);
     DP_LAUNCH_CHECK("expand_factor_kernel");
     return DP_OK;
 }
@@ -1056,48 +1165,105 @@ dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, in
 
 dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias, float *db,
                             int separate, float *sqnorm, long long sq_stride, int clip, float C_l, float *factor,
-                            float *clip_out, int *status_reset, cudaStream_t st) {
+                            float *clip_out, cudaStream_t st) {
+    DP_MAX_SHARED_CARVEOUT((dense_norm_kernel<float>));
+    DP_MAX_SHARED_CARVEOUT((dense_norm_kernel<__nv_bfloat16>));
     if (dtype == DP_F32)
         dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), Cin, Kout, has_bias, db,
-                                             separate, sqnorm, sq_stride, clip, C_l, factor, clip_out, status_reset);
+                                             separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
     else
         dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), Cin, Kout,
-                                             has_bias, db, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out, status_reset);
+                                             has_bias, db, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
     DP_LAUNCH_CHECK("dense_norm_kernel");
     return DP_OK;
 }
 
 template <typename T, int VEC>
 static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, int tcv, int pix, float *chunk_partial,
-                               float *dgamma, float *dbeta, float *partial2, bool &folded, cudaStream_t st) {
+                               float *dgamma, float *dbeta, float *partial2, bool &folded, AffineTail tail, cudaStream_t st) {
     const int cv = (C + VEC - 1) / VEC;
     const int chunks = (HW + pix - 1) / pix;
     const dim3 grid((cv + tcv - 1) / tcv, chunks, B);
     if (grid.y > 65535 || grid.z > 65535) return DP_ERR_UNSUPPORTED;
     const size_t smem = sizeof(float) * (size_t)(256 / tcv) * tcv * VEC * 2;
     folded = grid.x == 1 && chunks == 1;      // one block sees the whole example: it finishes the job itself
+    tail.blocks_per_example = (int)(grid.x * grid.y);
+    DP_MAX_SHARED_CARVEOUT((norm_affine_partial_kernel<T, VEC>));
     norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, pix, chunk_partial, chunks,
-                                                               folded ? dgamma : nullptr, dbeta, partial2);
+                                                               folded ? dgamma : nullptr, dbeta, partial2, tail);
     DP_LAUNCH_CHECK("norm_affine_partial_kernel");
     return DP_OK;
 }
 
-dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
-                             float *dgamma, float *dbeta, float *partial2, cudaStream_t st) {
-    dp_status rc;
-    bool folded = false;
+static dp_status norm_affine_dispatch(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
+                                      float *dgamma, float *dbeta, float *partial2, bool &folded, const AffineTail &tail,
+                                      cudaStream_t st) {
     int vec, tcv, pix;
     norm_shape(dtype, B, HW, C, vec, tcv, pix);
     if (dtype == DP_F32) {
-        if ((C & 3) == 0) rc = norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
-        else rc = norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
-    } else {
-        if ((C & 7) == 0) rc = norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
-        else rc = norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, st);
+        if ((C & 3) == 0) return norm_affine_t<float, 4>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, tail, st);
+        return norm_affine_t<float, 1>(static_cast<const float *>(X), static_cast<const float *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, tail, st);
     }
+    if ((C & 7) == 0) return norm_affine_t<__nv_bfloat16, 8>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, tail, st);
+    return norm_affine_t<__nv_bfloat16, 1>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), B, HW, C, tcv, pix, chunk_partial, dgamma, dbeta, partial2, folded, tail, st);
+}
+
+dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
+                             float *dgamma, float *dbeta, float *partial2, cudaStream_t st) {
+    bool folded = false;
+    AffineTail off = {};
+    const dp_status rc = norm_affine_dispatch(dtype, X, dY, B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, off, st);
     if (rc != DP_OK || folded) return rc;
-    norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, (HW + pix - 1) / pix, C, dgamma, dbeta, partial2);
+    DP_MAX_SHARED_CARVEOUT((norm_affine_fold_kernel));
+    norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, norm_chunks(dtype, B, HW, C), C, dgamma, dbeta, partial2);
     DP_LAUNCH_CHECK("norm_affine_fold_kernel");
+    return DP_OK;
+}
+
+// acc_w[c] += sum_n factor[2n] * dgamma[n, c] and acc_b[c] += sum_n factor[2n + 1] * dbeta[n, c] in one launch
+// (blockIdx.y picks the tensor).  Block = 32 channels x 8 example groups, groups folded in order.
+__global__ void __launch_bounds__(256)
+affine_accum_kernel(const float *__restrict__ dgamma, const float *__restrict__ dbeta, int B, int C,
+                    const float *__restrict__ factor, float *__restrict__ acc_w, float *__restrict__ acc_b) {
+    __shared__ float part[8][32];
+    const int lane = threadIdx.x & 31, q = threadIdx.x >> 5, which = blockIdx.y;
+    const float *v = which ? dbeta : dgamma;
+    const int c = blockIdx.x * 32 + lane;
+    float a = 0.f;
+    if (c < C) {
+#pragma unroll 8
+        for (int n = q; n < B; n += 8) a = fmaf(factor[2 * n + which], v[(long long)n * C + c], a);
+    }
+    part[q][lane] = a;
+    __syncthreads();
+    if (q == 0 && c < C) {
+        float t = part[0][lane];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) t += part[i][lane];
+        (which ? acc_b : acc_w)[c] += t;
+    }
+}
+
+bool affine_fused_eligible(int B) { return B + 1 <= kWsCounters; }
+
+// The whole layer call in one launch (two when the batch times the channel count is large): per-example gradients,
+// their squared norms, and for clip != 0 the factors against C_l and the clipped sums.  dgamma / dbeta: [B][C]
+// scratch or the caller's outputs; factor: [B][2] scratch; counters: B + 1 cleared tickets.
+dp_status launch_norm_affine_fused(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
+                                   float *dgamma, float *dbeta, float *factor, int *counters, int clip, float C_l,
+                                   int separate, float *sqnorm, long long sq_stride, float *clip_out, float *acc_w,
+                                   float *acc_b, cudaStream_t st) {
+    AffineTail t = {};
+    t.counters = counters; t.B = B; t.clip = clip; t.separate = separate; t.C_l = C_l;
+    t.accumulate_here = clip && (long long)B * C <= 16384;
+    t.sqnorm = sqnorm; t.sq_stride = sq_stride; t.clip_out = clip_out; t.factor = factor;
+    t.dgamma = dgamma; t.dbeta = dbeta; t.acc_w = acc_w; t.acc_b = acc_b;
+    bool folded = false;
+    const dp_status rc = norm_affine_dispatch(dtype, X, dY, B, HW, C, chunk_partial, dgamma, dbeta, nullptr, folded, t, st);
+    if (rc != DP_OK || !clip || t.accumulate_here) return rc;
+    DP_MAX_SHARED_CARVEOUT((affine_accum_kernel));
+    affine_accum_kernel<<<dim3((unsigned)((C + 31) / 32), 2), 256, 0, st>>>(dgamma, dbeta, B, C, factor, acc_w, acc_b);
+    DP_LAUNCH_CHECK("affine_accum_kernel");
     return DP_OK;
 }
 

@@ -34,7 +34,7 @@ dp_status launch_conv_thin(int dtype, const void *X, const void *dY, const ConvG
 // gradient and the published squared norms (sqnorm[n*sq_stride + {0,1}] when `separate`, else their sum) in one launch.
 bool rgb3_conv_eligible(const ConvGeom &g);
 dp_status launch_conv_rgb3(int dtype, const void *X, const void *dY, const ConvGeom &g, float *G_w, float *db,
-                           int has_bias, int separate, float *sqnorm, long long sq_stride, int *status_reset,
+                           int has_bias, int separate, float *sqnorm, long long sq_stride,
                            cudaStream_t stream);
 // db[n,k] = sum over pixels of dY; also sum_k db^2 per block into partial[n*slots + slot0 + block]
 dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, float *partial, int slots, int slot0,
@@ -42,7 +42,7 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
 // folds the partial slots of every example into sqnorm (and clip factors when clip != 0)
 dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
                           long long sq_stride, int clip, float C_l, float *factor, float *clip_out,
-                          cudaStream_t stream, int *status_reset = nullptr);
+                          cudaStream_t stream);
 // acc_b[k] += sum_n factor[n*2+which] * db[n,k]
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream,
                             int which = 1);
@@ -51,26 +51,33 @@ dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, co
                                   cudaStream_t stream);
 // dense layer: acc_w[o, i] += sum_n factor[n*f_stride] * dY[n, o] * X[n, i]
 dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, long long f_stride, int B,
-                                  int Cin, int Kout, float *acc_w, int *status_reset, cudaStream_t stream);
-// factor2[n] = (factor_w[n*stride], factor_b[n*stride]); optionally clears a status word
+                                  int Cin, int Kout, float *acc_w, cudaStream_t stream);
+// factor2[n] = (factor_w[n*stride], factor_b[n*stride])
 dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2,
-                               int *status_reset, cudaStream_t stream);
+                               cudaStream_t stream);
 
 dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, float *G_w,
                              float *G_b, cudaStream_t stream);
 // closed-form squared norms (|dY_n|^2 |X_n|^2 and |dY_n|^2), db = dY as fp32 (optional), norms and clip factors published
 dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias, float *db,
                             int separate, float *sqnorm, long long sq_stride, int clip, float C_l, float *factor,
-                            float *clip_out, int *status_reset, cudaStream_t stream);
+                            float *clip_out, cudaStream_t stream);
 
 // stage 1: per pixel-chunk partial sums; stage 2: fold, store, squared norms into partial2[n*2 + {0,1}]
 dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
                              float *dgamma, float *dbeta, float *partial2, cudaStream_t stream);
 
+// One-launch form of the normalisation layer (see the kernel): needs B + 1 cleared ticket counters.
+bool affine_fused_eligible(int B);
+dp_status launch_norm_affine_fused(int dtype, const void *X, const void *dY, int B, int HW, int C, float *chunk_partial,
+                                   float *dgamma, float *dbeta, float *factor, int *counters, int clip, float C_l,
+                                   int separate, float *sqnorm, long long sq_stride, float *clip_out, float *acc_w,
+                                   float *acc_b, cudaStream_t stream);
+
 // fused: factors from partial2 (two squared norms per example), publish norms / factors, accumulate both tensors
 dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int separate, float *sqnorm, long long sq_stride,
                                    float *clip_out, const float *dgamma, const float *dbeta, int C, float *acc_w,
-                                   float *acc_b, cudaStream_t stream, int *status_reset = nullptr);
+                                   float *acc_b, cudaStream_t stream);
 
 // Shape of the norm-affine reduction: channel vectors per block (tcv) and pixels per block (pix).  Starts from whole
 // channel rows and 256 pixels and narrows both until the grid has a couple of blocks per SM, so that layers with

@@ -21,6 +21,7 @@
 #include "wgrad_tc.cuh"
 #include <cuda.h>
 #include <mutex>
+#include <atomic>
 #include <algorithm>
 #include <array>
 #include <map>
@@ -31,6 +32,9 @@ constexpr int kRowBytes = 128;         // one pixel's slab of channels: 64 bf16 
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 200 * 1024;
 constexpr uint32_t kWaitPolls = 1u << 21;   // x ~1 us suspend hint: about two seconds before a wait gives up
+static std::atomic<uint32_t> g_wait_polls{kWaitPolls};
+void set_wait_polls(uint32_t polls) { g_wait_polls.store(polls, std::memory_order_relaxed); }
+uint32_t default_wait_polls() { return kWaitPolls; }
 
 struct TcPlan {
     bool ok;
@@ -56,7 +60,7 @@ struct TcParams {
     float *partial;             // [B][slots], slot = (mt*n_tiles + nt)*4 + epilogue warp
     int slots;
     int *status;
-    int reset_status;           // 1: this launch is the first of its call and clears the status word itself
+    uint32_t wait_polls;        // polls after which a wait gives up
     int total_tiles;            // work items: (example, tile) pairs, or (example range, tile) pairs in mode 2
     // mode 2: item = (split, tile); the CTA walks examples [split*per_split, ...) and keeps sum_n f_n D_n in registers
     int splits, per_split;
@@ -67,6 +71,9 @@ struct TcParams {
     float C_l;
     float *sqnorm; long long sq_stride; float *clip_out;
     float *sum_out;             // splits == 1: the accumulator (added to); else partial sums [splits][Kout*Ng]
+    // modes 0 / 1 with a ticket: counters[0] counts the CTAs that are done (zero on entry, left at zero); the last
+    // one folds every example's slots [0, w_slots) and [w_slots, slots) into sqnorm (two values when `separate`)
+    int *counters; int w_slots; int separate;
 };
 
 struct Item { int mt, nt, n_lo, n_hi, split; };
@@ -103,8 +110,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait expired).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    for (uint32_t it = 0; it < kWaitPolls; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t polls) {
+    for (uint32_t it = 0; it < polls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
@@ -189,8 +196,6 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const uint32_t tiles_u32 = smem_u32(tiles);
 
     if (threadIdx.x == 0) {
-        // a wait can only expire seconds from now, long after this store, so clearing here cannot hide a time-out
-        if (blockIdx.x == 0 && p.reset_status) *p.status = 0;
         // pull both tensor maps into the TMA descriptor cache before the first copy needs them
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
@@ -249,7 +254,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
                     bool ok = true;
                     if (lane == 0) {
-                        ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p);
+                        ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p, p.wait_polls);
                         if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -278,12 +283,12 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
               const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - it.nt * b_slabs_tile);
               const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, TF32 ? 2u : 1u);
               for (int n = it.n_lo; n < it.n_hi && live; ++n) {
-                if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p)) { live = false; break; }
+                if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p, p.wait_polls)) { live = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
                 uint32_t accumulate = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    if (!mbar_wait(smem_u32(TF32 ? &ready_bar[stage] : &full_bar[stage]), phase, abort_p)) { live = false; break; }
+                    if (!mbar_wait(smem_u32(TF32 ? &ready_bar[stage] : &full_bar[stage]), phase, abort_p, p.wait_polls)) { live = false; break; }
                     tc_fence_after();
                     const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
                     // descriptor low words: start address >> 4 in bits 0-13, slab stride >> 4 in bits 16-29
@@ -345,7 +350,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const int stage_count = (it.n_hi - it.n_lo) * p.k_tiles;
             for (int kt = 0; kt < stage_count; ++kt) {
                 if (turn == group) {
-                    const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p);
+                    const bool arrived = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p, p.wait_polls);
                     if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
                     uint8_t *base = tiles + (size_t)stage * p.stage_bytes;
                     // four 16-byte groups per thread and trip with all loads first, A region and B region in turn
@@ -407,7 +412,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 for (int i = 0; i < 128; ++i) run[CLIP ? i : 0] = 0.f;
             }
             for (int n = it.n_lo; n < it.n_hi; ++n) {
-                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p);
+                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
                 if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }   // the whole warp leaves together
                 full_phase ^= 1u << buf;
                 tc_fence_after();
@@ -480,7 +485,10 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
                     sq = warp_sum(sq);
-                    if (lane == 0) p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
+                    if (lane == 0) {
+                        p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
+                        if (p.counters) __threadfence();       // visible to the CTA that will fold the partial sums
+                    }
                 }
                 buf ^= 1;
             }
@@ -523,6 +531,33 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
     tc_fence_before();
     __syncthreads();
+    if (!CLIP && p.counters && !abort_flag) {
+        // The last CTA to finish (one ticket per CTA, nobody waits) folds every example's partial squared norms,
+        // bias slots included, in slot order and publishes the squared norm(s): no finalising launch.
+        __shared__ int last_cta;
+        if (threadIdx.x == 0) {
+            __threadfence();
+            last_cta = atomicAdd(&p.counters[0], 1) == (int)gridDim.x - 1;
+            if (last_cta) p.counters[0] = 0;
+        }
+        __syncthreads();
+        if (last_cta) {
+            __threadfence();
+            const int nwarps = blockDim.x >> 5;
+            for (int n = warp; n < p.B; n += nwarps) {
+                const float *pn = p.partial + (long long)n * p.slots;
+                double sw = 0.0, sb = 0.0;
+                for (int i = lane; i < p.w_slots; i += 32) sw += (double)__ldcg(pn + i);
+                for (int i = p.w_slots + lane; i < p.slots; i += 32) sb += (double)__ldcg(pn + i);
+                sw = warp_sum(sw); sb = warp_sum(sb);
+                if (lane == 0) {
+                    if (p.separate) { p.sqnorm[n * p.sq_stride] = (float)sw; p.sqnorm[n * p.sq_stride + 1] = (float)sb; }
+                    else p.sqnorm[n * p.sq_stride] = (float)(sw + sb);
+                }
+            }
+        }
+        __syncthreads();
+    }
     if (abort_flag) {
         // give copies still in flight time to land before shared memory is released
         if (threadIdx.x == 0) { *p.status = DP_ERR_TIMEOUT; __threadfence(); }
@@ -554,6 +589,8 @@ __global__ void fold_partial_sums_scalar_kernel(const float *__restrict__ part, 
 }
 
 dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream) {
+    DP_MAX_SHARED_CARVEOUT((fold_partial_sums_kernel));
+    DP_MAX_SHARED_CARVEOUT((fold_partial_sums_scalar_kernel));
     if (P % 4 == 0 && aligned(part, 16) && aligned(acc, 16))
         fold_partial_sums_kernel<<<(unsigned)((P / 4 + 255) / 256), 256, 0, stream>>>(part, splits, P, acc);
     else
@@ -650,18 +687,6 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-static int sm_count() {
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            sms = v;
-        else
-            return 148;
-    }
-    return sms;
-}
-
 // What the tensor-core kernel is actually given: the layer itself, or its unfolded 1x1 form.
 struct TcProblem {
     bool ok, unfold;
@@ -750,10 +775,13 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             // the 128 x NT accumulator: stores run at about 16 B/clk per SM when lanes write consecutive addresses
             // (rows of D are gradient columns) and about 7 B/clk otherwise; reading TMEM alone is cheap
             const double epilogue = (mode == 0) ? 128.0 * NT * 4.0 / (a_is_x ? 16.0 : 7.0) : (mode == 1 ? 6.0 * NT : 10.0 * NT);
-            for (int OHt = 1; OHt <= g.OH; ++OHt) {
-                if (OHt * g.stride > 256 || OHt * g.stride > g.H) break;
-                for (int OWt = 1; OWt <= g.OW; ++OWt) {
-                    if (OWt * g.stride > 256 || OWt * g.stride > g.W) break;
+            // a pixel tile may reach past the output plane (its rows there are zero-filled by TMA and add nothing):
+            // a 7 x 7 plane is one 8 x 8 tile of 64 reduction rows instead of four 4 x 4 tiles of 16
+            const int oh_max = std::min((g.OH + 7) / 8 * 8, 256 / g.stride), ow_max = std::min((g.OW + 7) / 8 * 8, 256 / g.stride);
+            for (int OHt = 1; OHt <= oh_max; ++OHt) {
+                for (int OWt = 1; OWt <= ow_max; ++OWt) {
+                    if (OWt > g.OW && OWt % 8) continue;      // overshoot only to the next multiple of eight
+                    if (OHt > g.OH && OHt % 8) continue;
                     const int Kt = OHt * OWt;
                     if (Kt % krows || Kt > 256) continue;
                     const int stage_bytes = slabs * Kt * kRowBytes * copies;
@@ -829,10 +857,10 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
     return bytes;
 }
 
-int tc_describe_plan(int dtype, const ConvGeom &g0, int *out, int n) {
+int tc_describe_plan(int dtype, const ConvGeom &g0, int epilogue, int *out, int n) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
-    const TcPlan pl = make_plan(dtype, pr.eff, 0);
+    const TcPlan pl = make_plan(dtype, pr.eff, epilogue);
     if (!pl.ok) return 0;
     const int v[12] = {pl.a_is_x, pl.a_ext, pl.b_ext, pl.m_tiles, pl.n_tiles, pl.NT, pl.OWt, pl.OHt, pl.Kt, pl.k_tiles,
                        pl.stages, pl.stage_bytes};
@@ -857,7 +885,7 @@ static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, in
 
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g_in, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace, int *status,
-                         cudaStream_t stream, bool second_pass, const TcInlineClip *inline_clip) {
+                         cudaStream_t stream, bool second_pass, const TcInlineClip *inline_clip, const TcPublish *publish) {
     const bool clip = epilogue == DP_EPI_CLIP_ACCUM;
     const ConvGeom &g0 = g_in;
     const TcProblem pr = tc_problem(dtype, g0);
@@ -874,6 +902,8 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
             const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / vec);
             const unsigned blocks = (unsigned)((total + 255) / 256);
             const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * (dtype == DP_BF16 ? 2 : 4);
+            DP_MAX_SHARED_CARVEOUT((unfold_rows_kernel<__nv_bfloat16, 8>));
+            DP_MAX_SHARED_CARVEOUT((unfold_rows_kernel<float, 4>));
             if (row_smem <= 40 * 1024 && g0.OH <= 0x7fffffff && g0.B <= 65535) {
                 const dim3 grid_rows(g0.OH, g0.B);
                 if (dtype == DP_BF16)
@@ -907,13 +937,18 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.single_pass = (dtype == DP_TF32) ? 1 : 0;
     p.mode = clip ? 2 : (epilogue == DP_EPI_STORE_NORM ? 0 : 1);
     p.G_w = G_w; p.partial = partial; p.slots = slots; p.status = status;
-    p.reset_status = second_pass ? 0 : 1;       // the second launch of a fused clip call must keep the first one's verdict
+    p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
     p.splits = 1; p.per_split = g.B; p.factor = factor; p.sum_out = acc_w;
     p.inline_factor = (clip && inline_clip) ? 1 : 0;
     p.C_l = inline_clip ? inline_clip->C_l : 0.f;
     p.sqnorm = inline_clip ? inline_clip->sqnorm : nullptr;
     p.sq_stride = inline_clip ? inline_clip->sq_stride : 0;
     p.clip_out = inline_clip ? inline_clip->clip_out : nullptr;
+    p.counters = nullptr; p.w_slots = 0; p.separate = 0;
+    if (!clip && publish) {
+        p.counters = publish->counters; p.w_slots = publish->w_slots; p.separate = publish->separate;
+        p.sqnorm = publish->sqnorm; p.sq_stride = publish->sq_stride;
+    }
     if (clip) {
         clip_split(g, pl, p.splits, p.per_split);
         if (p.splits > 1) p.sum_out = part_ws;

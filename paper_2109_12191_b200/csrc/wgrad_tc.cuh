@@ -12,15 +12,24 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g, int epilogue);
 // tiling chosen for the layer: {a_is_x, a_ext, b_ext, m_tiles, n_tiles, NT, OWt, OHt, Kt, k_tiles, stages, stage_bytes}
 // acc[i] += sum_s part[s][i] in index order of s (P a multiple of 4)
 dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream);
-int tc_describe_plan(int dtype, const ConvGeom &g, int *out, int n);
+int tc_describe_plan(int dtype, const ConvGeom &g, int epilogue, int *out, int n);
 // When given to a CLIP_ACCUM launch, the kernel derives each example's factor from the norm pass's partial sums
 // itself (threshold C_l) and writes sqnorm[n*sq_stride] and clip_out[n] (optional), so no finalising launch is needed.
 struct TcInlineClip { float C_l; float *sqnorm; long long sq_stride; float *clip_out; };
+
+// When given to a STORE_NORM / NORM_ONLY launch, the last CTA to finish folds every example's partial squared norms
+// (slots [0, w_slots) = weights, the rest = bias, written earlier in the stream) and writes sqnorm[n*sq_stride]
+// (+1 for the bias when `separate`), so no finalising launch is needed.  counters: one cleared ticket word.
+struct TcPublish { int *counters; int w_slots; int separate; float *sqnorm; long long sq_stride; };
 
 // epilogue as dp_epilogue; factor[n*2] scales example n (CLIP_ACCUM); status: device word set to nonzero on a timed-out wait
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
                          float *partial, int slots, const float *factor, float *acc_w, void *tc_workspace,
                          int *status, cudaStream_t stream, bool second_pass = false,
-                         const TcInlineClip *inline_clip = nullptr);
+                         const TcInlineClip *inline_clip = nullptr, const TcPublish *publish = nullptr);
+
+// Test hook: the number of polls after which a bounded wait of the kernel gives up (0 makes every wait give up at once).
+void set_wait_polls(uint32_t polls);
+uint32_t default_wait_polls();
 
 }  // namespace dp

@@ -22,3 +22,15 @@ def allreduce_accumulator(acc, dist=None):
     if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(acc, op=dist.ReduceOp.SUM)
     return acc
+
+
+def global_batch(local_examples: int, dist=None) -> int:
+    """|B| of the step: the examples all ranks processed together.  Shares may be uneven (shard_range), so every
+    rank contributes its own count instead of multiplying one rank's count by the number of ranks."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return int(local_examples)
+    import torch
+    backend = dist.get_backend()
+    t = torch.tensor([int(local_examples)], dtype=torch.int64, device="cuda" if backend == "nccl" else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return int(t.item())

@@ -34,6 +34,17 @@ def _tensors_of(layers):
     return out
 
 
+def _workspaces(nbytes, lanes, device):
+    """One initialised dp_per_example_wgrad workspace per lane (calls that may overlap need one each)."""
+    out = []
+    for _ in range(lanes):
+        w = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        b.check(b.dp_workspace_init(w), "dp_workspace_init")
+        out.append(w)
+    torch.cuda.synchronize()
+    return out
+
+
 class _NoiseKey:
     """Where the noise enters: once per step in finish() (default), or per example inside every chunk call, in which
     case the chunk calls need the step's total batch and key and finish() only divides."""
@@ -92,7 +103,7 @@ class GlobalClipStep:
         self.clip = torch.empty(B, dtype=torch.float32, device=device)
         ws = max([b.dp_workspace_bytes(d, e) for d in self.descs for e in (b.DP_EPI_STORE_NORM, b.DP_EPI_NORM_ONLY, b.DP_EPI_CLIP_ACCUM)] + [256])
         self.lanes = max(1, min(int(lanes), len(self.layers)))
-        self.ws_lane = [torch.empty(ws, dtype=torch.uint8, device=device) for _ in range(self.lanes)]
+        self.ws_lane = _workspaces(ws, self.lanes, device)
         self.ws = self.ws_lane[0]
         self._side = [torch.cuda.Stream(device=device) for _ in range(self.lanes - 1)] if self.lanes > 1 else []
         self.clip_ws = torch.empty(max(b.dp_clip_workspace_bytes(B, self.P_l), 256), dtype=torch.uint8, device=device)
@@ -212,9 +223,11 @@ class GlobalClipStep:
         for w in self.ws_lane:
             b.check(b.dp_wgrad_check(w), "dp_wgrad_check")
 
-    def finish(self, seed=0, step=0, world=1):
-        """world > 1: `acc` already holds the sum over all ranks (see sharding.allreduce_accumulator)."""
-        total = self.B * self.chunks_done * world
+    def finish(self, seed=0, step=0, total_batch=None):
+        """total_batch: |B| of the whole step.  Left out, it is what this object saw (one process).  With several
+        ranks `acc` already holds the sum over all of them (sharding.allreduce_accumulator) and the caller passes the
+        global count (sharding.global_batch): ranks may have run different numbers of chunks."""
+        total = self.B * self.chunks_done if total_batch is None else int(total_batch)
         sigma = self._noise.finish_sigma(self.sigma, total)
         b.check(b.dp_noise_average(self.acc, self.P, 0, sigma, self.C, total, seed, step, self.out), "dp_noise_average")
         return self.out
@@ -256,8 +269,9 @@ class FlatClipStep:
                                          self.clip, self.ws), "dp_clip_accumulate")
         self.chunks_done += 1
 
-    def finish(self, seed=0, step=0, world=1):
-        total = self.B * self.chunks_done * world
+    def finish(self, seed=0, step=0, total_batch=None):
+        """total_batch as for GlobalClipStep.finish (examples, not micro-batches)."""
+        total = self.B * self.chunks_done if total_batch is None else int(total_batch)
         sigma = self._noise.finish_sigma(self.sigma, total)
         b.check(b.dp_noise_average(self.acc, self.P, 0, sigma, self.C, total // self.micro, seed, step, self.out),
                 "dp_noise_average")
@@ -277,18 +291,30 @@ class PerLayerClipStep:
         self.L = len(self.tensors)
         self.C_l = self.C / math.sqrt(self.L)
         self.descs = [layer_desc(l, B, dtype, impl, 1) for l in self.layers]
-        self.acc_w = [torch.zeros(l.n_weight, dtype=torch.float32, device=device) for l in self.layers]
-        self.acc_b = [torch.zeros(l.n_bias, dtype=torch.float32, device=device) if l.n_bias else None for l in self.layers]
+        # one accumulator in parameter order (weight, then bias-like tensor, of each layer); the layer calls get views.
+        # A tensor that would start off a 16-byte boundary is padded forward (`self.offsets` keeps the true indices).
+        self.P = sum(t[2] for t in self.tensors)
+        starts, self.offsets, cur, true = [], [], 0, 0
+        for _, _, size in self.tensors:
+            cur = (cur + 3) // 4 * 4
+            starts.append(cur)
+            self.offsets.append(true)
+            cur += size
+            true += size
+        self.acc = torch.zeros(cur, dtype=torch.float32, device=device)
+        self.contiguous = cur == self.P                     # no padding: the accumulator IS the parameter vector
+        views = {(li, which): self.acc[s0:s0 + size] for (li, which, size), s0 in zip(self.tensors, starts)}
+        self.acc_w = [views[(li, "w")] for li in range(len(self.layers))]
+        self.acc_b = [views.get((li, "b")) for li in range(len(self.layers))]
         self.sq = torch.zeros((B, self.L), dtype=torch.float32, device=device)
         ws = max([b.dp_workspace_bytes(d, b.DP_EPI_CLIP_ACCUM) for d in self.descs] + [256])
         self.lanes = max(1, int(lanes))
-        self.ws_lane = [torch.empty(ws, dtype=torch.uint8, device=device) for _ in range(self.lanes)]
+        self.ws_lane = _workspaces(ws, self.lanes, device)
         self.ws = self.ws_lane[0]
         self._col, col = [], 0
         for l in self.layers:
             self._col.append(col)
             col += 2 if l.n_bias else 1
-        self.P = sum(t[2] for t in self.tensors)
         self.chunks_done = 0
         self._side = [torch.cuda.Stream(device=device) for _ in range(self.lanes - 1)] if self.lanes > 1 else []
         # layer -> lane: each call goes to the lane with the least work so far (a rough per-call cost is enough)
@@ -300,11 +326,7 @@ class PerLayerClipStep:
             self._lane_of.append(k)
 
     def begin(self):
-        for a in self.acc_w:
-            a.zero_()
-        for a in self.acc_b:
-            if a is not None:
-                a.zero_()
+        self.acc.zero_()
         self.chunks_done = 0
 
     def wgrad(self, li, X, dY, lane=0, stream=None):
@@ -341,13 +363,14 @@ class PerLayerClipStep:
         for w in self.ws_lane:
             b.check(b.dp_wgrad_check(w), "dp_wgrad_check")
 
-    def finish(self, seed=0, step=0):
-        """Noise uses the whole-gradient bound C (the per-tensor thresholds keep the sensitivity at C)."""
-        total, off = self.B * self.chunks_done, 0
-        for aw, ab in zip(self.acc_w, self.acc_b):
-            for a in (aw, ab):
-                if a is None:
-                    continue
-                b.check(b.dp_noise_average(a, a.numel(), off, self.sigma, self.C, total, seed, step, a), "dp_noise_average")
-                off += a.numel()
+    def finish(self, seed=0, step=0, total_batch=None):
+        """Noise uses the whole-gradient bound C (the per-tensor thresholds keep the sensitivity at C).
+        total_batch as for GlobalClipStep.finish."""
+        total = self.B * self.chunks_done if total_batch is None else int(total_batch)
+        if self.contiguous:
+            b.check(b.dp_noise_average(self.acc, self.P, 0, self.sigma, self.C, total, seed, step, self.acc), "dp_noise_average")
+            return self.acc_w, self.acc_b
+        views = [a for pair in zip(self.acc_w, self.acc_b) for a in pair if a is not None]
+        for a, off in zip(views, self.offsets):
+            b.check(b.dp_noise_average(a, a.numel(), off, self.sigma, self.C, total, seed, step, a), "dp_noise_average")
         return self.acc_w, self.acc_b

@@ -84,8 +84,9 @@ def gpu_layer(layer, inp, dtype, epilogue, impl=0, bias_separate=0, C_l=1.0, acc
     ws_bytes = b.dp_workspace_bytes(d, epilogue)
     assert ws_bytes > 0
     ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
-    ws.fill_(0xAB)                                   # the library must not rely on a zeroed workspace
+    ws.fill_(0xAB)                                   # beyond the header dp_workspace_init clears, nothing may be assumed
     guard = ws[ws_bytes:].clone()
+    b.check(b.dp_workspace_init(ws, ws_bytes), "dp_workspace_init")
     sq_ptr = sq.data_ptr() + 4 * sq_col
     st = b.dp_per_example_wgrad(d, X, dY, G_w, G_b, sq_ptr, sq_stride, epilogue, C_l, acc_w, acc_b, clip, ws, ws_bytes)
     if check_status:

@@ -90,6 +90,15 @@ def test_wgrad_rejects_bad_arguments_without_launching(b):
     assert b.dp_per_example_wgrad(forced, A, A, A, A, A, 1, 0, 1.0, None, None, None, A, 1 << 24, stream=0) == b.DP_ERR_UNSUPPORTED
 
 
+def test_workspace_init_rejects_bad_arguments(b):
+    A = 4096
+    assert b.dp_workspace_init(None, 1 << 20, stream=0) == b.DP_ERR_WORKSPACE
+    assert b.dp_workspace_init(A + 16, 1 << 20, stream=0) == b.DP_ERR_WORKSPACE     # not 256-byte aligned
+    assert b.dp_workspace_init(A, 1024, stream=0) == b.DP_ERR_WORKSPACE             # smaller than the header it clears
+    d = b.make_desc(b.DP_LAYER_DENSE, b.DP_F32, 1, 4, 4)
+    assert b.dp_workspace_bytes(d, b.DP_EPI_NORM_ONLY) >= 16384                     # every workspace holds the header
+
+
 def test_clip_rejects_bad_arguments(b):
     A = 4096
     P = [100, 7]

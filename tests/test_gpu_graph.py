@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2109_12191_b200 import synth
 from paper_2109_12191_b200.step import GlobalClipStep, PerLayerClipStep
-from gpu_util import dev_inputs, oracle_layer, rel_l2, TOL_NORM, TOL_ACC_BF16
+from gpu_util import dev_inputs, oracle_layer, rel_l2, TOL_NORM, TOL_ACC_BF16, TOL_ACC_F32
 
 pytestmark = pytest.mark.gpu
 
@@ -36,11 +36,73 @@ def test_graph_replay_equals_stream_launches():
     assert torch.equal(out, direct)
 
 
-@pytest.mark.parametrize("which", ["s0b0.c2", "s3b2.c3", "s2b0.gn2", "stem"])
-def test_per_layer_workload_full_size_layers(which):
-    """Layers of the per-layer ResNet-50 workload at full size (B = 32, threshold C/sqrt(161)), run from a replayed
-    CUDA graph as the benchmark does; the oracle checks every example's factor and the whole clipped sum."""
-    layer = next(l for l in synth.resnet50_gn_layers() if l.name == which)
+def test_small_cnn_step_as_benchmarked_matches_the_oracle():
+    """The composite the small-CNN benchmark times -- 256 examples, fp32 inputs taken as tf32, four streams, the
+    classifier's clipped sum recomputed instead of materialised, the whole step replayed from a CUDA graph --
+    against the oracle's privatisation step on the same inputs."""
+    cfg = synth.small_cnn()
+    layers, Bn = cfg["layers"], cfg["B"]
+    st = GlobalClipStep(layers, Bn, "tf32", cfg["C"], cfg["sigma"], lanes=4, recompute="auto")
+    assert st.recompute                                    # the classifier is not materialised
+    host = [synth.layer_inputs(l, Bn, "f32", 1, li, 0) for li, l in enumerate(layers)]
+    # N(0,1) inputs give whole-model norms near 3200, so every example would be clipped: spread them over the threshold
+    scale = (np.logspace(-0.8, 0.8, Bn) * cfg["C"] / 3200.0).astype(np.float32)
+    for h in host:
+        h["dY"] *= scale.reshape((Bn,) + (1,) * (h["dY"].ndim - 1))
+    ins = [dev_inputs(h, "f32") for h in host]
+
+    def step():
+        st.begin()
+        st.wgrad_all(ins)
+        st.clip_accumulate(inputs=ins)
+        return st.finish(seed=0, step=3)
+
+    step()                                                 # warm-up outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        out = step()
+    g.replay(); g.replay()
+    torch.cuda.synchronize()
+    st.check()
+    groups = []
+    for l, h in zip(layers, host):
+        dW, db = oracle_layer(l, h)
+        groups += [dW, db]
+    ref, ref_sq, ref_f = oracle.privatise([groups], cfg["C"], cfg["sigma"], "global", 0, 3)
+    ref_sq, ref_f = ref_sq[0], ref_f[0]                    # [B, L] squared norms and [B] factors of the one chunk
+    assert (ref_f == 1.0).any() and (ref_f < 1.0).any()
+    np.testing.assert_allclose(st.norms.cpu().numpy(), np.sqrt(ref_sq.sum(1)), rtol=TOL_NORM)
+    np.testing.assert_allclose(st.clip.cpu().numpy(), ref_f, rtol=TOL_NORM)
+    ref = np.concatenate(ref)
+    signal, _, _ = oracle.clipped_sum(groups, cfg["C"], "global")
+    signal = np.concatenate(signal) / Bn
+    got = out.cpu().numpy()
+    # the output is signal + noise; the noise is reproduced to 1e-5 of its scale, the signal to the tf32 bound
+    assert np.max(np.abs(got - ref)) <= 1e-5 * cfg["sigma"] * cfg["C"] / Bn + TOL_ACC_F32 * np.max(np.abs(signal))
+    assert rel_l2(got - (ref - signal), signal) <= TOL_ACC_F32
+
+
+def _distinct_resnet50_layers():
+    """One layer of every distinct shape of the per-layer ResNet-50 workload: 23 convolutions, the distinct
+    normalisation shapes and the classifier."""
+    seen, out = set(), []
+    for l in synth.resnet50_gn_layers():
+        key = (l.kind, l.Cin, l.Kout, l.R, l.stride, l.H)
+        if key not in seen:
+            seen.add(key)
+            out.append(l)
+    return out
+
+
+_DISTINCT = _distinct_resnet50_layers()
+
+
+@pytest.mark.parametrize("layer", _DISTINCT, ids=[f"{l.name}:{l.kind}{l.R}x{l.R}_{l.Cin}to{l.Kout}_s{l.stride}_at{l.H}" for l in _DISTINCT])
+def test_per_layer_workload_full_size_layers(layer):
+    """Every distinct layer shape of the per-layer ResNet-50 workload at full size (B = 32, threshold C/sqrt(161),
+    clip fused into the weight-gradient call), run from a replayed CUDA graph as the benchmark does; the oracle
+    checks every example's squared norm and factor and the whole clipped sum."""
     Bn, C_l = 32, 1.0 / math.sqrt(synth.RESNET50_GN_TENSORS)
     inp = synth.layer_inputs(layer, Bn, "bf16", 4, 7, 0)
     # norms of N(0,1) inputs are far above the threshold; scale so that they straddle it
@@ -59,17 +121,21 @@ def test_per_layer_workload_full_size_layers(which):
         st.wgrad(0, X, dYd)
     g.replay()
     torch.cuda.synchronize()
+    st.check()
     dW, db = oracle_layer(layer, inp)
     groups = [dW] + ([db] if db is not None else [])
     sq = st.sq.cpu().numpy()
+    factors = []
     for gi, grad in enumerate(groups):
         ref_sq = oracle.sqnorm(grad)
         np.testing.assert_allclose(sq[:, gi], ref_sq, rtol=TOL_NORM)
         f = oracle.clip_factor(ref_sq, C_l)
-        assert (f == 1.0).any() and (f < 1.0).any()
+        factors.append(f)
         got = (st.acc_w[0] if gi == 0 else st.acc_b[0]).cpu().numpy()
         # capturing records without running: the accumulator holds the single replay's contribution
         assert rel_l2(got, np.einsum("n,np->p", f, grad)) <= TOL_ACC_BF16
+    f = np.concatenate(factors)                            # (a classifier's bias gradient is small: never clipped)
+    assert (f == 1.0).any() and (f < 1.0).any()
 
 
 def test_layer_calls_spread_over_streams_give_the_same_bits():

@@ -41,6 +41,7 @@ def test_scaled_wgrad_matches_the_oracle(dtype, layer, impl):
         ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
         ws.fill_(0xAB)
         guard = ws[ws_bytes:].clone()
+        b.check(b.dp_workspace_init(ws, ws_bytes))
         table = torch.full((Bn, 3), float("nan"), device="cuda")          # factors at a stride, as in a [B, L] table
         table[:, 0] = dev(fw)
         table[:, 1] = dev(fb)
@@ -121,6 +122,7 @@ def test_argument_errors():
     d = make_desc(layer, 2, "f32", 0, 1)
     t = lambda *shape: torch.zeros(shape, device="cuda")
     ws = torch.empty(b.dp_workspace_bytes(d, b.DP_EPI_CLIP_ACCUM), dtype=torch.uint8, device="cuda")
+    b.check(b.dp_workspace_init(ws))
     ok = dict(desc=d, X=t(2, 16), dY=t(2, 4), factor_w=t(2), factor_b=None, factor_stride=1, acc_w=t(64), acc_b=t(4), workspace=ws)
     assert b.dp_per_example_wgrad_scaled(**ok) == b.DP_OK
     for bad in (dict(factor_w=None), dict(factor_stride=0), dict(acc_w=None), dict(acc_b=None), dict(X=None)):

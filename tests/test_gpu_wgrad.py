@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from paper_2109_12191_b200 import synth
-from gpu_util import (B, rel_l2, gpu_layer, oracle_layer, scaled_inputs, make_desc, TOL_NORM, TOL_FMA, TOL_ACC_BF16,
+from gpu_util import (B, rel_l2, gpu_layer, oracle_layer, scaled_inputs, make_desc, dev_inputs, TOL_NORM, TOL_FMA, TOL_ACC_BF16,
                       TOL_ACC_F32)
 
 pytestmark = pytest.mark.gpu
@@ -233,3 +233,32 @@ def test_tensor_core_rerun_is_bit_identical():
     b = gpu_layer(layer, inp, "bf16", STORE, TENSOR_CORE)
     np.testing.assert_array_equal(a["G_w"], b["G_w"])
     np.testing.assert_array_equal(a["sq"], b["sq"])
+
+
+def test_a_wait_that_runs_out_is_reported_and_later_calls_do_not_hide_it():
+    """Every wait of the tensor-core kernel is bounded.  With the poll limit at zero each role gives up before it
+    copies or multiplies anything, the kernel returns, and the workspace's status word says so; the word is sticky,
+    so a good call on the same workspace afterwards must not hide it, and reading it clears it."""
+    b = B()
+    layer = synth.conv(64, 64, 3, 1, 1, 14, name="c")
+    Bn = 4
+    inp = synth.layer_inputs(layer, Bn, "bf16", 955, 0)
+    X, dY = dev_inputs(inp, "bf16")
+    d = make_desc(layer, Bn, "bf16", b.DP_IMPL_TENSOR_CORE, 0)
+    ws = torch.empty(b.dp_workspace_bytes(d, b.DP_EPI_NORM_ONLY), dtype=torch.uint8, device="cuda")
+    b.check(b.dp_workspace_init(ws))
+    sq = torch.zeros((Bn, 1), device="cuda")
+    call = lambda: b.dp_per_example_wgrad(d, X, dY, None, None, sq, 1, b.DP_EPI_NORM_ONLY, 0.0, None, None, None, ws)
+    b.dp_debug_set_wait_polls(0)
+    try:
+        assert call() == b.DP_OK                           # the launch itself succeeds; the kernel gives up on the device
+        torch.cuda.synchronize()
+    finally:
+        b.dp_debug_set_wait_polls(-1)
+    assert call() == b.DP_OK                               # a good call on the same workspace ...
+    assert b.dp_wgrad_check(ws) == b.DP_ERR_TIMEOUT        # ... does not hide the earlier time-out
+    assert b.dp_wgrad_check(ws) == b.DP_OK                 # reported once, then the header starts over
+    assert call() == b.DP_OK
+    assert b.dp_wgrad_check(ws) == b.DP_OK
+    dW, _ = oracle_layer(layer, inp)
+    np.testing.assert_allclose(sq.cpu().numpy()[:, 0], oracle.sqnorm(dW), rtol=TOL_NORM)

@@ -10,7 +10,7 @@ import torch.multiprocessing as mp
 
 import oracle
 from paper_2109_12191_b200 import synth
-from paper_2109_12191_b200.sharding import shard_range, allreduce_accumulator
+from paper_2109_12191_b200.sharding import shard_range, allreduce_accumulator, global_batch
 
 SIZES, BN, CHUNKS, C, SIGMA = [300, 17], 4, 5, 0.3, 1.2
 
@@ -31,8 +31,10 @@ def _worker(rank, world, port, out):
         acc = [np.zeros(p) for p in SIZES]
     flat = torch.from_numpy(np.concatenate(acc))
     allreduce_accumulator(flat, dist)
-    res = oracle.noise_average(flat.numpy(), 0, SIGMA, C, BN * CHUNKS, 7, 3)
+    total = global_batch(BN * (hi - lo), dist)            # 5 chunks on 2 ranks: the shares are 3 and 2 chunks
+    res = oracle.noise_average(flat.numpy(), 0, SIGMA, C, total, 7, 3)
     out[rank] = res
+    out[f"total{rank}"] = total
     dist.barrier()
     dist.destroy_process_group()
 
@@ -58,5 +60,6 @@ def test_two_ranks_reproduce_the_single_process_step():
     ref, _, _ = oracle.privatise([_chunk(c) for c in range(CHUNKS)], C, SIGMA, "global", 7, 3)
     ref = np.concatenate(ref)
     for r in range(world):
+        assert out[f"total{r}"] == BN * CHUNKS             # uneven shares still add up to the step's batch
         np.testing.assert_allclose(out[r], ref, rtol=1e-12, atol=1e-15)
     np.testing.assert_array_equal(out[0], out[1])          # every rank holds the same noised average

@@ -5,13 +5,14 @@ memory pool that already owns the GPU, in callbacks that must not trigger cudaMa
 synchronisation, or in services that reserve all memory at start-up -- so they cannot provide the
 workspace dp_clip_accumulate asks for.  This entry point works in a fixed array inside the library.
 The test drives it through the C ABI twice in a row (the array keeps the first call's leftovers) and
-holds it to the results of the workspace-taking entry point.  The file sorts last so that a run that
+holds it to the results of the workspace-taking entry point and of the CPU oracle.  The file sorts last so that a run that
 stops at the first failure has already executed every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2109_12191_b200 import synth
 from gpu_util import B, dev, rel_l2, TOL_NORM, TOL_FMA
 
@@ -56,6 +57,12 @@ def test_static_scratch_variant_matches_the_workspace_variant_on_two_calls_in_a_
         np.testing.assert_allclose(clip_st, clip_ws, rtol=TOL_NORM)
         assert (clip_ws == 1.0).any() and (clip_ws < 1.0).any()
         for a, r in zip(acc_st, acc_ws):
+            assert rel_l2(a, r) <= TOL_FMA
+        ref_acc, ref_sq, ref_f = oracle.clipped_sum(groups, C, mode_name)
+        ref_norm = np.sqrt(ref_sq) if mode_name == "per_layer" else np.sqrt(ref_sq.sum(1))
+        np.testing.assert_allclose(norms_st, ref_norm, rtol=TOL_NORM)
+        np.testing.assert_allclose(clip_st, ref_f, rtol=TOL_NORM)
+        for a, r in zip(acc_st, ref_acc):
             assert rel_l2(a, r) <= TOL_FMA
 
 
