@@ -375,6 +375,8 @@ class PerLayer:
         self.cfg = self.config(synth)
         self.layers, self.B, self.G = self.cfg["layers"], self.cfg["B"], self.cfg["G"]
         self.lanes = int(os.environ.get("DP_BENCH_LANES", "4"))
+        self.sm_target = int(os.environ.get("DP_BENCH_SM_TARGET", "0"))
+        binding.check(binding.dp_set_sm_target(self.sm_target))
         self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"], lanes=self.lanes)
         self.examples_per_step = self.B * self.G
         g = torch.Generator(device="cuda"); g.manual_seed(4000 + rank)
@@ -813,8 +815,10 @@ def sweep(env, which, layer_sel, reps):
         layers = synth.resnet50_gn_layers()
     if which == "sweep_all_r101":
         layers = synth.resnet101_gn_layers()
-    if layer_sel:
-        layers = [layers[int(i)] for i in layer_sel.split(",")]
+    if layer_sel:                                          # indices or layer names
+        by_name = {l.name: l for l in layers}
+        layers = [by_name[i] if i in by_name else layers[int(i)] for i in layer_sel.split(",")]
+    b.check(b.dp_set_sm_target(int(os.environ.get("DP_BENCH_SM_TARGET", "0"))))
     Bn, dtype = 32, "bf16"
     flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")
     rows = []

@@ -95,6 +95,16 @@ DP_API int dp_layer_groups(const dp_layer_desc *desc);
  * for some paths, per-example bias gradients or clip factors. */
 DP_API size_t dp_workspace_bytes(const dp_layer_desc *desc, int epilogue);
 
+/* How many SMs one tensor-core launch of dp_per_example_wgrad(_scaled) should spread over (0 = all, the default).
+ * A chunk of few examples gives one layer only a few microseconds of work for a whole GPU, most of which a launch then
+ * spends starting and draining; a caller that runs several layer calls side by side on different streams gets more
+ * out of the GPU when each call takes a share of the SMs and keeps them busy for longer.  The value is process-wide,
+ * applies to launches made afterwards, and changes nothing but speed: results do not depend on it bit for bit only
+ * within one setting (the fused clipped sum splits the batch over thread blocks by it), so keep it fixed for a run that
+ * must be reproducible.  Workspace sizes depend on it: query dp_workspace_bytes after setting it.
+ * Errors: DP_ERR_INVALID_ARG for a negative value. */
+DP_API dp_status dp_set_sm_target(int sms);
+
 /* Prepares a freshly allocated (or otherwise overwritten) workspace of dp_per_example_wgrad /
  * dp_per_example_wgrad_scaled: clears its header, i.e. the status word dp_wgrad_check reports and the ticket
  * counters with which the last thread block to finish an example finds out that it is the last.  Call it once
@@ -320,6 +330,10 @@ DP_API dp_status dp_debug_noise_z(float *z, long long count, long long first_ind
  * sticky: kernels only ever set it, later calls do not hide it.  Reporting a time-out clears it and re-initialises
  * the workspace header, as dp_workspace_init does. */
 DP_API dp_status dp_wgrad_check(void *workspace, void *cuda_stream);
+
+/* Test hook: 0 makes DP_EPI_CLIP_ACCUM always run its two-pass form (norm pass, then clipped sum), 1 (the default)
+ * lets layers whose per-example gradient fits one thread-block cluster run the single-pass form.  Process-wide. */
+DP_API void dp_debug_set_single_pass(int on);
 
 /* Test hook: the number of polls (each about a microsecond) after which the bounded waits of the tensor-core kernel
  * give up; 0 makes every wait give up before anything is copied or multiplied, a negative value restores the

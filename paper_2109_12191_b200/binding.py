@@ -31,7 +31,7 @@ EXPORTS = ["dp_layer_groups", "dp_workspace_bytes", "dp_per_example_wgrad", "dp_
            "dp_clip_static_scratch_bytes", "dp_noise_average_sgd", "dp_clip_accumulate_noised",
            "dp_debug_example_noise_z", "dp_clip_accumulate_grouped", "dp_clip_accumulate_micro",
            "dp_per_example_wgrad_scaled", "dp_clip_factors", "dp_scale_accumulate", "dp_workspace_init",
-           "dp_debug_set_wait_polls"]
+           "dp_debug_set_wait_polls", "dp_set_sm_target", "dp_debug_set_single_pass"]
 
 
 class dp_layer_desc(ctypes.Structure):
@@ -90,6 +90,8 @@ _lib.dp_debug_noise_z.argtypes = [_vp, _ll, _ll, _ull, _ull, _vp]; _lib.dp_debug
 _lib.dp_wgrad_check.argtypes = [_vp, _vp]; _lib.dp_wgrad_check.restype = _i
 _lib.dp_workspace_init.argtypes = [_vp, _sz, _vp]; _lib.dp_workspace_init.restype = _i
 _lib.dp_debug_set_wait_polls.argtypes = [_ll]; _lib.dp_debug_set_wait_polls.restype = None
+_lib.dp_set_sm_target.argtypes = [_i]; _lib.dp_set_sm_target.restype = _i
+_lib.dp_debug_set_single_pass.argtypes = [_i]; _lib.dp_debug_set_single_pass.restype = None
 _lib.dp_status_string.argtypes = [_i]; _lib.dp_status_string.restype = ctypes.c_char_p
 _lib.dp_last_cuda_error.argtypes = []; _lib.dp_last_cuda_error.restype = ctypes.c_char_p
 _lib.dp_debug_launch_count.argtypes = []; _lib.dp_debug_launch_count.restype = _ull
@@ -257,6 +259,14 @@ def dp_workspace_init(workspace, workspace_bytes=None, stream=None):
     if workspace_bytes is None:
         workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else _nbytes(workspace)
     return _lib.dp_workspace_init(_ptr(workspace), workspace_bytes, _stream(stream))
+
+
+def dp_set_sm_target(sms):
+    return _lib.dp_set_sm_target(sms)
+
+
+def dp_debug_set_single_pass(on):
+    _lib.dp_debug_set_single_pass(int(on))
 
 
 def dp_debug_set_wait_polls(polls):

@@ -15,6 +15,10 @@ void note_error(const char *message);
 
 // Number of SMs of the current device (cached per device; 148 if the query fails).
 int sm_count();
+// Number of SMs one tensor-core launch should spread over: dp_set_sm_target()'s value, or all of them.
+int sm_target();
+// false while dp_debug_set_single_pass(0) holds: the fused clipped sum then always runs its two-pass form
+bool single_pass_enabled();
 
 // Every dp_per_example_wgrad workspace starts with this header, cleared by dp_workspace_init: the sticky status word
 // at byte 0 and, from byte 256, the ticket counters with which the last block to finish a unit of work finds out

@@ -21,6 +21,15 @@ dp_status cuda_fail(cudaError_t e, const char *where) {
 
 void note_error(const char *message) { snprintf(g_last_error, sizeof(g_last_error), "%s", message); }
 
+static std::atomic<int> g_sm_target{0};
+static std::atomic<int> g_single_pass{1};
+bool single_pass_enabled() { return g_single_pass.load(std::memory_order_relaxed) != 0; }
+
+int sm_target() {
+    const int all = sm_count(), t = g_sm_target.load(std::memory_order_relaxed);
+    return (t > 0 && t < all) ? t : all;
+}
+
 int sm_count() {
     static std::atomic<int> cached[64];
     int dev = 0;
@@ -187,6 +196,12 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             if (rc != DP_OK) return rc;
             return launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 0, 0.f, factor, nullptr, st);
         }
+        if (pl.use_tc && !d->has_bias && single_pass_enabled() && tc_clip_single_pass(d->dtype, g)) {
+            // per-layer clipping from ONE contraction: norm, factor and scaled sum come from the same accumulators
+            const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
+            return launch_conv_clip1(d->dtype, X, dY, g, partial, pl.slots, ic, acc_w, ws + pl.tc_off,
+                                     reinterpret_cast<int *>(ws + pl.status_off), st);
+        }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
         else rc = launch_conv_fma(storage_type(d), DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
@@ -298,7 +313,7 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
 }
 
 extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n) {
-    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 2 || !out || n <= 0) return 0;
+    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 3 || !out || n <= 0) return 0;   // 3: the single-pass form of the fused clip
     return tc_describe_plan(desc->dtype, geom_of(desc), epilogue, out, n);
 }
 
@@ -320,6 +335,14 @@ extern "C" dp_status dp_wgrad_check(void *workspace, void *cuda_stream) {
     DP_CUDA_TRY(cudaStreamSynchronize(st));
     return DP_ERR_TIMEOUT;
 }
+
+extern "C" dp_status dp_set_sm_target(int sms) {
+    if (sms < 0) return DP_ERR_INVALID_ARG;
+    dp::g_sm_target.store(sms, std::memory_order_relaxed);
+    return DP_OK;
+}
+
+extern "C" void dp_debug_set_single_pass(int on) { dp::g_single_pass.store(on ? 1 : 0, std::memory_order_relaxed); }
 
 extern "C" void dp_debug_set_wait_polls(long long polls) {
     set_wait_polls(polls < 0 ? default_wait_polls() : (uint32_t)(polls > 0xffffffffll ? 0xffffffffll : polls));

@@ -543,14 +543,23 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         __syncthreads();
         if (last_cta) {
             __threadfence();
-            const int nwarps = blockDim.x >> 5;
-            for (int n = warp; n < p.B; n += nwarps) {
-                const float *pn = p.partial + (long long)n * p.slots;
+            // eight lanes per example (slot i goes to lane i % 8, the eight sums are added by a butterfly), four
+            // examples per warp and trip: the walk is a chain of L2 round trips, so many examples go side by side
+            const int groups = (int)(blockDim.x >> 3), group = (int)(threadIdx.x >> 3), sub = lane & 7;
+            for (int n0 = 0; n0 < p.B; n0 += groups) {     // uniform trip count: the shuffles below need whole warps
+                const int n = n0 + group;
                 double sw = 0.0, sb = 0.0;
-                for (int i = lane; i < p.w_slots; i += 32) sw += (double)__ldcg(pn + i);
-                for (int i = p.w_slots + lane; i < p.slots; i += 32) sb += (double)__ldcg(pn + i);
-                sw = warp_sum(sw); sb = warp_sum(sb);
-                if (lane == 0) {
+                if (n < p.B) {
+                    const float *pn = p.partial + (long long)n * p.slots;
+                    for (int i = sub; i < p.w_slots; i += 8) sw += (double)__ldcg(pn + i);
+                    for (int i = p.w_slots + sub; i < p.slots; i += 8) sb += (double)__ldcg(pn + i);
+                }
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) {
+                    sw += __shfl_xor_sync(0xffffffffu, sw, o);
+                    sb += __shfl_xor_sync(0xffffffffu, sb, o);
+                }
+                if (n < p.B && sub == 0) {
                     if (p.separate) { p.sqnorm[n * p.sq_stride] = (float)sw; p.sqnorm[n * p.sq_stride + 1] = (float)sb; }
                     else p.sqnorm[n * p.sq_stride] = (float)(sw + sb);
                 }
@@ -564,6 +573,298 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         __nanosleep(200000);
         __syncthreads();
     }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
+
+// ----------------------------------------------------------------------------- single-pass fused clip (bf16)
+// Per-layer clipping needs an example's whole squared norm before any entry of its gradient can be scaled, so the
+// kernel above runs every contraction twice (a norm pass, then the clipped sum).  Here each contraction runs once:
+// a thread-block cluster owns ALL tiles of one example's gradient of this layer, one tile per CTA, kept in the CTA's
+// tensor memory.  Every CTA square-sums its tile, the CTAs exchange their partial sums through distributed shared
+// memory (plain remote stores plus a remote mbarrier arrival; every CTA loads its own operands, nothing is
+// multicast), every CTA then knows the example's norm and factor, scales its tile into a running sum held in
+// registers, and moves on to the cluster's next example while the tensor core already fills the other accumulator
+// buffer.  Clusters split the batch; with more than one cluster the running sums leave as partial sums, folded in
+// cluster order by the launch that follows.
+//
+// Roles (384 threads): warp 0 issues the TMA loads of the A slabs, warp 2 those of the B slabs, warp 1 allocates tensor
+// memory and issues the MMAs, warp 3 idles; warps 4-11 are the epilogue: warp w reads TMEM lanes 32*(w%4).. and the
+// 128-column half (w-4)/4 of the tile, so a thread holds 128 running sums.  The first warpgroup gives registers up
+// (setmaxnreg) and the epilogue warpgroups take them: 128*56 + 256*224 = 384*168, the launch's allocation.
+constexpr int kClipThreads = 384;
+constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
+static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
+constexpr int kMaxCluster = 8;
+
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                 "selp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t polls) {
+    for (uint32_t it = 0; it < polls; ++it) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((it & 63u) == 63u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__global__ void __launch_bounds__(kClipThreads, 1)
+conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2], norm_bar[2];
+    __shared__ float norm_part[2][kMaxCluster][8];      // [example parity][source CTA][source epilogue warp]
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t tiles_u32 = smem_u32(tiles);
+    const int cs = p.m_tiles * p.n_tiles;                 // cluster size = tiles of one example's gradient
+    const int rank = (int)cluster_rank();
+    const int mt = rank / p.n_tiles, nt = rank - mt * p.n_tiles;
+    const int split = (int)blockIdx.x / cs;
+    const int n_lo = split * p.per_split, n_hi = min(p.B, n_lo + p.per_split);
+
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 2); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 8);
+            mbar_init(smem_u32(&norm_bar[b]), (uint32_t)(cs * 8));
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                   // every CTA's barriers exist before anyone arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int *abort_p = &abort_flag;
+
+    const int slab_bytes = p.Kt * kRowBytes;
+    const int a_slabs_tile = 128 / p.slab_ch, b_slabs_tile = p.NT / p.slab_ch;
+    const int a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - mt * a_slabs_tile);
+    const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
+
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClipRegsControl));
+        if (warp == 0 || warp == 2) {
+            // ------------------------------------------------------------ TMA producers (A slabs / B slabs)
+            const bool is_a = warp == 0;
+            const bool active = is_a ? (lane < a_slabs) : (lane < b_slabs);
+            const bool is_x = is_a ? (p.a_is_x != 0) : (p.a_is_x == 0);
+            const int slab = (is_a ? mt * a_slabs_tile : nt * b_slabs_tile) + lane;
+            int c0, dw = 0, dh = 0, mul = 1;
+            if (is_x) {
+                const int j0 = slab * p.slab_ch;
+                const int tap = j0 / p.Cin;
+                c0 = j0 - tap * p.Cin;
+                const int r = tap / p.S;
+                dw = (tap - r * p.S) - p.pad;
+                dh = r - p.pad;
+                mul = p.stride;
+            } else {
+                c0 = slab * p.slab_ch;
+            }
+            const CUtensorMap *map = is_x ? &tmX : &tmY;
+            const uint32_t dst_off = (is_a ? 0u : (uint32_t)p.a_bytes) + (uint32_t)(lane * slab_bytes);
+            const uint32_t tx_bytes = (uint32_t)((is_a ? a_slabs : b_slabs) * slab_bytes);
+            int stage = 0; uint32_t phase = 0;
+            bool live = true;
+            for (int n = n_lo; n < n_hi && live; ++n) {
+                int ow0 = 0, oh0 = 0, tw = 0;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    bool ok = true;
+                    if (lane == 0) {
+                        ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p, p.wait_polls);
+                        if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { live = false; break; }
+                    if (active)
+                        tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
+                                    ow0 * mul + dw, oh0 * mul + dh, n);
+                    if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        } else if (warp == 1 && lane == 0) {
+            // ------------------------------------------------------------ MMA issuer (one lane)
+            int stage = 0; uint32_t phase = 0, acc_phase = 0;
+            int buf = 0;
+            bool live = true;
+            const uint64_t desc_base = operand_desc_base<false>((uint32_t)slab_bytes);
+            const uint32_t desc_lo = (uint32_t)desc_base, desc_hi32 = (uint32_t)(desc_base >> 32);
+            const int ksteps = p.Kt / p.krows;
+            constexpr uint32_t kadvance = (uint32_t)(16 * kRowBytes) >> 4;
+            const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, 1u);
+            for (int n = n_lo; n < n_hi && live; ++n) {
+                if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p, p.wait_polls)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                uint32_t accumulate = 0;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p, p.wait_polls)) { live = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
+                    uint32_t ad = desc_lo | ((a_src & 0x3FFFFu) >> 4);
+                    uint32_t bd = desc_lo | (((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
+#pragma unroll 4
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        umma<false>(d_tmem, ad, bd, desc_hi32, idesc, accumulate);
+                        accumulate = 1;
+                        ad += kadvance; bd += kadvance;
+                    }
+                    umma_commit(smem_u32(&empty_bar[stage]));
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (!live) break;
+                umma_commit(smem_u32(&tmem_full[buf]));
+                acc_phase ^= 1u << buf;
+                buf ^= 1;
+            }
+        }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kClipRegsEpilogue));
+        // ---------------------------------------------------------------- epilogue (8 warps)
+        const int e = warp - 4, q = e & 3, half = e >> 2;
+        const int row = q * 32 + lane;
+        const int a_rows = min(128, p.a_ext - mt * 128);
+        const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
+        const int my_cols = max(0, min(128, n_cols - half * 128));     // columns of this warp's half that exist
+        const int a_idx = mt * 128 + row;
+        const bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
+        float run[128];
+#pragma unroll
+        for (int i = 0; i < 128; ++i) run[i] = 0.f;
+        uint32_t full_phase = 0;
+        bool live = true;
+        int buf = 0;
+        for (int n = n_lo; n < n_hi; ++n) {
+            const int par = (n - n_lo) & 1;
+            const uint32_t use_parity = (uint32_t)(((n - n_lo) >> 1) & 1);
+            const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
+            if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+            full_phase ^= 1u << buf;
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
+            // pass 1: this warp's share of the example's squared norm
+            float sq = 0.f;
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                if (c4 * 32 < my_cols) {
+                    uint32_t v[32];
+                    tmem_ld32(t_addr + (uint32_t)(c4 * 32), v);
+                    if (row_ok) {      // (columns past the real ones of an unfolded thin layer hold exact zeros)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq = fmaf(f, f, sq); }
+                    }
+                }
+            }
+            sq = warp_sum(sq);
+            if (lane == 0) {
+                const uint32_t slot = smem_u32(&norm_part[par][rank][e]);
+                const uint32_t bar = smem_u32(&norm_bar[par]);
+                for (int r = 0; r < cs; ++r) {
+                    st_cluster_f32(map_to_cta(slot, (uint32_t)r), sq);
+                    mbar_arrive_remote(map_to_cta(bar, (uint32_t)r));
+                }
+            }
+            const bool all_in = mbar_wait_cluster(smem_u32(&norm_bar[par]), use_parity, abort_p, p.wait_polls);
+            if (!__all_sync(0xffffffffu, all_in)) { live = false; break; }
+            // the same order in every warp of every CTA: all of them apply the identical factor
+            double sn = 0.0;
+            for (int r = 0; r < cs; ++r)
+#pragma unroll
+                for (int w = 0; w < 8; ++w) sn += (double)norm_part[par][r][w];
+            const float f = clip_factor(sn, p.C_l);
+            if (rank == 0 && e == 0 && lane == 0) {
+                p.sqnorm[n * p.sq_stride] = (float)sn;
+                if (p.clip_out) p.clip_out[n] = f;
+            }
+            // pass 2: scale the tile into the running sum
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                if (c4 * 32 < my_cols) {
+                    uint32_t v[32];
+                    tmem_ld32(t_addr + (uint32_t)(c4 * 32), v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) run[c4 * 32 + i] = fmaf(f, __uint_as_float(v[i]), run[c4 * 32 + i]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            buf ^= 1;
+        }
+        if (live && row_ok) {
+            // one owner per output element: add straight into the accumulator, or leave a partial sum for the fold
+            const bool add = p.splits == 1;
+            float *base = p.sum_out + (add ? 0ll : (long long)split * p.Kout * p.Ng);
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                if (c4 * 32 < my_cols) {
+                    const int b_idx = nt * p.NT + half * 128 + c4 * 32;
+                    if (p.a_is_x) {
+                        float *dst = base + (long long)b_idx * p.Ng + a_idx;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            float *el = dst + (long long)i * p.Ng;
+                            const float r = run[c4 * 32 + i];
+                            *el = add ? *el + r : r;
+                        }
+                    } else if (!p.n_pad_cols) {
+                        float4 *dst = reinterpret_cast<float4 *>(base + (long long)a_idx * p.Ng + b_idx);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            float4 r = make_float4(run[c4 * 32 + 4 * i], run[c4 * 32 + 4 * i + 1], run[c4 * 32 + 4 * i + 2], run[c4 * 32 + 4 * i + 3]);
+                            if (add) { const float4 o = dst[i]; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
+                            dst[i] = r;
+                        }
+                    } else {
+                        float *dst = base + (long long)a_idx * p.Ng + b_idx;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (b_idx + i < p.Ng) dst[i] = add ? dst[i] + run[c4 * 32 + i] : run[c4 * 32 + i];
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag) {
+        if (threadIdx.x == 0) { *p.status = DP_ERR_TIMEOUT; __threadfence(); }
+        __nanosleep(200000);
+        __syncthreads();
+    }
+    cluster_sync_all();                                   // nobody leaves while a peer may still write to its shared memory
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
 }
 
@@ -730,12 +1031,21 @@ static double step_cycles(int dtype, int n_cols, double a_slabs_loaded, double b
 
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode);
 
+// single-pass clipped sum: how many clusters share the batch and how many examples each walks through
+static void cluster_split(int B, int cluster_size, int &splits, int &per_split) {
+    int want = sm_target() / cluster_size;
+    if (want < 1) want = 1;
+    if (want > B) want = B;
+    per_split = (B + want - 1) / want;
+    splits = (B + per_split - 1) / per_split;
+}
+
 // The tiling search is pure; its results are memoised per layer geometry (host side only).
 // mode: 0 gradients are stored, 1 norms only, 2 clipped sum (running sum in registers: at most 128 columns per tile)
 static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
     static std::mutex mu;
-    static std::map<std::array<int, 11>, TcPlan> memo;
-    const std::array<int, 11> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, mode};
+    static std::map<std::array<int, 12>, TcPlan> memo;
+    const std::array<int, 12> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, mode, sm_target()};
     std::lock_guard<std::mutex> lock(mu);
     auto it = memo.find(key);
     if (it != memo.end()) return it->second;
@@ -746,6 +1056,8 @@ static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
 
 // max_nt = 128 plans the clipped-sum mode: its running sum lives in registers (128 columns per thread) and the
 // work items are (example range, tile) pairs, so the wave count no longer depends on the batch size
+// mode 3 plans the single-pass clipped sum: all tiles of an example in one cluster (at most kMaxCluster of them), the
+// clusters share the batch, and what is minimised is SM time (clusters x CTAs x time), not the time of one launch
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
     const int max_nt = (mode == 2) ? 128 : 256;
     TcPlan best; best.ok = false;
@@ -753,7 +1065,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
     const int krows = (dtype == DP_BF16) ? 16 : 8;
     if (g.Cin % slab_ch || g.Kout % slab_ch) return best;
     if (g.stride > 8 || g.K < 1 || g.OH > 65535) return best;
-    const int sms = sm_count();
+    const int sms = sm_target();
     const int a_slabs_tile = 128 / slab_ch;
     const int copies = (dtype == DP_F32) ? 2 : 1;       // split tf32 keeps a hi and a lo copy of every stage
     double best_cost = 1e300;
@@ -766,15 +1078,24 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             const int slabs = a_slabs_tile + NT / slab_ch;
             const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
             if (total_tiles > 0x7fffffffLL) continue;
+            if (mode == 3 && m_tiles * n_tiles > kMaxCluster) continue;
             // per-CTA share of (example, tile) units: whole waves of tiles, or in clipped-sum mode an even share of the examples
-            const double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
-                                             : std::max(1.0, (double)total_tiles / sms);
+            double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
+                                       : std::max(1.0, (double)total_tiles / sms);
+            double sm_share = 1.0;
+            if (mode == 3) {
+                int splits, per;
+                cluster_split(g.B, m_tiles * n_tiles, splits, per);
+                waves = per;                                       // examples a cluster walks through
+                sm_share = (double)splits * m_tiles * n_tiles;      // SMs the launch holds meanwhile
+            }
             const double a_loaded = (double)(a_ext / slab_ch) / m_tiles, b_loaded = (double)(b_ext / slab_ch) / n_tiles;
             const double step = step_cycles(dtype, NT, a_loaded, b_loaded);
             // the epilogue of a tile overlaps the main loop of the next; what it costs depends on what it does with
             // the 128 x NT accumulator: stores run at about 16 B/clk per SM when lanes write consecutive addresses
             // (rows of D are gradient columns) and about 7 B/clk otherwise; reading TMEM alone is cheap
-            const double epilogue = (mode == 0) ? 128.0 * NT * 4.0 / (a_is_x ? 16.0 : 7.0) : (mode == 1 ? 6.0 * NT : 10.0 * NT);
+            const double epilogue = (mode == 0) ? 128.0 * NT * 4.0 / (a_is_x ? 16.0 : 7.0)
+                                  : (mode == 1 ? 6.0 * NT : (mode == 2 ? 10.0 * NT : 10.0 * std::min(NT, 128) + 600.0));
             // a pixel tile may reach past the output plane (its rows there are zero-filled by TMA and add nothing):
             // a 7 x 7 plane is one 8 x 8 tile of 64 reduction rows instead of four 4 x 4 tiles of 16
             const int oh_max = std::min((g.OH + 7) / 8 * 8, 256 / g.stride), ow_max = std::min((g.OW + 7) / 8 * 8, 256 / g.stride);
@@ -797,7 +1118,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
                         stage_cost = std::max(stage_cost, 0.5 * (1000.0 + (a_loaded + b_loaded) * Kt * 2.5));
                     double mainloop = stage_cost * tw * th;
                     if (stages < 3) mainloop *= 1.15;
-                    const double cost = (std::max(mainloop, epilogue) + 300.0) * waves;
+                    const double cost = ((std::max(mainloop, epilogue) + 300.0) * waves + (mode == 3 ? 4000.0 : 0.0)) * sm_share;
                     if (cost < best_cost) {
                         best_cost = cost;
                         best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
@@ -820,10 +1141,29 @@ bool tc_eligible(int dtype, const ConvGeom &g0, int epilogue) {
     return epilogue != DP_EPI_CLIP_ACCUM || make_plan(dtype, pr.eff, 2).ok;
 }
 
+// The single-pass kernel's register split only adds up when the launch allocates kClipRegsLaunch registers a thread.
+static bool clip1_registers_ok() {
+    static int ok = -1;
+    if (ok < 0) {
+        cudaFuncAttributes attr;
+        ok = (cudaFuncGetAttributes(&attr, conv_wgrad_clip1_kernel) == cudaSuccess && attr.numRegs == kClipRegsLaunch) ? 1 : 0;
+        if (!ok) (void)cudaGetLastError();
+    }
+    return ok == 1;
+}
+
+// true when the fused clipped sum of this layer runs as ONE contraction (bf16 inputs, the example's gradient fits the
+// tensor memory of one cluster)
+static bool clip1_plan(int dtype, const ConvGeom &eff, TcPlan &pl) {
+    if (dtype != DP_BF16) return false;
+    pl = make_plan(dtype, eff, 3);
+    return pl.ok;
+}
+
 // clipped-sum mode: how many example ranges each tile is cut into so that every SM has an item
 static void clip_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &per_split) {
     const int tiles = pl.m_tiles * pl.n_tiles;
-    int want = sm_count() / tiles;
+    int want = sm_target() / tiles;
     if (want < 1) want = 1;
     if (want > g.B) want = g.B;
     per_split = (g.B + want - 1) / want;
@@ -852,6 +1192,12 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
         if (!pl.ok) return 0;
         int splits, per;
         clip_split(pr.eff, pl, splits, per);
+        TcPlan one;
+        if (clip1_plan(dtype, pr.eff, one)) {              // room for either form: the single pass may be unavailable at run time
+            int s1, p1;
+            cluster_split(pr.eff.B, one.m_tiles * one.n_tiles, s1, p1);
+            splits = std::max(splits, s1);
+        }
         if (splits > 1) bytes += sizeof(float) * (size_t)splits * g0.M * g0.N;
     }
     return bytes;
@@ -966,7 +1312,7 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
         if (attr_err == cudaSuccess) attr_err = cudaFuncSetAttribute(conv_wgrad_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
-    const unsigned grid = (unsigned)std::min(p.total_tiles, sm_count());
+    const unsigned grid = (unsigned)std::min(p.total_tiles, sm_target());
     if (dtype == DP_BF16) {
         if (clip) conv_wgrad_tc_kernel<false, true><<<grid, 224, pl.smem, stream>>>(tmX, tmY, p);
         else conv_wgrad_tc_kernel<false, false><<<grid, 224, pl.smem, stream>>>(tmX, tmY, p);
@@ -976,6 +1322,71 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     }
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
     if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g0.M * g0.N, acc_w, stream);
+    return DP_OK;
+}
+
+bool tc_clip_single_pass(int dtype, const ConvGeom &g0) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    TcPlan pl;
+    return pr.ok && encode_fn() && clip1_plan(dtype, pr.eff, pl) && clip1_registers_ok();
+}
+
+dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const ConvGeom &g0, float *partial, int slots,
+                            const TcInlineClip &clipinfo, float *acc_w, void *tc_workspace, int *status, cudaStream_t stream) {
+    (void)partial; (void)slots;
+    const TcProblem pr = tc_problem(dtype, g0);
+    TcPlan pl;
+    if (!pr.ok || !encode_fn() || !clip1_plan(dtype, pr.eff, pl) || !clip1_registers_ok()) return DP_ERR_UNSUPPORTED;
+    const ConvGeom &g = pr.eff;
+    char *ws_bytes = static_cast<char *>(tc_workspace);
+    if (pr.unfold) {
+        const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * 2;
+        DP_MAX_SHARED_CARVEOUT((unfold_rows_kernel<__nv_bfloat16, 8>));
+        if (row_smem <= 40 * 1024 && g0.B <= 65535) {
+            unfold_rows_kernel<__nv_bfloat16, 8><<<dim3(g0.OH, g0.B), 256, row_smem, stream>>>(
+                static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad);
+        } else {
+            const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / 8);
+            unfold_small_channels_kernel<__nv_bfloat16, 8><<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+                static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad, total);
+        }
+        DP_LAUNCH_CHECK("unfold_small_channels_kernel");
+        X = ws_bytes;
+    }
+    float *part_ws = reinterpret_cast<float *>(ws_bytes + unfold_bytes(dtype, g0, pr));
+    CUtensorMap tmX, tmY;
+    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    TcParams p = {};
+    p.B = g.B; p.Kout = g.Kout; p.Ng = g0.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.n_pad_cols = (g.N != g0.N) ? 1 : 0;
+    p.slab_ch = 64; p.krows = 16;
+    p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
+    p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
+    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
+    p.mode = 3; p.status = status;
+    p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
+    p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
+    const int cs = pl.m_tiles * pl.n_tiles;
+    cluster_split(g.B, cs, p.splits, p.per_split);
+    p.sum_out = p.splits > 1 ? part_ws : acc_w;
+    p.total_tiles = p.splits * cs;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(conv_wgrad_clip1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.splits * cs)); cfg.blockDim = dim3(kClipThreads); cfg.dynamicSmemBytes = pl.smem; cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, conv_wgrad_clip1_kernel, tmX, tmY, p);
+    if (le != cudaSuccess) return cuda_fail(le, "conv_wgrad_clip1_kernel");
+    DP_LAUNCH_CHECK("conv_wgrad_clip1_kernel");
+    if (p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g0.M * g0.N, acc_w, stream);
     return DP_OK;
 }
 

@@ -28,6 +28,13 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
                          int *status, cudaStream_t stream, bool second_pass = false,
                          const TcInlineClip *inline_clip = nullptr, const TcPublish *publish = nullptr);
 
+// The fused clipped sum of a bf16 layer whose per-example gradient fits the tensor memory of one thread-block cluster
+// runs as ONE contraction (norm, factor and scaled sum from the same accumulators); tc_clip_single_pass says whether
+// this layer qualifies.  Writes sqnorm / clip_out like a CLIP_ACCUM launch with TcInlineClip; layers without bias only.
+bool tc_clip_single_pass(int dtype, const ConvGeom &g);
+dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const ConvGeom &g, float *partial, int slots,
+                            const TcInlineClip &clipinfo, float *acc_w, void *tc_workspace, int *status, cudaStream_t stream);
+
 // Test hook: the number of polls after which a bounded wait of the kernel gives up (0 makes every wait give up at once).
 void set_wait_polls(uint32_t polls);
 uint32_t default_wait_polls();

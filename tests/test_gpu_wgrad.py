@@ -55,6 +55,17 @@ def check_layer(layer, Bn, dtype, impl, key, bias_separate=0, spread=False, clip
     if db is not None:
         ref_acc_b = np.einsum("n,np->p", f[:, groups - 1], db)
         assert rel_l2(out_c["acc_b"], ref_acc_b) <= tol_for(out_c, dtype)
+    if out_c["uses_tc"] and db is None:
+        # the tensor-core clip has a single-pass form (taken when the layer qualifies) and a two-pass form: check the other too
+        b = B()
+        b.dp_debug_set_single_pass(0)
+        try:
+            out_2 = gpu_layer(layer, inp, dtype, CLIP, clip_impl if clip_impl is not None else impl, bias_separate, C_l=C_l)
+        finally:
+            b.dp_debug_set_single_pass(1)
+        np.testing.assert_allclose(out_2["clip"], f, rtol=TOL_NORM)
+        np.testing.assert_allclose(out_2["sq"], ref_sq, rtol=TOL_NORM)
+        assert rel_l2(out_2["acc_w"], ref_acc_w) <= tol_for(out_2, dtype)
     return out
 
 
@@ -262,3 +273,21 @@ def test_a_wait_that_runs_out_is_reported_and_later_calls_do_not_hide_it():
     assert b.dp_wgrad_check(ws) == b.DP_OK
     dW, _ = oracle_layer(layer, inp)
     np.testing.assert_allclose(sq.cpu().numpy()[:, 0], oracle.sqnorm(dW), rtol=TOL_NORM)
+
+
+def test_fused_clip_runs_one_contraction_where_the_gradient_fits_a_cluster():
+    """bf16 layers whose per-example gradient fits the tensor memory of one thread-block cluster take the single-pass
+    form of the fused clip: fewer launches than the two-pass form, same results (checked layer by layer above)."""
+    b = B()
+    layer = synth.conv(64, 128, 3, 1, 1, 14, name="c")
+    inp = scaled_inputs(layer, 6, "bf16", 956, 0, spread=True)
+    counts = []
+    for on in (1, 0):
+        b.dp_debug_set_single_pass(on)
+        try:
+            c0 = b.dp_debug_launch_count()
+            gpu_layer(layer, inp, "bf16", CLIP, AUTO, 0, C_l=1.0)
+            counts.append(b.dp_debug_launch_count() - c0)
+        finally:
+            b.dp_debug_set_single_pass(1)
+    assert counts[0] < counts[1]
