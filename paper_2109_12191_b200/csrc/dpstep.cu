@@ -187,7 +187,7 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         if (epi != DP_EPI_CLIP_ACCUM) {
             if (pl.use_tc) {
                 // one launch: the kernel's last CTA folds the partial norms (a ticket in the workspace header)
-                const TcPublish pub = {reinterpret_cast<int *>(ws + kWsCounterOffset), pl.w_slots, groups == 2, sqnorm, sqnorm_stride};
+                const TcPublish pub = {reinterpret_cast<int *>(ws + kWsCounterOffset), pl.w_slots, groups == 2, sqnorm, sqnorm_stride, nullptr, 0.f, nullptr};
                 return launch_conv_tc(d->dtype, epi, X, dY, g, G_w, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off,
                                       reinterpret_cast<int *>(ws + pl.status_off), st, false, nullptr, &pub);
             }
@@ -203,14 +203,20 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
                                      reinterpret_cast<int *>(ws + pl.status_off), st);
         }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
-        if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
-        else rc = launch_conv_fma(storage_type(d), DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
-        if (rc != DP_OK) return rc;
-        if (pl.use_tc && !d->has_bias) {
-            // no bias: the clipped-sum pass finalises the norms itself
-            const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
-            return launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, nullptr, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true, &ic);
+        if (pl.use_tc) {
+            // the norm pass's last CTA folds the partial norms (bias slots included) into norms and factors
+            const TcPublish pub = {reinterpret_cast<int *>(ws + kWsCounterOffset), pl.w_slots, groups == 2, sqnorm, sqnorm_stride, factor, C_l, clip_out};
+            rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off,
+                                reinterpret_cast<int *>(ws + pl.status_off), st, false, nullptr, &pub);
+            if (rc != DP_OK) return rc;
+            rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off,
+                                reinterpret_cast<int *>(ws + pl.status_off), st, true);
+            if (rc != DP_OK) return rc;
+            if (d->has_bias) return launch_bias_accum(db, d->B, d->K_out, factor, acc_b, st);
+            return DP_OK;
         }
+        rc = launch_conv_fma(storage_type(d), DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, nullptr, st);
+        if (rc != DP_OK) return rc;
         rc = launch_finalize(partial, d->B, pl.slots, pl.w_slots, groups == 2, sqnorm, sqnorm_stride, 1, C_l, factor, clip_out, st);
         if (rc != DP_OK) return rc;
         if (pl.use_tc) rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st, true);

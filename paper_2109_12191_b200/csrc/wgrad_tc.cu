@@ -74,6 +74,7 @@ struct TcParams {
     // modes 0 / 1 with a ticket: counters[0] counts the CTAs that are done (zero on entry, left at zero); the last
     // one folds every example's slots [0, w_slots) and [w_slots, slots) into sqnorm (two values when `separate`)
     int *counters; int w_slots; int separate;
+    float *factor_out;          // with the ticket: also the clip factors against C_l, [B][2] (weight, bias), and clip_out
 };
 
 struct Item { int mt, nt, n_lo, n_hi, split; };
@@ -150,6 +151,28 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint32_t a_lo, uint32_t b_
                      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
                      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
                      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Issue only: the registers hold the values after tmem_ld_wait32 on the same array.  Two loads in flight per thread
+// hide most of the tensor-memory round trip (a load-then-wait per 32 columns left the epilogue warps idle).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+// Waits for every tensor-memory load of this thread; the array rides along as in/out operands so that no use of its
+// registers can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait32(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -411,7 +434,13 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 #pragma unroll
                 for (int i = 0; i < 128; ++i) run[CLIP ? i : 0] = 0.f;
             }
+            float f_lane = 0.f;     // clip mode, known factors: lane l holds the factor of example n_base + l
+            int n_base = it.n_lo - 32;
             for (int n = it.n_lo; n < it.n_hi; ++n) {
+                if (CLIP && !p.inline_factor && n >= n_base + 32) {
+                    n_base = n;
+                    f_lane = (n + lane < it.n_hi) ? p.factor[2 * (n + lane)] : 0.f;    // one coalesced load per 32 examples
+                }
                 const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
                 if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }   // the whole warp leaves together
                 full_phase ^= 1u << buf;
@@ -431,30 +460,33 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                             if (p.clip_out) p.clip_out[n] = f;
                         }
                     } else {
-                        f = p.factor[2 * n];
+                        f = __shfl_sync(0xffffffffu, f_lane, n - n_base);
                     }
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        if (c4 * 32 < n_cols) {
-                            uint32_t v[32];
-                            tmem_ld32(t_addr + (uint32_t)(c4 * 32), v);
+                    for (int c2 = 0; c2 < 2; ++c2) {           // columns in pairs of 32: both loads in flight before the wait
+                        if (c2 * 64 < n_cols) {
+                            uint32_t v0[32], v1[32];
+                            tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                            tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);     // (NT is a multiple of 64 here)
+                            tmem_ld_wait32(v0); tmem_ld_wait32(v1);
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
-                                run[CLIP ? c4 * 32 + i : 0] = fmaf(f, __uint_as_float(v[i]), run[CLIP ? c4 * 32 + i : 0]);
+                                run[CLIP ? c2 * 64 + i : 0] = fmaf(f, __uint_as_float(v0[i]), run[CLIP ? c2 * 64 + i : 0]);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                run[CLIP ? c2 * 64 + 32 + i : 0] = fmaf(f, __uint_as_float(v1[i]), run[CLIP ? c2 * 64 + 32 + i : 0]);
                         }
                     }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
                 } else {
-                    float sq = 0.f;
+                    float sq4[4] = {0.f, 0.f, 0.f, 0.f};      // four chains: one accumulator would serialise 256 dependent FMAs
                     float *Gn = p.G_w + (long long)n * p.Kout * p.Ng;
-                    for (int cc = 0; cc < n_cols; cc += 32) {
-                        uint32_t v[32];
-                        tmem_ld32(t_addr + (uint32_t)cc, v);
+                    auto consume = [&](uint32_t (&v)[32], int cc) {
                         if (row_ok) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq = fmaf(f, f, sq); }
+                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
                             if (p.mode == 0) {
                                 const int b_idx = nt * p.NT + cc;
                                 if (p.a_is_x) {      // row = column j of G, tile column = output channel k: lanes write consecutive j
@@ -480,18 +512,27 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                             }
                             __syncwarp();
                         }
+                    };
+                    // columns in pairs of 32 with both loads in flight before the wait.  The second load of a tile with
+                    // an odd number of 32-column blocks reads columns of this accumulator buffer that nobody uses.
+                    for (int cc = 0; cc < n_cols; cc += 64) {
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32_issue(t_addr + (uint32_t)cc, v0);
+                        tmem_ld32_issue(t_addr + (uint32_t)(cc + 32), v1);
+                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+                        consume(v0, cc);
+                        if (cc + 32 < n_cols) consume(v1, cc + 32);
                     }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
-                    sq = warp_sum(sq);
-                    if (lane == 0) {
-                        p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
-                        if (p.counters) __threadfence();       // visible to the CTA that will fold the partial sums
-                    }
+                    const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
+                    if (lane == 0) p.partial[(long long)n * p.slots + (mt * p.n_tiles + nt) * 4 + q] = sq;
                 }
                 buf ^= 1;
             }
+            if (!CLIP && p.counters && lane == 0 && item + (int)gridDim.x >= p.total_tiles)
+                __threadfence();          // after this warp's last item: its partial sums are visible to the CTA that folds them
             if (CLIP && live && row_ok) {
                 // one owner per output element: add straight into the accumulator, or leave a partial sum for the fold
                 const bool add = p.splits == 1;
@@ -562,6 +603,15 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (n < p.B && sub == 0) {
                     if (p.separate) { p.sqnorm[n * p.sq_stride] = (float)sw; p.sqnorm[n * p.sq_stride + 1] = (float)sb; }
                     else p.sqnorm[n * p.sq_stride] = (float)(sw + sb);
+                    if (p.factor_out) {                    // the clipped-sum pass that follows reads its factors here
+                        const float fw = clip_factor(p.separate ? sw : sw + sb, p.C_l);
+                        const float fb = p.separate ? clip_factor(sb, p.C_l) : fw;
+                        p.factor_out[2 * n] = fw; p.factor_out[2 * n + 1] = fb;
+                        if (p.clip_out) {
+                            if (p.separate) { p.clip_out[2 * n] = fw; p.clip_out[2 * n + 1] = fb; }
+                            else p.clip_out[n] = fw;
+                        }
+                    }
                 }
             }
         }
@@ -774,19 +824,23 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
             tc_fence_after();
             const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
             // pass 1: this warp's share of the example's squared norm
-            float sq = 0.f;
+            float sq4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                if (c4 * 32 < my_cols) {
-                    uint32_t v[32];
-                    tmem_ld32(t_addr + (uint32_t)(c4 * 32), v);
+            for (int c2 = 0; c2 < 2; ++c2) {               // columns in pairs of 32, both loads in flight before the wait
+                if (c2 * 64 < my_cols) {                    // (my_cols is a multiple of 64)
+                    uint32_t v0[32], v1[32];
+                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                    tmem_ld_wait32(v0); tmem_ld_wait32(v1);
                     if (row_ok) {      // (columns past the real ones of an unfolded thin layer hold exact zeros)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v[i]); sq = fmaf(f, f, sq); }
+                        for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v0[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v1[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
                     }
                 }
             }
-            sq = warp_sum(sq);
+            const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
             if (lane == 0) {
                 const uint32_t slot = smem_u32(&norm_part[par][rank][e]);
                 const uint32_t bar = smem_u32(&norm_bar[par]);
@@ -809,12 +863,16 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
             }
             // pass 2: scale the tile into the running sum
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                if (c4 * 32 < my_cols) {
-                    uint32_t v[32];
-                    tmem_ld32(t_addr + (uint32_t)(c4 * 32), v);
+            for (int c2 = 0; c2 < 2; ++c2) {
+                if (c2 * 64 < my_cols) {
+                    uint32_t v0[32], v1[32];
+                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                    tmem_ld_wait32(v0); tmem_ld_wait32(v1);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) run[c4 * 32 + i] = fmaf(f, __uint_as_float(v[i]), run[c4 * 32 + i]);
+                    for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
                 }
             }
             tc_fence_before();
@@ -1032,8 +1090,9 @@ static double step_cycles(int dtype, int n_cols, double a_slabs_loaded, double b
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode);
 
 // single-pass clipped sum: how many clusters share the batch and how many examples each walks through
+static int max_active_clusters(int cluster_size);
 static void cluster_split(int B, int cluster_size, int &splits, int &per_split) {
-    int want = sm_target() / cluster_size;
+    int want = std::min(sm_target() / cluster_size, max_active_clusters(cluster_size));
     if (want < 1) want = 1;
     if (want > B) want = B;
     per_split = (B + want - 1) / want;
@@ -1150,6 +1209,29 @@ static bool clip1_registers_ok() {
         if (!ok) (void)cudaGetLastError();
     }
     return ok == 1;
+}
+
+// How many clusters of this size the GPU can hold at once (a cluster needs all its SMs free in one GPC at the same
+// time, so this is less than SMs / size); more clusters than that would run as a second wave.  Unknown (no device): no cap.
+static int max_active_clusters(int cluster_size) {
+    static std::mutex mu;
+    static int cached[kMaxCluster + 1] = {0};
+    if (cluster_size < 1 || cluster_size > kMaxCluster) return 1 << 30;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[cluster_size] == 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(cluster_size * 64)); cfg.blockDim = dim3(kClipThreads); cfg.dynamicSmemBytes = kSmemBudget + 1024;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = (unsigned)cluster_size; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        const bool ok = cudaFuncSetAttribute(conv_wgrad_clip1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048) == cudaSuccess &&
+                        cudaOccupancyMaxActiveClusters(&n, conv_wgrad_clip1_kernel, &cfg) == cudaSuccess && n > 0;
+        if (!ok) (void)cudaGetLastError();
+        cached[cluster_size] = ok ? n : -1;
+    }
+    return cached[cluster_size] > 0 ? cached[cluster_size] : 1 << 30;
 }
 
 // true when the fused clipped sum of this layer runs as ONE contraction (bf16 inputs, the example's gradient fits the
@@ -1290,10 +1372,11 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     p.sqnorm = inline_clip ? inline_clip->sqnorm : nullptr;
     p.sq_stride = inline_clip ? inline_clip->sq_stride : 0;
     p.clip_out = inline_clip ? inline_clip->clip_out : nullptr;
-    p.counters = nullptr; p.w_slots = 0; p.separate = 0;
+    p.counters = nullptr; p.w_slots = 0; p.separate = 0; p.factor_out = nullptr;
     if (!clip && publish) {
         p.counters = publish->counters; p.w_slots = publish->w_slots; p.separate = publish->separate;
         p.sqnorm = publish->sqnorm; p.sq_stride = publish->sq_stride;
+        p.factor_out = publish->factor_out; p.C_l = publish->C_l; p.clip_out = publish->clip_out;
     }
     if (clip) {
         clip_split(g, pl, p.splits, p.per_split);

@@ -20,7 +20,8 @@ struct TcInlineClip { float C_l; float *sqnorm; long long sq_stride; float *clip
 // When given to a STORE_NORM / NORM_ONLY launch, the last CTA to finish folds every example's partial squared norms
 // (slots [0, w_slots) = weights, the rest = bias, written earlier in the stream) and writes sqnorm[n*sq_stride]
 // (+1 for the bias when `separate`), so no finalising launch is needed.  counters: one cleared ticket word.
-struct TcPublish { int *counters; int w_slots; int separate; float *sqnorm; long long sq_stride; };
+// factor_out (optional): also the clip factors against C_l, [B][2] = (weight, bias), and clip_out as dp_per_example_wgrad defines it.
+struct TcPublish { int *counters; int w_slots; int separate; float *sqnorm; long long sq_stride; float *factor_out; float C_l; float *clip_out; };
 
 // epilogue as dp_epilogue; factor[n*2] scales example n (CLIP_ACCUM); status: device word set to nonzero on a timed-out wait
 dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY, const ConvGeom &g, float *G_w,
