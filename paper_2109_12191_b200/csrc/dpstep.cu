@@ -202,6 +202,12 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             return launch_conv_clip1(d->dtype, X, dY, g, partial, pl.slots, ic, acc_w, ws + pl.tc_off,
                                      reinterpret_cast<int *>(ws + pl.status_off), st);
         }
+        if (pl.use_tc && !d->has_bias && single_pass_enabled() && tc_clip_grid_pass(d->dtype, g)) {
+            // ... also where the gradient is too large for a cluster: partial norms meet in global memory instead
+            const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
+            return launch_conv_clip2(d->dtype, X, dY, g, partial, factor, reinterpret_cast<int *>(ws + kWsCounterOffset), ic, acc_w,
+                                     reinterpret_cast<int *>(ws + pl.status_off), st);
+        }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) {
             // the norm pass's last CTA folds the partial norms (bias slots included) into norms and factors
@@ -319,7 +325,7 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
 }
 
 extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n) {
-    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 3 || !out || n <= 0) return 0;   // 3: the single-pass form of the fused clip
+    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 4 || !out || n <= 0) return 0;   // 3, 4: the single-pass forms of the fused clip (cluster, grid)
     return tc_describe_plan(desc->dtype, geom_of(desc), epilogue, out, n);
 }
 

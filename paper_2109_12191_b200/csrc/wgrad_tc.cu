@@ -926,6 +926,281 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
 }
 
+
+// ----------------------------------------------------------------------------- grid-synchronised single-pass fused clip (bf16)
+// Layers whose per-example gradient is too large for one cluster's tensor memory (few pixels, many channels: the 7 x 7
+// and 14 x 14 layers of a ResNet) still run ONE contraction: the grid has one CTA per 128 x 128 tile of the gradient,
+// every CTA walks all examples for its tile, and the CTAs exchange each example's partial squared norms through global
+// memory: a CTA hands in its partial sum with a ticket, the last one to do so folds all of them in tile order and
+// publishes the example's factor with a release store, the others poll that flag (bounded; all CTAs are resident at
+// once because the launch is cooperative).  The round trip through L2 costs a few microseconds, so the tile of an
+// example stays in tensor memory while the next three examples' tiles are computed and square-summed (four accumulator
+// buffers of 128 columns): a CTA scales example m only after handing in example m + 3.  Every CTA owns its tile of the
+// clipped sum for the whole batch, so the sums go straight into the accumulator: no partial sums, no fold.
+constexpr int kClip2Lag = 3;      // examples handed in before the oldest one's factor is needed (buffers = lag + 1)
+
+__device__ __forceinline__ int ld_acquire_gpu(const int *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int *p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(224, 1)
+conv_wgrad_clip2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[kClip2Lag + 1], tmem_empty[kClip2Lag + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t tiles_u32 = smem_u32(tiles);
+    const int n_tiles_total = p.m_tiles * p.n_tiles;
+    const int tile = (int)blockIdx.x;
+    const int mt = tile / p.n_tiles, nt = tile - mt * p.n_tiles;
+    int *tickets = p.counters, *ready = p.counters + p.B, *exit_ticket = p.counters + 2 * p.B;
+
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 2); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int b = 0; b <= kClip2Lag; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int *abort_p = &abort_flag;
+
+    const int slab_bytes = p.Kt * kRowBytes;
+    const int a_slabs_tile = 128 / p.slab_ch, b_slabs_tile = p.NT / p.slab_ch;
+    const int a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - mt * a_slabs_tile);
+    const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
+
+    if (warp == 0 || warp == 6) {
+        // ------------------------------------------------------------ TMA producers (A slabs / B slabs)
+        const bool is_a = warp == 0;
+        const bool active = is_a ? (lane < a_slabs) : (lane < b_slabs);
+        const bool is_x = is_a ? (p.a_is_x != 0) : (p.a_is_x == 0);
+        const int slab = (is_a ? mt * a_slabs_tile : nt * b_slabs_tile) + lane;
+        int c0, dw = 0, dh = 0, mul = 1;
+        if (is_x) {
+            const int j0 = slab * p.slab_ch;
+            const int tap = j0 / p.Cin;
+            c0 = j0 - tap * p.Cin;
+            const int r = tap / p.S;
+            dw = (tap - r * p.S) - p.pad;
+            dh = r - p.pad;
+            mul = p.stride;
+        } else {
+            c0 = slab * p.slab_ch;
+        }
+        const CUtensorMap *map = is_x ? &tmX : &tmY;
+        const uint32_t dst_off = (is_a ? 0u : (uint32_t)p.a_bytes) + (uint32_t)(lane * slab_bytes);
+        const uint32_t tx_bytes = (uint32_t)((is_a ? a_slabs : b_slabs) * slab_bytes);
+        int stage = 0; uint32_t phase = 0;
+        bool live = true;
+        for (int n = 0; n < p.B && live; ++n) {
+            int ow0 = 0, oh0 = 0, tw = 0;
+            for (int kt = 0; kt < p.k_tiles; ++kt) {
+                bool ok = true;
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p, p.wait_polls);
+                    if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { live = false; break; }
+                if (active)
+                    tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
+                                ow0 * mul + dw, oh0 * mul + dh, n);
+                if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool live = true;
+            const uint64_t desc_base = operand_desc_base<false>((uint32_t)slab_bytes);
+            const uint32_t desc_lo = (uint32_t)desc_base, desc_hi32 = (uint32_t)(desc_base >> 32);
+            const int ksteps = p.Kt / p.krows;
+            constexpr uint32_t kadvance = (uint32_t)(16 * kRowBytes) >> 4;
+            const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, 1u);
+            for (int n = 0; n < p.B && live; ++n) {
+                const int buf = n & kClip2Lag;                       // lag + 1 = 4 buffers
+                const uint32_t use = (uint32_t)(n >> 2);
+                if (!mbar_wait(smem_u32(&tmem_empty[buf]), (use & 1u) ^ 1u, abort_p, p.wait_polls)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 128);
+                uint32_t accumulate = 0;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p, p.wait_polls)) { live = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
+                    uint32_t ad = desc_lo | ((a_src & 0x3FFFFu) >> 4);
+                    uint32_t bd = desc_lo | (((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
+#pragma unroll 4
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        umma<false>(d_tmem, ad, bd, desc_hi32, idesc, accumulate);
+                        accumulate = 1;
+                        ad += kadvance; bd += kadvance;
+                    }
+                    umma_commit(smem_u32(&empty_bar[stage]));
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (!live) break;
+                umma_commit(smem_u32(&tmem_full[buf]));
+            }
+        }
+    } else if (warp >= 2 && warp <= 5) {
+        // ------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
+        static_assert(kClip2Lag == 3, "buffer index arithmetic assumes four accumulator buffers");
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const int a_rows = min(128, p.a_ext - mt * 128);
+        const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
+        const int a_idx = mt * 128 + row;
+        const bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
+        const int slots = n_tiles_total * 4;                 // partial sums per example: (tile, epilogue warp)
+        float run[128];
+#pragma unroll
+        for (int i = 0; i < 128; ++i) run[i] = 0.f;
+        bool live = true;
+        for (int step = 0; step < p.B + kClip2Lag && live; ++step) {
+            if (step < p.B) {
+                // hand in example `step`: square-sum its tile, leave the partial sum, take a ticket
+                const int n = step, buf = n & 3;
+                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (uint32_t)((n >> 2) & 1), abort_p, p.wait_polls);
+                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+                tc_fence_after();
+                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 128) + ((uint32_t)(q * 32) << 16);
+                float sq4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    if (c2 * 64 < n_cols) {
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+                        if (row_ok) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v0[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v1[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
+                        }
+                    }
+                }
+                const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
+                int last = 0;
+                if (lane == 0) {
+                    p.partial[(long long)n * slots + tile * 4 + q] = sq;
+                    __threadfence();
+                    last = atomicAdd(&tickets[n], 1) == slots - 1;
+                }
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    // everyone's partial sums of example n are in: fold them in slot order, publish norm and factor
+                    __threadfence();
+                    const float *pn = p.partial + (long long)n * slots;
+                    double sn = 0.0;
+                    for (int i = lane; i < slots; i += 32) sn += (double)__ldcg(pn + i);
+                    sn = warp_sum(sn);
+                    if (lane == 0) {
+                        const float f = clip_factor(sn, p.C_l);
+                        p.sqnorm[n * p.sq_stride] = (float)sn;
+                        if (p.clip_out) p.clip_out[n] = f;
+                        p.factor_out[n] = f;
+                        tickets[n] = 0;
+                        st_release_gpu(&ready[n], 1);
+                    }
+                }
+            }
+            if (step >= kClip2Lag) {
+                // scale example m, handed in three steps ago, once its factor is known
+                const int m = step - kClip2Lag, buf = m & 3;
+                int ok = 0;
+                if (lane == 0) {
+                    for (uint32_t it = 0; it < p.wait_polls; ++it) {
+                        if (ld_acquire_gpu(&ready[m]) != 0) { ok = 1; break; }
+                        if ((it & 63u) == 63u && *abort_p) break;
+                        __nanosleep(64);
+                    }
+                    if (!ok) *abort_p = 1;
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { live = false; break; }
+                const float f = __ldcg(p.factor_out + m);
+                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 128) + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    if (c2 * 64 < n_cols) {
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            }
+        }
+        if (live && row_ok) {
+            // this CTA owns its tile of the clipped sum for the whole batch: add straight into the accumulator
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                if (c4 * 32 < n_cols) {
+                    const int b_idx = nt * p.NT + c4 * 32;
+                    if (p.a_is_x) {
+                        float *dst = p.sum_out + (long long)b_idx * p.Ng + a_idx;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) dst[(long long)i * p.Ng] += run[c4 * 32 + i];
+                    } else if (!p.n_pad_cols) {
+                        float4 *dst = reinterpret_cast<float4 *>(p.sum_out + (long long)a_idx * p.Ng + b_idx);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            float4 o = dst[i];
+                            o.x += run[c4 * 32 + 4 * i]; o.y += run[c4 * 32 + 4 * i + 1]; o.z += run[c4 * 32 + 4 * i + 2]; o.w += run[c4 * 32 + 4 * i + 3];
+                            dst[i] = o;
+                        }
+                    } else {
+                        float *dst = p.sum_out + (long long)a_idx * p.Ng + b_idx;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (b_idx + i < p.Ng) dst[i] += run[c4 * 32 + i];
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag) {
+        if (threadIdx.x == 0) { *p.status = DP_ERR_TIMEOUT; __threadfence(); }
+        __nanosleep(200000);
+        __syncthreads();
+    } else if (threadIdx.x == 0) {
+        // the last CTA to leave clears the flags for the next call: by then every CTA has read all of them
+        if (atomicAdd(exit_ticket, 1) == (int)gridDim.x - 1) {
+            for (int n = 0; n < p.B; ++n) ready[n] = 0;
+            *exit_ticket = 0;
+        }
+    }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
 // acc[i] += sum over splits of part[s][i], splits in index order (P a multiple of 4, both 16-byte aligned)
 __global__ void __launch_bounds__(256)
 fold_partial_sums_kernel(const float *__restrict__ part, int splits, long long P, float *__restrict__ acc) {
@@ -1118,7 +1393,7 @@ static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
 // mode 3 plans the single-pass clipped sum: all tiles of an example in one cluster (at most kMaxCluster of them), the
 // clusters share the batch, and what is minimised is SM time (clusters x CTAs x time), not the time of one launch
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
-    const int max_nt = (mode == 2) ? 128 : 256;
+    const int max_nt = (mode == 2 || mode == 4) ? 128 : 256;
     TcPlan best; best.ok = false;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
@@ -1138,10 +1413,15 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
             if (total_tiles > 0x7fffffffLL) continue;
             if (mode == 3 && m_tiles * n_tiles > kMaxCluster) continue;
+            if (mode == 4 && m_tiles * n_tiles > sm_count()) continue;      // one resident CTA per tile
             // per-CTA share of (example, tile) units: whole waves of tiles, or in clipped-sum mode an even share of the examples
             double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
                                        : std::max(1.0, (double)total_tiles / sms);
             double sm_share = 1.0;
+            if (mode == 4) {
+                waves = g.B;                                       // every CTA walks the whole batch for its tile
+                sm_share = (double)m_tiles * n_tiles;
+            }
             if (mode == 3) {
                 int splits, per;
                 cluster_split(g.B, m_tiles * n_tiles, splits, per);
@@ -1154,7 +1434,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             // the 128 x NT accumulator: stores run at about 16 B/clk per SM when lanes write consecutive addresses
             // (rows of D are gradient columns) and about 7 B/clk otherwise; reading TMEM alone is cheap
             const double epilogue = (mode == 0) ? 128.0 * NT * 4.0 / (a_is_x ? 16.0 : 7.0)
-                                  : (mode == 1 ? 6.0 * NT : (mode == 2 ? 10.0 * NT : 10.0 * std::min(NT, 128) + 600.0));
+                                  : (mode == 1 ? 6.0 * NT : (mode == 2 ? 10.0 * NT : (mode == 4 ? 9.0 * NT : 10.0 * std::min(NT, 128) + 600.0)));
             // a pixel tile may reach past the output plane (its rows there are zero-filled by TMA and add nothing):
             // a 7 x 7 plane is one 8 x 8 tile of 64 reduction rows instead of four 4 x 4 tiles of 16
             const int oh_max = std::min((g.OH + 7) / 8 * 8, 256 / g.stride), ow_max = std::min((g.OW + 7) / 8 * 8, 256 / g.stride);
@@ -1177,7 +1457,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
                         stage_cost = std::max(stage_cost, 0.5 * (1000.0 + (a_loaded + b_loaded) * Kt * 2.5));
                     double mainloop = stage_cost * tw * th;
                     if (stages < 3) mainloop *= 1.15;
-                    const double cost = ((std::max(mainloop, epilogue) + 300.0) * waves + (mode == 3 ? 4000.0 : 0.0)) * sm_share;
+                    const double cost = ((std::max(mainloop, epilogue) + 300.0) * waves + (mode >= 3 ? 4000.0 : 0.0)) * sm_share;
                     if (cost < best_cost) {
                         best_cost = cost;
                         best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
@@ -1242,6 +1522,14 @@ static bool clip1_plan(int dtype, const ConvGeom &eff, TcPlan &pl) {
     return pl.ok;
 }
 
+// true when the fused clipped sum of this layer runs as one contraction with the grid-wide exchange of partial norms
+// (bf16 inputs, one resident CTA per 128-column tile, tickets and flags for B examples in the workspace header)
+static bool clip2_plan(int dtype, const ConvGeom &eff, TcPlan &pl) {
+    if (dtype != DP_BF16 || 2 * eff.B + 1 > kWsCounters) return false;
+    pl = make_plan(dtype, eff, 4);
+    return pl.ok;
+}
+
 // clipped-sum mode: how many example ranges each tile is cut into so that every SM has an item
 static void clip_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &per_split) {
     const int tiles = pl.m_tiles * pl.n_tiles;
@@ -1256,7 +1544,10 @@ int tc_norm_slots(int dtype, const ConvGeom &g0, int epilogue) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
     const TcPlan pl = make_plan(dtype, pr.eff, epilogue == DP_EPI_STORE_NORM ? 0 : 1);
-    return pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
+    int slots = pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
+    TcPlan two;
+    if (epilogue == DP_EPI_CLIP_ACCUM && clip2_plan(dtype, pr.eff, two)) slots = std::max(slots, two.m_tiles * two.n_tiles * 4);
+    return slots;
 }
 
 static size_t unfold_bytes(int dtype, const ConvGeom &g0, const TcProblem &pr) {
@@ -1405,6 +1696,59 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     }
     DP_LAUNCH_CHECK("conv_wgrad_tc_kernel");
     if (clip && p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g0.M * g0.N, acc_w, stream);
+    return DP_OK;
+}
+
+int tc_clip_grid_pass(int dtype, const ConvGeom &g0) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    TcPlan pl;
+    if (!pr.ok || pr.unfold || !encode_fn() || !clip2_plan(dtype, pr.eff, pl)) return 0;
+    static int coop = -1;
+    if (coop < 0) {
+        int dev = 0, v = 0;
+        coop = (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : 0;
+    }
+    return coop;
+}
+
+dp_status launch_conv_clip2(int dtype, const void *X, const void *dY, const ConvGeom &g0, float *partial, float *factor,
+                            int *counters, const TcInlineClip &clipinfo, float *acc_w, int *status, cudaStream_t stream) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    TcPlan pl;
+    if (!pr.ok || pr.unfold || !encode_fn() || !clip2_plan(dtype, pr.eff, pl)) return DP_ERR_UNSUPPORTED;
+    const ConvGeom &g = pr.eff;
+    CUtensorMap tmX, tmY;
+    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    TcParams p = {};
+    p.B = g.B; p.Kout = g.Kout; p.Ng = g0.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.n_pad_cols = 0;
+    p.slab_ch = 64; p.krows = 16;
+    p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
+    p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
+    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
+    p.mode = 4; p.status = status;
+    p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
+    p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
+    p.partial = partial; p.slots = pl.m_tiles * pl.n_tiles * 4;
+    p.factor_out = factor; p.counters = counters;
+    p.splits = 1; p.per_split = g.B; p.sum_out = acc_w;
+    p.total_tiles = pl.m_tiles * pl.n_tiles;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(conv_wgrad_clip2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.total_tiles); cfg.blockDim = dim3(224); cfg.dynamicSmemBytes = pl.smem; cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;       // all CTAs resident at once: the ones that poll can rely on the others running
+    at[0].val.cooperative = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, conv_wgrad_clip2_kernel, tmX, tmY, p);
+    if (le != cudaSuccess) return cuda_fail(le, "conv_wgrad_clip2_kernel");
+    DP_LAUNCH_CHECK("conv_wgrad_clip2_kernel");
     return DP_OK;
 }
 
