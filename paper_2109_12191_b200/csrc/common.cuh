@@ -17,6 +17,7 @@ void note_error(const char *message);
 int sm_count();
 // Number of SMs one tensor-core launch should spread over: dp_set_sm_target()'s value, or all of them.
 int sm_target();
+bool sm_target_set();   // true once dp_set_sm_target() was given a positive value: the caller runs calls side by side
 // false while dp_debug_set_single_pass(0) holds: the fused clipped sum then always runs its two-pass form
 bool single_pass_enabled();
 

@@ -25,6 +25,8 @@ static std::atomic<int> g_sm_target{0};
 static std::atomic<int> g_single_pass{1};
 bool single_pass_enabled() { return g_single_pass.load(std::memory_order_relaxed) != 0; }
 
+bool sm_target_set() { return g_sm_target.load(std::memory_order_relaxed) > 0; }
+
 int sm_target() {
     const int all = sm_count(), t = g_sm_target.load(std::memory_order_relaxed);
     return (t > 0 && t < all) ? t : all;
@@ -202,12 +204,6 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             return launch_conv_clip1(d->dtype, X, dY, g, partial, pl.slots, ic, acc_w, ws + pl.tc_off,
                                      reinterpret_cast<int *>(ws + pl.status_off), st);
         }
-        if (pl.use_tc && !d->has_bias && single_pass_enabled() && tc_clip_grid_pass(d->dtype, g)) {
-            // ... also where the gradient is too large for a cluster: partial norms meet in global memory instead
-            const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
-            return launch_conv_clip2(d->dtype, X, dY, g, partial, factor, reinterpret_cast<int *>(ws + kWsCounterOffset), ic, acc_w,
-                                     reinterpret_cast<int *>(ws + pl.status_off), st);
-        }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) {
             // the norm pass's last CTA folds the partial norms (bias slots included) into norms and factors
@@ -215,6 +211,8 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off,
                                 reinterpret_cast<int *>(ws + pl.status_off), st, false, nullptr, &pub);
             if (rc != DP_OK) return rc;
+            if (!d->has_bias && single_pass_enabled() && tc_clip_scaled_sum(d->dtype, g))
+                return launch_conv_ssum(d->dtype, X, dY, g, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
             rc = launch_conv_tc(d->dtype, DP_EPI_CLIP_ACCUM, X, dY, g, nullptr, partial, pl.slots, factor, acc_w, ws + pl.tc_off,
                                 reinterpret_cast<int *>(ws + pl.status_off), st, true);
             if (rc != DP_OK) return rc;
@@ -325,7 +323,7 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
 }
 
 extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n) {
-    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 4 || !out || n <= 0) return 0;   // 3, 4: the single-pass forms of the fused clip (cluster, grid)
+    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 4 || !out || n <= 0) return 0;   // 3: the single-pass form of the fused clip, 4: the clipped sum as one product
     return tc_describe_plan(desc->dtype, geom_of(desc), epilogue, out, n);
 }
 

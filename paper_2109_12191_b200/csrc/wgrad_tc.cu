@@ -646,6 +646,7 @@ constexpr int kClipThreads = 384;
 constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
 static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
 constexpr int kMaxCluster = 8;
+constexpr int kMinExamplesPerCluster = 4;   // with an SM target set (calls run side by side)
 
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -927,48 +928,35 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
 }
 
 
-// ----------------------------------------------------------------------------- grid-synchronised single-pass fused clip (bf16)
-// Layers whose per-example gradient is too large for one cluster's tensor memory (few pixels, many channels: the 7 x 7
-// and 14 x 14 layers of a ResNet) still run ONE contraction: the grid has one CTA per 128 x 128 tile of the gradient,
-// every CTA walks all examples for its tile, and the CTAs exchange each example's partial squared norms through global
-// memory: a CTA hands in its partial sum with a ticket, the last one to do so folds all of them in tile order and
-// publishes the example's factor with a release store, the others poll that flag (bounded; all CTAs are resident at
-// once because the launch is cooperative).  The round trip through L2 costs a few microseconds, so the tile of an
-// example stays in tensor memory while the next three examples' tiles are computed and square-summed (four accumulator
-// buffers of 128 columns): a CTA scales example m only after handing in example m + 3.  Every CTA owns its tile of the
-// clipped sum for the whole batch, so the sums go straight into the accumulator: no partial sums, no fold.
-constexpr int kClip2Lag = 3;      // examples handed in before the oldest one's factor is needed (buffers = lag + 1)
 
-__device__ __forceinline__ int ld_acquire_gpu(const int *p) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release_gpu(int *p, int v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-
+// ----------------------------------------------------------------------------- clipped sum as ONE matrix product (bf16)
+// With the factors known, sum_n f_n dY_n^T Xcol_n is a single matrix product whose reduction runs over (example, pixel)
+// once every row of dY carries its example's factor: the tensor core then adds all examples into one accumulator and
+// nothing is read back from tensor memory per example (reading a 128 x 256 tile back costs as much as eight MMAs,
+// which is what bounds a per-example clipped sum on layers with few pixels).  f_n * dY does not fit bf16, so a small
+// launch before this one splits it into hi + lo (both bf16, hi = the rounded product, lo = the rounded remainder: what
+// is lost is below 2^-17 of each product) and every k-step issues two MMAs, X with hi and X with lo.  A work item is a
+// tile for a range of examples; with more than one range the tiles leave as partial sums for the fold.
+// Roles as in the kernel at the top: warp 0 / 6 TMA (the warp that loads dY loads both copies), warp 1 MMA, warps 2-5 epilogue.
 __global__ void __launch_bounds__(224, 1)
-conv_wgrad_clip2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
+conv_wgrad_ssum_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmYhi,
+                       const __grid_constant__ CUtensorMap tmYlo, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[kClip2Lag + 1], tmem_empty[kClip2Lag + 1];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t tiles_u32 = smem_u32(tiles);
-    const int n_tiles_total = p.m_tiles * p.n_tiles;
-    const int tile = (int)blockIdx.x;
-    const int mt = tile / p.n_tiles, nt = tile - mt * p.n_tiles;
-    int *tickets = p.counters, *ready = p.counters + p.B, *exit_ticket = p.counters + 2 * p.B;
 
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmYhi)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmYlo)) : "memory");
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 2); mbar_init(smem_u32(&empty_bar[s]), 1); }
-        for (int b = 0; b <= kClip2Lag; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
@@ -980,208 +968,153 @@ conv_wgrad_clip2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
 
     const int slab_bytes = p.Kt * kRowBytes;
     const int a_slabs_tile = 128 / p.slab_ch, b_slabs_tile = p.NT / p.slab_ch;
-    const int a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - mt * a_slabs_tile);
-    const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - nt * b_slabs_tile);
+    const bool a_is_y = p.a_is_x == 0;                        // which operand is dY (and so has a lo copy)
 
     if (warp == 0 || warp == 6) {
-        // ------------------------------------------------------------ TMA producers (A slabs / B slabs)
-        const bool is_a = warp == 0;
-        const bool active = is_a ? (lane < a_slabs) : (lane < b_slabs);
-        const bool is_x = is_a ? (p.a_is_x != 0) : (p.a_is_x == 0);
-        const int slab = (is_a ? mt * a_slabs_tile : nt * b_slabs_tile) + lane;
-        int c0, dw = 0, dh = 0, mul = 1;
-        if (is_x) {
-            const int j0 = slab * p.slab_ch;
-            const int tap = j0 / p.Cin;
-            c0 = j0 - tap * p.Cin;
-            const int r = tap / p.S;
-            dw = (tap - r * p.S) - p.pad;
-            dh = r - p.pad;
-            mul = p.stride;
-        } else {
-            c0 = slab * p.slab_ch;
-        }
-        const CUtensorMap *map = is_x ? &tmX : &tmY;
-        const uint32_t dst_off = (is_a ? 0u : (uint32_t)p.a_bytes) + (uint32_t)(lane * slab_bytes);
-        const uint32_t tx_bytes = (uint32_t)((is_a ? a_slabs : b_slabs) * slab_bytes);
+        // ------------------------------------------------------------ TMA producers
         int stage = 0; uint32_t phase = 0;
         bool live = true;
-        for (int n = 0; n < p.B && live; ++n) {
-            int ow0 = 0, oh0 = 0, tw = 0;
-            for (int kt = 0; kt < p.k_tiles; ++kt) {
-                bool ok = true;
-                if (lane == 0) {
-                    ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p, p.wait_polls);
-                    if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+        for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
+            const Item it = decode_item(p, item);
+            const int a_slab0 = it.mt * a_slabs_tile, a_slabs = min(a_slabs_tile, p.a_ext / p.slab_ch - a_slab0);
+            const int b_slab0 = it.nt * b_slabs_tile, b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - b_slab0);
+            const bool is_a = warp == 0;
+            const bool is_y = is_a == a_is_y;
+            const int mine = is_a ? a_slabs : b_slabs;       // slabs of this warp's operand; a dY warp issues each twice (hi, lo)
+            const bool second = is_y && lane >= mine;        // lanes [mine, 2*mine) of a dY warp load the lo copies
+            const int local = second ? lane - mine : lane;
+            const bool active = lane < (is_y ? 2 * mine : mine);
+            const int slab = (is_a ? a_slab0 : b_slab0) + local;
+            int c0, dw = 0, dh = 0, mul = 1;
+            if (!is_y) {
+                const int j0 = slab * p.slab_ch;
+                const int tap = j0 / p.Cin;
+                c0 = j0 - tap * p.Cin;
+                const int r = tap / p.S;
+                dw = (tap - r * p.S) - p.pad;
+                dh = r - p.pad;
+                mul = p.stride;
+            } else {
+                c0 = slab * p.slab_ch;
+            }
+            const CUtensorMap *map = !is_y ? &tmX : (second ? &tmYlo : &tmYhi);
+            const uint32_t dst_off = (second ? (uint32_t)p.lo_offset : (is_a ? 0u : (uint32_t)p.a_bytes)) + (uint32_t)(local * slab_bytes);
+            const uint32_t tx_bytes = (uint32_t)((is_y ? 2 * mine : mine) * slab_bytes);
+            for (int n = it.n_lo; n < it.n_hi && live; ++n) {
+                int ow0 = 0, oh0 = 0, tw = 0;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    bool ok = true;
+                    if (lane == 0) {
+                        ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p, p.wait_polls);
+                        if (ok) mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { live = false; break; }
+                    if (active)
+                        tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
+                                    ow0 * mul + dw, oh0 * mul + dh, n);
+                    if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) { live = false; break; }
-                if (active)
-                    tma_load_4d(tiles_u32 + stage * p.stage_bytes + dst_off, map, smem_u32(&full_bar[stage]), c0,
-                                ow0 * mul + dw, oh0 * mul + dh, n);
-                if (++tw == p.tiles_w) { tw = 0; ow0 = 0; oh0 += p.OHt; } else { ow0 += p.OWt; }
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (one lane)
         if (lane == 0) {
-            int stage = 0; uint32_t phase = 0;
+            int stage = 0; uint32_t phase = 0, acc_phase = 0;
+            int buf = 0;
             bool live = true;
             const uint64_t desc_base = operand_desc_base<false>((uint32_t)slab_bytes);
             const uint32_t desc_lo = (uint32_t)desc_base, desc_hi32 = (uint32_t)(desc_base >> 32);
             const int ksteps = p.Kt / p.krows;
             constexpr uint32_t kadvance = (uint32_t)(16 * kRowBytes) >> 4;
-            const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, 1u);
-            for (int n = 0; n < p.B && live; ++n) {
-                const int buf = n & kClip2Lag;                       // lag + 1 = 4 buffers
-                const uint32_t use = (uint32_t)(n >> 2);
-                if (!mbar_wait(smem_u32(&tmem_empty[buf]), (use & 1u) ^ 1u, abort_p, p.wait_polls)) break;
+            for (int item = blockIdx.x; item < p.total_tiles && live; item += gridDim.x) {
+                const Item it = decode_item(p, item);
+                const int b_slabs = min(b_slabs_tile, p.b_ext / p.slab_ch - it.nt * b_slabs_tile);
+                const uint32_t idesc = instr_desc(b_slabs * p.slab_ch, 1u);
+                if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p, p.wait_polls)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 128);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
                 uint32_t accumulate = 0;
-                for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p, p.wait_polls)) { live = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_src = tiles_u32 + stage * p.stage_bytes;
-                    uint32_t ad = desc_lo | ((a_src & 0x3FFFFu) >> 4);
-                    uint32_t bd = desc_lo | (((a_src + p.a_bytes) & 0x3FFFFu) >> 4);
-#pragma unroll 4
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        umma<false>(d_tmem, ad, bd, desc_hi32, idesc, accumulate);
-                        accumulate = 1;
-                        ad += kadvance; bd += kadvance;
+                for (int n = it.n_lo; n < it.n_hi && live; ++n) {
+                    for (int kt = 0; kt < p.k_tiles; ++kt) {
+                        if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p, p.wait_polls)) { live = false; break; }
+                        tc_fence_after();
+                        const uint32_t src = tiles_u32 + stage * p.stage_bytes;
+                        uint32_t ad = desc_lo | ((src & 0x3FFFFu) >> 4);
+                        uint32_t bd = desc_lo | (((src + p.a_bytes) & 0x3FFFFu) >> 4);
+                        uint32_t ld = desc_lo | (((src + p.lo_offset) & 0x3FFFFu) >> 4);
+#pragma unroll 2
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            umma<false>(d_tmem, ad, bd, desc_hi32, idesc, accumulate);                               // X with hi(f dY)
+                            if (a_is_y) umma<false>(d_tmem, ld, bd, desc_hi32, idesc, 1u);                           // X with lo(f dY)
+                            else umma<false>(d_tmem, ad, ld, desc_hi32, idesc, 1u);
+                            accumulate = 1;
+                            ad += kadvance; bd += kadvance; ld += kadvance;
+                        }
+                        umma_commit(smem_u32(&empty_bar[stage]));
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                     }
-                    umma_commit(smem_u32(&empty_bar[stage]));
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!live) break;
                 umma_commit(smem_u32(&tmem_full[buf]));
+                acc_phase ^= 1u << buf;
+                buf ^= 1;
             }
         }
     } else if (warp >= 2 && warp <= 5) {
-        // ------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
-        static_assert(kClip2Lag == 3, "buffer index arithmetic assumes four accumulator buffers");
+        // ------------------------------------------------------------ epilogue: one read of the finished tile per item
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        const int a_rows = min(128, p.a_ext - mt * 128);
-        const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
-        const int a_idx = mt * 128 + row;
-        const bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
-        const int slots = n_tiles_total * 4;                 // partial sums per example: (tile, epilogue warp)
-        float run[128];
+        uint32_t full_phase = 0;
+        int buf = 0;
+        for (int item = blockIdx.x; item < p.total_tiles; item += gridDim.x) {
+            const Item it = decode_item(p, item);
+            const int mt = it.mt, nt = it.nt;
+            const int a_rows = min(128, p.a_ext - mt * 128);
+            const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
+            const int a_idx = mt * 128 + row;
+            const bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
+            const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
+            if (!__all_sync(0xffffffffu, arrived)) break;
+            full_phase ^= 1u << buf;
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256) + ((uint32_t)(q * 32) << 16);
+            const bool add = p.splits == 1;
+            float *base = p.sum_out + (add ? 0ll : (long long)it.split * p.Kout * p.Ng);
+            auto put = [&](uint32_t (&v)[32], int cc) {
+                if (!row_ok) return;
+                const int b_idx = nt * p.NT + cc;
+                if (p.a_is_x) {
+                    float *dst = base + (long long)b_idx * p.Ng + a_idx;
 #pragma unroll
-        for (int i = 0; i < 128; ++i) run[i] = 0.f;
-        bool live = true;
-        for (int step = 0; step < p.B + kClip2Lag && live; ++step) {
-            if (step < p.B) {
-                // hand in example `step`: square-sum its tile, leave the partial sum, take a ticket
-                const int n = step, buf = n & 3;
-                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (uint32_t)((n >> 2) & 1), abort_p, p.wait_polls);
-                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
-                tc_fence_after();
-                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 128) + ((uint32_t)(q * 32) << 16);
-                float sq4[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int i = 0; i < 32; ++i) {
+                        float *el = dst + (long long)i * p.Ng;
+                        const float r = __uint_as_float(v[i]);
+                        *el = add ? *el + r : r;
+                    }
+                } else {
+                    float4 *dst = reinterpret_cast<float4 *>(base + (long long)a_idx * p.Ng + b_idx);
 #pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
-                    if (c2 * 64 < n_cols) {
-                        uint32_t v0[32], v1[32];
-                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
-                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
-                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
-                        if (row_ok) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v0[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v1[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
-                        }
+                    for (int i = 0; i < 8; ++i) {
+                        float4 r = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                        if (add) { const float4 o = dst[i]; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
+                        dst[i] = r;
                     }
                 }
-                const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
-                int last = 0;
-                if (lane == 0) {
-                    p.partial[(long long)n * slots + tile * 4 + q] = sq;
-                    __threadfence();
-                    last = atomicAdd(&tickets[n], 1) == slots - 1;
-                }
-                last = __shfl_sync(0xffffffffu, last, 0);
-                if (last) {
-                    // everyone's partial sums of example n are in: fold them in slot order, publish norm and factor
-                    __threadfence();
-                    const float *pn = p.partial + (long long)n * slots;
-                    double sn = 0.0;
-                    for (int i = lane; i < slots; i += 32) sn += (double)__ldcg(pn + i);
-                    sn = warp_sum(sn);
-                    if (lane == 0) {
-                        const float f = clip_factor(sn, p.C_l);
-                        p.sqnorm[n * p.sq_stride] = (float)sn;
-                        if (p.clip_out) p.clip_out[n] = f;
-                        p.factor_out[n] = f;
-                        tickets[n] = 0;
-                        st_release_gpu(&ready[n], 1);
-                    }
-                }
+            };
+            for (int cc = 0; cc < n_cols; cc += 64) {
+                uint32_t v0[32], v1[32];
+                tmem_ld32_issue(t_addr + (uint32_t)cc, v0);
+                tmem_ld32_issue(t_addr + (uint32_t)(cc + 32), v1);
+                tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+                put(v0, cc);
+                if (cc + 32 < n_cols) put(v1, cc + 32);
             }
-            if (step >= kClip2Lag) {
-                // scale example m, handed in three steps ago, once its factor is known
-                const int m = step - kClip2Lag, buf = m & 3;
-                int ok = 0;
-                if (lane == 0) {
-                    for (uint32_t it = 0; it < p.wait_polls; ++it) {
-                        if (ld_acquire_gpu(&ready[m]) != 0) { ok = 1; break; }
-                        if ((it & 63u) == 63u && *abort_p) break;
-                        __nanosleep(64);
-                    }
-                    if (!ok) *abort_p = 1;
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) { live = false; break; }
-                const float f = __ldcg(p.factor_out + m);
-                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 128) + ((uint32_t)(q * 32) << 16);
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
-                    if (c2 * 64 < n_cols) {
-                        uint32_t v0[32], v1[32];
-                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
-                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
-                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
-            }
-        }
-        if (live && row_ok) {
-            // this CTA owns its tile of the clipped sum for the whole batch: add straight into the accumulator
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                if (c4 * 32 < n_cols) {
-                    const int b_idx = nt * p.NT + c4 * 32;
-                    if (p.a_is_x) {
-                        float *dst = p.sum_out + (long long)b_idx * p.Ng + a_idx;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) dst[(long long)i * p.Ng] += run[c4 * 32 + i];
-                    } else if (!p.n_pad_cols) {
-                        float4 *dst = reinterpret_cast<float4 *>(p.sum_out + (long long)a_idx * p.Ng + b_idx);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            float4 o = dst[i];
-                            o.x += run[c4 * 32 + 4 * i]; o.y += run[c4 * 32 + 4 * i + 1]; o.z += run[c4 * 32 + 4 * i + 2]; o.w += run[c4 * 32 + 4 * i + 3];
-                            dst[i] = o;
-                        }
-                    } else {
-                        float *dst = p.sum_out + (long long)a_idx * p.Ng + b_idx;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (b_idx + i < p.Ng) dst[i] += run[c4 * 32 + i];
-                    }
-                }
-            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            buf ^= 1;
         }
     }
 
@@ -1191,14 +1124,28 @@ conv_wgrad_clip2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         if (threadIdx.x == 0) { *p.status = DP_ERR_TIMEOUT; __threadfence(); }
         __nanosleep(200000);
         __syncthreads();
-    } else if (threadIdx.x == 0) {
-        // the last CTA to leave clears the flags for the next call: by then every CTA has read all of them
-        if (atomicAdd(exit_ticket, 1) == (int)gridDim.x - 1) {
-            for (int n = 0; n < p.B; ++n) ready[n] = 0;
-            *exit_ticket = 0;
-        }
     }
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
+// hi[i] = bf16(f_n y[i]), lo[i] = bf16(f_n y[i] - hi[i]) for every entry of example n (eight entries per thread)
+__global__ void __launch_bounds__(256)
+scale_split_kernel(const __nv_bfloat16 *__restrict__ y, const float *__restrict__ factor, long long per_example, long long total8,
+                   __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo) {
+    const long long i8 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i8 >= total8) return;
+    const long long i = i8 * 8;
+    const float f = factor[2 * (i / per_example)];
+    __nv_bfloat16 v[8], h[8], l[8];
+    *reinterpret_cast<uint4 *>(v) = *reinterpret_cast<const uint4 *>(y + i);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const float x = f * __bfloat162float(v[e]);
+        h[e] = __float2bfloat16_rn(x);
+        l[e] = __float2bfloat16_rn(x - __bfloat162float(h[e]));
+    }
+    *reinterpret_cast<uint4 *>(hi + i) = *reinterpret_cast<const uint4 *>(h);
+    *reinterpret_cast<uint4 *>(lo + i) = *reinterpret_cast<const uint4 *>(l);
 }
 
 // acc[i] += sum over splits of part[s][i], splits in index order (P a multiple of 4, both 16-byte aligned)
@@ -1328,11 +1275,21 @@ struct TcProblem {
     int n_pad;          // unfolded row length (columns incl. zero padding)
 };
 
+// A 1 x 1 convolution with stride 1 is a plain product over the pixels, whatever their arrangement: its planes are
+// flattened to one row of H*W pixels, so that a pixel tile is any run of pixels (no width / height rounding: 14 x 14
+// is 208 reduction rows instead of 240) and a TMA box is one long run instead of many short rows.
+static void flatten_pointwise(ConvGeom &e) {
+    if (e.R == 1 && e.S == 1 && e.stride == 1 && e.pad == 0 && e.H > 1) {
+        e.W = e.H * e.W; e.H = 1;
+        e.OW = e.OH * e.OW; e.OH = 1;
+    }
+}
+
 static TcProblem tc_problem(int dtype, const ConvGeom &g) {
     TcProblem pr; pr.ok = false; pr.unfold = false; pr.eff = g; pr.n_pad = g.N;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     if (g.Kout % slab_ch) return pr;
-    if (g.Cin % slab_ch == 0) { pr.ok = true; return pr; }
+    if (g.Cin % slab_ch == 0) { pr.ok = true; flatten_pointwise(pr.eff); return pr; }
     // small-channel layers only: the unfolded copy costs N/C_in times the input, which is only worth it for thin inputs
     if (g.Cin > 8 || g.N > 512) return pr;
     pr.unfold = true;
@@ -1340,6 +1297,7 @@ static TcProblem tc_problem(int dtype, const ConvGeom &g) {
     ConvGeom e = g;
     e.H = g.OH; e.W = g.OW; e.Cin = pr.n_pad; e.R = 1; e.S = 1; e.stride = 1; e.pad = 0;
     e.N = pr.n_pad;
+    flatten_pointwise(e);
     pr.eff = e;
     pr.ok = true;
     return pr;
@@ -1365,9 +1323,23 @@ static double step_cycles(int dtype, int n_cols, double a_slabs_loaded, double b
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode);
 
 // single-pass clipped sum: how many clusters share the batch and how many examples each walks through
+// scaled-sum product: example ranges per tile.  A launch that already has a CTA for a quarter of the SMs keeps whole
+// tiles (no partial sums to fold); fewer tiles are cut up to half of the SMs.
+static void ssum_split(int B, int tiles, int &splits, int &per_split) {
+    const int sms = sm_target();
+    int want = (tiles * 4 >= sms) ? 1 : (sms / 2) / tiles;
+    if (want < 1) want = 1;
+    if (want > B) want = B;
+    per_split = (B + want - 1) / want;
+    splits = (B + per_split - 1) / per_split;
+}
+
 static int max_active_clusters(int cluster_size);
 static void cluster_split(int B, int cluster_size, int &splits, int &per_split) {
     int want = std::min(sm_target() / cluster_size, max_active_clusters(cluster_size));
+    // A caller that set an SM target runs calls side by side: what counts then is SM time, and a cluster that walks
+    // through several examples spends its start-up, its first loads and its final stores once for all of them.
+    if (sm_target_set()) want = std::min(want, std::max(1, B / kMinExamplesPerCluster));
     if (want < 1) want = 1;
     if (want > B) want = B;
     per_split = (B + want - 1) / want;
@@ -1379,7 +1351,7 @@ static void cluster_split(int B, int cluster_size, int &splits, int &per_split) 
 static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
     static std::mutex mu;
     static std::map<std::array<int, 12>, TcPlan> memo;
-    const std::array<int, 12> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, mode, sm_target()};
+    const std::array<int, 12> key = {dtype, g.H, g.W, g.Cin, g.Kout, g.R, g.S, g.stride, g.pad, g.B, mode, sm_target_set() ? -sm_target() : sm_target()};
     std::lock_guard<std::mutex> lock(mu);
     auto it = memo.find(key);
     if (it != memo.end()) return it->second;
@@ -1393,7 +1365,7 @@ static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
 // mode 3 plans the single-pass clipped sum: all tiles of an example in one cluster (at most kMaxCluster of them), the
 // clusters share the batch, and what is minimised is SM time (clusters x CTAs x time), not the time of one launch
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
-    const int max_nt = (mode == 2 || mode == 4) ? 128 : 256;
+    const int max_nt = (mode == 2) ? 128 : 256;
     TcPlan best; best.ok = false;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
@@ -1413,14 +1385,16 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
             if (total_tiles > 0x7fffffffLL) continue;
             if (mode == 3 && m_tiles * n_tiles > kMaxCluster) continue;
-            if (mode == 4 && m_tiles * n_tiles > sm_count()) continue;      // one resident CTA per tile
+            const int y_slabs = (mode == 4) ? (a_is_x ? NT / slab_ch : a_slabs_tile) : 0;     // second (lo) copy of the dY slabs
             // per-CTA share of (example, tile) units: whole waves of tiles, or in clipped-sum mode an even share of the examples
             double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
                                        : std::max(1.0, (double)total_tiles / sms);
             double sm_share = 1.0;
             if (mode == 4) {
-                waves = g.B;                                       // every CTA walks the whole batch for its tile
-                sm_share = (double)m_tiles * n_tiles;
+                int splits, per;
+                ssum_split(g.B, m_tiles * n_tiles, splits, per);
+                waves = per;
+                sm_share = (double)std::min(splits * m_tiles * n_tiles, sms);
             }
             if (mode == 3) {
                 int splits, per;
@@ -1429,22 +1403,22 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
                 sm_share = (double)splits * m_tiles * n_tiles;      // SMs the launch holds meanwhile
             }
             const double a_loaded = (double)(a_ext / slab_ch) / m_tiles, b_loaded = (double)(b_ext / slab_ch) / n_tiles;
-            const double step = step_cycles(dtype, NT, a_loaded, b_loaded);
+            const double step = step_cycles(dtype, NT, a_loaded, b_loaded) * (mode == 4 ? 2.0 : 1.0);
             // the epilogue of a tile overlaps the main loop of the next; what it costs depends on what it does with
             // the 128 x NT accumulator: stores run at about 16 B/clk per SM when lanes write consecutive addresses
             // (rows of D are gradient columns) and about 7 B/clk otherwise; reading TMEM alone is cheap
             const double epilogue = (mode == 0) ? 128.0 * NT * 4.0 / (a_is_x ? 16.0 : 7.0)
-                                  : (mode == 1 ? 6.0 * NT : (mode == 2 ? 10.0 * NT : (mode == 4 ? 9.0 * NT : 10.0 * std::min(NT, 128) + 600.0)));
+                                  : (mode == 1 ? 6.0 * NT : (mode == 2 ? 10.0 * NT : (mode == 4 ? 0.0 : 10.0 * std::min(NT, 128) + 600.0)));
             // a pixel tile may reach past the output plane (its rows there are zero-filled by TMA and add nothing):
             // a 7 x 7 plane is one 8 x 8 tile of 64 reduction rows instead of four 4 x 4 tiles of 16
-            const int oh_max = std::min((g.OH + 7) / 8 * 8, 256 / g.stride), ow_max = std::min((g.OW + 7) / 8 * 8, 256 / g.stride);
+            const int oh_max = std::min((g.OH + 7) / 8 * 8, 256 / g.stride), ow_max = std::min((g.OW + 15) / 16 * 16, 256 / g.stride);
             for (int OHt = 1; OHt <= oh_max; ++OHt) {
                 for (int OWt = 1; OWt <= ow_max; ++OWt) {
                     if (OWt > g.OW && OWt % 8) continue;      // overshoot only to the next multiple of eight
                     if (OHt > g.OH && OHt % 8) continue;
                     const int Kt = OHt * OWt;
                     if (Kt % krows || Kt > 256) continue;
-                    const int stage_bytes = slabs * Kt * kRowBytes * copies;
+                    const int stage_bytes = (slabs + y_slabs) * Kt * kRowBytes * copies;
                     int stages = kSmemBudget / stage_bytes;
                     if (stages < 2) continue;
                     if (stages > kMaxStages) stages = kMaxStages;
@@ -1457,7 +1431,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
                         stage_cost = std::max(stage_cost, 0.5 * (1000.0 + (a_loaded + b_loaded) * Kt * 2.5));
                     double mainloop = stage_cost * tw * th;
                     if (stages < 3) mainloop *= 1.15;
-                    const double cost = ((std::max(mainloop, epilogue) + 300.0) * waves + (mode >= 3 ? 4000.0 : 0.0)) * sm_share;
+                    const double cost = ((std::max(mainloop, epilogue) + 300.0) * waves + (mode == 3 ? 4000.0 : (mode == 4 ? 6000.0 : 0.0))) * sm_share;
                     if (cost < best_cost) {
                         best_cost = cost;
                         best.ok = true; best.a_is_x = a_is_x; best.a_ext = a_ext; best.b_ext = b_ext;
@@ -1522,14 +1496,6 @@ static bool clip1_plan(int dtype, const ConvGeom &eff, TcPlan &pl) {
     return pl.ok;
 }
 
-// true when the fused clipped sum of this layer runs as one contraction with the grid-wide exchange of partial norms
-// (bf16 inputs, one resident CTA per 128-column tile, tickets and flags for B examples in the workspace header)
-static bool clip2_plan(int dtype, const ConvGeom &eff, TcPlan &pl) {
-    if (dtype != DP_BF16 || 2 * eff.B + 1 > kWsCounters) return false;
-    pl = make_plan(dtype, eff, 4);
-    return pl.ok;
-}
-
 // clipped-sum mode: how many example ranges each tile is cut into so that every SM has an item
 static void clip_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &per_split) {
     const int tiles = pl.m_tiles * pl.n_tiles;
@@ -1544,10 +1510,7 @@ int tc_norm_slots(int dtype, const ConvGeom &g0, int epilogue) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
     const TcPlan pl = make_plan(dtype, pr.eff, epilogue == DP_EPI_STORE_NORM ? 0 : 1);
-    int slots = pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
-    TcPlan two;
-    if (epilogue == DP_EPI_CLIP_ACCUM && clip2_plan(dtype, pr.eff, two)) slots = std::max(slots, two.m_tiles * two.n_tiles * 4);
-    return slots;
+    return pl.ok ? pl.m_tiles * pl.n_tiles * 4 : 0;
 }
 
 static size_t unfold_bytes(int dtype, const ConvGeom &g0, const TcProblem &pr) {
@@ -1555,7 +1518,10 @@ static size_t unfold_bytes(int dtype, const ConvGeom &g0, const TcProblem &pr) {
     return round_up((size_t)g0.B * g0.OH * g0.OW * pr.n_pad * (dtype == DP_BF16 ? 2 : 4), 1024);
 }
 
-// layout: [unfolded input, if any][partial sums of the clipped-sum mode, if any]
+static size_t ssum_copy_bytes(const ConvGeom &g) { return round_up((size_t)g.B * g.OH * g.OW * g.Kout * 2, 1024); }
+bool tc_clip_scaled_sum(int dtype, const ConvGeom &g0);
+
+// layout: [unfolded input, if any][partial sums of the clipped-sum mode, if any], or the scaled copies of dY and partial sums
 size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
@@ -1571,7 +1537,14 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
             cluster_split(pr.eff.B, one.m_tiles * one.n_tiles, s1, p1);
             splits = std::max(splits, s1);
         }
-        if (splits > 1) bytes += sizeof(float) * (size_t)splits * g0.M * g0.N;
+        size_t clip_bytes = splits > 1 ? sizeof(float) * (size_t)splits * g0.M * g0.N : 0;
+        if (tc_clip_scaled_sum(dtype, g0)) {
+            const TcPlan sp = make_plan(dtype, pr.eff, 4);
+            int s4, p4;
+            ssum_split(pr.eff.B, sp.m_tiles * sp.n_tiles, s4, p4);
+            clip_bytes = std::max(clip_bytes, 2 * ssum_copy_bytes(pr.eff) + (s4 > 1 ? sizeof(float) * (size_t)s4 * g0.M * g0.N : 0));
+        }
+        bytes += clip_bytes;
     }
     return bytes;
 }
@@ -1699,56 +1672,53 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
     return DP_OK;
 }
 
-int tc_clip_grid_pass(int dtype, const ConvGeom &g0) {
+// The fused clipped sum of a bf16 layer that does not fit a cluster: norm pass, then ONE matrix product over all examples.
+bool tc_clip_scaled_sum(int dtype, const ConvGeom &g0) {
     const TcProblem pr = tc_problem(dtype, g0);
-    TcPlan pl;
-    if (!pr.ok || pr.unfold || !encode_fn() || !clip2_plan(dtype, pr.eff, pl)) return 0;
-    static int coop = -1;
-    if (coop < 0) {
-        int dev = 0, v = 0;
-        coop = (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : 0;
-    }
-    return coop;
+    return dtype == DP_BF16 && pr.ok && !pr.unfold && encode_fn() && g0.Kout % 8 == 0 && make_plan(dtype, pr.eff, 4).ok;
 }
 
-dp_status launch_conv_clip2(int dtype, const void *X, const void *dY, const ConvGeom &g0, float *partial, float *factor,
-                            int *counters, const TcInlineClip &clipinfo, float *acc_w, int *status, cudaStream_t stream) {
+dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvGeom &g0, const float *factor, float *acc_w,
+                           void *tc_workspace, int *status, cudaStream_t stream) {
+    if (!tc_clip_scaled_sum(dtype, g0)) return DP_ERR_UNSUPPORTED;
     const TcProblem pr = tc_problem(dtype, g0);
-    TcPlan pl;
-    if (!pr.ok || pr.unfold || !encode_fn() || !clip2_plan(dtype, pr.eff, pl)) return DP_ERR_UNSUPPORTED;
     const ConvGeom &g = pr.eff;
-    CUtensorMap tmX, tmY;
+    const TcPlan pl = make_plan(dtype, g, 4);
+    char *ws_bytes = static_cast<char *>(tc_workspace);
+    __nv_bfloat16 *hi = reinterpret_cast<__nv_bfloat16 *>(ws_bytes), *lo = reinterpret_cast<__nv_bfloat16 *>(ws_bytes + ssum_copy_bytes(g));
+    float *part_ws = reinterpret_cast<float *>(ws_bytes + 2 * ssum_copy_bytes(g));
+    {
+        const long long per_example = (long long)g.OH * g.OW * g.Kout, total8 = per_example * g.B / 8;
+        DP_MAX_SHARED_CARVEOUT((scale_split_kernel));
+        scale_split_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, stream>>>(static_cast<const __nv_bfloat16 *>(dY), factor, per_example, total8, hi, lo);
+        DP_LAUNCH_CHECK("scale_split_kernel");
+    }
+    CUtensorMap tmX, tmYhi, tmYlo;
     if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
-    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    if (!encode_nhwc(&tmYhi, dtype, hi, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY hi)");
+    if (!encode_nhwc(&tmYlo, dtype, lo, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY lo)");
     TcParams p = {};
-    p.B = g.B; p.Kout = g.Kout; p.Ng = g0.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
-    p.n_pad_cols = 0;
+    p.B = g.B; p.Kout = g.Kout; p.Ng = g.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
     p.slab_ch = 64; p.krows = 16;
     p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
     p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
-    p.mode = 4; p.status = status;
+    p.lo_offset = pl.a_bytes + (pl.NT / 64) * pl.Kt * kRowBytes;      // after the A and B slabs
+    p.mode = 2; p.status = status;                                    // items are (example range, tile) pairs
     p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
-    p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
-    p.partial = partial; p.slots = pl.m_tiles * pl.n_tiles * 4;
-    p.factor_out = factor; p.counters = counters;
-    p.splits = 1; p.per_split = g.B; p.sum_out = acc_w;
-    p.total_tiles = pl.m_tiles * pl.n_tiles;
+    ssum_split(g.B, pl.m_tiles * pl.n_tiles, p.splits, p.per_split);
+    p.sum_out = p.splits > 1 ? part_ws : acc_w;
+    p.total_tiles = p.splits * pl.m_tiles * pl.n_tiles;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(conv_wgrad_clip2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        attr_err = cudaFuncSetAttribute(conv_wgrad_ssum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)p.total_tiles); cfg.blockDim = dim3(224); cfg.dynamicSmemBytes = pl.smem; cfg.stream = stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeCooperative;       // all CTAs resident at once: the ones that poll can rely on the others running
-    at[0].val.cooperative = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    const cudaError_t le = cudaLaunchKernelEx(&cfg, conv_wgrad_clip2_kernel, tmX, tmY, p);
-    if (le != cudaSuccess) return cuda_fail(le, "conv_wgrad_clip2_kernel");
-    DP_LAUNCH_CHECK("conv_wgrad_clip2_kernel");
+    const unsigned grid = (unsigned)std::min(p.total_tiles, sm_target());
+    conv_wgrad_ssum_kernel<<<grid, 224, pl.smem, stream>>>(tmX, tmYhi, tmYlo, p);
+    DP_LAUNCH_CHECK("conv_wgrad_ssum_kernel");
+    if (p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g.M * g.N, acc_w, stream);
     return DP_OK;
 }
 

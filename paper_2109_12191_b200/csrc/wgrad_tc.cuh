@@ -36,12 +36,11 @@ bool tc_clip_single_pass(int dtype, const ConvGeom &g);
 dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const ConvGeom &g, float *partial, int slots,
                             const TcInlineClip &clipinfo, float *acc_w, void *tc_workspace, int *status, cudaStream_t stream);
 
-// Layers too large for one cluster run the single contraction with a grid-wide exchange of partial norms instead (a
-// cooperative launch, one CTA per 128-column tile).  partial: [B][tiles*4] floats (tc_norm_slots covers it), factor: [B]
-// floats, counters: 2*B + 1 cleared ints.  Layers without bias, not unfolded.
-int tc_clip_grid_pass(int dtype, const ConvGeom &g);
-dp_status launch_conv_clip2(int dtype, const void *X, const void *dY, const ConvGeom &g, float *partial, float *factor,
-                            int *counters, const TcInlineClip &clipinfo, float *acc_w, int *status, cudaStream_t stream);
+// bf16 layers too large for one cluster: after the norm pass has published the factors (factor[2n]), the clipped sum is
+// ONE matrix product over all examples with f_n dY split into hi + lo bf16 copies (kept in tc_workspace).  No bias, not unfolded.
+bool tc_clip_scaled_sum(int dtype, const ConvGeom &g);
+dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvGeom &g, const float *factor, float *acc_w,
+                           void *tc_workspace, int *status, cudaStream_t stream);
 
 // Test hook: the number of polls after which a bounded wait of the kernel gives up (0 makes every wait give up at once).
 void set_wait_polls(uint32_t polls);
