@@ -127,6 +127,8 @@ class SmallCnn:
         self.cfg = synth.small_cnn()
         self.layers, self.B = self.cfg["layers"], self.cfg["B"]
         self.lanes = int(os.environ.get("DP_BENCH_LANES", "4"))
+        from paper_2109_12191_b200 import binding
+        binding.check(binding.dp_set_sm_target(0))
         # layers whose per-example gradients outweigh their inputs (conv3, the classifier) are not materialised
         self.recompute = os.environ.get("DP_BENCH_RECOMPUTE", "auto")
         # fp32 inputs; tensor-core layers take them as tf32 (one pass, the precision class the accuracy bounds name)
@@ -374,8 +376,13 @@ class PerLayer:
         self.torch, self.synth, self.dist, self.world, self.b = torch, synth, dist, world, binding
         self.cfg = self.config(synth)
         self.layers, self.B, self.G = self.cfg["layers"], self.cfg["B"], self.cfg["G"]
-        self.lanes = int(os.environ.get("DP_BENCH_LANES", "4"))
-        self.sm_target = int(os.environ.get("DP_BENCH_SM_TARGET", "0"))
+        only = os.environ.get("DP_BENCH_ONLY")           # experiments: time one layer kind alone ("conv", "norm")
+        if only:
+            self.layers = [l for l in self.layers if l.kind == only]
+        # the layer calls of a chunk run side by side on 16 streams; the SM target (here: all SMs, which still switches
+        # the library's tiling from "fastest single call" to "least SM time") is set for that
+        self.lanes = int(os.environ.get("DP_BENCH_LANES", "16"))
+        self.sm_target = int(os.environ.get("DP_BENCH_SM_TARGET", str(torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count)))
         binding.check(binding.dp_set_sm_target(self.sm_target))
         self.step_obj = PerLayerClipStep(self.layers, self.B, "bf16", self.cfg["C"], self.cfg["sigma"], lanes=self.lanes)
         self.examples_per_step = self.B * self.G
@@ -413,7 +420,7 @@ class PerLayer:
         return {"workload": self.workload_text(self.layers, self.step_obj.L),
                 "examples_per_step": self.examples_per_step, "params": self.step_obj.P,
                 "l2": f"one chunk of inputs is {self.in_bytes / 1e9:.2f} GB, far larger than L2",
-                "streams": self.lanes}
+                "streams": self.lanes, "sm_target": self.sm_target}
 
     def run(self, i, rec=None):
         """With a recorder the calls run one after the other on one stream so that each can be timed; otherwise the
@@ -454,11 +461,35 @@ class PerLayer:
     def algorithmic_bytes(self, call):
         return self.bytes_kind[call] if call < 4 else 2 * self.step_obj.P * 4
 
+    def class_times_ms(self, reps=20):
+        """ms per chunk of each kind of layer call on its own, in the launch mode of the timed region (the chunk's calls
+        of that kind captured into a CUDA graph over the step object's streams, replayed `reps` times between two events)."""
+        t, st, out = self.torch, self.step_obj, []
+        for kind in range(4):
+            only = {li for li, k in enumerate(self.kind_of) if k == kind}
+            if not only:
+                out.append(0.0)
+                continue
+            g = t.cuda.CUDAGraph()
+            with t.cuda.graph(g):
+                st.chunk_calls(self.inputs, only=only)
+            for _ in range(3):
+                g.replay()
+            e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                g.replay()
+            e1.record()
+            t.cuda.synchronize()
+            out.append(e0.elapsed_time(e1) / reps)
+        return out
+
     def roofline(self, dom, totals, prof_steps, peaks):
         """Tensor-core convs are reported against the sustained bf16 tensor peak (they are timed inside a long step;
         flops counted once even where a two-pass scheme executes them twice); the normalisation layers against HBM;
         and the whole chunk against the sum over layers of max(HBM time, tensor time) at the measured peaks."""
-        per_chunk = [t / (prof_steps * self.G) for t in totals]          # ms per chunk of each call class, one stream
+        per_chunk = self.class_times_ms()                                 # ms per chunk of each call class, replayed alone
+        dom = max(range(4), key=lambda k: per_chunk[k])
         gn_gbs = self.bytes_kind[2] / (per_chunk[2] / 1e3) / 1e9 if per_chunk[2] > 0 else 0.0
         ceiling_ms = 0.0
         for l, (x, y), k in zip(self.layers, self.inputs, self.kind_of):
@@ -468,14 +499,20 @@ class PerLayer:
         extra = {"norm_affine": {"bound": "hbm", "achieved": round(gn_gbs, 1), "peak": peaks["hbm"], "unit": "GB/s",
                                  "frac": round(gn_gbs / peaks["hbm"], 4), "algorithmic_bytes": self.bytes_kind[2],
                                  "avg_ms_per_chunk": round(per_chunk[2], 5)},
-                 "chunk_ceiling": {"ms_at_measured_peaks": round(ceiling_ms, 4), "ms_one_stream": round(sum(per_chunk[:4]), 4),
-                                   "frac": round(ceiling_ms / max(sum(per_chunk[:4]), 1e-9), 4)}}
+                 "chunk_ceiling": {"ms_at_measured_peaks": round(ceiling_ms, 4), "ms_classes_alone": round(sum(per_chunk[:4]), 4),
+                                   "frac": round(ceiling_ms / max(sum(per_chunk[:4]), 1e-9), 4)},
+                 "class_ms_per_chunk": {n: round(v, 4) for n, v in zip(self.call_names[:4], per_chunk)},
+                 "how": "each kind of layer call captured alone into a CUDA graph over the same streams and replayed; "
+                        "`shares` come from the eager one-stream pass and include host launch gaps"}
         if dom != 0:
             return extra
         tf = self.flops_tc / (per_chunk[0] / 1e3) / 1e12
-        return dict(extra, bound="tensor", achieved=round(tf, 1), peak=peaks["bf16_sustained"], unit="TFLOP/s",
+        n_tc = max(1, sum(1 for k in self.kind_of if k == 0))
+        return dict(extra, bound="tensor", kernel="wgrad:conv (tensor core): the chunk's %d fused clip calls" % n_tc,
+                    achieved=round(tf, 1), peak=peaks["bf16_sustained"], unit="TFLOP/s",
                     frac=round(tf / peaks["bf16_sustained"], 4), algorithmic_flops=self.flops_tc,
-                    avg_ms_per_launch=round(per_chunk[0] / max(1, sum(1 for k in self.kind_of if k == 0)), 5))
+                    algorithmic_bytes=self.bytes_kind[0], avg_ms_per_launch=round(per_chunk[0], 5),
+                    launch="one launch = the chunk's tensor-core calls replayed as one graph")
 
     def e2e_prepare(self):
         t = self.torch

@@ -552,7 +552,6 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
         sq = sq_ws;
     }
     if (!stage3_only) {
-        DP_MAX_SHARED_CARVEOUT((clip_factor_kernel));
         const long long count = per_layer ? (long long)B * L : B;
         if (var.groups)
             clip_factor_grouped_kernel<<<(unsigned)B, 128, 0, stream>>>(sq, L, *var.groups, C, factor_ws, norms_out, clip_out);
@@ -568,8 +567,6 @@ static dp_status clip_accumulate_impl(int mode, int B, int L, const float *const
             SegTable t;
             const int blocks = fill(l0, t, false, cursor);
             if (t.nseg == 0) return DP_ERR_UNSUPPORTED;
-            DP_MAX_SHARED_CARVEOUT((scale_accumulate_rowsplit_kernel));
-            DP_MAX_SHARED_CARVEOUT((scale_accumulate_kernel<8>));
             if (noise) scale_accumulate_noised_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer, *noise);
             else if (split) scale_accumulate_rowsplit_kernel<<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
             else scale_accumulate_kernel<8><<<(unsigned)blocks, 256, 0, stream>>>(t, factor, B, L, per_layer);
@@ -595,7 +592,6 @@ extern "C" dp_status dp_clip_factors(int mode, int B, int L, const float *sqnorm
     if (!dp::aligned(sqnorm, 4) || !dp::aligned(factors_out, 4) || (norms_out && !dp::aligned(norms_out, 4))) return DP_ERR_INVALID_ARG;
     const int per_layer = (mode == DP_CLIP_PER_LAYER);
     const long long count = per_layer ? (long long)B * L : B;
-    DP_MAX_SHARED_CARVEOUT((dp::clip_factor_kernel));
     dp::clip_factor_kernel<<<(unsigned)((count + 127) / 128), 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         sqnorm, B, L, per_layer, C, factors_out, norms_out, nullptr);
     DP_LAUNCH_CHECK("clip_factor_kernel");

@@ -40,17 +40,6 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Host-side count of kernel launches made by this process (read by dp_debug_launch_count).
 void count_launch();
 
-// Before a launch: asks once for the largest shared-memory carve-out for this kernel.  The tensor-core kernel needs
-// nearly all of an SM's shared memory; an SM whose L1 / shared-memory split has to change between two kernels must
-// drain first, which serialises kernels that could otherwise follow or overlap each other.  With every kernel of the
-// library on the same split no such change happens.  (A hint: its failure is ignored.)
-#define DP_MAX_SHARED_CARVEOUT(kern)                                                                              \
-    do {                                                                                                          \
-        static const cudaError_t carve__ = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, \
-                                                                (int)cudaSharedmemCarveoutMaxShared);            \
-        (void)carve__;                                                                                            \
-    } while (0)
-
 // After a kernel launch: picks up launch-configuration errors without synchronising.
 #define DP_LAUNCH_CHECK(name)                                          \
     do {                                                               \

@@ -488,8 +488,6 @@ dp_status launch_conv_rgb3(int dtype, const void *X, const void *dY, const ConvG
                            int has_bias, int separate, float *sqnorm, long long sq_stride,
                            cudaStream_t st) {
     const size_t smem = rgb3_smem_bytes(g);
-    DP_MAX_SHARED_CARVEOUT((conv_wgrad_rgb3_kernel<float>));
-    DP_MAX_SHARED_CARVEOUT((conv_wgrad_rgb3_kernel<__nv_bfloat16>));
     if (dtype == DP_F32)
         conv_wgrad_rgb3_kernel<float><<<g.B, 256, smem, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), g,
                                                               G_w, db, has_bias, separate, sqnorm, sq_stride);
@@ -1021,7 +1019,6 @@ affine_clip_accum_kernel(const float *__restrict__ partial2, int B, float C_l, i
 dp_status launch_affine_clip_accum(const float *partial2, int B, float C_l, int separate, float *sqnorm, long long sq_stride,
                                    float *clip_out, const float *dgamma, const float *dbeta, int C, float *acc_w,
                                    float *acc_b, cudaStream_t st) {
-    DP_MAX_SHARED_CARVEOUT((affine_clip_accum_kernel));
     affine_clip_accum_kernel<<<(C + 127) / 128, 128, 0, st>>>(partial2, B, C_l, separate, sqnorm, sq_stride, clip_out, dgamma,
                                                             dbeta, C, acc_w, acc_b);
     DP_LAUNCH_CHECK("affine_clip_accum_kernel");
@@ -1060,7 +1057,6 @@ static dp_status conv_fma_t(int mode, const T *X, const T *dY, const ConvGeom &g
     DP_LAUNCH_CHECK("conv_wgrad_fma_kernel");
     if (mode == 2 && splits > 1) {
         const long long P = (long long)g.M * g.N;
-        DP_MAX_SHARED_CARVEOUT((fold_sums_kernel));
         fold_sums_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(sum_ws, splits, P, acc_w);
         DP_LAUNCH_CHECK("fold_sums_kernel");
     }
@@ -1079,8 +1075,6 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
     const int vec = (dtype == DP_F32) ? 4 : 8;
     if (g.Kout % vec == 0 && g.Kout / vec <= 256 && bias_blocks(g) <= 256) {
         const size_t smem = sizeof(float) * (size_t)(256 / (g.Kout / vec)) * g.Kout;
-        DP_MAX_SHARED_CARVEOUT((bias_vec_kernel<float, 4>));
-        DP_MAX_SHARED_CARVEOUT((bias_vec_kernel<__nv_bfloat16, 8>));
         if (dtype == DP_F32)
             bias_vec_kernel<float, 4><<<g.B, 256, smem, st>>>(static_cast<const float *>(dY), g.K, g.Kout, db, partial, slots, slot0, bias_blocks(g));
         else
@@ -1098,14 +1092,12 @@ dp_status launch_bias(int dtype, const void *dY, const ConvGeom &g, float *db, f
 
 dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, int separate, float *sqnorm,
                           long long sq_stride, int clip, float C_l, float *factor, float *clip_out, cudaStream_t st) {
-    DP_MAX_SHARED_CARVEOUT((finalize_norm_kernel));
     finalize_norm_kernel<<<B, 128, 0, st>>>(partial, slots, w_slots, separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
     DP_LAUNCH_CHECK("finalize_norm_kernel");
     return DP_OK;
 }
 
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t st, int which) {
-    DP_MAX_SHARED_CARVEOUT((bias_accum_kernel<float>));
     bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(db, B, Kout, factor + which, 2, acc_b);
     DP_LAUNCH_CHECK("bias_accum_kernel");
     return DP_OK;
@@ -1125,8 +1117,6 @@ dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, cons
                                   int Cin, int Kout, float *acc_w, cudaStream_t st) {
     const dim3 grid((unsigned)((Cin + 31) / 32), (unsigned)((Kout + kDenseOT - 1) / kDenseOT));
     if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
-    DP_MAX_SHARED_CARVEOUT((dense_scaled_sum_kernel<float>));
-    DP_MAX_SHARED_CARVEOUT((dense_scaled_sum_kernel<__nv_bfloat16>));
     if (dtype == DP_F32)
         dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, f_stride, B, Cin, Kout, acc_w);
     else
@@ -1136,7 +1126,6 @@ dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, cons
 }
 
 dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2, cudaStream_t st) {
-    DP_MAX_SHARED_CARVEOUT((expand_factor_kernel));
     expand_factor_kernel<<<(B + 127) / 128, 128, 0, st>>>(factor_w, factor_b, stride, B, factor2);
     DP_LAUNCH_CHECK("expand_factor_kernel");
     return DP_OK;
@@ -1166,8 +1155,6 @@ dp_status launch_dense_store(int dtype, const void *X, const void *dY, int B, in
 dp_status launch_dense_norm(int dtype, const void *X, const void *dY, int B, int Cin, int Kout, int has_bias, float *db,
                             int separate, float *sqnorm, long long sq_stride, int clip, float C_l, float *factor,
                             float *clip_out, cudaStream_t st) {
-    DP_MAX_SHARED_CARVEOUT((dense_norm_kernel<float>));
-    DP_MAX_SHARED_CARVEOUT((dense_norm_kernel<__nv_bfloat16>));
     if (dtype == DP_F32)
         dense_norm_kernel<<<B, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), Cin, Kout, has_bias, db,
                                              separate, sqnorm, sq_stride, clip, C_l, factor, clip_out);
@@ -1188,7 +1175,6 @@ static dp_status norm_affine_t(const T *X, const T *dY, int B, int HW, int C, in
     const size_t smem = sizeof(float) * (size_t)(256 / tcv) * tcv * VEC * 2;
     folded = grid.x == 1 && chunks == 1;      // one block sees the whole example: it finishes the job itself
     tail.blocks_per_example = (int)(grid.x * grid.y);
-    DP_MAX_SHARED_CARVEOUT((norm_affine_partial_kernel<T, VEC>));
     norm_affine_partial_kernel<T, VEC><<<grid, 256, smem, st>>>(X, dY, HW, C, tcv, pix, chunk_partial, chunks,
                                                                folded ? dgamma : nullptr, dbeta, partial2, tail);
     DP_LAUNCH_CHECK("norm_affine_partial_kernel");
@@ -1214,7 +1200,6 @@ dp_status launch_norm_affine(int dtype, const void *X, const void *dY, int B, in
     AffineTail off = {};
     const dp_status rc = norm_affine_dispatch(dtype, X, dY, B, HW, C, chunk_partial, dgamma, dbeta, partial2, folded, off, st);
     if (rc != DP_OK || folded) return rc;
-    DP_MAX_SHARED_CARVEOUT((norm_affine_fold_kernel));
     norm_affine_fold_kernel<<<B, 256, 0, st>>>(chunk_partial, norm_chunks(dtype, B, HW, C), C, dgamma, dbeta, partial2);
     DP_LAUNCH_CHECK("norm_affine_fold_kernel");
     return DP_OK;
@@ -1261,7 +1246,6 @@ dp_status launch_norm_affine_fused(int dtype, const void *X, const void *dY, int
     bool folded = false;
     const dp_status rc = norm_affine_dispatch(dtype, X, dY, B, HW, C, chunk_partial, dgamma, dbeta, nullptr, folded, t, st);
     if (rc != DP_OK || !clip || t.accumulate_here) return rc;
-    DP_MAX_SHARED_CARVEOUT((affine_accum_kernel));
     affine_accum_kernel<<<dim3((unsigned)((C + 31) / 32), 2), 256, 0, st>>>(dgamma, dbeta, B, C, factor, acc_w, acc_b);
     DP_LAUNCH_CHECK("affine_accum_kernel");
     return DP_OK;

@@ -1170,8 +1170,6 @@ __global__ void fold_partial_sums_scalar_kernel(const float *__restrict__ part, 
 }
 
 dp_status launch_fold_partial_sums(const float *part, int splits, long long P, float *acc, cudaStream_t stream) {
-    DP_MAX_SHARED_CARVEOUT((fold_partial_sums_kernel));
-    DP_MAX_SHARED_CARVEOUT((fold_partial_sums_scalar_kernel));
     if (P % 4 == 0 && aligned(part, 16) && aligned(acc, 16))
         fold_partial_sums_kernel<<<(unsigned)((P / 4 + 255) / 256), 256, 0, stream>>>(part, splits, P, acc);
     else
@@ -1594,8 +1592,6 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
             const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / vec);
             const unsigned blocks = (unsigned)((total + 255) / 256);
             const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * (dtype == DP_BF16 ? 2 : 4);
-            DP_MAX_SHARED_CARVEOUT((unfold_rows_kernel<__nv_bfloat16, 8>));
-            DP_MAX_SHARED_CARVEOUT((unfold_rows_kernel<float, 4>));
             if (row_smem <= 40 * 1024 && g0.OH <= 0x7fffffff && g0.B <= 65535) {
                 const dim3 grid_rows(g0.OH, g0.B);
                 if (dtype == DP_BF16)
@@ -1689,7 +1685,6 @@ dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvG
     float *part_ws = reinterpret_cast<float *>(ws_bytes + 2 * ssum_copy_bytes(g));
     {
         const long long per_example = (long long)g.OH * g.OW * g.Kout, total8 = per_example * g.B / 8;
-        DP_MAX_SHARED_CARVEOUT((scale_split_kernel));
         scale_split_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, stream>>>(static_cast<const __nv_bfloat16 *>(dY), factor, per_example, total8, hi, lo);
         DP_LAUNCH_CHECK("scale_split_kernel");
     }
@@ -1738,7 +1733,6 @@ dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const Conv
     char *ws_bytes = static_cast<char *>(tc_workspace);
     if (pr.unfold) {
         const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * 2;
-        DP_MAX_SHARED_CARVEOUT((unfold_rows_kernel<__nv_bfloat16, 8>));
         if (row_smem <= 40 * 1024 && g0.B <= 65535) {
             unfold_rows_kernel<__nv_bfloat16, 8><<<dim3(g0.OH, g0.B), 256, row_smem, stream>>>(
                 static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad);

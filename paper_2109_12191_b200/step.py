@@ -334,11 +334,13 @@ class PerLayerClipStep:
                                        b.DP_EPI_CLIP_ACCUM, self.C_l, self.acc_w[li], self.acc_b[li], None,
                                        self.ws_lane[lane], stream=stream), "dp_per_example_wgrad")
 
-    def chunk_calls(self, inputs):
-        """The layer calls of one chunk: in order on the current stream, or forked over the lanes and joined again."""
+    def chunk_calls(self, inputs, only=None):
+        """The layer calls of one chunk: in order on the current stream, or forked over the lanes and joined again.
+        only: a set of layer indices to restrict the chunk to (measurements of one kind of layer)."""
         if self.lanes == 1:
             for li, (X, dY) in enumerate(inputs):
-                self.wgrad(li, X, dY)
+                if only is None or li in only:
+                    self.wgrad(li, X, dY)
             return
         main = torch.cuda.current_stream()
         fork = torch.cuda.Event()
@@ -347,6 +349,8 @@ class PerLayerClipStep:
         for s in self._side:
             s.wait_event(fork)
         for li, (X, dY) in enumerate(inputs):
+            if only is not None and li not in only:
+                continue
             k = self._lane_of[li]
             self.wgrad(li, X, dY, lane=k, stream=streams[k])
         for s in self._side:
