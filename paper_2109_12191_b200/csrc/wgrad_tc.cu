@@ -646,7 +646,7 @@ constexpr int kClipThreads = 384;
 constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
 static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
 constexpr int kMaxCluster = 8;
-constexpr int kMinExamplesPerCluster = 4;   // with an SM target set (calls run side by side)
+constexpr int kMinExamplesPerCluster = 8;   // with an SM target set (calls run side by side)
 
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -684,8 +684,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 __global__ void __launch_bounds__(kClipThreads, 1)
 conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2], norm_bar[2];
-    __shared__ float norm_part[2][kMaxCluster][8];      // [example parity][source CTA][source epilogue warp]
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2], norm_bar[4];
+    __shared__ float norm_part[4][kMaxCluster][8];      // [example mod 4][source CTA][source epilogue warp]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -703,10 +703,8 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 2); mbar_init(smem_u32(&empty_bar[s]), 1); }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 8);
-            mbar_init(smem_u32(&norm_bar[b]), (uint32_t)(cs * 8));
-        }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 8); }
+        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&norm_bar[b]), (uint32_t)(cs * 8));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
@@ -813,73 +811,78 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         float run[128];
 #pragma unroll
         for (int i = 0; i < 128; ++i) run[i] = 0.f;
-        uint32_t full_phase = 0;
         bool live = true;
-        int buf = 0;
-        for (int n = n_lo; n < n_hi; ++n) {
-            const int par = (n - n_lo) & 1;
-            const uint32_t use_parity = (uint32_t)(((n - n_lo) >> 1) & 1);
-            const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
-            if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
-            full_phase ^= 1u << buf;
-            tc_fence_after();
-            const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
-            // pass 1: this warp's share of the example's squared norm
-            float sq4[4] = {0.f, 0.f, 0.f, 0.f};
+        // One step behind: an example's partial sums travel through the cluster while the next example's tile is being
+        // square-summed, and its tile is scaled after that.  Step s hands in example s and then scales example s - 1.
+        // Slots and barriers of the exchange come in fours: a slot of example j is overwritten by example j + 4, which a
+        // warp sends only after it has scaled example j + 2, i.e. after every warp of the cluster has sent example
+        // j + 2, which each of them did after scaling (and so after reading the slots of) example j.
+        const int count = n_hi - n_lo;
+        for (int step = 0; step <= count && live; ++step) {
+            if (step < count) {
+                const int buf = step & 1, slot = step & 3;
+                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (uint32_t)((step >> 1) & 1), abort_p, p.wait_polls);
+                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+                tc_fence_after();
+                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
+                // pass 1: this warp's share of the example's squared norm
+                float sq4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c2 = 0; c2 < 2; ++c2) {               // columns in pairs of 32, both loads in flight before the wait
-                if (c2 * 64 < my_cols) {                    // (my_cols is a multiple of 64)
-                    uint32_t v0[32], v1[32];
-                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
-                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
-                    tmem_ld_wait32(v0); tmem_ld_wait32(v1);
-                    if (row_ok) {      // (columns past the real ones of an unfolded thin layer hold exact zeros)
+                for (int c2 = 0; c2 < 2; ++c2) {           // columns in pairs of 32, both loads in flight before the wait
+                    if (c2 * 64 < my_cols) {                // (my_cols is a multiple of 64)
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+                        if (row_ok) {      // (columns past the real ones of an unfolded thin layer hold exact zeros)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v0[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
+                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v0[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v1[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
+                            for (int i = 0; i < 32; ++i) { const float f = __uint_as_float(v1[i]); sq4[i & 3] = fmaf(f, f, sq4[i & 3]); }
+                        }
                     }
                 }
-            }
-            const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
-            if (lane == 0) {
-                const uint32_t slot = smem_u32(&norm_part[par][rank][e]);
-                const uint32_t bar = smem_u32(&norm_bar[par]);
-                for (int r = 0; r < cs; ++r) {
-                    st_cluster_f32(map_to_cta(slot, (uint32_t)r), sq);
-                    mbar_arrive_remote(map_to_cta(bar, (uint32_t)r));
+                const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
+                if (lane < cs) {
+                    // lane r tells CTA r (every lane holds the warp's sum): the remote store and the remote arrival that
+                    // releases it cost a round trip through the cluster each, so the peers are served side by side, not in turn
+                    st_cluster_f32(map_to_cta(smem_u32(&norm_part[slot][rank][e]), (uint32_t)lane), sq);
+                    mbar_arrive_remote(map_to_cta(smem_u32(&norm_bar[slot]), (uint32_t)lane));
                 }
             }
-            const bool all_in = mbar_wait_cluster(smem_u32(&norm_bar[par]), use_parity, abort_p, p.wait_polls);
-            if (!__all_sync(0xffffffffu, all_in)) { live = false; break; }
-            // the same order in every warp of every CTA: all of them apply the identical factor
-            double sn = 0.0;
-            for (int r = 0; r < cs; ++r)
+            if (step >= 1) {
+                const int j = step - 1, n = n_lo + j, buf = j & 1, slot = j & 3;
+                const bool all_in = mbar_wait_cluster(smem_u32(&norm_bar[slot]), (uint32_t)((j >> 2) & 1), abort_p, p.wait_polls);
+                if (!__all_sync(0xffffffffu, all_in)) { live = false; break; }
+                // the same order in every warp of every CTA: all of them apply the identical factor
+                double sn = 0.0;
+                for (int r = 0; r < cs; ++r)
 #pragma unroll
-                for (int w = 0; w < 8; ++w) sn += (double)norm_part[par][r][w];
-            const float f = clip_factor(sn, p.C_l);
-            if (rank == 0 && e == 0 && lane == 0) {
-                p.sqnorm[n * p.sq_stride] = (float)sn;
-                if (p.clip_out) p.clip_out[n] = f;
-            }
-            // pass 2: scale the tile into the running sum
-#pragma unroll
-            for (int c2 = 0; c2 < 2; ++c2) {
-                if (c2 * 64 < my_cols) {
-                    uint32_t v0[32], v1[32];
-                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
-                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
-                    tmem_ld_wait32(v0); tmem_ld_wait32(v1);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
+                    for (int w = 0; w < 8; ++w) sn += (double)norm_part[slot][r][w];
+                const float f = clip_factor(sn, p.C_l);
+                if (rank == 0 && e == 0 && lane == 0) {
+                    p.sqnorm[n * p.sq_stride] = (float)sn;
+                    if (p.clip_out) p.clip_out[n] = f;
                 }
+                // pass 2: scale the tile into the running sum
+                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    if (c2 * 64 < my_cols) {
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
-            buf ^= 1;
         }
         if (live && row_ok) {
             // one owner per output element: add straight into the accumulator, or leave a partial sum for the fold
