@@ -646,7 +646,7 @@ constexpr int kClipThreads = 384;
 constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
 static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
 constexpr int kMaxCluster = 8;
-constexpr int kMinExamplesPerCluster = 8;   // with an SM target set (calls run side by side)
+constexpr int kMinExamplesPerCluster = 8;   // examples a cluster walks through when an SM target is set (calls run side by side)
 
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -1336,11 +1336,17 @@ static void ssum_split(int B, int tiles, int &splits, int &per_split) {
 }
 
 static int max_active_clusters(int cluster_size);
-static void cluster_split(int B, int cluster_size, int &splits, int &per_split) {
+// K, NT: pixels per example and columns per tile (for a rough time of one example in one CTA)
+static void cluster_split(int B, int cluster_size, int K, int NT, int &splits, int &per_split) {
     int want = std::min(sm_target() / cluster_size, max_active_clusters(cluster_size));
     // A caller that set an SM target runs calls side by side: what counts then is SM time, and a cluster that walks
-    // through several examples spends its start-up, its first loads and its final stores once for all of them.
-    if (sm_target_set()) want = std::min(want, std::max(1, B / kMinExamplesPerCluster));
+    // through several examples spends its start-up, its first loads and its final stores once for all of them -- up
+    // to eight examples, and not beyond some 30 microseconds a launch, so that no call holds its stream up for long.
+    if (sm_target_set()) {
+        const double cycles = (K / 16.0) * std::max(NT / 2.0, 64.0) * 1.5;
+        const int per = std::max(1, std::min(kMinExamplesPerCluster, (int)(60000.0 / cycles)));
+        want = std::min(want, std::max(1, B / per));
+    }
     if (want < 1) want = 1;
     if (want > B) want = B;
     per_split = (B + want - 1) / want;
@@ -1399,7 +1405,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             }
             if (mode == 3) {
                 int splits, per;
-                cluster_split(g.B, m_tiles * n_tiles, splits, per);
+                cluster_split(g.B, m_tiles * n_tiles, g.K, NT, splits, per);
                 waves = per;                                       // examples a cluster walks through
                 sm_share = (double)splits * m_tiles * n_tiles;      // SMs the launch holds meanwhile
             }
@@ -1535,7 +1541,7 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
         TcPlan one;
         if (clip1_plan(dtype, pr.eff, one)) {              // room for either form: the single pass may be unavailable at run time
             int s1, p1;
-            cluster_split(pr.eff.B, one.m_tiles * one.n_tiles, s1, p1);
+            cluster_split(pr.eff.B, one.m_tiles * one.n_tiles, pr.eff.K, one.NT, s1, p1);
             splits = std::max(splits, s1);
         }
         size_t clip_bytes = splits > 1 ? sizeof(float) * (size_t)splits * g0.M * g0.N : 0;
@@ -1762,7 +1768,7 @@ dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const Conv
     p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
     p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
     const int cs = pl.m_tiles * pl.n_tiles;
-    cluster_split(g.B, cs, p.splits, p.per_split);
+    cluster_split(g.B, cs, g.K, pl.NT, p.splits, p.per_split);
     p.sum_out = p.splits > 1 ? part_ws : acc_w;
     p.total_tiles = p.splits * cs;
     static std::once_flag once;
