@@ -322,18 +322,19 @@ class FlatGrad:
         return 2 * self.P * 4
 
     def roofline(self, dom, totals, prof_steps, peaks):
-        """Per-example noise draws B*P normals per chunk and is bound by integer and transcendental arithmetic: about
-        45 instructions per normal (a quarter of a ten-round Philox block, half a Box-Muller pair, the scaled add), so
-        the ceiling is SMs x 128 lanes x SM clock / 45 normals per second."""
+        """Per-example noise draws B*P normals per chunk and is bound by integer and transcendental arithmetic: 54
+        thread instructions per normal (a quarter of a ten-round Philox block, half a Box-Muller pair, the scaled add;
+        counted by ncu: smsp__thread_inst_executed.sum = 27.63 G for 512 M normals), so the ceiling is
+        SMs x 128 lanes x SM clock / 54 normals per second."""
         if self.variant != "per_example_noise" or dom != 0:
             return None
         avg_ms_per_chunk = totals[0] / (prof_steps * self.G)
         props = self.torch.cuda.get_device_properties(self.torch.cuda.current_device())
         sms, ghz = props.multi_processor_count, peaks.get("sm_max_mhz", 1965.0) / 1e3
-        peak = sms * 128 * ghz * 1e9 / 45.0 / 1e9
+        peak = sms * 128 * ghz * 1e9 / 54.0 / 1e9
         got = self.B * self.P / (avg_ms_per_chunk / 1e3) / 1e9
         return {"bound": "alu", "achieved": round(got, 1), "peak": round(peak, 1),
-                "peak_source": f"derived: {sms} SMs x 128 lanes x {ghz:.3f} GHz / 45 instructions per normal (an estimate of the instruction count)",
+                "peak_source": f"derived: {sms} SMs x 128 lanes x {ghz:.3f} GHz / 54 thread instructions per normal (ncu count)",
                 "unit": "Gnormal/s", "frac": round(got / peak, 4)}
 
     def e2e_prepare(self):

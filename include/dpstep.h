@@ -293,6 +293,9 @@ DP_API size_t dp_clip_static_scratch_bytes(void);
  *   u1 = ((r_a >> 9) + 0.5) * 2^-23, u2 = (r_b >> 8) * 2^-24, radius = sqrt(-2 ln u1),
  *   lane g%4 = 0,2 takes radius*cos(2 pi u2), lane 1,3 takes radius*sin(2 pi u2).
  * sigma = 0 adds nothing, whatever C is; with sigma > 0, C must be finite.
+ * seed and step are call arguments: a call captured into a CUDA graph keeps the values it was captured with, so
+ * replaying it repeats the same draw.  Keep this call outside graphs that are replayed across training steps (or
+ * update the kernel node's parameters), or every step gets the same noise and the privacy guarantee is void.
  * In per-layer mode C is still the whole-gradient bound (the per-group thresholds are chosen so
  * that the whole gradient keeps sensitivity C).
  * Errors: DP_ERR_INVALID_ARG for P <= 0, param_offset < 0, total_batch <= 0, sigma < 0, C <= 0. */
