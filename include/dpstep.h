@@ -355,6 +355,9 @@ DP_API const char *dp_last_cuda_error(void);
 /* Test / report hook: the tiling the tensor-core kernel would use for a conv layer and epilogue, as up to 12 ints
  * {rows-are-input-columns, row extent, column extent, row tiles, column tiles, columns per tile,
  *  pixel-tile width, pixel-tile height, pixels per stage, pixel tiles, pipeline stages, bytes per stage}.
+ * `epilogue` is a dp_epilogue value, or 3 (the fused clip as one contraction per cluster), 4 (the clipped sum as one
+ * product over all examples) or 5 (norms from the pixel Gram matrices: row and column extent = pixels of the box,
+ * pixel tiles = loads per row tile).
  * Returns the number of values available (0 when the layer is not eligible). `out` is host memory. */
 DP_API int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n);
 

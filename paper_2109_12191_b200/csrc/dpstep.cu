@@ -206,6 +206,13 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
         }
         // per-layer clipping: norms of every example first, then the clipped sum with the factors known
         if (pl.use_tc) {
+            if (!d->has_bias && single_pass_enabled() && tc_clip_scaled_sum(d->dtype, g) && tc_gram_norm(d->dtype, g)) {
+                // small planes: norms and factors from the pixel Gram matrices, then the clipped sum as one product
+                const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
+                rc = launch_conv_gram_norm(d->dtype, X, dY, g, ic, factor, reinterpret_cast<int *>(ws + pl.status_off), st);
+                if (rc != DP_OK) return rc;
+                return launch_conv_ssum(d->dtype, X, dY, g, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
+            }
             // the norm pass's last CTA folds the partial norms (bias slots included) into norms and factors
             const TcPublish pub = {reinterpret_cast<int *>(ws + kWsCounterOffset), pl.w_slots, groups == 2, sqnorm, sqnorm_stride, factor, C_l, clip_out};
             rc = launch_conv_tc(d->dtype, DP_EPI_NORM_ONLY, X, dY, g, nullptr, partial, pl.slots, nullptr, nullptr, ws + pl.tc_off,
@@ -323,7 +330,7 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
 }
 
 extern "C" int dp_debug_wgrad_plan(const dp_layer_desc *desc, int epilogue, int *out, int n) {
-    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 4 || !out || n <= 0) return 0;   // 3: the single-pass form of the fused clip, 4: the clipped sum as one product
+    if (!valid_desc(desc) || desc->kind != DP_LAYER_CONV2D || epilogue < 0 || epilogue > 5 || !out || n <= 0) return 0;   // 3: the single-pass form of the fused clip, 4: the clipped sum as one product, 5: norms from Gram matrices
     return tc_describe_plan(desc->dtype, geom_of(desc), epilogue, out, n);
 }
 

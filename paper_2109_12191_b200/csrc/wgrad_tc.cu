@@ -1131,6 +1131,211 @@ conv_wgrad_ssum_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
 }
 
+// ----------------------------------------------------------------------------- norms from Gram matrices
+// For a layer whose gradient is far larger than its pixel count squared, the squared norm of example n comes cheaper
+// from the identity  ||dY_n^T Xcol_n||_F^2 = sum_{p,q} (dY_n dY_n^T)[p,q] (Xcol_n Xcol_n^T)[p,q]  over pixel pairs
+// (the norm the clip factor of the paper's section 2 needs, without the gradient itself): two Gram matrices of
+// [pixels x pixels], each a product over channels, and Xcol's is the sum over the taps of the Gram matrices of the
+// shifted inputs.  Here the SAME shared-memory tiles as above (one TMA box = pixels x 64 channels, 128-byte rows,
+// 128-byte swizzle) are read as K-major operands: the pixel is the M / N index and the channel the reduction index,
+// and one tile serves as both A and B.  One CTA per example; a plane of up to 256 pixels (box rows, a multiple of 16)
+// is one or two row tiles of 128, and since both matrices are symmetric the second row tile only needs the columns
+// from 128 on, the first one counting its columns from 128 on twice.
+// Roles (192 threads): warp 0 TMA, warp 1 MMA issue, warps 2-5 read both matrices back and sum their products.
+struct GramParams {
+    int B, Cin, Kout, S, taps, stride, pad;
+    int rows;                   // pixels of the box (zero rows past the plane included), a multiple of 16, <= 256
+    int m_tiles, stages, stage_bytes;
+    float C_l;
+    float *sqnorm; long long sq_stride; float *factor_out; float *clip_out;
+    int *status;
+    uint32_t wait_polls;
+};
+
+// K-major operand of 128-byte rows with the 128-byte swizzle: 8-row groups 1024 B apart; the leading offset is unused
+// because one instruction's 32 bytes of K lie inside one swizzle row.
+__device__ __forceinline__ uint64_t kmajor_desc_base() {
+    uint64_t d = (uint64_t)1 << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n_cols
+__device__ __forceinline__ uint32_t instr_desc_kmajor(int n_cols) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(192, 1)
+conv_gram_norm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const GramParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ __align__(8) uint64_t norm_bar;
+    __shared__ double warp_part[4][4];      // [example & 3][quadrant]: a warp may run up to three examples ahead of the one that adds up
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t tiles_u32 = smem_u32(tiles);
+
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 4); }
+        mbar_init(smem_u32(&norm_bar), 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int *abort_p = &abort_flag;
+
+    // tensor memory: one or two buffers of 256 columns; in a buffer dY's matrix first, then Xcol's
+    const int nbuf = p.rows > 128 ? 1 : 2;
+    const uint32_t x_col = p.rows > 128 ? 256u : 128u;
+    const int y_slabs = p.Kout / 64, c_slabs = p.Cin / 64;
+    const int slabs = y_slabs + p.taps * c_slabs;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer: one box per stage
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool live = true;
+            const uint32_t tx_bytes = (uint32_t)(p.rows * kRowBytes);
+            for (int n = blockIdx.x; n < p.B && live; n += gridDim.x) {
+                for (int mt = 0; mt < p.m_tiles && live; ++mt) {
+                    int tap = 0, cs = 0;
+                    for (int s = 0; s < slabs; ++s) {
+                        if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_p, p.wait_polls)) { live = false; break; }
+                        mbar_expect_tx(smem_u32(&full_bar[stage]), tx_bytes);
+                        const uint32_t dst = tiles_u32 + stage * p.stage_bytes;
+                        if (s < y_slabs) {
+                            tma_load_4d(dst, &tmY, smem_u32(&full_bar[stage]), s * 64, 0, 0, n);
+                        } else {
+                            const int r = tap / p.S;
+                            tma_load_4d(dst, &tmX, smem_u32(&full_bar[stage]), cs * 64, (tap - r * p.S) - p.pad, r - p.pad, n);
+                            if (++cs == c_slabs) { cs = 0; ++tap; }
+                        }
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0, acc_phase = 0;
+            int buf = 0;
+            bool live = true;
+            const uint64_t desc_base = kmajor_desc_base();
+            const uint32_t desc_lo = (uint32_t)desc_base, desc_hi32 = (uint32_t)(desc_base >> 32);
+            for (int n = blockIdx.x; n < p.B && live; n += gridDim.x) {
+                for (int mt = 0; mt < p.m_tiles && live; ++mt) {
+                    const int col0 = mt * 128;                       // the tile's columns start at its own first row
+                    const uint32_t idesc = instr_desc_kmajor(p.rows - col0);
+                    if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p, p.wait_polls)) { live = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_y = tmem_base + (uint32_t)(buf * 256), d_x = d_y + x_col;
+                    for (int s = 0; s < slabs; ++s) {
+                        if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_p, p.wait_polls)) { live = false; break; }
+                        tc_fence_after();
+                        const uint32_t src = tiles_u32 + stage * p.stage_bytes + (uint32_t)(col0 * kRowBytes);
+                        uint32_t ad = desc_lo | ((src & 0x3FFFFu) >> 4);
+                        const bool is_y = s < y_slabs;
+                        const uint32_t d_tmem = is_y ? d_y : d_x;
+                        uint32_t accumulate = (s == 0 || s == y_slabs) ? 0u : 1u;
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {             // 64 channels = four steps of 16, 32 bytes apart in the row
+                            umma<false>(d_tmem, ad, ad, desc_hi32, idesc, accumulate);
+                            accumulate = 1;
+                            ad += 2;
+                        }
+                        umma_commit(smem_u32(&empty_bar[stage]));
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!live) break;
+                    umma_commit(smem_u32(&tmem_full[buf]));
+                    acc_phase ^= 1u << buf;
+                    if (nbuf == 2) buf ^= 1;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: sum over the tile of G_Y .* G_X
+        const int q = warp & 3;
+        uint32_t full_phase = 0;
+        int buf = 0;
+        bool live = true;
+        int trip = 0;
+        for (int n = blockIdx.x; n < p.B && live; n += gridDim.x) {
+            double acc = 0.0;
+            for (int mt = 0; mt < p.m_tiles; ++mt) {
+                const int col0 = mt * 128, n_cols = p.rows - col0;
+                const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
+                if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+                full_phase ^= 1u << buf;
+                tc_fence_after();
+                const int row = col0 + q * 32 + lane;
+                if (col0 + q * 32 < p.rows) {                        // warps whose rows all lie past the box read nothing
+                    const uint32_t t_y = tmem_base + (uint32_t)(buf * 256) + ((uint32_t)(q * 32) << 16), t_x = t_y + x_col;
+                    float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};     // columns below / from 128
+                    for (int cc = 0; cc < n_cols; cc += 32) {
+                        uint32_t vy[32], vx[32];
+                        tmem_ld32_issue(t_y + (uint32_t)cc, vy);
+                        tmem_ld32_issue(t_x + (uint32_t)cc, vx);
+                        tmem_ld_wait32(vy); tmem_ld_wait32(vx);
+                        const bool twice = cc >= 128;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float pr = (cc + i < n_cols) ? __uint_as_float(vy[i]) * __uint_as_float(vx[i]) : 0.f;
+                            if (twice) s2[i & 3] += pr; else s1[i & 3] += pr;
+                        }
+                    }
+                    if (row < p.rows)
+                        acc += ((double)s1[0] + (double)s1[1]) + ((double)s1[2] + (double)s1[3]) +
+                               2.0 * (((double)s2[0] + (double)s2[1]) + ((double)s2[2] + (double)s2[3]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+                if (nbuf == 2) buf ^= 1;
+            }
+            if (!live) break;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            // the four warps hand their sums to the one that publishes through a barrier word (no warp waits for
+            // another except that one, and its wait is bounded like every other)
+            if (lane == 0) { warp_part[trip & 3][q] = acc; mbar_arrive(smem_u32(&norm_bar)); }
+            if (q == 0) {
+                if (!mbar_wait(smem_u32(&norm_bar), (uint32_t)(trip & 1), abort_p, p.wait_polls)) { live = false; break; }
+                if (lane == 0) {
+                    const double *w = warp_part[trip & 3];
+                    const double sq = (w[0] + w[1]) + (w[2] + w[3]);
+                    p.sqnorm[n * p.sq_stride] = (float)sq;
+                    const float f = clip_factor(sq, p.C_l);
+                    if (p.factor_out) { p.factor_out[2 * n] = f; p.factor_out[2 * n + 1] = f; }
+                    if (p.clip_out) p.clip_out[n] = f;
+                }
+            }
+            ++trip;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag) {
+        if (threadIdx.x == 0) { *p.status = DP_ERR_TIMEOUT; __threadfence(); }
+        __nanosleep(200000);
+        __syncthreads();
+    }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
 // hi[i] = bf16(f_n y[i]), lo[i] = bf16(f_n y[i] - hi[i]) for every entry of example n (eight entries per thread)
 __global__ void __launch_bounds__(256)
 scale_split_kernel(const __nv_bfloat16 *__restrict__ y, const float *__restrict__ factor, long long per_example, long long total8,
@@ -1556,9 +1761,11 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
     return bytes;
 }
 
+static int gram_describe(int dtype, const ConvGeom &g0, int *out, int n);
 int tc_describe_plan(int dtype, const ConvGeom &g0, int epilogue, int *out, int n) {
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
+    if (epilogue == 5) return gram_describe(dtype, g0, out, n);
     const TcPlan pl = make_plan(dtype, pr.eff, epilogue);
     if (!pl.ok) return 0;
     const int v[12] = {pl.a_is_x, pl.a_ext, pl.b_ext, pl.m_tiles, pl.n_tiles, pl.NT, pl.OWt, pl.OHt, pl.Kt, pl.k_tiles,
@@ -1723,6 +1930,73 @@ dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvG
     conv_wgrad_ssum_kernel<<<grid, 224, pl.smem, stream>>>(tmX, tmYhi, tmYlo, p);
     DP_LAUNCH_CHECK("conv_wgrad_ssum_kernel");
     if (p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g.M * g.N, acc_w, stream);
+    return DP_OK;
+}
+
+// ---- norms from Gram matrices (conv_gram_norm_kernel): the whole output plane as one pixel box
+struct GramPlan { bool ok; ConvGeom g; int OWb, OHb, rows, m_tiles, stages, stage_bytes; size_t smem; };
+
+static GramPlan gram_plan(int dtype, const ConvGeom &g0) {
+    GramPlan gp = {};
+    const TcProblem pr = tc_problem(dtype, g0);
+    if (dtype != DP_BF16 || !pr.ok || pr.unfold || !encode_fn()) return gp;
+    gp.g = pr.eff;
+    const ConvGeom &g = gp.g;
+    if (g.stride > 8) return gp;
+    int best = 1 << 30;
+    // the smallest box over the plane whose pixel count is a multiple of 16 (rows past the plane are zero-filled)
+    for (int OHb = g.OH; OHb <= g.OH + 15; ++OHb)
+        for (int OWb = g.OW; OWb <= g.OW + 15; ++OWb) {
+            const int rows = OHb * OWb;
+            if (rows % 16 || rows > 256 || OWb * g.stride > 256 || OHb * g.stride > 256 || rows >= best) continue;
+            best = rows; gp.OWb = OWb; gp.OHb = OHb;
+        }
+    if (best > 256) return gp;
+    gp.rows = best;
+    gp.m_tiles = (best + 127) / 128;
+    gp.stage_bytes = gp.m_tiles * 128 * kRowBytes;      // a row tile always reads 128 rows, whatever the box holds
+    gp.stages = std::min(kMaxStages, kSmemBudget / gp.stage_bytes);
+    gp.smem = (size_t)gp.stages * gp.stage_bytes + 1024;
+    gp.ok = true;
+    return gp;
+}
+
+bool tc_gram_norm(int dtype, const ConvGeom &g0) { return gram_plan(dtype, g0).ok; }
+
+// {1, pixels of the box, same, row tiles, 1, columns of the first row tile, box width, box height, pixels per stage,
+//  loads per row tile, stages, bytes per stage}
+static int gram_describe(int dtype, const ConvGeom &g0, int *out, int n) {
+    const GramPlan gp = gram_plan(dtype, g0);
+    if (!gp.ok) return 0;
+    const int v[12] = {1, gp.rows, gp.rows, gp.m_tiles, 1, gp.rows, gp.OWb, gp.OHb, gp.rows,
+                       gp.g.Kout / 64 + gp.g.R * gp.g.S * (gp.g.Cin / 64), gp.stages, gp.stage_bytes};
+    for (int i = 0; i < n && i < 12; ++i) out[i] = v[i];
+    return 12;
+}
+
+dp_status launch_conv_gram_norm(int dtype, const void *X, const void *dY, const ConvGeom &g0, const TcInlineClip &clipinfo,
+                                float *factor_out, int *status, cudaStream_t stream) {
+    const GramPlan gp = gram_plan(dtype, g0);
+    if (!gp.ok) return DP_ERR_UNSUPPORTED;
+    const ConvGeom &g = gp.g;
+    CUtensorMap tmX, tmY;
+    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, gp.OWb, gp.OHb, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, gp.OWb, gp.OHb, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    GramParams p = {};
+    p.B = g.B; p.Cin = g.Cin; p.Kout = g.Kout; p.S = g.S; p.taps = g.R * g.S; p.stride = g.stride; p.pad = g.pad;
+    p.rows = gp.rows; p.m_tiles = gp.m_tiles; p.stages = gp.stages; p.stage_bytes = gp.stage_bytes;
+    p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
+    p.factor_out = factor_out; p.status = status;
+    p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(conv_gram_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
+    const unsigned grid = (unsigned)std::min(g.B, sm_target());
+    conv_gram_norm_kernel<<<grid, 192, gp.smem, stream>>>(tmX, tmY, p);
+    DP_LAUNCH_CHECK("conv_gram_norm_kernel");
     return DP_OK;
 }
 

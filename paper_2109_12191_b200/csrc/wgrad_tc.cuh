@@ -42,6 +42,13 @@ bool tc_clip_scaled_sum(int dtype, const ConvGeom &g);
 dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvGeom &g, const float *factor, float *acc_w,
                            void *tc_workspace, int *status, cudaStream_t stream);
 
+// bf16 layers whose whole output plane is at most 256 pixels: per-example squared norms (and factors against
+// clipinfo.C_l into factor_out[2n], factor_out[2n+1], when given) from the Gram matrices of dY and of the unfolded
+// input over the pixels, without forming the gradient.  Weight group only; not for unfolded layers.
+bool tc_gram_norm(int dtype, const ConvGeom &g);
+dp_status launch_conv_gram_norm(int dtype, const void *X, const void *dY, const ConvGeom &g, const TcInlineClip &clipinfo,
+                                float *factor_out, int *status, cudaStream_t stream);
+
 // Test hook: the number of polls after which a bounded wait of the kernel gives up (0 makes every wait give up at once).
 void set_wait_polls(uint32_t polls);
 uint32_t default_wait_polls();

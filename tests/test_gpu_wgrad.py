@@ -291,3 +291,60 @@ def test_fused_clip_runs_one_contraction_where_the_gradient_fits_a_cluster():
         finally:
             b.dp_debug_set_single_pass(1)
     assert counts[0] < counts[1]
+
+
+GRAM_CONVS = [
+    # Cin, Kout, R, stride, pad, H: gradients too large for a cluster, output planes of at most 256 pixels
+    (128, 256, 3, 1, 1, 14),      # 196 pixels in a 16 x 14 box: two row tiles, the second with 96 rows
+    (128, 256, 3, 1, 1, 10),      # 100 pixels in a 12 x 12 box: second row tile of 16 rows
+    (128, 256, 3, 1, 1, 5),       # 25 pixels in a 48-row box: one row tile, mostly zero rows
+    (128, 256, 3, 2, 1, 14),      # strided taps, 7 x 7 output in an 8 x 8 box
+    (512, 1024, 1, 2, 0, 14),     # strided 1 x 1
+    (1024, 512, 1, 1, 0, 14),     # 1 x 1 with flattened pixels: 196 -> 208 rows
+    (256, 1152, 1, 1, 0, 16),     # exactly 256 pixels: two full row tiles
+]
+
+
+def gram_plan(b, layer, Bn):
+    plan = b.dp_debug_wgrad_plan(make_desc(layer, Bn, "bf16", b.DP_IMPL_AUTO, 0), epilogue=5)
+    return None if plan is None else list(plan.values())
+
+
+@pytest.mark.parametrize("case", GRAM_CONVS)
+def test_conv_norms_from_pixel_gram_matrices(case):
+    """Large layers over small planes take their norms from the Gram matrices of dY and of the unfolded input over
+    the pixels; norms, factors and the clipped sum are held to the same bounds as every other route, and
+    check_layer also runs the route that forms the gradients."""
+    Cin, Kout, R, stride, pad, H = case
+    b = B()
+    layer = synth.conv(Cin, Kout, R, stride, pad, H, False, name=str(case))
+    plan = gram_plan(b, layer, 5)
+    assert plan is not None and plan[1] % 16 == 0 and plan[1] <= 256
+    c0 = b.dp_debug_launch_count()
+    out = check_layer(layer, 5, "bf16", AUTO, (960, sum(case)), spread=True)
+    assert out["uses_tc"]
+    assert b.dp_debug_launch_count() > c0
+
+
+def test_gram_norm_waits_are_bounded():
+    """The Gram-matrix kernel's waits give up like the others: poll limit zero, the kernels return, the status word says so."""
+    b = B()
+    layer = synth.conv(128, 256, 3, 1, 1, 14, name="c")
+    Bn = 3
+    assert gram_plan(b, layer, Bn) is not None
+    inp = synth.layer_inputs(layer, Bn, "bf16", 961, 0)
+    X, dY = dev_inputs(inp, "bf16")
+    d = make_desc(layer, Bn, "bf16", b.DP_IMPL_AUTO, 0)
+    ws = torch.empty(b.dp_workspace_bytes(d, b.DP_EPI_CLIP_ACCUM), dtype=torch.uint8, device="cuda")
+    b.check(b.dp_workspace_init(ws))
+    sq = torch.zeros((Bn, 1), device="cuda")
+    acc = torch.zeros(layer.n_weight, device="cuda")
+    call = lambda: b.dp_per_example_wgrad(d, X, dY, None, None, sq, 1, b.DP_EPI_CLIP_ACCUM, 1.0, acc, None, None, ws)
+    b.dp_debug_set_wait_polls(0)
+    try:
+        assert call() == b.DP_OK
+        torch.cuda.synchronize()
+    finally:
+        b.dp_debug_set_wait_polls(-1)
+    assert b.dp_wgrad_check(ws) == b.DP_ERR_TIMEOUT
+    assert b.dp_wgrad_check(ws) == b.DP_OK
