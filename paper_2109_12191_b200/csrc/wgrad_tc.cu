@@ -75,7 +75,19 @@ struct TcParams {
     // one folds every example's slots [0, w_slots) and [w_slots, slots) into sqnorm (two values when `separate`)
     int *counters; int w_slots; int separate;
     float *factor_out;          // with the ticket: also the clip factors against C_l, [B][2] (weight, bias), and clip_out
+    // space-to-depth form of a thin strided layer (s2d_st > 0): row j' of D is (r2, s2, dy, dx, c) of the regrouped
+    // input and maps to column ((st*r2+dy)*s2d_S + st*s2d+dx)*s2d_Cin + c of the gradient, or to nothing
+    int s2d_st, s2d_R, s2d_S, s2d_Cin;
 };
+
+// column of the gradient that row j of the space-to-depth product stands for, or -1 (a tap or channel that does not exist)
+__device__ __forceinline__ int s2d_column(const TcParams &p, int j) {
+    const int r2 = j >> 6, s2 = (j >> 4) & 3, ch = j & 15;
+    const int q = ch / p.s2d_Cin, c = ch - q * p.s2d_Cin;
+    const int dy = q / p.s2d_st, dx = q - dy * p.s2d_st;
+    const int r = p.s2d_st * r2 + dy, s = p.s2d_st * s2 + dx;
+    return (dy < p.s2d_st && r < p.s2d_R && s < p.s2d_S) ? (r * p.s2d_S + s) * p.s2d_Cin + c : -1;
+}
 
 struct Item { int mt, nt, n_lo, n_hi, split; };
 __device__ __forceinline__ Item decode_item(const TcParams &p, int item) {
@@ -806,8 +818,12 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         const int a_rows = min(128, p.a_ext - mt * 128);
         const int n_cols = min(p.NT, p.b_ext - nt * p.NT);
         const int my_cols = max(0, min(128, n_cols - half * 128));     // columns of this warp's half that exist
-        const int a_idx = mt * 128 + row;
-        const bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
+        int a_idx = mt * 128 + row;
+        bool row_ok = row < a_rows && (!p.a_is_x || a_idx < p.Ng);
+        if (p.s2d_st) {                                    // (rows are input columns in this form)
+            a_idx = row < a_rows ? s2d_column(p, a_idx) : -1;
+            row_ok = a_idx >= 0;
+        }
         float run[128];
 #pragma unroll
         for (int i = 0; i < 128; ++i) run[i] = 0.f;
@@ -1418,42 +1434,80 @@ unfold_small_channels_kernel(const T *__restrict__ X, T *__restrict__ Xcol, cons
 }
 
 // Same unfolding, one block per (output row, example): the R input rows the output row touches are staged in
-// shared memory (zero rows for the padding), then every thread assembles 16-byte groups of columns from them.
+// shared memory with their zero padding written out (so no window needs a bounds check), then every thread
+// assembles 16-byte groups of columns from them through a table  column j -> offset inside the staged rows.
 // Within one filter row r the (s, c) columns of a pixel are a contiguous run of the input row.
+constexpr int kUnfoldMaxCols = 512;
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
 unfold_rows_kernel(const T *__restrict__ X, T *__restrict__ Xcol, const ConvGeom g, int n_pad) {
     extern __shared__ __align__(16) unsigned char unfold_smem[];
-    T *rows = reinterpret_cast<T *>(unfold_smem);          // [R][W*Cin]
+    __shared__ __align__(16) short col_off[kUnfoldMaxCols];
+    T *rows = reinterpret_cast<T *>(unfold_smem);          // [R][Wp*Cin], Wp = (OW-1)*stride + S padded pixels
     const int oh = blockIdx.x, n = blockIdx.y;
-    const int row_len = g.W * g.Cin;
+    const int row_p = ((g.OW - 1) * g.stride + g.S) * g.Cin, row_len = g.W * g.Cin, shift = g.pad * g.Cin;
+    const int tap_row = g.S * g.Cin;
+    for (int j = threadIdx.x; j < n_pad; j += 256) {
+        const int r = j / tap_row;
+        col_off[j] = (j < g.N) ? (short)(r * row_p + (j - r * tap_row)) : (short)-1;
+    }
     for (int r = 0; r < g.R; ++r) {
         const int ih = oh * g.stride + r - g.pad;
         const bool inside = ih >= 0 && ih < g.H;
         const T *src = X + ((long long)n * g.H + (inside ? ih : 0)) * row_len;
-        for (int i = threadIdx.x; i < row_len; i += 256) rows[r * row_len + i] = inside ? src[i] : T(0.f);
+        for (int i = threadIdx.x; i < row_p; i += 256) {
+            const int col = i - shift;
+            rows[r * row_p + i] = (inside && col >= 0 && col < row_len) ? src[col] : T(0.f);
+        }
     }
     __syncthreads();
-    const int groups = n_pad / VEC, tap_row = g.S * g.Cin;
+    const int groups = n_pad / VEC, step = g.stride * g.Cin;
     T *dst = Xcol + ((long long)n * g.OH + oh) * g.OW * n_pad;
     for (int chunk = threadIdx.x; chunk < g.OW * groups; chunk += 256) {
         const int ow = chunk / groups;
         const int j0 = (chunk - ow * groups) * VEC;
-        const int base = (ow * g.stride - g.pad) * g.Cin;
-        int r = j0 / tap_row, jj = j0 - r * tap_row;
-        T v[VEC];
+        const T *win = rows + ow * step;
+        __align__(16) short off[VEC];
+        if (VEC == 8) *reinterpret_cast<uint4 *>(off) = *reinterpret_cast<const uint4 *>(col_off + j0);
+        else *reinterpret_cast<uint2 *>(off) = *reinterpret_cast<const uint2 *>(col_off + j0);
+        __align__(16) T v[VEC];
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) {
-            T x = T(0.f);
-            if (j0 + e < g.N) {
-                const int col = base + jj;
-                if (col >= 0 && col < row_len) x = rows[r * row_len + col];
-            }
-            v[e] = x;
-            if (++jj == tap_row) { jj = 0; ++r; }
-        }
+        for (int e = 0; e < VEC; ++e) v[e] = off[e] >= 0 ? win[off[e]] : T(0.f);
         *reinterpret_cast<uint4 *>(dst + (long long)chunk * VEC) = *reinterpret_cast<const uint4 *>(v);
     }
+}
+
+// Space-to-depth regrouping of a thin strided input (C_in * stride^2 <= 16 channels): pixel (a, b) of the result
+// holds the stride x stride block of padded-input pixels (stride*a + dy, stride*b + dx) as channels
+// (dy*stride + dx)*C_in + c, zero-filled up to 16.  The strided R x S convolution over the input is then a
+// stride-1 convolution with ceil(R/stride) x ceil(S/stride) taps over 16-channel pixels, and the (at most four)
+// taps of one filter row are 64 contiguous values: one 128-byte operand row per output pixel, read straight
+// from this buffer by a tensor map whose pixel stride (32 bytes) is smaller than its row (128 bytes).
+__global__ void __launch_bounds__(256)
+space_to_depth_kernel(const __nv_bfloat16 *__restrict__ X, __nv_bfloat16 *__restrict__ Xs, const ConvGeom g, int Hs, int Ws, long long total) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // one output pixel each
+    if (idx >= total) return;
+    const int b = (int)(idx % Ws);
+    const long long t = idx / Ws;
+    const int a = (int)(t % Hs);
+    const long long n = t / Hs;
+    __align__(16) __nv_bfloat16 v[16];
+#pragma unroll
+    for (int ch = 0; ch < 16; ++ch) v[ch] = __float2bfloat16(0.f);
+    const int st = g.stride;
+    for (int dy = 0; dy < st; ++dy) {
+        const int ih = st * a + dy - g.pad;
+        if (ih < 0 || ih >= g.H) continue;
+        for (int dx = 0; dx < st; ++dx) {
+            const int iw = st * b + dx - g.pad;
+            if (iw < 0 || iw >= g.W) continue;
+            const __nv_bfloat16 *src = X + ((n * g.H + ih) * g.W + iw) * g.Cin;
+            for (int c = 0; c < g.Cin; ++c) v[(dy * st + dx) * g.Cin + c] = src[c];
+        }
+    }
+    uint4 *dst = reinterpret_cast<uint4 *>(Xs + idx * 16);
+    dst[0] = *reinterpret_cast<const uint4 *>(v);
+    dst[1] = *reinterpret_cast<const uint4 *>(v + 8);
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -1578,6 +1632,8 @@ static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
 // clusters share the batch, and what is minimised is SM time (clusters x CTAs x time), not the time of one launch
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
     const int max_nt = (mode == 2) ? 128 : 256;
+    const bool rows_are_inputs = mode == 6;              // mode 6: mode 3 with the rows of D fixed to the input columns
+    if (mode == 6) mode = 3;
     TcPlan best; best.ok = false;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
@@ -1587,7 +1643,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
     const int a_slabs_tile = 128 / slab_ch;
     const int copies = (dtype == DP_F32) ? 2 : 1;       // split tf32 keeps a hi and a lo copy of every stage
     double best_cost = 1e300;
-    for (int a_is_x = 0; a_is_x < 2; ++a_is_x) {
+    for (int a_is_x = rows_are_inputs ? 1 : 0; a_is_x < 2; ++a_is_x) {
         const int a_ext = a_is_x ? g.N : g.M, b_ext = a_is_x ? g.M : g.N;
         for (int NT = slab_ch; NT <= max_nt; NT += slab_ch) {
             if (NT != 32 && NT % 64) continue;
@@ -1700,11 +1756,35 @@ static int max_active_clusters(int cluster_size) {
     return cached[cluster_size] > 0 ? cached[cluster_size] : 1 << 30;
 }
 
-// true when the fused clipped sum of this layer runs as ONE contraction (bf16 inputs, the example's gradient fits the
-// tensor memory of one cluster)
-static bool clip1_plan(int dtype, const ConvGeom &eff, TcPlan &pl) {
-    if (dtype != DP_BF16) return false;
-    pl = make_plan(dtype, eff, 3);
+// Thin strided layers (a 7 x 7 stride-2 stem on RGB) in space-to-depth form, see space_to_depth_kernel: the geometry the
+// kernel tiles is a stride-1 convolution with ceil(R/stride) x 1 taps of 64 "channels" (one filter row's window).
+struct S2dProblem { bool ok; int R2, Hs, Ws; ConvGeom eff; };
+static S2dProblem s2d_problem(int dtype, const ConvGeom &g, const TcProblem &pr) {
+    S2dProblem sp = {};
+    if (dtype != DP_BF16 || !pr.ok || !pr.unfold || g.stride < 2 || g.Cin * g.stride * g.stride > 16 || g.Kout % 64) return sp;
+    if ((g.S + g.stride - 1) / g.stride > 4) return sp;
+    sp.R2 = (g.R + g.stride - 1) / g.stride;
+    sp.Hs = g.OH + sp.R2 - 1; sp.Ws = g.OW + 3;
+    if ((size_t)sp.Hs * sp.Ws * 32 > (size_t)g.OH * g.OW * pr.n_pad * 2) return sp;     // lives in the unfolded copy's room
+    ConvGeom e = g;
+    e.Cin = 64; e.R = sp.R2; e.S = 1; e.stride = 1; e.pad = 0; e.H = sp.Hs; e.W = g.OW;
+    e.N = sp.R2 * 64;
+    sp.eff = e; sp.ok = true;
+    return sp;
+}
+
+// The single-pass plan of a layer and the geometry it tiles: bf16 inputs, the example's gradient fits the tensor memory
+// of one cluster.  Thin strided layers take the space-to-depth form when that has a plan (rows of D = input columns).
+static bool clip1_plan(int dtype, const ConvGeom &g0, const TcProblem &pr, TcPlan &pl, ConvGeom &g, bool &s2d) {
+    s2d = false;
+    if (dtype != DP_BF16 || !pr.ok) return false;
+    const S2dProblem sp = s2d_problem(dtype, g0, pr);
+    if (sp.ok) {
+        pl = make_plan(dtype, sp.eff, 6);
+        if (pl.ok) { g = sp.eff; s2d = true; return true; }
+    }
+    g = pr.eff;
+    pl = make_plan(dtype, pr.eff, 3);
     return pl.ok;
 }
 
@@ -1730,6 +1810,15 @@ static size_t unfold_bytes(int dtype, const ConvGeom &g0, const TcProblem &pr) {
     return round_up((size_t)g0.B * g0.OH * g0.OW * pr.n_pad * (dtype == DP_BF16 ? 2 : 4), 1024);
 }
 
+// the row-staging form of the unfolding: its staged rows must fit shared memory and its offsets 16 bits
+static size_t unfold_rows_smem(int dtype, const ConvGeom &g) {
+    return (size_t)g.R * ((size_t)(g.OW - 1) * g.stride + g.S) * g.Cin * (dtype == DP_BF16 ? 2 : 4);
+}
+static bool unfold_rows_ok(int dtype, const ConvGeom &g, int n_pad) {
+    const size_t bytes = unfold_rows_smem(dtype, g);
+    return bytes <= 40 * 1024 && bytes / (dtype == DP_BF16 ? 2 : 4) < 32768 && n_pad <= kUnfoldMaxCols && g.B <= 65535;
+}
+
 static size_t ssum_copy_bytes(const ConvGeom &g) { return round_up((size_t)g.B * g.OH * g.OW * g.Kout * 2, 1024); }
 bool tc_clip_scaled_sum(int dtype, const ConvGeom &g0);
 
@@ -1743,10 +1832,10 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
         if (!pl.ok) return 0;
         int splits, per;
         clip_split(pr.eff, pl, splits, per);
-        TcPlan one;
-        if (clip1_plan(dtype, pr.eff, one)) {              // room for either form: the single pass may be unavailable at run time
+        TcPlan one; ConvGeom og; bool s2d;
+        if (clip1_plan(dtype, g0, pr, one, og, s2d)) {     // room for either form: the single pass may be unavailable at run time
             int s1, p1;
-            cluster_split(pr.eff.B, one.m_tiles * one.n_tiles, pr.eff.K, one.NT, s1, p1);
+            cluster_split(og.B, one.m_tiles * one.n_tiles, og.K, one.NT, s1, p1);
             splits = std::max(splits, s1);
         }
         size_t clip_bytes = splits > 1 ? sizeof(float) * (size_t)splits * g0.M * g0.N : 0;
@@ -1766,7 +1855,13 @@ int tc_describe_plan(int dtype, const ConvGeom &g0, int epilogue, int *out, int 
     const TcProblem pr = tc_problem(dtype, g0);
     if (!pr.ok) return 0;
     if (epilogue == 5) return gram_describe(dtype, g0, out, n);
-    const TcPlan pl = make_plan(dtype, pr.eff, epilogue);
+    TcPlan pl;
+    if (epilogue == 3) {
+        ConvGeom g; bool s2d;
+        if (!clip1_plan(dtype, g0, pr, pl, g, s2d)) return 0;
+    } else {
+        pl = make_plan(dtype, pr.eff, epilogue);
+    }
     if (!pl.ok) return 0;
     const int v[12] = {pl.a_is_x, pl.a_ext, pl.b_ext, pl.m_tiles, pl.n_tiles, pl.NT, pl.OWt, pl.OHt, pl.Kt, pl.k_tiles,
                        pl.stages, pl.stage_bytes};
@@ -1807,8 +1902,8 @@ dp_status launch_conv_tc(int dtype, int epilogue, const void *X, const void *dY,
             const int vec = (dtype == DP_BF16) ? 8 : 4;
             const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / vec);
             const unsigned blocks = (unsigned)((total + 255) / 256);
-            const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * (dtype == DP_BF16 ? 2 : 4);
-            if (row_smem <= 40 * 1024 && g0.OH <= 0x7fffffff && g0.B <= 65535) {
+            const size_t row_smem = unfold_rows_smem(dtype, g0);
+            if (unfold_rows_ok(dtype, g0, pr.n_pad)) {
                 const dim3 grid_rows(g0.OH, g0.B);
                 if (dtype == DP_BF16)
                     unfold_rows_kernel<__nv_bfloat16, 8><<<grid_rows, 256, row_smem, stream>>>(
@@ -2002,22 +2097,35 @@ dp_status launch_conv_gram_norm(int dtype, const void *X, const void *dY, const 
 
 bool tc_clip_single_pass(int dtype, const ConvGeom &g0) {
     const TcProblem pr = tc_problem(dtype, g0);
-    TcPlan pl;
-    return pr.ok && encode_fn() && clip1_plan(dtype, pr.eff, pl) && clip1_registers_ok();
+    TcPlan pl; ConvGeom g; bool s2d;
+    return pr.ok && encode_fn() && clip1_plan(dtype, g0, pr, pl, g, s2d) && clip1_registers_ok();
 }
 
 dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const ConvGeom &g0, float *partial, int slots,
                             const TcInlineClip &clipinfo, float *acc_w, void *tc_workspace, int *status, cudaStream_t stream) {
     (void)partial; (void)slots;
     const TcProblem pr = tc_problem(dtype, g0);
-    TcPlan pl;
-    if (!pr.ok || !encode_fn() || !clip1_plan(dtype, pr.eff, pl) || !clip1_registers_ok()) return DP_ERR_UNSUPPORTED;
-    const ConvGeom &g = pr.eff;
+    TcPlan pl; ConvGeom g; bool s2d;
+    if (!pr.ok || !encode_fn() || !clip1_plan(dtype, g0, pr, pl, g, s2d) || !clip1_registers_ok()) return DP_ERR_UNSUPPORTED;
     char *ws_bytes = static_cast<char *>(tc_workspace);
-    if (pr.unfold) {
-        const size_t row_smem = (size_t)g0.R * g0.W * g0.Cin * 2;
-        if (row_smem <= 40 * 1024 && g0.B <= 65535) {
-            unfold_rows_kernel<__nv_bfloat16, 8><<<dim3(g0.OH, g0.B), 256, row_smem, stream>>>(
+    CUtensorMap tmX, tmY;
+    if (s2d) {
+        const S2dProblem sp = s2d_problem(dtype, g0, pr);
+        const long long total = (long long)g0.B * sp.Hs * sp.Ws;
+        space_to_depth_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, sp.Hs, sp.Ws, total);
+        DP_LAUNCH_CHECK("space_to_depth_kernel");
+        // one operand row per output pixel: 64 values from pixel ow on, pixels 16 values apart
+        const cuuint64_t dims[4] = {64, (cuuint64_t)g.OW, (cuuint64_t)sp.Hs, (cuuint64_t)g.B};
+        const cuuint64_t strides[3] = {32, (cuuint64_t)sp.Ws * 32, (cuuint64_t)sp.Hs * sp.Ws * 32};
+        const cuuint32_t box[4] = {64, (cuuint32_t)pl.OWt, (cuuint32_t)pl.OHt, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (encode_fn()(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, ws_bytes, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(space-to-depth X)");
+    } else if (pr.unfold) {
+        if (unfold_rows_ok(dtype, g0, pr.n_pad)) {
+            unfold_rows_kernel<__nv_bfloat16, 8><<<dim3(g0.OH, g0.B), 256, unfold_rows_smem(dtype, g0), stream>>>(
                 static_cast<const __nv_bfloat16 *>(X), reinterpret_cast<__nv_bfloat16 *>(ws_bytes), g0, pr.n_pad);
         } else {
             const long long total = (long long)g0.B * g0.OH * g0.OW * (pr.n_pad / 8);
@@ -2028,8 +2136,7 @@ dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const Conv
         X = ws_bytes;
     }
     float *part_ws = reinterpret_cast<float *>(ws_bytes + unfold_bytes(dtype, g0, pr));
-    CUtensorMap tmX, tmY;
-    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!s2d && !encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
     if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
     TcParams p = {};
     p.B = g.B; p.Kout = g.Kout; p.Ng = g0.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
@@ -2039,6 +2146,7 @@ dp_status launch_conv_clip1(int dtype, const void *X, const void *dY, const Conv
     p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
     p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
     p.mode = 3; p.status = status;
+    if (s2d) { p.s2d_st = g0.stride; p.s2d_R = g0.R; p.s2d_S = g0.S; p.s2d_Cin = g0.Cin; }
     p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
     p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
     const int cs = pl.m_tiles * pl.n_tiles;

@@ -183,7 +183,11 @@ TC_CONVS = [
     ("f32", 64, 128, 3, 2, 1, 16, True),       # third conv of the small CNN
     ("f32", 32, 32, 1, 1, 0, 8, False),
     ("f32", 96, 160, 3, 1, 1, 9, False),       # extents that are multiples of 32 but not of 64 or 128
-    ("bf16", 3, 64, 7, 2, 3, 30, False),       # stem: 3 input channels are unfolded to 147 (+45 zero) columns first
+    ("bf16", 3, 64, 7, 2, 3, 30, False),       # stem: 3 input channels are unfolded to 147 (+45 zero) columns first;
+                                               # its fused clip regroups 2 x 2 pixel blocks into channels instead
+    ("bf16", 4, 64, 5, 2, 2, 21, False),       # ... 16 regrouped channels exactly, three of the four window taps exist
+    ("bf16", 3, 128, 3, 2, 1, 17, False),      # ... two taps a row, odd input size
+    ("bf16", 1, 64, 7, 4, 3, 29, False),       # ... stride 4: 4 x 4 blocks of a single channel
     ("f32", 3, 32, 3, 1, 1, 32, True),         # first conv of the small CNN: 27 (+5 zero) columns
     ("bf16", 4, 128, 3, 1, 1, 9, True),        # 36 columns, rows of the gradient not 16-byte aligned
     ("f32", 1, 64, 5, 2, 2, 13, False),        # single input channel
