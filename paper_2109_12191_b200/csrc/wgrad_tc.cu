@@ -658,7 +658,7 @@ constexpr int kClipThreads = 384;
 constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
 static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
 constexpr int kMaxCluster = 8;
-constexpr int kMinExamplesPerCluster = 8;   // examples a cluster walks through when an SM target is set (calls run side by side)
+constexpr int kMinExamplesPerCluster = 16;   // examples a cluster walks through when an SM target is set (calls run side by side)
 
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -1587,7 +1587,8 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode);
 // tiles (no partial sums to fold); fewer tiles are cut up to half of the SMs.
 static void ssum_split(int B, int tiles, int &splits, int &per_split) {
     const int sms = sm_target();
-    int want = (tiles * 4 >= sms) ? 1 : (sms / 2) / tiles;
+    // (side by side with other calls, under an SM target, a quarter: fewer partial sums to write and fold)
+    int want = (tiles * 4 >= sms) ? 1 : (sms / (sm_target_set() ? 4 : 2)) / tiles;
     if (want < 1) want = 1;
     if (want > B) want = B;
     per_split = (B + want - 1) / want;
@@ -1600,10 +1601,10 @@ static void cluster_split(int B, int cluster_size, int K, int NT, int &splits, i
     int want = std::min(sm_target() / cluster_size, max_active_clusters(cluster_size));
     // A caller that set an SM target runs calls side by side: what counts then is SM time, and a cluster that walks
     // through several examples spends its start-up, its first loads and its final stores once for all of them -- up
-    // to eight examples, and not beyond some 30 microseconds a launch, so that no call holds its stream up for long.
+    // to sixteen examples, and not beyond some 60 microseconds a launch, so that no call holds its stream up for long.
     if (sm_target_set()) {
         const double cycles = (K / 16.0) * std::max(NT / 2.0, 64.0) * 1.5;
-        const int per = std::max(1, std::min(kMinExamplesPerCluster, (int)(60000.0 / cycles)));
+        const int per = std::max(1, std::min(kMinExamplesPerCluster, (int)(120000.0 / cycles)));
         want = std::min(want, std::max(1, B / per));
     }
     if (want < 1) want = 1;

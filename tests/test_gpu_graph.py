@@ -101,7 +101,7 @@ _DISTINCT = _distinct_resnet50_layers()
 @pytest.mark.parametrize("layer", _DISTINCT, ids=[f"{l.name}:{l.kind}{l.R}x{l.R}_{l.Cin}to{l.Kout}_s{l.stride}_at{l.H}" for l in _DISTINCT])
 def test_per_layer_workload_full_size_layers(layer):
     """Every distinct layer shape of the per-layer ResNet-50 workload at full size (B = 32, threshold C/sqrt(161),
-    clip fused into the weight-gradient call), run from a replayed CUDA graph as the benchmark does; the oracle
+    clip fused into the weight-gradient call), run from a replayed CUDA graph under an SM target as the benchmark does; the oracle
     checks every example's squared norm and factor and the whole clipped sum."""
     Bn, C_l = 32, 1.0 / math.sqrt(synth.RESNET50_GN_TENSORS)
     inp = synth.layer_inputs(layer, Bn, "bf16", 4, 7, 0)
@@ -109,19 +109,26 @@ def test_per_layer_workload_full_size_layers(layer):
     s = (np.logspace(-0.5, 0.5, Bn) * C_l / math.sqrt(layer.flops() / 2)).astype(np.float32)
     dY = inp["dY"] * s.reshape((Bn,) + (1,) * (inp["dY"].ndim - 1))
     inp["dY_bits"], inp["dY"] = synth.round_to_bf16(dY)
-    st = PerLayerClipStep([layer], Bn, "bf16", 1.0, 1.0)
-    st.C_l = C_l                                           # the threshold of the 161-tensor model, not of this one layer
-    X, dYd = dev_inputs(inp, "bf16")
-    st.begin()
-    st.wgrad(0, X, dYd)                                    # warm-up launch (sets kernel attributes before capture)
-    torch.cuda.synchronize()
-    st.begin()
-    g = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g):
-        st.wgrad(0, X, dYd)
-    g.replay()
-    torch.cuda.synchronize()
-    st.check()
+    # the benchmark sets an SM target (its calls run side by side), which changes how a call splits the batch over
+    # thread blocks: the same setting here, queried before the workspace is sized
+    from paper_2109_12191_b200 import binding
+    binding.check(binding.dp_set_sm_target(torch.cuda.get_device_properties(0).multi_processor_count))
+    try:
+        st = PerLayerClipStep([layer], Bn, "bf16", 1.0, 1.0)
+        st.C_l = C_l                                       # the threshold of the 161-tensor model, not of this one layer
+        X, dYd = dev_inputs(inp, "bf16")
+        st.begin()
+        st.wgrad(0, X, dYd)                                # warm-up launch (sets kernel attributes before capture)
+        torch.cuda.synchronize()
+        st.begin()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            st.wgrad(0, X, dYd)
+        g.replay()
+        torch.cuda.synchronize()
+        st.check()
+    finally:
+        binding.check(binding.dp_set_sm_target(0))
     dW, db = oracle_layer(layer, inp)
     groups = [dW] + ([db] if db is not None else [])
     sq = st.sq.cpu().numpy()

@@ -352,3 +352,18 @@ def test_gram_norm_waits_are_bounded():
         b.dp_debug_set_wait_polls(-1)
     assert b.dp_wgrad_check(ws) == b.DP_ERR_TIMEOUT
     assert b.dp_wgrad_check(ws) == b.DP_OK
+
+
+@pytest.mark.parametrize("case", [(64, 128, 3, 1, 1, 14), (128, 256, 3, 1, 1, 14), (3, 64, 7, 2, 3, 30), (256, 64, 1, 1, 0, 28)])
+def test_fused_clip_under_an_sm_target_with_a_ragged_batch(case):
+    """With an SM target set (calls meant to run side by side) a cluster walks through up to sixteen examples and the
+    one-product clipped sum takes fewer example ranges: 37 examples leave a ragged last range in both."""
+    Cin, Kout, R, stride, pad, H = case
+    b = B()
+    layer = synth.conv(Cin, Kout, R, stride, pad, H, False, name=str(case))
+    b.check(b.dp_set_sm_target(torch.cuda.get_device_properties(0).multi_processor_count))
+    try:
+        out = check_layer(layer, 37, "bf16", AUTO, (962, sum(case)), spread=True)
+    finally:
+        b.check(b.dp_set_sm_target(0))
+    assert out["uses_tc"]
