@@ -1156,11 +1156,14 @@ conv_wgrad_ssum_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 // 128-byte swizzle) are read as K-major operands: the pixel is the M / N index and the channel the reduction index,
 // and one tile serves as both A and B.  One CTA per example; a plane of up to 256 pixels (box rows, a multiple of 16)
 // is one or two row tiles of 128, and since both matrices are symmetric the second row tile only needs the columns
-// from 128 on, the first one counting its columns from 128 on twice.
+// from 128 on, the first one counting its columns from 128 on twice.  Planes of 64 box pixels go two examples to a tile
+// (one TMA box over two examples): the small MMAs of a single 64-pixel example are bound by their issue rate.
 // Roles (192 threads): warp 0 TMA, warp 1 MMA issue, warps 2-5 read both matrices back and sum their products.
 struct GramParams {
     int B, Cin, Kout, S, taps, stride, pad;
     int rows;                   // pixels of the box (zero rows past the plane included), a multiple of 16, <= 256
+    int pack;                   // examples per tile: 2 when rows == 64 (two examples fill the 128 rows of an MMA; only the
+                                // diagonal 64 x 64 blocks of the products are read), else 1
     int m_tiles, stages, stage_bytes;
     float C_l;
     float *sqnorm; long long sq_stride; float *factor_out; float *clip_out;
@@ -1222,8 +1225,8 @@ conv_gram_norm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool live = true;
-            const uint32_t tx_bytes = (uint32_t)(p.rows * kRowBytes);
-            for (int n = blockIdx.x; n < p.B && live; n += gridDim.x) {
+            const uint32_t tx_bytes = (uint32_t)(p.pack * p.rows * kRowBytes);
+            for (int n = blockIdx.x * p.pack; n < p.B && live; n += gridDim.x * p.pack) {
                 for (int mt = 0; mt < p.m_tiles && live; ++mt) {
                     int tap = 0, cs = 0;
                     for (int s = 0; s < slabs; ++s) {
@@ -1250,10 +1253,10 @@ conv_gram_norm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             bool live = true;
             const uint64_t desc_base = kmajor_desc_base();
             const uint32_t desc_lo = (uint32_t)desc_base, desc_hi32 = (uint32_t)(desc_base >> 32);
-            for (int n = blockIdx.x; n < p.B && live; n += gridDim.x) {
+            for (int n = blockIdx.x * p.pack; n < p.B && live; n += gridDim.x * p.pack) {
                 for (int mt = 0; mt < p.m_tiles && live; ++mt) {
                     const int col0 = mt * 128;                       // the tile's columns start at its own first row
-                    const uint32_t idesc = instr_desc_kmajor(p.rows - col0);
+                    const uint32_t idesc = instr_desc_kmajor(p.pack * p.rows - col0);
                     if (!mbar_wait(smem_u32(&tmem_empty[buf]), ((acc_phase >> buf) & 1u) ^ 1u, abort_p, p.wait_polls)) { live = false; break; }
                     tc_fence_after();
                     const uint32_t d_y = tmem_base + (uint32_t)(buf * 256), d_x = d_y + x_col;
@@ -1288,19 +1291,22 @@ conv_gram_norm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         int buf = 0;
         bool live = true;
         int trip = 0;
-        for (int n = blockIdx.x; n < p.B && live; n += gridDim.x) {
+        for (int n = blockIdx.x * p.pack; n < p.B && live; n += gridDim.x * p.pack) {
             double acc = 0.0;
             for (int mt = 0; mt < p.m_tiles; ++mt) {
-                const int col0 = mt * 128, n_cols = p.rows - col0;
+                const int col0 = mt * 128;
                 const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (full_phase >> buf) & 1u, abort_p, p.wait_polls);
                 if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
                 full_phase ^= 1u << buf;
                 tc_fence_after();
                 const int row = col0 + q * 32 + lane;
-                if (col0 + q * 32 < p.rows) {                        // warps whose rows all lie past the box read nothing
+                // packed: quadrants 0, 1 hold the first example (columns 0..63), quadrants 2, 3 the second (64..127)
+                const int c_lo = p.pack == 2 ? (q >> 1) * 64 : 0;
+                const int c_hi = p.pack == 2 ? c_lo + 64 : p.rows - col0;
+                if (col0 + q * 32 < p.pack * p.rows) {               // warps whose rows all lie past the box read nothing
                     const uint32_t t_y = tmem_base + (uint32_t)(buf * 256) + ((uint32_t)(q * 32) << 16), t_x = t_y + x_col;
                     float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};     // columns below / from 128
-                    for (int cc = 0; cc < n_cols; cc += 32) {
+                    for (int cc = c_lo; cc < c_hi; cc += 32) {
                         uint32_t vy[32], vx[32];
                         tmem_ld32_issue(t_y + (uint32_t)cc, vy);
                         tmem_ld32_issue(t_x + (uint32_t)cc, vx);
@@ -1308,11 +1314,11 @@ conv_gram_norm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                         const bool twice = cc >= 128;
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
-                            const float pr = (cc + i < n_cols) ? __uint_as_float(vy[i]) * __uint_as_float(vx[i]) : 0.f;
+                            const float pr = (cc + i < c_hi) ? __uint_as_float(vy[i]) * __uint_as_float(vx[i]) : 0.f;
                             if (twice) s2[i & 3] += pr; else s1[i & 3] += pr;
                         }
                     }
-                    if (row < p.rows)
+                    if (row < p.pack * p.rows)
                         acc += ((double)s1[0] + (double)s1[1]) + ((double)s1[2] + (double)s1[3]) +
                                2.0 * (((double)s2[0] + (double)s2[1]) + ((double)s2[2] + (double)s2[3]));
                 }
@@ -1329,13 +1335,14 @@ conv_gram_norm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             if (lane == 0) { warp_part[trip & 3][q] = acc; mbar_arrive(smem_u32(&norm_bar)); }
             if (q == 0) {
                 if (!mbar_wait(smem_u32(&norm_bar), (uint32_t)(trip & 1), abort_p, p.wait_polls)) { live = false; break; }
-                if (lane == 0) {
+                if (lane < p.pack && n + lane < p.B) {
                     const double *w = warp_part[trip & 3];
-                    const double sq = (w[0] + w[1]) + (w[2] + w[3]);
-                    p.sqnorm[n * p.sq_stride] = (float)sq;
+                    const double sq = p.pack == 2 ? w[2 * lane] + w[2 * lane + 1] : (w[0] + w[1]) + (w[2] + w[3]);
+                    const int m = n + lane;
+                    p.sqnorm[m * p.sq_stride] = (float)sq;
                     const float f = clip_factor(sq, p.C_l);
-                    if (p.factor_out) { p.factor_out[2 * n] = f; p.factor_out[2 * n + 1] = f; }
-                    if (p.clip_out) p.clip_out[n] = f;
+                    if (p.factor_out) { p.factor_out[2 * m] = f; p.factor_out[2 * m + 1] = f; }
+                    if (p.clip_out) p.clip_out[m] = f;
                 }
             }
             ++trip;
@@ -1872,11 +1879,11 @@ int tc_describe_plan(int dtype, const ConvGeom &g0, int epilogue, int *out, int 
 
 // channels-last [B, H, W, C] tensor, box = {one slab of channels, boxW, boxH, 1 example}; `step` > 1 walks every
 // step-th pixel (the box then spans boxW*step pixels and delivers boxW of them)
-static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, int W, int H, int Bn, int boxW, int boxH, int step) {
+static bool encode_nhwc(CUtensorMap *map, int dtype, const void *base, int C, int W, int H, int Bn, int boxW, int boxH, int step, int boxN = 1) {
     const cuuint64_t es = (dtype == DP_BF16) ? 2 : 4;
     const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)Bn};
     const cuuint64_t strides[3] = {(cuuint64_t)C * es, (cuuint64_t)W * C * es, (cuuint64_t)H * W * C * es};
-    const cuuint32_t box[4] = {(cuuint32_t)(kRowBytes / es), (cuuint32_t)(boxW * step), (cuuint32_t)(boxH * step), 1};
+    const cuuint32_t box[4] = {(cuuint32_t)(kRowBytes / es), (cuuint32_t)(boxW * step), (cuuint32_t)(boxH * step), (cuuint32_t)boxN};
     const cuuint32_t estr[4] = {1, (cuuint32_t)step, (cuuint32_t)step, 1};
     return encode_fn()(map, dtype == DP_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
                        const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -2030,7 +2037,7 @@ dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvG
 }
 
 // ---- norms from Gram matrices (conv_gram_norm_kernel): the whole output plane as one pixel box
-struct GramPlan { bool ok; ConvGeom g; int OWb, OHb, rows, m_tiles, stages, stage_bytes; size_t smem; };
+struct GramPlan { bool ok; ConvGeom g; int OWb, OHb, rows, pack, m_tiles, stages, stage_bytes; size_t smem; };
 
 static GramPlan gram_plan(int dtype, const ConvGeom &g0) {
     GramPlan gp = {};
@@ -2049,6 +2056,7 @@ static GramPlan gram_plan(int dtype, const ConvGeom &g0) {
         }
     if (best > 256) return gp;
     gp.rows = best;
+    gp.pack = (best == 64) ? 2 : 1;
     gp.m_tiles = (best + 127) / 128;
     gp.stage_bytes = gp.m_tiles * 128 * kRowBytes;      // a row tile always reads 128 rows, whatever the box holds
     gp.stages = std::min(kMaxStages, kSmemBudget / gp.stage_bytes);
@@ -2076,11 +2084,11 @@ dp_status launch_conv_gram_norm(int dtype, const void *X, const void *dY, const 
     if (!gp.ok) return DP_ERR_UNSUPPORTED;
     const ConvGeom &g = gp.g;
     CUtensorMap tmX, tmY;
-    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, gp.OWb, gp.OHb, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
-    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, gp.OWb, gp.OHb, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, gp.OWb, gp.OHb, g.stride, gp.pack)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, gp.OWb, gp.OHb, 1, gp.pack)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
     GramParams p = {};
     p.B = g.B; p.Cin = g.Cin; p.Kout = g.Kout; p.S = g.S; p.taps = g.R * g.S; p.stride = g.stride; p.pad = g.pad;
-    p.rows = gp.rows; p.m_tiles = gp.m_tiles; p.stages = gp.stages; p.stage_bytes = gp.stage_bytes;
+    p.rows = gp.rows; p.pack = gp.pack; p.m_tiles = gp.m_tiles; p.stages = gp.stages; p.stage_bytes = gp.stage_bytes;
     p.C_l = clipinfo.C_l; p.sqnorm = clipinfo.sqnorm; p.sq_stride = clipinfo.sq_stride; p.clip_out = clipinfo.clip_out;
     p.factor_out = factor_out; p.status = status;
     p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
@@ -2090,7 +2098,7 @@ dp_status launch_conv_gram_norm(int dtype, const void *X, const void *dY, const 
         attr_err = cudaFuncSetAttribute(conv_gram_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
-    const unsigned grid = (unsigned)std::min(g.B, sm_target());
+    const unsigned grid = (unsigned)std::min((g.B + gp.pack - 1) / gp.pack, sm_target());
     conv_gram_norm_kernel<<<grid, 192, gp.smem, stream>>>(tmX, tmY, p);
     DP_LAUNCH_CHECK("conv_gram_norm_kernel");
     return DP_OK;
