@@ -211,6 +211,8 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
                 const TcInlineClip ic = {C_l, sqnorm, sqnorm_stride, clip_out};
                 rc = launch_conv_gram_norm(d->dtype, X, dY, g, ic, factor, reinterpret_cast<int *>(ws + pl.status_off), st);
                 if (rc != DP_OK) return rc;
+                if (tc_clip_scaled_tiles(d->dtype, g))     // enough pixels an example: scaled per example out of tensor memory
+                    return launch_conv_scaled_tiles(d->dtype, X, dY, g, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
                 return launch_conv_ssum(d->dtype, X, dY, g, factor, acc_w, ws + pl.tc_off, reinterpret_cast<int *>(ws + pl.status_off), st);
             }
             // the norm pass's last CTA folds the partial norms (bias slots included) into norms and factors

@@ -705,7 +705,9 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t tiles_u32 = smem_u32(tiles);
     const int cs = p.m_tiles * p.n_tiles;                 // cluster size = tiles of one example's gradient
-    const int rank = (int)cluster_rank();
+    // With the factors known beforehand (p.factor) nothing is exchanged: the launch has no clusters and any number of tiles
+    const bool known = p.factor != nullptr;
+    const int rank = known ? (int)(blockIdx.x % (unsigned)cs) : (int)cluster_rank();
     const int mt = rank / p.n_tiles, nt = rank - mt * p.n_tiles;
     const int split = (int)blockIdx.x / cs;
     const int n_lo = split * p.per_split, n_hi = min(p.B, n_lo + p.per_split);
@@ -834,7 +836,32 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         // warp sends only after it has scaled example j + 2, i.e. after every warp of the cluster has sent example
         // j + 2, which each of them did after scaling (and so after reading the slots of) example j.
         const int count = n_hi - n_lo;
-        for (int step = 0; step <= count && live; ++step) {
+        for (int step = 0; known && step < count && live; ++step) {
+            // factors known: one read of the finished tile per example, scaled into the running sum
+            const int buf = step & 1;
+            const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (uint32_t)((step >> 1) & 1), abort_p, p.wait_polls);
+            if (!__all_sync(0xffffffffu, arrived)) { live = false; break; }
+            tc_fence_after();
+            const float f = __ldg(p.factor + 2 * (n_lo + step));
+            const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2) {
+                if (c2 * 64 < my_cols) {
+                    uint32_t v0[32], v1[32];
+                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                    tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                    tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+        }
+        for (int step = 0; !known && step <= count && live; ++step) {
             if (step < count) {
                 const int buf = step & 1, slot = step & 3;
                 const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (uint32_t)((step >> 1) & 1), abort_p, p.wait_polls);
@@ -1641,7 +1668,8 @@ static TcPlan make_plan(int dtype, const ConvGeom &g, int mode) {
 static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
     const int max_nt = (mode == 2) ? 128 : 256;
     const bool rows_are_inputs = mode == 6;              // mode 6: mode 3 with the rows of D fixed to the input columns
-    if (mode == 6) mode = 3;
+    const bool any_tiles = mode == 7;                    // mode 7: mode 3 without clusters (factors known): any number of tiles
+    if (mode == 6 || mode == 7) mode = 3;
     TcPlan best; best.ok = false;
     const int slab_ch = (dtype == DP_BF16) ? 64 : 32;
     const int krows = (dtype == DP_BF16) ? 16 : 8;
@@ -1660,7 +1688,7 @@ static TcPlan search_plan(int dtype, const ConvGeom &g, int mode) {
             const int slabs = a_slabs_tile + NT / slab_ch;
             const long long total_tiles = (long long)g.B * m_tiles * n_tiles;
             if (total_tiles > 0x7fffffffLL) continue;
-            if (mode == 3 && m_tiles * n_tiles > kMaxCluster) continue;
+            if (mode == 3 && !any_tiles && m_tiles * n_tiles > kMaxCluster) continue;
             const int y_slabs = (mode == 4) ? (a_is_x ? NT / slab_ch : a_slabs_tile) : 0;     // second (lo) copy of the dY slabs
             // per-CTA share of (example, tile) units: whole waves of tiles, or in clipped-sum mode an even share of the examples
             double waves = (mode != 2) ? (double)((total_tiles + sms - 1) / sms)
@@ -1829,6 +1857,8 @@ static bool unfold_rows_ok(int dtype, const ConvGeom &g, int n_pad) {
 
 static size_t ssum_copy_bytes(const ConvGeom &g) { return round_up((size_t)g.B * g.OH * g.OW * g.Kout * 2, 1024); }
 bool tc_clip_scaled_sum(int dtype, const ConvGeom &g0);
+bool tc_clip_scaled_tiles(int dtype, const ConvGeom &g0);
+static void scaled_tiles_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &per);
 
 // layout: [unfolded input, if any][partial sums of the clipped-sum mode, if any], or the scaled copies of dY and partial sums
 size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
@@ -1852,6 +1882,11 @@ size_t tc_workspace_bytes(int dtype, const ConvGeom &g0, int epilogue) {
             int s4, p4;
             ssum_split(pr.eff.B, sp.m_tiles * sp.n_tiles, s4, p4);
             clip_bytes = std::max(clip_bytes, 2 * ssum_copy_bytes(pr.eff) + (s4 > 1 ? sizeof(float) * (size_t)s4 * g0.M * g0.N : 0));
+        }
+        if (tc_clip_scaled_tiles(dtype, g0)) {
+            int s7, p7;
+            scaled_tiles_split(pr.eff, make_plan(dtype, pr.eff, 7), s7, p7);
+            clip_bytes = std::max(clip_bytes, s7 > 1 ? sizeof(float) * (size_t)s7 * g0.M * g0.N : (size_t)0);
         }
         bytes += clip_bytes;
     }
@@ -2032,6 +2067,54 @@ dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvG
     const unsigned grid = (unsigned)std::min(p.total_tiles, sm_target());
     conv_wgrad_ssum_kernel<<<grid, 224, pl.smem, stream>>>(tmX, tmYhi, tmYlo, p);
     DP_LAUNCH_CHECK("conv_wgrad_ssum_kernel");
+    if (p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g.M * g.N, acc_w, stream);
+    return DP_OK;
+}
+
+// ---- clipped sum with the factors known, per example through tensor memory (the single-pass kernel without its norm
+// pass and exchange): one tile per CTA, the CTA walks a range of examples, reads each finished tile once and keeps
+// sum_n f_n D_n in registers.  Pays where an example has enough pixels that its MMAs outlast the read-back of the tile
+// (some nine steps of 16 pixels); below that the one-product form above is the better one.
+constexpr int kScaledTilesMinPixels = 128;
+bool tc_clip_scaled_tiles(int dtype, const ConvGeom &g0) {
+    const TcProblem pr = tc_problem(dtype, g0);
+    return dtype == DP_BF16 && pr.ok && !pr.unfold && encode_fn() && pr.eff.K >= kScaledTilesMinPixels &&
+           make_plan(dtype, pr.eff, 7).ok && clip1_registers_ok();
+}
+
+static void scaled_tiles_split(const ConvGeom &g, const TcPlan &pl, int &splits, int &per) {
+    cluster_split(g.B, pl.m_tiles * pl.n_tiles, g.K, pl.NT, splits, per);
+}
+
+dp_status launch_conv_scaled_tiles(int dtype, const void *X, const void *dY, const ConvGeom &g0, const float *factor, float *acc_w,
+                                   void *tc_workspace, int *status, cudaStream_t stream) {
+    if (!tc_clip_scaled_tiles(dtype, g0)) return DP_ERR_UNSUPPORTED;
+    const TcProblem pr = tc_problem(dtype, g0);
+    const ConvGeom &g = pr.eff;
+    const TcPlan pl = make_plan(dtype, g, 7);
+    CUtensorMap tmX, tmY;
+    if (!encode_nhwc(&tmX, dtype, X, g.Cin, g.W, g.H, g.B, pl.OWt, pl.OHt, g.stride)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(X)");
+    if (!encode_nhwc(&tmY, dtype, dY, g.Kout, g.OW, g.OH, g.B, pl.OWt, pl.OHt, 1)) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(dY)");
+    TcParams p = {};
+    p.B = g.B; p.Kout = g.Kout; p.Ng = g.N; p.Cin = g.Cin; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.slab_ch = 64; p.krows = 16;
+    p.a_is_x = pl.a_is_x; p.a_ext = pl.a_ext; p.b_ext = pl.b_ext; p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles; p.NT = pl.NT;
+    p.OWt = pl.OWt; p.OHt = pl.OHt; p.tiles_w = pl.tiles_w; p.Kt = pl.Kt; p.k_tiles = pl.k_tiles;
+    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.a_bytes = pl.a_bytes;
+    p.mode = 3; p.status = status; p.factor = factor;
+    p.wait_polls = g_wait_polls.load(std::memory_order_relaxed);
+    const int tiles = pl.m_tiles * pl.n_tiles;
+    scaled_tiles_split(g, pl, p.splits, p.per_split);
+    p.sum_out = p.splits > 1 ? static_cast<float *>(tc_workspace) : acc_w;
+    p.total_tiles = p.splits * tiles;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(conv_wgrad_clip1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute");
+    conv_wgrad_clip1_kernel<<<(unsigned)p.total_tiles, kClipThreads, pl.smem, stream>>>(tmX, tmY, p);
+    DP_LAUNCH_CHECK("conv_wgrad_clip1_kernel");
     if (p.splits > 1) return launch_fold_partial_sums(p.sum_out, p.splits, (long long)g.M * g.N, acc_w, stream);
     return DP_OK;
 }

@@ -42,6 +42,12 @@ bool tc_clip_scaled_sum(int dtype, const ConvGeom &g);
 dp_status launch_conv_ssum(int dtype, const void *X, const void *dY, const ConvGeom &g, const float *factor, float *acc_w,
                            void *tc_workspace, int *status, cudaStream_t stream);
 
+// The same clipped sum with known factors, per example through tensor memory (one tile per CTA, an example range per
+// CTA, each finished tile read once and scaled into registers): the better form when an example has 128 pixels or more.
+bool tc_clip_scaled_tiles(int dtype, const ConvGeom &g);
+dp_status launch_conv_scaled_tiles(int dtype, const void *X, const void *dY, const ConvGeom &g, const float *factor, float *acc_w,
+                                   void *tc_workspace, int *status, cudaStream_t stream);
+
 // bf16 layers whose whole output plane is at most 256 pixels: per-example squared norms (and factors against
 // clipinfo.C_l into factor_out[2n], factor_out[2n+1], when given) from the Gram matrices of dY and of the unfolded
 // input over the pixels, without forming the gradient.  Weight group only; not for unfolded layers.
