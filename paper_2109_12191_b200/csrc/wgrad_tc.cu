@@ -830,11 +830,12 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
 #pragma unroll
         for (int i = 0; i < 128; ++i) run[i] = 0.f;
         bool live = true;
-        // One step behind: an example's partial sums travel through the cluster while the next example's tile is being
-        // square-summed, and its tile is scaled after that.  Step s hands in example s and then scales example s - 1.
+        // One step behind, with two tiles of tensor memory: step s first finishes example s - 1 (waits for its partial sums
+        // from the whole cluster, scales its tile into the running sum and hands the tile's columns back to the MMA warp,
+        // which starts on example s + 1), then square-sums example s and sends its partial sums on their way.
         // Slots and barriers of the exchange come in fours: a slot of example j is overwritten by example j + 4, which a
-        // warp sends only after it has scaled example j + 2, i.e. after every warp of the cluster has sent example
-        // j + 2, which each of them did after scaling (and so after reading the slots of) example j.
+        // warp sends only after it has scaled example j + 3, i.e. after every warp of the cluster has sent example
+        // j + 3, which each of them did after scaling (and so after reading the slots of) example j + 2 and before it j.
         const int count = n_hi - n_lo;
         for (int step = 0; known && step < count && live; ++step) {
             // factors known: one read of the finished tile per example, scaled into the running sum
@@ -862,6 +863,43 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
             if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
         }
         for (int step = 0; !known && step <= count && live; ++step) {
+            if (step >= 1) {
+                // finish example step - 1 first: its tile leaves tensor memory before this step's tile is touched, so the
+                // MMAs of the example after this one run while this step's tile is being square-summed
+                const int j = step - 1, n = n_lo + j, buf = j & 1, slot = j & 3;
+                const bool all_in = mbar_wait_cluster(smem_u32(&norm_bar[slot]), (uint32_t)((j >> 2) & 1), abort_p, p.wait_polls);
+                if (!__all_sync(0xffffffffu, all_in)) { live = false; break; }
+                // the same tree in every warp of every CTA (two entries a lane, then a butterfly): all of them apply the
+                // identical factor
+                const float *parts = &norm_part[slot][0][0];
+                const int entries = cs * 8;
+                double sn = (lane < entries ? (double)parts[lane] : 0.0) + (lane + 32 < entries ? (double)parts[lane + 32] : 0.0);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) sn += __shfl_xor_sync(0xffffffffu, sn, o);
+                const float f = clip_factor(sn, p.C_l);
+                if (rank == 0 && e == 0 && lane == 0) {
+                    p.sqnorm[n * p.sq_stride] = (float)sn;
+                    if (p.clip_out) p.clip_out[n] = f;
+                }
+                // pass 2: scale the tile into the running sum
+                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    if (c2 * 64 < my_cols) {
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
+                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
+                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            }
             if (step < count) {
                 const int buf = step & 1, slot = step & 3;
                 const bool arrived = mbar_wait(smem_u32(&tmem_full[buf]), (uint32_t)((step >> 1) & 1), abort_p, p.wait_polls);
@@ -892,39 +930,6 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
                     st_cluster_f32(map_to_cta(smem_u32(&norm_part[slot][rank][e]), (uint32_t)lane), sq);
                     mbar_arrive_remote(map_to_cta(smem_u32(&norm_bar[slot]), (uint32_t)lane));
                 }
-            }
-            if (step >= 1) {
-                const int j = step - 1, n = n_lo + j, buf = j & 1, slot = j & 3;
-                const bool all_in = mbar_wait_cluster(smem_u32(&norm_bar[slot]), (uint32_t)((j >> 2) & 1), abort_p, p.wait_polls);
-                if (!__all_sync(0xffffffffu, all_in)) { live = false; break; }
-                // the same order in every warp of every CTA: all of them apply the identical factor
-                double sn = 0.0;
-                for (int r = 0; r < cs; ++r)
-#pragma unroll
-                    for (int w = 0; w < 8; ++w) sn += (double)norm_part[slot][r][w];
-                const float f = clip_factor(sn, p.C_l);
-                if (rank == 0 && e == 0 && lane == 0) {
-                    p.sqnorm[n * p.sq_stride] = (float)sn;
-                    if (p.clip_out) p.clip_out[n] = f;
-                }
-                // pass 2: scale the tile into the running sum
-                const uint32_t t_addr = tmem_base + (uint32_t)(buf * 256 + half * 128) + ((uint32_t)(q * 32) << 16);
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
-                    if (c2 * 64 < my_cols) {
-                        uint32_t v0[32], v1[32];
-                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64), v0);
-                        tmem_ld32_issue(t_addr + (uint32_t)(c2 * 64 + 32), v1);
-                        tmem_ld_wait32(v0); tmem_ld_wait32(v1);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) run[c2 * 64 + i] = fmaf(f, __uint_as_float(v0[i]), run[c2 * 64 + i]);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) run[c2 * 64 + 32 + i] = fmaf(f, __uint_as_float(v1[i]), run[c2 * 64 + 32 + i]);
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
             }
         }
         if (live && row_ok) {
