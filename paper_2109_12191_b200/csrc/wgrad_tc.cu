@@ -673,6 +673,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
+// one-way remote store that reports its bytes to a barrier of the receiving CTA (no separate arrival to release it)
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(cluster_addr), "r"(__float_as_uint(v)), "r"(cluster_bar) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
@@ -696,8 +701,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 __global__ void __launch_bounds__(kClipThreads, 1)
 conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2], norm_bar[4];
-    __shared__ float norm_part[4][kMaxCluster][8];      // [example mod 4][source CTA][source epilogue warp]
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2], norm_bar[4], warp_bar[4];
+    __shared__ float warp_part[4][8];                   // [example mod 4][epilogue warp]: this CTA's partial sums
+    __shared__ float norm_part[4][kMaxCluster];         // [example mod 4][source CTA]: every CTA's sum, sent by its first epilogue warp
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -718,7 +724,7 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 2); mbar_init(smem_u32(&empty_bar[s]), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&tmem_full[b]), 1); mbar_init(smem_u32(&tmem_empty[b]), 8); }
-        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&norm_bar[b]), (uint32_t)(cs * 8));
+        for (int b = 0; b < 4; ++b) { mbar_init(smem_u32(&norm_bar[b]), 1); mbar_init(smem_u32(&warp_bar[b]), 8); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
@@ -871,12 +877,13 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
                 if (!__all_sync(0xffffffffu, all_in)) { live = false; break; }
                 // the same tree in every warp of every CTA (two entries a lane, then a butterfly): all of them apply the
                 // identical factor
-                const float *parts = &norm_part[slot][0][0];
-                const int entries = cs * 8;
-                double sn = (lane < entries ? (double)parts[lane] : 0.0) + (lane + 32 < entries ? (double)parts[lane + 32] : 0.0);
+                double sn = lane < cs ? (double)norm_part[slot][lane] : 0.0;
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) sn += __shfl_xor_sync(0xffffffffu, sn, o);
-                const float f = clip_factor(sn, p.C_l);
+                for (int o = 4; o > 0; o >>= 1) sn += __shfl_xor_sync(0xffffffffu, sn, o);      // (at most eight CTAs)
+                sn = __shfl_sync(0xffffffffu, sn, 0);
+                // min(1, C_l / sqrt(sn)) in single precision here: the double-precision square root and division are
+                // some hundreds of cycles on the path every example waits on
+                const float f = (sn <= (double)p.C_l * (double)p.C_l) ? 1.0f : p.C_l / sqrtf((float)sn);
                 if (rank == 0 && e == 0 && lane == 0) {
                     p.sqnorm[n * p.sq_stride] = (float)sn;
                     if (p.clip_out) p.clip_out[n] = f;
@@ -924,11 +931,20 @@ conv_wgrad_clip1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
                     }
                 }
                 const float sq = warp_sum((sq4[0] + sq4[1]) + (sq4[2] + sq4[3]));
-                if (lane < cs) {
-                    // lane r tells CTA r (every lane holds the warp's sum): the remote store and the remote arrival that
-                    // releases it cost a round trip through the cluster each, so the peers are served side by side, not in turn
-                    st_cluster_f32(map_to_cta(smem_u32(&norm_part[slot][rank][e]), (uint32_t)lane), sq);
-                    mbar_arrive_remote(map_to_cta(smem_u32(&norm_bar[slot]), (uint32_t)lane));
+                // The CTA's eight partial sums meet in its own shared memory first; its first epilogue warp adds them and
+                // tells the cluster: lane r sends the sum to CTA r with a store that reports its bytes to that CTA's barrier
+                // (one way; a plain remote store followed by a releasing remote arrival costs a round trip more).
+                if (lane == 0) { warp_part[slot][e] = sq; mbar_arrive(smem_u32(&warp_bar[slot])); }
+                if (e == 0) {
+                    const bool mine_in = mbar_wait(smem_u32(&warp_bar[slot]), (uint32_t)((step >> 2) & 1), abort_p, p.wait_polls);
+                    if (!__all_sync(0xffffffffu, mine_in)) { live = false; break; }
+                    const float *w = warp_part[slot];
+                    const float cta_sq = ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
+                    // this CTA expects one float from every CTA of the cluster (its own included) in this slot's phase
+                    if (lane == 0) mbar_expect_tx(smem_u32(&norm_bar[slot]), (uint32_t)(cs * 4));
+                    if (lane < cs)
+                        st_async_f32(map_to_cta(smem_u32(&norm_part[slot][rank]), (uint32_t)lane), cta_sq,
+                                     map_to_cta(smem_u32(&norm_bar[slot]), (uint32_t)lane));
                 }
             }
         }
