@@ -187,6 +187,12 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             if (rc != DP_OK) return rc;
         }
         if (epi != DP_EPI_CLIP_ACCUM) {
+            if (pl.use_tc && epi == DP_EPI_NORM_ONLY && !d->has_bias && single_pass_enabled() && tc_gram_norm(d->dtype, g) &&
+                !tc_clip_single_pass(d->dtype, g)) {
+                // norms only, a large gradient over a small plane: from the pixel Gram matrices, without forming the gradient
+                const TcInlineClip ic = {0.f, sqnorm, sqnorm_stride, nullptr};
+                return launch_conv_gram_norm(d->dtype, X, dY, g, ic, nullptr, reinterpret_cast<int *>(ws + pl.status_off), st);
+            }
             if (pl.use_tc) {
                 // one launch: the kernel's last CTA folds the partial norms (a ticket in the workspace header)
                 const TcPublish pub = {reinterpret_cast<int *>(ws + kWsCounterOffset), pl.w_slots, groups == 2, sqnorm, sqnorm_stride, nullptr, 0.f, nullptr};
