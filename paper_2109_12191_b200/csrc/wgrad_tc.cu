@@ -658,7 +658,7 @@ constexpr int kClipThreads = 384;
 constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
 static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
 constexpr int kMaxCluster = 8;
-constexpr int kMinExamplesPerCluster = 16;   // examples a cluster walks through when an SM target is set (calls run side by side)
+constexpr int kMinExamplesPerCluster = 32;   // examples a cluster walks through when an SM target is set (calls run side by side)
 
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -1656,7 +1656,8 @@ static void cluster_split(int B, int cluster_size, int K, int NT, int &splits, i
     int want = std::min(sm_target() / cluster_size, max_active_clusters(cluster_size));
     // A caller that set an SM target runs calls side by side: what counts then is SM time, and a cluster that walks
     // through several examples spends its start-up, its first loads and its final stores once for all of them -- up
-    // to sixteen examples, and not beyond some 60 microseconds a launch, so that no call holds its stream up for long.
+    // to thirty-two examples (a whole chunk of the per-layer workload: one example range, nothing to fold), and not
+    // beyond some 60 microseconds a launch, so that no call holds its stream up for long.
     if (sm_target_set()) {
         const double cycles = (K / 16.0) * std::max(NT / 2.0, 64.0) * 1.5;
         const int per = std::max(1, std::min(kMinExamplesPerCluster, (int)(120000.0 / cycles)));

@@ -356,7 +356,7 @@ def test_gram_norm_waits_are_bounded():
 
 @pytest.mark.parametrize("case", [(64, 128, 3, 1, 1, 14), (128, 256, 3, 1, 1, 14), (3, 64, 7, 2, 3, 30), (256, 64, 1, 1, 0, 28)])
 def test_fused_clip_under_an_sm_target_with_a_ragged_batch(case):
-    """With an SM target set (calls meant to run side by side) a cluster walks through up to sixteen examples and the
+    """With an SM target set (calls meant to run side by side) a cluster walks through up to thirty-two examples and the
     one-product clipped sum takes fewer example ranges: 37 examples leave a ragged last range in both."""
     Cin, Kout, R, stride, pad, H = case
     b = B()
