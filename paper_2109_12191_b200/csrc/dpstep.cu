@@ -187,9 +187,10 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
             if (rc != DP_OK) return rc;
         }
         if (epi != DP_EPI_CLIP_ACCUM) {
-            if (pl.use_tc && epi == DP_EPI_NORM_ONLY && !d->has_bias && single_pass_enabled() && tc_gram_norm(d->dtype, g) &&
-                !tc_clip_single_pass(d->dtype, g)) {
-                // norms only, a large gradient over a small plane: from the pixel Gram matrices, without forming the gradient
+            if (pl.use_tc && epi == DP_EPI_NORM_ONLY && !d->has_bias && single_pass_enabled() && sm_target_set() &&
+                tc_gram_norm(d->dtype, g) && !tc_clip_single_pass(d->dtype, g)) {
+                // norms only, a large gradient over a small plane, calls running side by side: from the pixel Gram matrices,
+                // without forming the gradient (far less SM time; a call that has the GPU to itself is quicker on all SMs)
                 const TcInlineClip ic = {0.f, sqnorm, sqnorm_stride, nullptr};
                 return launch_conv_gram_norm(d->dtype, X, dY, g, ic, nullptr, reinterpret_cast<int *>(ws + pl.status_off), st);
             }
