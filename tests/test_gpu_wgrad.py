@@ -367,3 +367,23 @@ def test_fused_clip_under_an_sm_target_with_a_ragged_batch(case):
     finally:
         b.check(b.dp_set_sm_target(0))
     assert out["uses_tc"]
+
+
+@pytest.mark.parametrize("case", [(128, 256, 3, 1, 1, 14), (512, 512, 3, 1, 1, 7), (256, 1024, 1, 1, 0, 14), (3, 64, 7, 2, 3, 30)])
+@pytest.mark.parametrize("target", [0, 1])
+def test_fused_clip_rerun_is_bit_identical(case, target):
+    """Norms from Gram matrices, the known-factor and one-product clipped sums, the cluster exchange and the
+    space-to-depth stem add in a fixed order: a second run gives the same bits, with and without an SM target."""
+    Cin, Kout, R, stride, pad, H = case
+    b = B()
+    layer = synth.conv(Cin, Kout, R, stride, pad, H, False, name=str(case))
+    inp = scaled_inputs(layer, 9, "bf16", 963, sum(case), spread=True)
+    b.check(b.dp_set_sm_target(torch.cuda.get_device_properties(0).multi_processor_count if target else 0))
+    try:
+        one = gpu_layer(layer, inp, "bf16", CLIP, AUTO, 0, C_l=0.7)
+        two = gpu_layer(layer, inp, "bf16", CLIP, AUTO, 0, C_l=0.7)
+    finally:
+        b.check(b.dp_set_sm_target(0))
+    np.testing.assert_array_equal(one["acc_w"], two["acc_w"])
+    np.testing.assert_array_equal(one["sq"], two["sq"])
+    np.testing.assert_array_equal(one["clip"], two["clip"])
