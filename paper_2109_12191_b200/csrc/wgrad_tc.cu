@@ -643,12 +643,13 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 // Per-layer clipping needs an example's whole squared norm before any entry of its gradient can be scaled, so the
 // kernel above runs every contraction twice (a norm pass, then the clipped sum).  Here each contraction runs once:
 // a thread-block cluster owns ALL tiles of one example's gradient of this layer, one tile per CTA, kept in the CTA's
-// tensor memory.  Every CTA square-sums its tile, the CTAs exchange their partial sums through distributed shared
-// memory (plain remote stores plus a remote mbarrier arrival; every CTA loads its own operands, nothing is
-// multicast), every CTA then knows the example's norm and factor, scales its tile into a running sum held in
-// registers, and moves on to the cluster's next example while the tensor core already fills the other accumulator
-// buffer.  Clusters split the batch; with more than one cluster the running sums leave as partial sums, folded in
-// cluster order by the launch that follows.
+// tensor memory.  Every CTA square-sums its tile, the CTAs exchange their sums through distributed shared memory
+// (one remote store per pair of CTAs that reports its bytes to the receiver's barrier; every CTA loads its own
+// operands, nothing is multicast), every CTA then knows the example's norm and factor, scales its tile into a running
+// sum held in registers, and moves on to the cluster's next example while the tensor core already fills the other
+// accumulator buffer.  Clusters split the batch; with more than one cluster the running sums leave as partial sums,
+// folded in cluster order by the launch that follows.  Given the factors beforehand (norms from the Gram-matrix kernel
+// below) the same kernel runs without clusters and without the norm pass: one tile a CTA, any number of tiles.
 //
 // Roles (384 threads): warp 0 issues the TMA loads of the A slabs, warp 2 those of the B slabs, warp 1 allocates tensor
 // memory and issues the MMAs, warp 3 idles; warps 4-11 are the epilogue: warp w reads TMEM lanes 32*(w%4).. and the
@@ -658,7 +659,7 @@ constexpr int kClipThreads = 384;
 constexpr int kClipRegsLaunch = 168, kClipRegsControl = 56, kClipRegsEpilogue = 224;
 static_assert(128 * kClipRegsControl + 256 * kClipRegsEpilogue == kClipThreads * kClipRegsLaunch, "register split must add up");
 constexpr int kMaxCluster = 8;
-constexpr int kMinExamplesPerCluster = 32;   // examples a cluster walks through when an SM target is set (calls run side by side)
+constexpr int kMaxExamplesPerCluster = 32;   // examples a cluster walks through when an SM target is set (calls run side by side)
 
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -670,16 +671,10 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
 // one-way remote store that reports its bytes to a barrier of the receiving CTA (no separate arrival to release it)
 __device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
                  ::"r"(cluster_addr), "r"(__float_as_uint(v)), "r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -1660,7 +1655,7 @@ static void cluster_split(int B, int cluster_size, int K, int NT, int &splits, i
     // beyond some 60 microseconds a launch, so that no call holds its stream up for long.
     if (sm_target_set()) {
         const double cycles = (K / 16.0) * std::max(NT / 2.0, 64.0) * 1.5;
-        const int per = std::max(1, std::min(kMinExamplesPerCluster, (int)(120000.0 / cycles)));
+        const int per = std::max(1, std::min(kMaxExamplesPerCluster, (int)(120000.0 / cycles)));
         want = std::min(want, std::max(1, B / per));
     }
     if (want < 1) want = 1;
