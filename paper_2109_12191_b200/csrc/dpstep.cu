@@ -256,10 +256,9 @@ extern "C" dp_status dp_per_example_wgrad(const dp_layer_desc *d, const void *X,
                                sqnorm_stride, clip, C_l, factor, clip_out, st);
         if (rc != DP_OK || !clip) return rc;
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis
-        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor, 2, d->B, d->C_in, d->K_out, acc_w, st);
-        if (rc != DP_OK) return rc;
-        if (d->has_bias) return launch_bias_accum(db_ws, d->B, d->K_out, factor, acc_b, st);
-        return DP_OK;
+        // (the bias gradient of a dense layer is dY: its clipped sum rides in the same launch, with the bias factor)
+        return launch_dense_scaled_sum(storage_type(d), X, dY, factor, 2, d->B, d->C_in, d->K_out, acc_w, st,
+                                       d->has_bias ? factor + 1 : nullptr, 2, d->has_bias ? acc_b : nullptr);
     }
 
     // normalisation affine
@@ -305,11 +304,9 @@ extern "C" dp_status dp_per_example_wgrad_scaled(const dp_layer_desc *d, const v
     dp_status rc;
     if (d->kind == DP_LAYER_DENSE) {
         // sum_n f_n dY_n^T X_n is one matrix product with the batch as the reduction axis; the bias gradient is dY itself.
-        // Both kernels read the caller's factors in place.
-        rc = launch_dense_scaled_sum(storage_type(d), X, dY, factor_w, factor_stride, d->B, d->C_in, d->K_out, acc_w, st);
-        if (rc != DP_OK) return rc;
-        if (d->has_bias) rc = launch_dense_bias_accum(storage_type(d), dY, d->B, d->K_out, factor_b, factor_stride, acc_b, st);
-        return rc;
+        // One launch does both and reads the caller's factors in place.
+        return launch_dense_scaled_sum(storage_type(d), X, dY, factor_w, factor_stride, d->B, d->C_in, d->K_out, acc_w, st,
+                                       d->has_bias ? factor_b : nullptr, factor_stride, d->has_bias ? acc_b : nullptr);
     }
     // the clipped-sum kernels read one (weight, bias) pair of factors per example
     rc = launch_expand_factor(factor_w, factor_b, factor_stride, d->B, factor, st);

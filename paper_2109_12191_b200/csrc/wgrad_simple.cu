@@ -541,11 +541,21 @@ bias_vec_kernel(const T *__restrict__ dY, int K, int Kout, float *__restrict__ d
     for (int v = 0; v < VEC; ++v) a[v] = 0.f;
     if (prow < rows) {
         const T *base = dY + (long long)n * K * Kout + kv * VEC;
-        for (int pix = prow; pix < K; pix += rows) {
-            T g[VEC];
-            *reinterpret_cast<uint4 *>(g) = __ldcs(reinterpret_cast<const uint4 *>(base + (long long)pix * Kout));
+        // eight pixels per trip, all loads issued before any addition (a block is one example: few threads, so the
+        // loads in flight per thread are what hides the memory latency); pixels still add in pixel order
+        for (int pix = prow; pix < K; pix += 8 * rows) {
+            uint4 g[8];
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) a[v] += to_float(g[v]);
+            for (int u = 0; u < 8; ++u)
+                if (pix + u * rows < K) g[u] = __ldcs(reinterpret_cast<const uint4 *>(base + (long long)(pix + u * rows) * Kout));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (pix + u * rows < K) {
+                    const T *gv = reinterpret_cast<const T *>(&g[u]);
+#pragma unroll
+                    for (int v = 0; v < VEC; ++v) a[v] += to_float(gv[v]);
+                }
+            }
         }
 #pragma unroll
         for (int v = 0; v < VEC; ++v) red[prow * Kout + kv * VEC + v] = a[v];
@@ -626,9 +636,29 @@ constexpr int kDenseOT = 16;
 template <typename T>
 __global__ void __launch_bounds__(256)
 dense_scaled_sum_kernel(const T *__restrict__ X, const T *__restrict__ dY, const float *__restrict__ factor,
-                        long long f_stride, int B, int Cin, int Kout, float *__restrict__ acc) {
+                        long long f_stride, int B, int Cin, int Kout, float *__restrict__ acc,
+                        const float *__restrict__ factor_b, long long fb_stride, float *__restrict__ acc_b) {
     __shared__ __align__(16) float fy[256][kDenseOT];
     __shared__ float part[8][kDenseOT][32];
+    __shared__ float bsum[16][kDenseOT];
+    // the bias gradient of a dense layer is dY itself: the first column block of every output group also adds
+    // acc_b[o] += sum_n fb_n dY[n, o] (16 outputs x 16 example groups, groups folded in order), which saves a launch
+    if (acc_b && blockIdx.x == 0) {
+        const int o = threadIdx.x & (kDenseOT - 1), gq = threadIdx.x >> 4, oo = blockIdx.y * kDenseOT + o;
+        float sum = 0.f;
+        if (oo < Kout) {
+#pragma unroll 8
+            for (int n = gq; n < B; n += 16) sum = fmaf(factor_b[n * fb_stride], to_float(dY[(long long)n * Kout + oo]), sum);
+        }
+        bsum[gq][o] = sum;
+        __syncthreads();
+        if (threadIdx.x < kDenseOT && blockIdx.y * kDenseOT + threadIdx.x < Kout) {
+            float t = bsum[0][threadIdx.x];
+#pragma unroll
+            for (int g2 = 1; g2 < 16; ++g2) t += bsum[g2][threadIdx.x];
+            acc_b[blockIdx.y * kDenseOT + threadIdx.x] += t;
+        }
+    }
     const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
     const int i = blockIdx.x * 32 + lane, o0 = blockIdx.y * kDenseOT;
     float a[kDenseOT];
@@ -1103,24 +1133,15 @@ dp_status launch_bias_accum(const float *db, int B, int Kout, const float *facto
     return DP_OK;
 }
 
-dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *f, long long f_stride, float *acc_b,
-                                  cudaStream_t st) {
-    if (dtype == DP_F32)
-        bias_accum_kernel<float><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const float *>(dY), B, Kout, f, f_stride, acc_b);
-    else
-        bias_accum_kernel<__nv_bfloat16><<<(Kout + 31) / 32, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(dY), B, Kout, f, f_stride, acc_b);
-    DP_LAUNCH_CHECK("bias_accum_kernel");
-    return DP_OK;
-}
-
 dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, long long f_stride, int B,
-                                  int Cin, int Kout, float *acc_w, cudaStream_t st) {
+                                  int Cin, int Kout, float *acc_w, cudaStream_t st, const float *factor_b, long long fb_stride,
+                                  float *acc_b) {
     const dim3 grid((unsigned)((Cin + 31) / 32), (unsigned)((Kout + kDenseOT - 1) / kDenseOT));
     if (grid.y > 65535) return DP_ERR_UNSUPPORTED;
     if (dtype == DP_F32)
-        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, f_stride, B, Cin, Kout, acc_w);
+        dense_scaled_sum_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(dY), factor, f_stride, B, Cin, Kout, acc_w, factor_b, fb_stride, acc_b);
     else
-        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, f_stride, B, Cin, Kout, acc_w);
+        dense_scaled_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(dY), factor, f_stride, B, Cin, Kout, acc_w, factor_b, fb_stride, acc_b);
     DP_LAUNCH_CHECK("dense_scaled_sum_kernel");
     return DP_OK;
 }

@@ -46,12 +46,11 @@ dp_status launch_finalize(const float *partial, int B, int slots, int w_slots, i
 // acc_b[k] += sum_n factor[n*2+which] * db[n,k]
 dp_status launch_bias_accum(const float *db, int B, int Kout, const float *factor, float *acc_b, cudaStream_t stream,
                             int which = 1);
-// dense layer, db = dY: acc_b[k] += sum_n f[n*f_stride] * dY[n,k]
-dp_status launch_dense_bias_accum(int dtype, const void *dY, int B, int Kout, const float *f, long long f_stride, float *acc_b,
-                                  cudaStream_t stream);
-// dense layer: acc_w[o, i] += sum_n factor[n*f_stride] * dY[n, o] * X[n, i]
+// dense layer: acc_w[o, i] += sum_n factor[n*f_stride] * dY[n, o] * X[n, i]; with acc_b also (same launch)
+// acc_b[o] += sum_n factor_b[n*fb_stride] * dY[n, o]
 dp_status launch_dense_scaled_sum(int dtype, const void *X, const void *dY, const float *factor, long long f_stride, int B,
-                                  int Cin, int Kout, float *acc_w, cudaStream_t stream);
+                                  int Cin, int Kout, float *acc_w, cudaStream_t stream, const float *factor_b = nullptr,
+                                  long long fb_stride = 0, float *acc_b = nullptr);
 // factor2[n] = (factor_w[n*stride], factor_b[n*stride])
 dp_status launch_expand_factor(const float *factor_w, const float *factor_b, long long stride, int B, float *factor2,
                                cudaStream_t stream);
