@@ -128,7 +128,10 @@ class SmallCnn:
         self.layers, self.B = self.cfg["layers"], self.cfg["B"]
         self.lanes = int(os.environ.get("DP_BENCH_LANES", "4"))
         from paper_2109_12191_b200 import binding
-        binding.check(binding.dp_set_sm_target(0))
+        # the two tensor-core convolutions run side by side on their own streams: each is told to take half of the SMs
+        # (a call that spreads over all of them makes the other wait for its turn)
+        self.sm_target = int(os.environ.get("DP_BENCH_SM_TARGET", str(torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count // 2)))
+        binding.check(binding.dp_set_sm_target(self.sm_target))
         # layers whose per-example gradients outweigh their inputs (conv3, the classifier) are not materialised
         self.recompute = os.environ.get("DP_BENCH_RECOMPUTE", "auto")
         # fp32 inputs; tensor-core layers take them as tf32 (one pass, the precision class the accuracy bounds name)
@@ -156,7 +159,7 @@ class SmallCnn:
                 "examples_per_step": self.B, "params": self.step_obj.P,
                 "l2": f"inputs rotate over {self.n_sets} resident sets ({self.n_sets * self.in_bytes / 1e6:.0f} MB) and "
                       f"{sum(self.step_obj.P_l[i] for i in self.step_obj._kept) * self.B * 4 / 1e6:.0f} MB of per-example gradients are written and re-read per step",
-                "streams": self.lanes,
+                "streams": self.lanes, "sm_target": self.sm_target,
                 "recomputed_layers": [self.layers[i].name for i in sorted(self.step_obj.recompute)]}
 
     def run(self, i, rec=None):

@@ -37,11 +37,21 @@ def test_graph_replay_equals_stream_launches():
 
 
 def test_small_cnn_step_as_benchmarked_matches_the_oracle():
-    """The composite the small-CNN benchmark times -- 256 examples, fp32 inputs taken as tf32, four streams, the
-    classifier's clipped sum recomputed instead of materialised, the whole step replayed from a CUDA graph --
-    against the oracle's privatisation step on the same inputs."""
+    """The composite the small-CNN benchmark times -- 256 examples, fp32 inputs taken as tf32, four streams, an SM target
+    of half the SMs, the classifier's clipped sum recomputed instead of materialised, the whole step replayed from a
+    CUDA graph -- against the oracle's privatisation step on the same inputs."""
+    from paper_2109_12191_b200 import binding
     cfg = synth.small_cnn()
     layers, Bn = cfg["layers"], cfg["B"]
+    # as in the benchmark: the convolutions run side by side, each told to take half of the SMs
+    binding.check(binding.dp_set_sm_target(torch.cuda.get_device_properties(0).multi_processor_count // 2))
+    try:
+        _small_cnn_as_benchmarked(cfg, layers, Bn)
+    finally:
+        binding.check(binding.dp_set_sm_target(0))
+
+
+def _small_cnn_as_benchmarked(cfg, layers, Bn):
     st = GlobalClipStep(layers, Bn, "tf32", cfg["C"], cfg["sigma"], lanes=4, recompute="auto")
     assert st.recompute                                    # the classifier is not materialised
     host = [synth.layer_inputs(l, Bn, "f32", 1, li, 0) for li, l in enumerate(layers)]
